@@ -1,0 +1,226 @@
+/*
+ * typhoon_mla.h -- C ABI of the B200 (sm_100a) MLA decode-attention library.
+ *
+ * The operation is the decode attention of Multi-Head Latent Attention when
+ * many requests share a long prefix of the KV cache (Algorithm 1, "TyphoonMLA
+ * Decode Attention Kernel"):
+ *
+ *   - the shared prefix is attended in the naive formulation over per-head
+ *     keys/values that were expanded once from the shared latent cache
+ *     (Section 3.1 "Prefill"; Algorithm 1 line 4);
+ *   - each request's own suffix is attended in the absorb formulation: q_nope
+ *     is moved through W_UK (= W_KVb1) into the latent space, attention runs
+ *     over the paged latent cache plus the rope keys, and the latent output is
+ *     projected through W_UV (= W_KVb2) (Algorithm 1 lines 5-7);
+ *   - the two normalised partial results are merged by their log-sum-exps
+ *     (Algorithm 1 line 8; Section 3.2 "CombineLSE");
+ *   - below a batch threshold the whole context runs in absorb form
+ *     (Section 3.1 "Fall-back to Absorb"; Eq. 1).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - Tensors are bf16 (raw uint16 storage) unless stated; accumulation,
+ *     softmax statistics, split partials and the combine are fp32.
+ *   - q_pe and all cached rope keys arrive already rotated: no RoPE is applied.
+ *   - softmax_scale multiplies the sum of the nope and the rope logits.
+ *   - Log-sum-exps are natural logarithms of sum(exp(scaled logit)).
+ *   - A single decode query attends to every cached token (no mask).
+ *   - Every call returns a status (0 = OK); nothing throws, aborts or traps.
+ *     Work is enqueued on the given cudaStream_t (passed as void*) and the call
+ *     returns without synchronising unless stated.
+ *   - Inputs are never modified.  `out` rows 0..B-1 are fully overwritten.
+ *   - There is no CPU fallback: without a CUDA device every compute entry
+ *     point returns TYPHOON_MLA_ERR_CUDA.
+ *
+ * Supported dimensions: d_nope = 128, d_rope = 64, d_v = 128,
+ * kv_lora_rank = 512, num_heads a multiple of 16 up to 128 (DeepSeek-v3: 128,
+ * Kimi-K2: 64), page_size 64 or 128, base pointers 16-byte aligned.
+ */
+#ifndef TYPHOON_MLA_H_
+#define TYPHOON_MLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct typhoon_mla_shared typhoon_mla_shared_t; /* opaque host object */
+
+typedef struct {
+    int32_t num_heads;     /* H   */
+    int32_t d_nope;        /* D_n */
+    int32_t d_rope;        /* D_r */
+    int32_t d_v;           /* D_v */
+    int32_t kv_lora_rank;  /* D_l */
+} typhoon_mla_dims_t;
+
+enum {
+    TYPHOON_MLA_OK = 0,
+    TYPHOON_MLA_ERR_INVALID_ARG = 1,
+    TYPHOON_MLA_ERR_UNSUPPORTED_DIMS = 2,
+    TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL = 3,
+    TYPHOON_MLA_ERR_ALLOC = 4,
+    TYPHOON_MLA_ERR_CUDA = 5,
+    TYPHOON_MLA_ERR_DEVICE_CHECK = 6
+};
+
+enum {
+    TYPHOON_MLA_MODE_AUTO = 0,   /* crossover rule decides (ABSORB or HYBRID; NAIVE if max_pages == 0) */
+    TYPHOON_MLA_MODE_ABSORB = 1, /* whole context in absorb form (the fall-back) */
+    TYPHOON_MLA_MODE_HYBRID = 2, /* Algorithm 1: naive over the prefix, absorb over the suffix */
+    TYPHOON_MLA_MODE_NAIVE = 3   /* shared prefix only (Algorithm 1 line 4 + combine); suffixes ignored */
+};
+
+/* Kinds for typhoon_mla_cost_model (rows of Table 1). */
+enum { TYPHOON_MLA_COST_NAIVE = 0, TYPHOON_MLA_COST_ABSORB = 1, TYPHOON_MLA_COST_TYPHOON = 2 };
+
+/*
+ * Expand the shared prefix (Section 3.1 "Prefill": the shared part of the
+ * latent cache is passed through the up-projection to form per-head K and V).
+ *
+ *   ckv_shared  bf16 [Ls, 512], row stride ld_ckv elements (>= 512)
+ *   kpe_shared  bf16 [Ls, 64],  row stride ld_kpe elements (>= 64)
+ *   w_uk        bf16 [H, 128, 512] contiguous   (W_KVb1)
+ *   w_uv        bf16 [H, 128, 512] contiguous   (W_KVb2)
+ *
+ * The handle OWNS (cudaMalloc) the expanded per-head keys K_nope [H, Ls', 128],
+ * the expanded values stored transposed V^T [H, 128, Ls'], a copy of the shared
+ * latent cache and rope keys, and a transposed copy of W_UK; Ls' is Ls rounded
+ * up to a multiple of 128, the padding is zero.  It BORROWS w_uv: the caller
+ * keeps w_uv alive and unchanged until typhoon_mla_free.  Ls may be 0.
+ * The work is enqueued on `stream`; the handle may be used on that stream at
+ * once, on other streams after the caller has ordered them behind it.
+ * Errors: NULL arguments or bad strides -> INVALID_ARG; other dimensions ->
+ * UNSUPPORTED_DIMS; cudaMalloc failure -> ALLOC (nothing is leaked).
+ */
+int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims /* host */,
+                               const void* ckv_shared, const void* kpe_shared,
+                               int64_t Ls, int64_t ld_ckv, int64_t ld_kpe,
+                               const void* w_uk, const void* w_uv,
+                               void* stream, typhoon_mla_shared_t** out_handle /* host */);
+
+/* Release the handle and the device memory it owns (synchronises the device).
+ * NULL is accepted. */
+int typhoon_mla_free(typhoon_mla_shared_t* shared);
+
+/* Bytes of scratch typhoon_mla_decode needs for this problem size in the worst
+ * case over modes (host, pure).  Returns 0 on invalid arguments. */
+size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* shared, int32_t B,
+                                   int32_t max_pages, int32_t page_size);
+
+/*
+ * One decode-attention step for B requests (Algorithm 1).
+ *
+ *   q_nope       bf16 [B, H, 128] contiguous
+ *   q_pe         bf16 [B, H, 64]  contiguous, RoPE already applied
+ *   ckv_pages    bf16 latent cache, token (page p, slot s) at
+ *                ckv_pages + (p * page_size + s) * ckv_token_stride, 512 wide
+ *   kpe_pages    bf16 rope keys, same addressing with kpe_token_stride, 64 wide
+ *                (strides in elements, multiples of 8; a fused 576-wide page
+ *                layout can be passed by pointing both into it)
+ *   block_table  int32 [B, max_pages]: physical page of each logical page;
+ *                entries at or beyond ceil(seq_lens[b] / page_size) are ignored
+ *   seq_lens     int32 [B]: suffix length of each request, may be 0; values
+ *                above max_pages * page_size are clamped to it
+ *   out          bf16 [B, H, 128]
+ *   lse_out      optional fp32 [B, H] (NULL to skip): ln sum exp over the whole
+ *                context of each (request, head)
+ *   workspace    at least typhoon_mla_workspace_bytes() bytes, 256-byte
+ *                aligned; contents are scratch.  Calls that overlap in time
+ *                need distinct workspaces.
+ *
+ * Token slots past a request's length and unused block-table entries are never
+ * read into the result.  A request with no context at all (Ls = 0 and
+ * seq_lens[b] = 0) gets a zero output row and lse = -inf.
+ * The call never allocates and never synchronises.
+ * Errors: INVALID_ARG (NULL/misaligned pointers, B < 1, bad mode or page size),
+ * WORKSPACE_TOO_SMALL, CUDA (launch failure; see typhoon_mla_last_cuda_error).
+ */
+int typhoon_mla_decode(const typhoon_mla_shared_t* shared,
+                       const void* q_nope, const void* q_pe, int32_t B,
+                       const void* ckv_pages, const void* kpe_pages,
+                       int64_t ckv_token_stride, int64_t kpe_token_stride,
+                       int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                       const int32_t* seq_lens,
+                       float softmax_scale, int32_t mode,
+                       void* out, float* lse_out,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of device staging typhoon_mla_decode_host needs (host, pure). */
+size_t typhoon_mla_host_staging_bytes(const typhoon_mla_shared_t* shared, int32_t B, int32_t max_pages);
+
+/*
+ * The same step with the per-step tensors in HOST memory (pinned memory makes
+ * the copies asynchronous): q_nope, q_pe, block_table, seq_lens are copied to
+ * `staging` (device), the step runs, and `out` (host, bf16 [B, H, 128]) is
+ * copied back, all on `stream`.  The caches (ckv_pages, kpe_pages) stay device
+ * pointers.  The call returns after enqueueing; synchronise the stream before
+ * reading `out`.
+ */
+int typhoon_mla_decode_host(const typhoon_mla_shared_t* shared,
+                            const void* q_nope_host, const void* q_pe_host, int32_t B,
+                            const void* ckv_pages, const void* kpe_pages,
+                            int64_t ckv_token_stride, int64_t kpe_token_stride,
+                            int32_t page_size, const int32_t* block_table_host, int32_t max_pages,
+                            const int32_t* seq_lens_host,
+                            float softmax_scale, int32_t mode,
+                            void* out_host,
+                            void* staging, size_t staging_bytes,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Crossover rule (Section 3.1 "Fall-back to Absorb"; Eq. 1), host, pure.
+ * Returns TYPHOON_MLA_MODE_ABSORB or _HYBRID (or _NAIVE when
+ * total_suffix_tokens == 0 and Ls > 0) for a batch of B requests against this
+ * prefix; total_suffix_tokens < 0 means unknown.  The rule compares modelled
+ * times t_hybrid and t_absorb built from the Table 1 work terms, the hardware
+ * model set by typhoon_mla_set_hw_model and a fixed per-launch cost; ties go
+ * to ABSORB.
+ */
+int typhoon_mla_choose_mode(const typhoon_mla_shared_t* shared, int32_t B, int64_t total_suffix_tokens);
+
+/* The same rule from the dimensions and the prefix length alone (no handle, no device). */
+int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims /* host */, int64_t Ls, int32_t B,
+                                int64_t total_suffix_tokens);
+
+/* Hardware model of the crossover rule: sustained tensor throughput in FLOP/s,
+ * HBM bandwidth in bytes/s, fixed cost of the extra hybrid launches in
+ * seconds.  Non-positive values restore the defaults (B200 measured values).
+ * Process-wide; not thread-safe against concurrent decode calls. */
+int typhoon_mla_set_hw_model(double tensor_flops, double hbm_bytes_per_s, double hybrid_fixed_s);
+
+/* Eq. 1: B_theta = (D_qk + D_v) / (S_q (2 D_l + D_r)) * T / M.  Host, pure. */
+double typhoon_mla_batch_threshold(const typhoon_mla_dims_t* dims /* host */, int32_t S_q, double T, double M);
+
+/* Table 1: MACs and HBM words of the attention part for one of the three
+ * formulations (kind = TYPHOON_MLA_COST_*).  Host, pure.  L_n is the suffix
+ * length of every request. */
+int typhoon_mla_cost_model(const typhoon_mla_dims_t* dims /* host */, int32_t kind,
+                           int64_t B, int64_t S_q, int64_t L_s, int64_t L_n,
+                           int64_t* macs /* host */, int64_t* hbm_words /* host */);
+
+/* Read-only views of what the handle owns (for tests and accounting):
+ * k_nope bf16 [H, Ls_padded, 128]; v_t bf16 [H, 128, Ls_padded]. */
+int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
+                            const void** k_nope, const void** v_t,
+                            int64_t* Ls /* host */, int64_t* Ls_padded /* host */,
+                            int64_t* owned_bytes /* host */);
+
+/* Copy the expanded caches into caller buffers of H * Ls_padded * 128 bf16
+ * elements each (device memory), on `stream`. */
+int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_dst, void* v_t_dst, void* stream);
+
+/* Number of kernels the last typhoon_mla_decode call of this thread launched. */
+int typhoon_mla_last_launch_count(void);
+
+/* The cudaError_t (as int) behind the last TYPHOON_MLA_ERR_CUDA of this thread. */
+int typhoon_mla_last_cuda_error(void);
+
+const char* typhoon_mla_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TYPHOON_MLA_H_ */

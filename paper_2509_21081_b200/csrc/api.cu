@@ -1,0 +1,436 @@
+// C ABI of the library: argument validation, the prepared-prefix handle, the
+// workspace plan, the crossover rule (Eq. 1 / Table 1) and the launch sequence
+// of one decode step (Algorithm 1).
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/typhoon_mla.h"
+#include "kernels.h"
+
+using namespace tmla;
+
+struct typhoon_mla_shared {
+    typhoon_mla_dims_t dims;
+    int64_t Ls, Ls_pad;
+    void* k_nope;   // bf16 [H, Ls_pad, 128]
+    void* v_t;      // bf16 [H, 128, Ls_pad]
+    void* ckv;      // bf16 [Ls_pad, 512]
+    void* kpe;      // bf16 [Ls_pad, 64]
+    void* w_uk_t;   // bf16 [H, 512, 128]
+    const void* w_uv;  // borrowed, bf16 [H, 128, 512]
+    size_t owned_bytes;
+    int device;
+};
+
+namespace {
+
+thread_local int g_last_launches = 0;
+thread_local int g_last_cuda_error = 0;
+
+// Hardware model of the crossover rule (defaults: measured on B200).
+double g_tensor_flops = 1.0e15;      // sustained rate the attention kernels reach, FLOP/s
+double g_hbm_bytes = 6.0e12;         // bytes/s
+double g_hybrid_fixed_s = 6.0e-6;    // extra launches + combine of the hybrid path
+constexpr double kDefTensor = 1.0e15, kDefHbm = 6.0e12, kDefFixed = 6.0e-6;
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool dims_supported(const typhoon_mla_dims_t& d) {
+    return d.d_nope == 128 && d.d_rope == 64 && d.d_v == 128 && d.kv_lora_rank == 512 && d.num_heads >= 16 &&
+           d.num_heads <= 128 && d.num_heads % 16 == 0;
+}
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return TYPHOON_MLA_ERR_CUDA;
+}
+
+// ---- workspace plan --------------------------------------------------------
+struct Plan {
+    int mode;
+    int n_split_naive;       // KV splits of the naive kernel
+    int chunk;               // tokens per absorb chunk
+    int n_shared_chunks;     // absorb chunks over the shared prefix (ABSORB mode)
+    int n_suffix_chunks;
+    // byte offsets into the workspace
+    size_t off_qabs, off_opart_a, off_lsepart_a, off_olat, off_lse_a, off_oabs, off_opart_n, off_lsepart_n, total;
+};
+
+constexpr int kNumSM = 148;
+
+int naive_splits(int B, int H, int64_t Ls) {
+    if (Ls <= 0) return 0;
+    int n_tiles = (int)((Ls + 63) / 64);
+    int base = ((B + 63) / 64) * H;
+    int want = (4 * kNumSM + base - 1) / base;
+    return std::max(1, std::min({want, n_tiles, 64}));
+}
+
+void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chunk, int* n_sh, int* n_sf) {
+    int units = B * ((H + 63) / 64);
+    int target = std::max(1, (2 * kNumSM + units - 1) / units);
+    int64_t longest = std::max<int64_t>(std::max(Ls_absorb, cap_suffix), 1);
+    int64_t c = round_up((longest + target - 1) / target, 64);
+    c = std::max<int64_t>(c, 256);
+    *chunk = (int)c;
+    *n_sh = (int)((Ls_absorb + c - 1) / c);
+    *n_sf = (int)((cap_suffix + c - 1) / c);
+}
+
+Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size, int mode) {
+    Plan p{};
+    const int H = sh->dims.num_heads;
+    p.mode = mode;
+    const int64_t cap = (int64_t)max_pages * page_size;
+    const bool use_naive = (mode != TYPHOON_MLA_MODE_ABSORB) && sh->Ls > 0;
+    const bool use_absorb = (mode != TYPHOON_MLA_MODE_NAIVE);
+    p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls) : 0;
+    if (use_absorb) {
+        absorb_chunks(B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
+                      &p.n_suffix_chunks);
+    }
+    const int n_chunks = p.n_shared_chunks + p.n_suffix_chunks;
+    const size_t BH = (size_t)B * H;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off += round_up((int64_t)bytes, 256);
+        return o;
+    };
+    p.off_qabs = take(BH * 512 * 2);
+    p.off_opart_a = take((size_t)n_chunks * BH * 512 * 4);
+    p.off_lsepart_a = take((size_t)n_chunks * BH * 4);
+    p.off_olat = take(BH * 512 * 2);
+    p.off_lse_a = take(BH * 4);
+    p.off_oabs = take(BH * 128 * 4);
+    p.off_opart_n = take((size_t)p.n_split_naive * BH * 128 * 4);
+    p.off_lsepart_n = take((size_t)p.n_split_naive * BH * 4);
+    p.total = off;
+    return p;
+}
+
+int resolve_mode(const typhoon_mla_shared* sh, int B, int max_pages, int mode) {
+    if (mode == TYPHOON_MLA_MODE_AUTO) {
+        if (max_pages == 0 && sh->Ls > 0) return TYPHOON_MLA_MODE_NAIVE;
+        return typhoon_mla_choose_mode(sh, B, -1);
+    }
+    if (mode == TYPHOON_MLA_MODE_HYBRID && sh->Ls == 0) return TYPHOON_MLA_MODE_ABSORB;
+    return mode;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* typhoon_mla_status_string(int status) {
+    switch (status) {
+        case TYPHOON_MLA_OK: return "ok";
+        case TYPHOON_MLA_ERR_INVALID_ARG: return "invalid argument";
+        case TYPHOON_MLA_ERR_UNSUPPORTED_DIMS: return "unsupported dimensions";
+        case TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case TYPHOON_MLA_ERR_ALLOC: return "device allocation failed";
+        case TYPHOON_MLA_ERR_CUDA: return "CUDA error";
+        case TYPHOON_MLA_ERR_DEVICE_CHECK: return "device-side check failed";
+        default: return "unknown status";
+    }
+}
+
+int typhoon_mla_last_launch_count(void) { return g_last_launches; }
+int typhoon_mla_last_cuda_error(void) { return g_last_cuda_error; }
+
+double typhoon_mla_batch_threshold(const typhoon_mla_dims_t* d, int32_t S_q, double T, double M) {
+    if (!d || S_q < 1 || !(M > 0.0)) return -1.0;
+    const double d_qk = (double)d->d_nope + d->d_rope;
+    return (d_qk + d->d_v) / ((double)S_q * (2.0 * d->kv_lora_rank + d->d_rope)) * (T / M);
+}
+
+int typhoon_mla_cost_model(const typhoon_mla_dims_t* d, int32_t kind, int64_t B, int64_t S_q, int64_t L_s,
+                           int64_t L_n, int64_t* macs, int64_t* hbm_words) {
+    if (!d || B < 0 || S_q < 1 || L_s < 0 || L_n < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const int64_t H = d->num_heads;
+    const int64_t w_naive = H * ((int64_t)d->d_nope + d->d_rope + d->d_v);      // per (query, token) / per token
+    const int64_t w_abs_mac = H * (2 * (int64_t)d->kv_lora_rank + d->d_rope);
+    const int64_t w_abs_mem = (int64_t)d->kv_lora_rank + d->d_rope;
+    int64_t m, w;
+    switch (kind) {
+        case TYPHOON_MLA_COST_NAIVE:
+            m = B * S_q * (L_s + L_n) * w_naive;
+            w = (L_s + B * L_n) * w_naive;
+            break;
+        case TYPHOON_MLA_COST_ABSORB:
+            m = B * S_q * (L_s + L_n) * w_abs_mac;
+            w = (L_s + B * L_n) * w_abs_mem;
+            break;
+        case TYPHOON_MLA_COST_TYPHOON:
+            m = B * S_q * (L_s * w_naive + L_n * w_abs_mac);
+            w = L_s * w_naive + B * L_n * w_abs_mem;
+            break;
+        default: return TYPHOON_MLA_ERR_INVALID_ARG;
+    }
+    if (macs) *macs = m;
+    if (hbm_words) *hbm_words = w;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_set_hw_model(double tensor_flops, double hbm_bytes_per_s, double hybrid_fixed_s) {
+    g_tensor_flops = tensor_flops > 0 ? tensor_flops : kDefTensor;
+    g_hbm_bytes = hbm_bytes_per_s > 0 ? hbm_bytes_per_s : kDefHbm;
+    g_hybrid_fixed_s = hybrid_fixed_s >= 0 ? hybrid_fixed_s : kDefFixed;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int32_t B, int64_t total_suffix_tokens) {
+    if (!dims || B < 1 || Ls <= 0) return TYPHOON_MLA_MODE_ABSORB;
+    if (total_suffix_tokens == 0) return TYPHOON_MLA_MODE_NAIVE;
+    // Shared-prefix part only: the suffix part is identical in both modes.
+    // Work terms are Table 1's, with the rope keys of the expanded cache read
+    // once per token instead of once per head.
+    const typhoon_mla_dims_t& d = *dims;
+    const double H = d.num_heads, L = (double)Ls;
+    const double f_naive = 2.0 * B * H * L * (d.d_nope + d.d_rope + d.d_v);
+    const double f_absorb = 2.0 * B * H * L * (2.0 * d.kv_lora_rank + d.d_rope);
+    const double by_naive = 2.0 * L * (H * (d.d_nope + d.d_v) + d.d_rope);
+    const double by_absorb = 2.0 * L * (d.kv_lora_rank + d.d_rope);
+    const double t_hybrid = std::max(f_naive / g_tensor_flops, by_naive / g_hbm_bytes) + g_hybrid_fixed_s;
+    const double t_absorb = std::max(f_absorb / g_tensor_flops, by_absorb / g_hbm_bytes);
+    return t_hybrid < t_absorb ? TYPHOON_MLA_MODE_HYBRID : TYPHOON_MLA_MODE_ABSORB;
+}
+
+int typhoon_mla_choose_mode(const typhoon_mla_shared_t* sh, int32_t B, int64_t total_suffix_tokens) {
+    if (!sh) return TYPHOON_MLA_MODE_ABSORB;
+    return typhoon_mla_choose_mode_for(&sh->dims, sh->Ls, B, total_suffix_tokens);
+}
+
+int typhoon_mla_free(typhoon_mla_shared_t* sh) {
+    if (!sh) return TYPHOON_MLA_OK;
+    cudaDeviceSynchronize();
+    cudaFree(sh->k_nope);
+    cudaFree(sh->v_t);
+    cudaFree(sh->ckv);
+    cudaFree(sh->kpe);
+    cudaFree(sh->w_uk_t);
+    delete sh;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_shared, const void* kpe_shared,
+                               int64_t Ls, int64_t ld_ckv, int64_t ld_kpe, const void* w_uk, const void* w_uv,
+                               void* stream, typhoon_mla_shared_t** out_handle) {
+    if (!dims || !out_handle || !w_uk || !w_uv || Ls < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    *out_handle = nullptr;
+    if (!dims_supported(*dims)) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;
+    if (Ls > 0 && (!ckv_shared || !kpe_shared || ld_ckv < 512 || ld_kpe < 64 || ld_ckv % 8 || ld_kpe % 8 ||
+                   !aligned16(ckv_shared) || !aligned16(kpe_shared)))
+        return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!aligned16(w_uk) || !aligned16(w_uv) || Ls > (int64_t)1 << 24) return TYPHOON_MLA_ERR_INVALID_ARG;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    typhoon_mla_shared* sh = new (std::nothrow) typhoon_mla_shared();
+    if (!sh) return TYPHOON_MLA_ERR_ALLOC;
+    std::memset(sh, 0, sizeof(*sh));
+    sh->dims = *dims;
+    sh->Ls = Ls;
+    sh->Ls_pad = round_up(Ls, 128);
+    sh->w_uv = w_uv;
+    sh->device = dev;
+    const int H = dims->num_heads;
+    const size_t Lp = (size_t)sh->Ls_pad;
+    const size_t b_k = (size_t)H * Lp * 128 * 2, b_ckv = Lp * 512 * 2, b_kpe = Lp * 64 * 2,
+                 b_w = (size_t)H * 512 * 128 * 2;
+    auto alloc = [&](void** p, size_t bytes) {
+        if (bytes == 0) { *p = nullptr; return true; }
+        if (cudaMalloc(p, bytes) != cudaSuccess) { cudaGetLastError(); *p = nullptr; return false; }
+        sh->owned_bytes += bytes;
+        return true;
+    };
+    if (!alloc(&sh->k_nope, b_k) || !alloc(&sh->v_t, b_k) || !alloc(&sh->ckv, b_ckv) || !alloc(&sh->kpe, b_kpe) ||
+        !alloc(&sh->w_uk_t, b_w)) {
+        typhoon_mla_free(sh);
+        return TYPHOON_MLA_ERR_ALLOC;
+    }
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    e = launch_transpose_bf16(w_uk, sh->w_uk_t, 128, 512, H, s);
+    if (e == cudaSuccess && Ls > 0) {
+        e = launch_copy_pad_rows(ckv_shared, ld_ckv, sh->ckv, (int)Ls, (int)Lp, 512, s);
+        if (e == cudaSuccess) e = launch_copy_pad_rows(kpe_shared, ld_kpe, sh->kpe, (int)Ls, (int)Lp, 64, s);
+        if (e == cudaSuccess) {  // K_nope[h] = ckv * W_UK[h]^T
+            GemmTN g{sh->ckv, 512, 0, w_uk, 512, 128 * 512, sh->k_nope, 128, (int64_t)Lp * 128,
+                     (int)Lp, 128, 512, H, false};
+            e = launch_gemm_tn(g, s);
+        }
+        if (e == cudaSuccess) {  // V^T[h] = W_UV[h] * ckv^T
+            GemmTN g{w_uv, 512, 128 * 512, sh->ckv, 512, 0, sh->v_t, (int64_t)Lp, (int64_t)(128 * Lp),
+                     128, (int)Lp, 512, H, false};
+            e = launch_gemm_tn(g, s);
+        }
+    }
+    if (e != cudaSuccess) {
+        typhoon_mla_free(sh);
+        return cuda_fail(e);
+    }
+    *out_handle = sh;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_shared_view(const typhoon_mla_shared_t* sh, const void** k_nope, const void** v_t, int64_t* Ls,
+                            int64_t* Ls_padded, int64_t* owned_bytes) {
+    if (!sh) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (k_nope) *k_nope = sh->k_nope;
+    if (v_t) *v_t = sh->v_t;
+    if (Ls) *Ls = sh->Ls;
+    if (Ls_padded) *Ls_padded = sh->Ls_pad;
+    if (owned_bytes) *owned_bytes = (int64_t)sh->owned_bytes;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_shared_export(const typhoon_mla_shared_t* sh, void* k_nope_dst, void* v_t_dst, void* stream) {
+    if (!sh || !k_nope_dst || !v_t_dst) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)sh->dims.num_heads * (size_t)sh->Ls_pad * 128 * 2;
+    if (bytes == 0) return TYPHOON_MLA_OK;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(k_nope_dst, sh->k_nope, bytes, cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(v_t_dst, sh->v_t, bytes, cudaMemcpyDeviceToDevice, s);
+    return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
+}
+
+size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* sh, int32_t B, int32_t max_pages, int32_t page_size) {
+    if (!sh || B < 1 || max_pages < 0 || (page_size != 64 && page_size != 128)) return 0;
+    size_t a = make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_ABSORB).total;
+    size_t h = make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID).total;
+    return std::max(a, h) + 256;
+}
+
+int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
+                       const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
+                       int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                       const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    g_last_launches = 0;
+    if (!sh || !q_nope || !q_pe || !out || B < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (mode < TYPHOON_MLA_MODE_AUTO || mode > TYPHOON_MLA_MODE_NAIVE) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!(softmax_scale == softmax_scale)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    mode = resolve_mode(sh, B, max_pages, mode);
+    const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
+    if (use_absorb && max_pages > 0) {
+        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens) return TYPHOON_MLA_ERR_INVALID_ARG;
+        if (!aligned16(ckv_pages) || !aligned16(kpe_pages) || ckv_token_stride < 512 || kpe_token_stride < 64 ||
+            ckv_token_stride % 8 || kpe_token_stride % 8)
+            return TYPHOON_MLA_ERR_INVALID_ARG;
+    }
+    if (mode == TYPHOON_MLA_MODE_NAIVE && sh->Ls == 0) max_pages = 0;
+    const Plan pl = make_plan(sh, B, use_absorb ? max_pages : 0, page_size, mode);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
+
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = reinterpret_cast<char*>(workspace);
+    const int H = sh->dims.num_heads;
+    cudaError_t e = cudaSuccess;
+    int launches = 0;
+
+    float* o_part_n = reinterpret_cast<float*>(ws + pl.off_opart_n);
+    float* lse_part_n = reinterpret_cast<float*>(ws + pl.off_lsepart_n);
+    float* o_abs = reinterpret_cast<float*>(ws + pl.off_oabs);
+    float* lse_a = reinterpret_cast<float*>(ws + pl.off_lse_a);
+
+    // --- naive shared-prefix attention (Algorithm 1 line 4)
+    if (pl.n_split_naive > 0) {
+        NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad,
+                     pl.n_split_naive, softmax_scale, o_part_n, lse_part_n};
+        e = launch_naive_attn_mma(na, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+    }
+    const int n_chunks = pl.n_shared_chunks + pl.n_suffix_chunks;
+    const bool have_absorb = use_absorb && n_chunks > 0;
+    if (have_absorb) {
+        // --- query absorption Q_A = Q_N W_UK (Algorithm 1 line 5)
+        void* q_abs = ws + pl.off_qabs;
+        GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,
+                  B, 512, 128, H, false};
+        e = launch_gemm_tn(g1, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+        // --- absorb attention over latent tokens (Algorithm 1 line 6)
+        float* o_part_a = reinterpret_cast<float*>(ws + pl.off_opart_a);
+        float* lse_part_a = reinterpret_cast<float*>(ws + pl.off_lsepart_a);
+        AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
+                      ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
+                      seq_lens, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
+                      o_part_a, lse_part_a};
+        e = launch_absorb_attn_mma(ab, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+        void* o_lat = ws + pl.off_olat;
+        e = launch_merge_latent(o_part_a, lse_part_a, n_chunks, B, H, o_lat, lse_a, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+        // --- output projection O_A W_UV^T (Algorithm 1 line 7)
+        GemmTN g2{o_lat, (int64_t)H * 512, 512, sh->w_uv, 512, 128 * 512, o_abs, (int64_t)H * 128, 128,
+                  B, 128, 512, H, true};
+        e = launch_gemm_tn(g2, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+    }
+    // --- LSE combine (Algorithm 1 line 8)
+    e = launch_combine(o_part_n, lse_part_n, pl.n_split_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
+                       lse_out, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    ++launches;
+    g_last_launches = launches;
+    return TYPHOON_MLA_OK;
+}
+
+size_t typhoon_mla_host_staging_bytes(const typhoon_mla_shared_t* sh, int32_t B, int32_t max_pages) {
+    if (!sh || B < 1 || max_pages < 0) return 0;
+    const size_t BH = (size_t)B * sh->dims.num_heads;
+    return round_up(BH * 128 * 2, 256) + round_up(BH * 64 * 2, 256) + round_up((size_t)B * std::max(max_pages, 1) * 4, 256) +
+           round_up((size_t)B * 4, 256) + round_up(BH * 128 * 2, 256);
+}
+
+int typhoon_mla_decode_host(const typhoon_mla_shared_t* sh, const void* q_nope_host, const void* q_pe_host, int32_t B,
+                            const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
+                            int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table_host,
+                            int32_t max_pages, const int32_t* seq_lens_host, float softmax_scale, int32_t mode,
+                            void* out_host, void* staging, size_t staging_bytes, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+    if (!sh || !q_nope_host || !q_pe_host || !out_host || !staging || B < 1 || max_pages < 0)
+        return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (max_pages > 0 && (!block_table_host || !seq_lens_host)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (staging_bytes < typhoon_mla_host_staging_bytes(sh, B, max_pages)) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(staging) & 255u) return TYPHOON_MLA_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t BH = (size_t)B * sh->dims.num_heads;
+    char* st = reinterpret_cast<char*>(staging);
+    char* d_qn = st;
+    char* d_qp = d_qn + round_up(BH * 128 * 2, 256);
+    char* d_bt = d_qp + round_up(BH * 64 * 2, 256);
+    char* d_sl = d_bt + round_up((size_t)B * std::max(max_pages, 1) * 4, 256);
+    char* d_out = d_sl + round_up((size_t)B * 4, 256);
+    cudaError_t e = cudaMemcpyAsync(d_qn, q_nope_host, BH * 128 * 2, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(d_qp, q_pe_host, BH * 64 * 2, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && max_pages > 0) {
+        e = cudaMemcpyAsync(d_bt, block_table_host, (size_t)B * max_pages * 4, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(d_sl, seq_lens_host, (size_t)B * 4, cudaMemcpyHostToDevice, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    int st_code = typhoon_mla_decode(sh, d_qn, d_qp, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride,
+                                     page_size, reinterpret_cast<const int32_t*>(d_bt), max_pages,
+                                     reinterpret_cast<const int32_t*>(d_sl), softmax_scale, mode, d_out, nullptr,
+                                     workspace, workspace_bytes, stream);
+    if (st_code != TYPHOON_MLA_OK) return st_code;
+    e = cudaMemcpyAsync(out_host, d_out, BH * 128 * 2, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return TYPHOON_MLA_OK;
+}
+
+}  // extern "C"

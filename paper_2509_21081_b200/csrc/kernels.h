@@ -1,0 +1,59 @@
+// Internal launch interfaces between the C ABI (api.cu) and the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tmla {
+
+// C[z][m][n] = sum_k A[z][m][k] * B[z][n][k]   (both operands K-major, bf16, fp32 accumulate)
+struct GemmTN {
+    const void* A; int64_t lda; int64_t a_batch;   // elements
+    const void* B; int64_t ldb; int64_t b_batch;
+    void* C; int64_t ldc; int64_t c_batch;
+    int M, N, K, batch;
+    bool out_fp32;
+};
+cudaError_t launch_gemm_tn(const GemmTN& g, cudaStream_t s);
+
+// Naive shared-prefix attention partials (Algorithm 1 line 4).
+struct NaiveAttn {
+    const void* q_nope; const void* q_pe;          // [B,H,128], [B,H,64]
+    const void* k_nope; const void* v_t; const void* kpe;  // [H,Lp,128], [H,128,Lp], [Lp,64]
+    int B, H; int Ls, Ls_pad; int n_split;
+    float scale;
+    float* o_part;   // [n_split][B][H][128], each normalised
+    float* lse_part; // [n_split][B][H], natural log
+};
+cudaError_t launch_naive_attn_mma(const NaiveAttn& p, cudaStream_t s);
+
+// Absorb attention partials over latent tokens (Algorithm 1 line 6).
+struct AbsorbAttn {
+    const void* q_abs; const void* q_pe;           // [B,H,512], [B,H,64]
+    const void* ckv_shared; const void* kpe_shared; int Ls_absorb;  // shared prefix handled here (ABSORB mode) or 0
+    const void* ckv_pages; const void* kpe_pages;
+    int64_t ckv_stride, kpe_stride; int page_size;
+    const int32_t* block_table; int max_pages; const int32_t* seq_lens;
+    int B, H; int chunk;                           // tokens per chunk
+    int n_shared_chunks, n_suffix_chunks;
+    float scale;
+    float* o_part;   // [n_chunks][B][H][512], each normalised
+    float* lse_part; // [n_chunks][B][H]
+};
+cudaError_t launch_absorb_attn_mma(const AbsorbAttn& p, cudaStream_t s);
+
+// Merge absorb chunk partials -> bf16 latent output [B,H,512] + lse [B,H].
+cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,
+                                void* o_lat_bf16, float* lse, cudaStream_t s);
+
+// Final LSE combine (Algorithm 1 line 8) of n_naive naive partials and an optional absorb partial.
+cudaError_t launch_combine(const float* o_naive, const float* lse_naive, int n_naive,
+                           const float* o_abs, const float* lse_abs,
+                           int B, int H, void* out_bf16, float* lse_out, cudaStream_t s);
+
+// out[c][r] = in[r][c] for each of `batch` matrices [R][C] bf16.
+cudaError_t launch_transpose_bf16(const void* in, void* out, int R, int C, int batch, cudaStream_t s);
+
+// rows [L, W] with stride ld_in -> contiguous padded [Lp, W] (padding zero), bf16
+cudaError_t launch_copy_pad_rows(const void* in, int64_t ld_in, void* out, int L, int Lp, int W, cudaStream_t s);
+
+}  // namespace tmla

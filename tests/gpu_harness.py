@@ -1,0 +1,81 @@
+"""Helpers of the GPU parity tests: upload a seeded problem, run the library, run the CPU checker."""
+import math
+
+import numpy as np
+import torch
+
+from oracle import mla_oracle as O
+from paper_2509_21081_b200 import inputs as I
+
+MAX_ABS_TOL = 2e-2      # bar on max |gpu - oracle| over the output tensor
+REL_FRO_TOL = 5e-3      # bar on ||gpu - oracle||_F / ||oracle||_F
+LSE_TOL = 2e-2          # natural-log LSE; bf16 inputs, fp32 statistics
+
+
+def run_gpu(inp, mode, page_size=None, pages=None, want_lse=True, poison=True, min_max_pages=0,
+            force_max_pages=None):
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    cfg = inp.cfg
+    ps = page_size or cfg.page_size
+    pc = pages or I.build_pages(inp, page_size=ps, poison=poison, min_max_pages=min_max_pages)
+    dev = "cuda"
+    max_pages = pc.block_table.shape[1] if force_max_pages is None else force_max_pages
+    dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev),
+                            inp.w_uv.to(dev), inp.scale, cfg.B, max_pages, ps)
+    lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device=dev) if want_lse else None
+    if force_max_pages == 0:
+        out = dec.decode(inp.q_nope.to(dev), inp.q_pe.to(dev), None, None, None, None, mode=mode, lse_out=lse)
+    else:
+        out = dec.decode(inp.q_nope.to(dev), inp.q_pe.to(dev), pc.ckv_pages.to(dev), pc.kpe_pages.to(dev),
+                         pc.block_table.to(dev), pc.seq_lens.to(dev), mode=mode, lse_out=lse)
+    torch.cuda.synchronize()
+    launches = b.typhoon_mla_last_launch_count()
+    res = out.float().cpu().double().numpy(), (lse.cpu().double().numpy() if want_lse else None), launches
+    dec.close()
+    return res
+
+
+def run_oracle(inp, pairs=None, drop_suffix=False):
+    f = I.to_f64
+    ckv_suf = [f(x[:0] if drop_suffix else x) for x in inp.ckv_suffix]
+    kpe_suf = [f(x[:0] if drop_suffix else x) for x in inp.kpe_suffix]
+    return O.mla_decode(f(inp.q_nope), f(inp.q_pe), f(inp.ckv_shared), f(inp.kpe_shared), ckv_suf, kpe_suf,
+                        f(inp.w_uk), f(inp.w_uv), inp.scale, pairs=pairs)
+
+
+def errors(gpu, ref, mask=None):
+    if mask is not None:
+        gpu, ref = gpu[mask], ref[mask]
+    d = gpu - ref
+    max_abs = float(np.max(np.abs(d))) if d.size else 0.0
+    denom = float(np.linalg.norm(ref))
+    rel = float(np.linalg.norm(d)) / denom if denom > 0 else float(np.linalg.norm(d))
+    return max_abs, rel
+
+
+def assert_parity(gpu_out, ref_out, gpu_lse=None, ref_lse=None, mask=None, what=""):
+    assert np.isfinite(gpu_out if mask is None else gpu_out[mask]).all(), f"{what}: non-finite output"
+    max_abs, rel = errors(gpu_out, ref_out, mask)
+    assert max_abs <= MAX_ABS_TOL, f"{what}: max-abs {max_abs:.3e} > {MAX_ABS_TOL}"
+    assert rel <= REL_FRO_TOL, f"{what}: rel-Frobenius {rel:.3e} > {REL_FRO_TOL}"
+    # no single (b, h) row may hide behind the aggregate: per-row relative error bar (looser)
+    if mask is None:
+        rows_g = gpu_out.reshape(-1, gpu_out.shape[-1]); rows_r = ref_out.reshape(-1, ref_out.shape[-1])
+    else:
+        rows_g, rows_r = gpu_out[mask], ref_out[mask]
+    rn = np.linalg.norm(rows_r, axis=1)
+    re = np.linalg.norm(rows_g - rows_r, axis=1)
+    ok = rn > 0
+    if ok.any():
+        worst = float(np.max(re[ok] / rn[ok]))
+        assert worst <= 4 * REL_FRO_TOL, f"{what}: worst row rel error {worst:.3e}"
+    if gpu_lse is not None:
+        gl = gpu_lse if mask is None else gpu_lse[mask]
+        rl = ref_lse if mask is None else ref_lse[mask]
+        inf = np.isinf(rl)
+        assert np.array_equal(np.isinf(gl), inf), f"{what}: -inf pattern of lse differs"
+        if (~inf).any():
+            e = float(np.max(np.abs(gl[~inf] - rl[~inf])))
+            assert e <= LSE_TOL, f"{what}: lse error {e:.3e}"
+    return max_abs, rel

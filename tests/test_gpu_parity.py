@@ -1,0 +1,274 @@
+"""GPU parity: the CUDA library (through the C ABI) against the float64 CPU
+checker on the same seeded inputs.  Bars (bf16 inputs, fp32 accumulation):
+max-abs <= 2e-2 and relative Frobenius <= 5e-3 on the output, 2e-2 on the LSE.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_21081_b200 import inputs as I
+from tests import gpu_harness as G
+
+pytestmark = pytest.mark.gpu
+
+ABSORB, HYBRID, AUTO, NAIVE = 1, 2, 0, 3
+
+
+def _cfg(name, B, H, Ls, lo, hi, seed, page_size=64):
+    return I.MLAConfig(name, B=B, H=H, Ls=Ls, suffix_lo=lo, suffix_hi=hi, seed=seed, page_size=page_size)
+
+
+@pytest.mark.parametrize("mode", [HYBRID, ABSORB, AUTO])
+def test_cfg0_tiny(mode):
+    inp = I.make_inputs(I.CONFIGS["cfg0"])
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, launches = G.run_gpu(inp, mode)
+    assert launches > 0
+    G.assert_parity(out, ref, lse, ref_lse, what=f"cfg0 mode {mode}")
+
+
+@pytest.mark.parametrize("mode", [HYBRID, ABSORB])
+@pytest.mark.parametrize("page_size", [64, 128])
+def test_ragged_small(mode, page_size):
+    """Ragged prefix (not a tile multiple), ragged suffixes with empty / one-token / page-edge lengths,
+    NaN-poisoned page tails and spare pages, -1 in unused block-table slots."""
+    cfg = _cfg("ragged", B=9, H=16, Ls=331, lo=0, hi=0, seed=21, page_size=page_size)
+    inp = I.make_inputs(cfg, suffix_lens=[0, 1, 63, 64, 65, 127, 129, 300, 777])
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, mode, page_size=page_size)
+    G.assert_parity(out, ref, lse, ref_lse, what=f"ragged mode {mode} ps {page_size}")
+
+
+@pytest.mark.parametrize("H", [16, 48, 64, 128])
+def test_head_counts_and_batch_tail(H):
+    """B not a multiple of the row tile; several head counts (incl. a ragged head group)."""
+    cfg = _cfg("heads", B=70 if H <= 64 else 37, H=H, Ls=520, lo=40, hi=200, seed=22 + H)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    for mode in (HYBRID, ABSORB):
+        out, lse, _ = G.run_gpu(inp, mode)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"H={H} mode {mode}")
+
+
+def test_no_prefix():
+    """Ls = 0: absorb path alone (Algorithm 1 lines 5-7)."""
+    cfg = _cfg("noprefix", B=6, H=32, Ls=0, lo=1, hi=400, seed=23)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    for mode in (HYBRID, ABSORB, AUTO):
+        out, lse, _ = G.run_gpu(inp, mode)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"Ls=0 mode {mode}")
+
+
+def test_no_suffix():
+    """All suffixes empty: naive path alone (Algorithm 1 line 4) -- with a page table of zero
+    lengths, with no page table at all, and in NAIVE mode."""
+    cfg = _cfg("nosuffix", B=5, H=32, Ls=1000, lo=0, hi=0, seed=24)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, HYBRID, min_max_pages=3)
+    G.assert_parity(out, ref, lse, ref_lse, what="Ln=0 hybrid")
+    out, lse, _ = G.run_gpu(inp, AUTO, force_max_pages=0)
+    G.assert_parity(out, ref, lse, ref_lse, what="Ln=0 auto, no page table")
+    out, lse, _ = G.run_gpu(inp, NAIVE)
+    G.assert_parity(out, ref, lse, ref_lse, what="Ln=0 naive")
+    out, lse, _ = G.run_gpu(inp, ABSORB, min_max_pages=2)
+    G.assert_parity(out, ref, lse, ref_lse, what="Ln=0 absorb")
+
+
+def test_naive_mode_ignores_suffix():
+    cfg = _cfg("naiveonly", B=4, H=16, Ls=300, lo=10, hi=90, seed=25)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp, drop_suffix=True)
+    out, lse, _ = G.run_gpu(inp, NAIVE)
+    G.assert_parity(out, ref, lse, ref_lse, what="naive mode")
+
+
+def test_empty_context_rows():
+    """No prefix and some empty suffixes: those rows are zero with lse = -inf, no NaN anywhere."""
+    cfg = _cfg("empty", B=4, H=16, Ls=0, lo=0, hi=0, seed=26)
+    inp = I.make_inputs(cfg, suffix_lens=[0, 5, 0, 70])
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, HYBRID)
+    G.assert_parity(out, ref, lse, ref_lse, what="empty rows")
+    assert np.all(out[0] == 0) and np.all(out[2] == 0) and np.all(np.isneginf(lse[0]))
+
+
+@pytest.mark.parametrize("mult", [4.0, 8.0])
+def test_peaked_softmax(mult):
+    """Queries scaled up so that a few tokens dominate: sometimes in the prefix, sometimes in the
+    suffix.  A mis-masked or dropped token shows here, where diffuse attention would hide it."""
+    cfg = _cfg("peaked", B=8, H=16, Ls=700, lo=50, hi=600, seed=27)
+    inp = I.make_inputs(cfg)
+    inp.q_nope = (inp.q_nope.float() * mult).to(torch.bfloat16)
+    inp.q_pe = (inp.q_pe.float() * mult).to(torch.bfloat16)
+    ref, ref_lse = G.run_oracle(inp)
+    for mode in (HYBRID, ABSORB):
+        out, lse, _ = G.run_gpu(inp, mode)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"peaked x{mult} mode {mode}")
+
+
+def test_dominant_token_in_suffix_and_prefix():
+    """One token carries (almost) all the weight; output must be its decompressed value."""
+    cfg = _cfg("dominant", B=2, H=16, Ls=200, lo=100, hi=100, seed=28)
+    inp = I.make_inputs(cfg)
+    inp.q_pe[:] = 0
+    inp.q_pe[:, :, 0] = 8.0
+    inp.kpe_shared[:] = 0
+    for b in range(2):
+        inp.kpe_suffix[b][:] = 0
+    inp.kpe_suffix[0][77, 0] = 64.0      # request 0: winner in the suffix
+    inp.kpe_shared[123, 0] = 0.0
+    ref, ref_lse = G.run_oracle(inp)
+    for mode in (HYBRID, ABSORB):
+        out, lse, _ = G.run_gpu(inp, mode)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"dominant suffix mode {mode}")
+    inp.kpe_suffix[0][77, 0] = 0.0
+    inp.kpe_shared[123, 0] = 64.0        # both requests: winner in the prefix
+    ref, ref_lse = G.run_oracle(inp)
+    for mode in (HYBRID, ABSORB):
+        out, lse, _ = G.run_gpu(inp, mode)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"dominant prefix mode {mode}")
+
+
+def test_metamorphic_paging_and_modes():
+    """Permuting physical pages, switching the page size and switching mode leave the result
+    unchanged (within tolerance); repeating a call is bitwise identical."""
+    cfg = _cfg("meta", B=6, H=32, Ls=450, lo=30, hi=500, seed=29)
+    inp = I.make_inputs(cfg)
+    ref, _ = G.run_oracle(inp)
+    a, _, _ = G.run_gpu(inp, HYBRID, pages=I.build_pages(inp, 64, seed=1))
+    b, _, _ = G.run_gpu(inp, HYBRID, pages=I.build_pages(inp, 64, seed=2))
+    c, _, _ = G.run_gpu(inp, HYBRID, page_size=128, pages=I.build_pages(inp, 128, seed=3))
+    d, _, _ = G.run_gpu(inp, ABSORB, pages=I.build_pages(inp, 64, seed=1))
+    a2, _, _ = G.run_gpu(inp, HYBRID, pages=I.build_pages(inp, 64, seed=1))
+    assert np.array_equal(a, a2), "run-to-run results differ bitwise"
+    assert np.array_equal(a, b), "page permutation changed the result"
+    for x, name in ((a, "a"), (c, "page128"), (d, "absorb")):
+        G.assert_parity(x, ref, what=f"meta {name}")
+    assert G.errors(d, a)[1] < G.REL_FRO_TOL
+
+
+def test_moving_tokens_between_prefix_and_suffix():
+    """The same total context split at a different point between shared prefix and suffixes."""
+    cfg = _cfg("move", B=3, H=16, Ls=384, lo=64, hi=64, seed=30)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    moved = I.make_inputs(cfg)
+    k = 100
+    moved.ckv_suffix = [torch.cat([inp.ckv_shared[-k:], x]) for x in inp.ckv_suffix]
+    moved.kpe_suffix = [torch.cat([inp.kpe_shared[-k:], x]) for x in inp.kpe_suffix]
+    moved.ckv_shared, moved.kpe_shared = inp.ckv_shared[:-k].contiguous(), inp.kpe_shared[:-k].contiguous()
+    moved.suffix_lens = [n + k for n in inp.suffix_lens]
+    out, lse, _ = G.run_gpu(moved, HYBRID)
+    G.assert_parity(out, ref, lse, ref_lse, what="moved split")
+
+
+def test_expansion_matches_plain_matmul():
+    """Shared-prefix expansion against a float64 matmul: within one bf16 rounding of the exact value."""
+    from oracle import mla_oracle as O
+    from paper_2509_21081_b200 import binding as b
+    cfg = _cfg("expand", B=1, H=16, Ls=333, lo=0, hi=0, seed=31)
+    inp = I.make_inputs(cfg)
+    dims = b.make_dims(cfg.H)
+    w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
+    sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    k, vt = b.typhoon_mla_shared_export(sh)
+    Ls, Lp, owned = b.typhoon_mla_shared_view(sh)
+    torch.cuda.synchronize()
+    assert (Ls, Lp) == (333, 384) and owned >= 2 * cfg.H * Lp * 128 * 2
+    k = k.float().cpu().double().numpy(); v = vt.float().cpu().double().numpy().transpose(0, 2, 1)
+    sh.free()
+    kr = O.expand_shared(I.to_f64(inp.ckv_shared), I.to_f64(inp.w_uk))
+    vr = O.expand_shared(I.to_f64(inp.ckv_shared), I.to_f64(inp.w_uv))
+    for got, ref in ((k, kr), (v, vr)):
+        assert np.all(got[:, 333:, :] == 0), "padding not zero"
+        err = np.abs(got[:, :333, :] - ref)
+        bound = np.abs(ref) * 2.0 ** -8 + 1e-6     # half-ulp of bf16 is 2^-9 relative; allow one ulp
+        assert np.all(err <= bound), f"expansion error {err.max():.3e}"
+
+
+def test_decode_host_matches_device_call():
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    cfg = _cfg("host", B=5, H=16, Ls=260, lo=10, hi=150, seed=32)
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp)
+    dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(),
+                            inp.scale, cfg.B, pc.block_table.shape[1])
+    ckv_p, kpe_p = pc.ckv_pages.cuda(), pc.kpe_pages.cuda()
+    ref = dec.decode(inp.q_nope.cuda(), inp.q_pe.cuda(), ckv_p, kpe_p, pc.block_table.cuda(), pc.seq_lens.cuda(),
+                     mode=HYBRID).cpu()
+    out_h = torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16).pin_memory()
+    dec.decode_host(inp.q_nope.pin_memory(), inp.q_pe.pin_memory(), ckv_p, kpe_p, pc.block_table.pin_memory(),
+                    pc.seq_lens.pin_memory(), out_h, mode=HYBRID)
+    torch.cuda.synchronize()
+    assert torch.equal(out_h, ref)
+    dec.close()
+
+
+def test_invalid_arguments():
+    from paper_2509_21081_b200 import binding as b
+    cfg = _cfg("inval", B=2, H=16, Ls=64, lo=8, hi=8, seed=33)
+    inp = I.make_inputs(cfg)
+    with pytest.raises(b.TyphoonMLAError) as e:
+        b.typhoon_mla_prepare_shared(b.make_dims(17), inp.ckv_shared.cuda(), inp.kpe_shared.cuda(),
+                                     inp.w_uk.cuda(), inp.w_uv.cuda())
+    assert e.value.status == 2
+    sh = b.typhoon_mla_prepare_shared(b.make_dims(16), inp.ckv_shared.cuda(), inp.kpe_shared.cuda(),
+                                      inp.w_uk.cuda(), inp.w_uv.cuda())
+    pc = I.build_pages(inp)
+    out = torch.empty(2, 16, 128, dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(b.TyphoonMLAError) as e:
+        b.typhoon_mla_decode(sh, inp.q_nope.cuda(), inp.q_pe.cuda(), pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), 64,
+                             pc.block_table.cuda(), pc.seq_lens.cuda(), inp.scale, out, small, mode=HYBRID)
+    assert e.value.status == 3
+    with pytest.raises(b.TyphoonMLAError) as e:
+        b.typhoon_mla_decode(sh, inp.q_nope.cuda(), inp.q_pe.cuda(), pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), 48,
+                             pc.block_table.cuda(), pc.seq_lens.cuda(), inp.scale, out, small, mode=HYBRID)
+    assert e.value.status == 1
+    sh.free()
+
+
+# ------------------------------------------------------------ full-size configs
+def _sampled_pairs(cfg, n, seed):
+    r = np.random.default_rng(seed)
+    pairs = {(int(r.integers(cfg.B)), int(r.integers(cfg.H))) for _ in range(n)}
+    return sorted(pairs)
+
+
+def _full_size_sampled(cfg, modes, n_pairs, extremes=False):
+    inp = I.make_inputs(cfg)
+    pairs = _sampled_pairs(cfg, n_pairs, cfg.seed)
+    if extremes:  # always include the shortest and the longest suffix
+        for b in (int(np.argmin(inp.suffix_lens)), int(np.argmax(inp.suffix_lens))):
+            pairs += [(b, 0), (b, cfg.H - 1)]
+    ref, ref_lse = G.run_oracle(inp, pairs=pairs)
+    mask = ~np.isnan(ref_lse)
+    res = {}
+    for mode in modes:
+        out, lse, launches = G.run_gpu(inp, mode)
+        assert np.isfinite(out).all()
+        res[mode] = G.assert_parity(out, ref, lse, ref_lse, mask=mask, what=f"{cfg.name} mode {mode}")
+    return res
+
+
+def test_cfg1_full_size_sampled():
+    """DeepSeek-v3 dims, B=64, Ls=4096, Ln=512 -- the benchmark's launch configuration, checked on
+    sampled (request, head) rows computed one by one by the CPU checker."""
+    _full_size_sampled(I.CONFIGS["cfg1"], (HYBRID, ABSORB, AUTO), 48)
+
+
+def test_cfg3_kimi_like_sampled():
+    _full_size_sampled(I.CONFIGS["cfg3"], (HYBRID,), 24, extremes=True)
+
+
+def test_cfg2_long_prompt_sampled():
+    _full_size_sampled(I.CONFIGS["cfg2"], (HYBRID,), 16, extremes=True)
+
+
+@pytest.mark.parametrize("B", [1, 8, 128])
+def test_cfg4_fanout_sampled(B):
+    _full_size_sampled(I.CONFIGS["cfg4"].with_batch(B), (AUTO, HYBRID), 8)

@@ -1,0 +1,107 @@
+"""CPU-only tests of the library's host side: the shared object loads and exports every symbol the
+header declares; cost model and Eq. 1 agree with the paper's printed constants; the crossover rule
+behaves as the paper describes.  No compute entry point is called (no GPU here)."""
+import ctypes
+import json
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+GOLD = os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2509_21081_b200 import build
+    build.build()
+    from paper_2509_21081_b200 import binding
+    return binding
+
+
+def test_exports_every_declared_symbol(b):
+    hdr = open(os.path.join(ROOT, "include", "typhoon_mla.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(typhoon_mla_[a-z_0-9]+)\s*\(", hdr))
+    assert {"typhoon_mla_prepare_shared", "typhoon_mla_decode", "typhoon_mla_free"} <= names
+    lib = ctypes.CDLL(b.LIB_PATH)
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} declared in the header but not exported"
+
+
+def test_status_strings(b):
+    assert b._lib.typhoon_mla_status_string(0) == b"ok"
+    assert b"workspace" in b._lib.typhoon_mla_status_string(3)
+
+
+def test_eq1_printed_value(b):
+    g = json.load(open(os.path.join(GOLD, "eq1_batch_threshold.json")))
+    bt = b.typhoon_mla_batch_threshold(b.make_dims(128), g["S_q"], g["T"], g["M"])
+    assert int(bt) == g["B_theta_printed"]
+    assert abs(b.typhoon_mla_batch_threshold(b.make_dims(128), 2, g["T"], g["M"]) - bt / 2) < 1e-9
+    # no head-count dependence in Eq. 1
+    assert b.typhoon_mla_batch_threshold(b.make_dims(64), 1, g["T"], g["M"]) == bt
+
+
+def test_table1_printed_constants(b):
+    g = json.load(open(os.path.join(GOLD, "table1_constants.json")))
+    d = b.make_dims(g["dims"]["H"])
+    B, Ls, Ln = 7, 1000, 300
+    mn, wn = b.typhoon_mla_cost_model(d, b.COST_NAIVE, B, 1, Ls, Ln)
+    ma, wa = b.typhoon_mla_cost_model(d, b.COST_ABSORB, B, 1, Ls, Ln)
+    mt, wt = b.typhoon_mla_cost_model(d, b.COST_TYPHOON, B, 1, Ls, Ln)
+    k = 1024
+    assert mn == g["mac_per_token_x1024"]["naive"] * k * B * (Ls + Ln)
+    assert ma == g["mac_per_token_x1024"]["absorb"] * k * B * (Ls + Ln)
+    assert mt == 40 * k * B * Ls + 136 * k * B * Ln
+    assert wn == 40 * k * (Ls + B * Ln)
+    assert wa == int(g["hbm_per_token_x1024"]["absorb_exact"] * k) * (Ls + B * Ln)
+    assert wt == 40 * k * Ls + 576 * B * Ln
+    m3, _ = b.typhoon_mla_cost_model(d, b.COST_TYPHOON, B, 3, Ls, Ln)
+    assert m3 == 3 * mt
+
+
+def test_cost_model_matches_checker(b):
+    """Same Table 1 terms as the CPU checker's independent helper."""
+    from oracle import mla_oracle as O
+    for H in (64, 128):
+        d = b.make_dims(H)
+        kw = dict(H=H, D_qk=192, D_v=128, D_l=512, D_r=64)
+        for kind, name in ((b.COST_NAIVE, "naive"), (b.COST_ABSORB, "absorb"), (b.COST_TYPHOON, "typhoon")):
+            m, w = b.typhoon_mla_cost_model(d, kind, 33, 2, 4096, 512)
+            assert m == O.macs(name, 33, 2, 4096, 512, **kw)
+            assert w == O.hbm_words(name, 33, 4096, 512, **kw)
+
+
+def test_crossover_rule(b):
+    d = b.make_dims(128)
+    # zero fixed cost and the paper's NPU numbers: the switch happens where Eq. 1 says, up to the
+    # rope keys being read once per token instead of once per head (256.5 vs 320 words per head-token)
+    b.typhoon_mla_set_hw_model(376e12, 1.8e12, 0.0)
+    modes = [b.typhoon_mla_choose_mode_for(d, 4096, B) for B in range(1, 200)]
+    first_hybrid = modes.index(b.MODE_HYBRID) + 1
+    assert all(m == b.MODE_ABSORB for m in modes[: first_hybrid - 1])
+    assert all(m == b.MODE_HYBRID for m in modes[first_hybrid - 1:])
+    bt = b.typhoon_mla_batch_threshold(d, 1, 376e12, 1.8e12)
+    assert bt * 256.5 / 320 - 1 <= first_hybrid <= bt + 1
+    # a fixed cost pushes short prefixes to absorb, leaves long ones alone
+    b.typhoon_mla_set_hw_model(376e12, 1.8e12, 50e-6)
+    assert b.typhoon_mla_choose_mode_for(d, 64, 100) == b.MODE_ABSORB
+    assert b.typhoon_mla_choose_mode_for(d, 65536, 100) == b.MODE_HYBRID
+    # empty suffixes -> naive only; no prefix -> absorb
+    assert b.typhoon_mla_choose_mode_for(d, 4096, 8, 0) == b.MODE_NAIVE
+    assert b.typhoon_mla_choose_mode_for(d, 0, 512) == b.MODE_ABSORB
+    b.typhoon_mla_set_hw_model(0, 0, -1)   # restore defaults
+    # defaults (B200): tiny batches fall back, large batches go hybrid
+    assert b.typhoon_mla_choose_mode_for(d, 16384, 1) == b.MODE_ABSORB
+    assert b.typhoon_mla_choose_mode_for(d, 16384, 8) == b.MODE_ABSORB
+    assert b.typhoon_mla_choose_mode_for(d, 16384, 512) == b.MODE_HYBRID
+
+
+def test_pure_entry_points_reject_bad_arguments(b):
+    assert b._lib.typhoon_mla_workspace_bytes(None, 4, 4, 64) == 0
+    assert b._lib.typhoon_mla_free(None) == 0
+    assert b.typhoon_mla_batch_threshold(b.make_dims(128), 0, 1.0, 1.0) < 0
+    with pytest.raises(b.TyphoonMLAError):
+        b.typhoon_mla_cost_model(b.make_dims(128), 9, 1, 1, 1, 1)
