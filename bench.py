@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the MLA shared-prefix decode attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg1] [--mode auto|hybrid|absorb]
+    python bench.py --impl reference ...      # the float64 CPU checker on the host cores
+    python bench.py --sweep                   # config 4 fan-out sweep (one JSON line per batch size)
+
+One step = one pass of the whole path (Algorithm 1 lines 4-8: naive shared attention, query
+absorption, absorb suffix attention, split merge, W_UV projection, LSE combine) over one batch of
+synthetic requests.  Metric: decode-attention queries/s (one query = one request's token across
+all heads).  Prints one JSON line.  With N > 1 (torchrun) every rank runs an independent replica
+on its own requests (the path shards by request with no exchange): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mla_decode_attention_queries_per_s"
+UNIT = "queries/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (key: (config, kernel)); None where no capture exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------ work accounting
+def algorithmic_work(cfg, suffix_lens, mode_name):
+    """Algorithmic flops and bytes of one step (Table 1 terms plus the once-only reads of q and the
+    weights and the write of out)."""
+    H, B, Ls = cfg.H, cfg.B, cfg.Ls
+    sum_ln = sum(suffix_lens)
+    W = 4 * H * 65536
+    if mode_name == "absorb":
+        flops = H * (2176 * (B * Ls + sum_ln) + 4 * 65536 * B)
+        bytes_ = 1152 * Ls + W + 1152 * sum_ln + 640 * H * B
+    else:
+        flops = H * (640 * B * Ls + 2176 * sum_ln + 4 * 65536 * B)
+        bytes_ = (512 * H + 128) * Ls + W + 1152 * sum_ln + 640 * H * B
+    return flops, bytes_
+
+
+def dominant_kernel(cfg, suffix_lens, mode_name):
+    """(kernel id, name, bound, algorithmic bytes per launch, flops per launch) of the kernel that
+    carries most of the step's roofline time."""
+    H, B, Ls = cfg.H, cfg.B, cfg.Ls
+    sum_ln = sum(suffix_lens)
+    naive_bytes = (512 * H + 128) * Ls + 384 * B * H          # expanded K/V + rope keys once, q once
+    naive_flops = 640 * B * H * Ls
+    if mode_name == "absorb":
+        absorb_bytes = 1152 * (B * Ls + sum_ln) + 1152 * B * H   # latent tokens per request + Q_A|q_pe
+        absorb_flops = 2176 * H * (B * Ls + sum_ln)
+        return 2, "absorb_attn", absorb_bytes, absorb_flops
+    absorb_bytes = 1152 * sum_ln + 1152 * B * H
+    absorb_flops = 2176 * H * sum_ln
+    pk = _peaks()
+    t_naive = max(naive_bytes / (pk["hbm_gbs"] * 1e9), naive_flops / (pk["bf16_tflops"] * 1e12))
+    t_abs = max(absorb_bytes / (pk["hbm_gbs"] * 1e9), absorb_flops / (pk["bf16_tflops"] * 1e12))
+    if t_naive >= t_abs:
+        return 0, "naive_attn", naive_bytes, naive_flops
+    return 2, "absorb_attn", absorb_bytes, absorb_flops
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {}
+        for k in dir(nv):
+            if k.startswith("nvmlClocksEventReason") or k.startswith("nvmlClocksThrottleReason"):
+                v = getattr(nv, k)
+                if isinstance(v, int) and v:
+                    names.setdefault(v, k.replace("nvmlClocksEventReason", "").replace("nvmlClocksThrottleReason", ""))
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons", None)
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                if get_reasons:
+                    r = int(get_reasons(self.h))
+                    for bit, name in names.items():
+                        if bit and (r & bit) == bit and bin(bit).count("1") == 1:
+                            self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        if self._thr:
+            self._stop.set()
+            self._thr.join()
+
+    def summary(self):
+        idle = {"GpuIdle", "None", "ApplicationsClocksSetting"}
+        return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
+                "reasons": sorted(r for r in self.reasons if r not in idle)}
+
+
+# ------------------------------------------------------------------ CPU checker timing
+def time_oracle_sample(inp, heads, target_requests=None):
+    """Times the float64 CPU checker, as it stands, on all requests x the first `heads` heads and
+    scales to all heads.  Returns (queries/s, seconds, cores, sample description)."""
+    import numpy as np  # noqa: F401
+    from oracle import mla_oracle as O
+    from paper_2509_21081_b200 import inputs as I
+    cfg = inp.cfg
+    f = I.to_f64
+    nb = cfg.B if target_requests is None else min(cfg.B, target_requests)
+    args = (f(inp.q_nope), f(inp.q_pe), f(inp.ckv_shared), f(inp.kpe_shared),
+            [f(x) for x in inp.ckv_suffix], [f(x) for x in inp.kpe_suffix], f(inp.w_uk), f(inp.w_uv), inp.scale)
+    pairs = [(b, h) for h in range(heads) for b in range(nb)]
+    t0 = time.perf_counter()
+    O.mla_decode(*args, pairs=pairs)
+    dt = time.perf_counter() - t0
+    scaled = dt * (cfg.H / heads)
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count()])
+    except Exception:
+        cores = os.cpu_count()
+    return nb / scaled, dt, int(cores), f"{nb} requests x {heads} of {cfg.H} heads, time scaled by {cfg.H / heads:g}"
+
+
+# ------------------------------------------------------------------ main arms
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2509_21081_b200 import inputs as I
+    cfg = I.CONFIGS[args.config]
+    inp = I.make_inputs(cfg)
+    # Size the per-step sample (heads) so that the K timed steps take about two minutes in total.
+    _, t1, _, _ = time_oracle_sample(inp, 1)
+    for _ in range(max(args.warmup - 1, 0)):
+        time_oracle_sample(inp, 1)
+    K = max(args.steps, 1)
+    heads = max(1, min(cfg.H, args.ref_heads, int(120.0 / (K * max(t1, 1e-3)))))
+    vals = []
+    for _ in range(K):
+        qps, dt, cores, sample = time_oracle_sample(inp, heads)
+        vals.append((qps, dt))
+    qps = statistics.median(v[0] for v in vals)
+    ms = cfg.B / qps * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": _workload_name(cfg)},
+            "cpu_baseline": {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def _workload_name(cfg):
+    return (f"{cfg.name}: B={cfg.B} H={cfg.H} Ls={cfg.Ls} Ln=[{cfg.suffix_lo},{cfg.suffix_hi}] "
+            f"page={cfg.page_size} d=(128,64,128,512) bf16")
+
+
+def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with_e2e=True):
+    import torch
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200 import inputs as I
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+
+    dev = "cuda"
+    # Each rank draws its own requests (seed shifted by rank); the prefix and weights are replicated.
+    rcfg = cfg if rank == 0 else dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+    inp = I.make_inputs(rcfg)
+    pc = I.build_pages(inp, poison=False)
+    max_pages = pc.block_table.shape[1]
+    # Two full copies of everything a step touches, used alternately, so that no step finds the
+    # previous step's data in the 126 MB L2 (each copy alone is larger than L2 for configs 1-4).
+    n_sets = 2
+    sets = []
+    for _ in range(n_sets):
+        dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev),
+                                inp.w_uv.to(dev), inp.scale, cfg.B, max_pages, pc.page_size)
+        sets.append(dict(dec=dec, q_nope=inp.q_nope.to(dev), q_pe=inp.q_pe.to(dev), ckv=pc.ckv_pages.to(dev),
+                         kpe=pc.kpe_pages.to(dev), bt=pc.block_table.to(dev), sl=pc.seq_lens.to(dev),
+                         out=torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16, device=dev)))
+    resolved = mode if mode != b.MODE_AUTO else sets[0]["dec"].choose_mode(cfg.B, sum(inp.suffix_lens))
+    mode_name = b.MODE_NAMES[resolved]
+
+    def step(i):
+        s = sets[i % n_sets]
+        s["dec"].decode(s["q_nope"], s["q_pe"], s["ckv"], s["kpe"], s["bt"], s["sl"], mode=mode, out=s["out"])
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    W, K = max(args.warmup, 3), max(args.steps, 1)
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    launches_per_step = b.typhoon_mla_last_launch_count()
+    kid, kname, k_bytes, k_flops = dominant_kernel(cfg, inp.suffix_lens, mode_name)
+
+    # ---- device-resident timing
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b.typhoon_mla_profile_begin(kid, K)
+    barrier()
+    with ClockSampler(device_index) as clocks:
+        ev0.record()
+        for i in range(K):
+            step(i)
+        ev1.record()
+        barrier()
+    total_ms = ev0.elapsed_time(ev1)
+    k_ms, k_n = b.typhoon_mla_profile_end()
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    value = world * cfg.B / (ms_per_step * 1e-3)
+
+    # ---- roofline of the dominant kernel
+    pk = _peaks()
+    k_avg_s = (k_ms / max(k_n, 1)) * 1e-3
+    t_mem = k_bytes / (pk["hbm_gbs"] * 1e9)
+    t_cmp = k_flops / (pk["bf16_tflops_sustained"] * 1e12)
+    if t_mem >= t_cmp:
+        achieved = k_bytes / k_avg_s / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / pk["hbm_gbs"]}
+    else:
+        achieved = k_flops / k_avg_s / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / pk["bf16_tflops_sustained"]}
+    roof.update({"traffic": NCU_TRAFFIC_BYTES.get((cfg.name, kname)), "kernel": kname,
+                 "kernel_ms": k_avg_s * 1e3, "launches_timed": k_n, "peak_source": pk["source"],
+                 "algorithmic_bytes": k_bytes, "algorithmic_flops": k_flops})
+    flops, bytes_ = algorithmic_work(cfg, inp.suffix_lens, mode_name)
+    t_lb = max(flops / (pk["bf16_tflops"] * 1e12), bytes_ / (pk["hbm_gbs"] * 1e9))
+    roof["step_frac_of_combined_roofline"] = t_lb / (ms_per_step * 1e-3)
+
+    # ---- end to end: per-step tensors from pinned host memory, result read back, every step
+    e2e = None
+    if with_e2e:
+        hq = [(inp.q_nope.pin_memory(), inp.q_pe.pin_memory(), pc.block_table.pin_memory(), pc.seq_lens.pin_memory(),
+               torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16).pin_memory()) for _ in range(n_sets)]
+
+        def step_host(i):
+            s, h = sets[i % n_sets], hq[i % n_sets]
+            s["dec"].decode_host(h[0], h[1], s["ckv"], s["kpe"], h[2], h[3], h[4], mode=mode)
+
+        for i in range(W):
+            step_host(i)
+        barrier()
+        ev0.record()
+        for i in range(K):
+            step_host(i)
+        ev1.record()
+        barrier()
+        t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        e_ms = float(t.item()) / K
+        h2d = inp.q_nope.numel() * 2 + inp.q_pe.numel() * 2 + pc.block_table.numel() * 4 + pc.seq_lens.numel() * 4
+        d2h = cfg.B * cfg.H * 128 * 2
+        e2e = {"value": world * cfg.B / (e_ms * 1e-3), "unit": UNIT, "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    cpu = None
+    if with_cpu and rank == 0 and world == 1:
+        heads = max(1, min(cfg.H, args.ref_heads))
+        qps, dt, cores, sample = time_oracle_sample(inp, heads)
+        cpu = {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": dt}
+
+    for s in sets:
+        s["dec"].close()
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": _workload_name(cfg), "mode": mode_name, "requested_mode": b.MODE_NAMES[mode],
+                       "parallelism": f"replicas x{world} (shard by request, no exchange)",
+                       "l2": f"{n_sets} full input sets used alternately, each larger than the 126 MB L2"},
+            "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches_per_step * K,
+            "roofline": roof, "cpu_baseline": cpu}
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--mode", default="auto", choices=["auto", "absorb", "hybrid", "naive"])
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (config 4 sweep)")
+    ap.add_argument("--sweep", action="store_true", help="config 4 fan-out sweep over batch sizes and modes")
+    ap.add_argument("--ref-heads", type=int, default=64, help="heads the CPU checker is timed on (scaled up)")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200 import inputs as I
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
+    mode = {"auto": b.MODE_AUTO, "absorb": b.MODE_ABSORB, "hybrid": b.MODE_HYBRID, "naive": b.MODE_NAIVE}[args.mode]
+
+    if args.sweep:
+        base = I.CONFIGS["cfg4"]
+        for B in I.CFG4_BATCHES:
+            for m in (b.MODE_ABSORB, b.MODE_HYBRID, b.MODE_AUTO):
+                line = bench_config(base.with_batch(B), args, m, rank, world, local, with_cpu=False, with_e2e=False)
+                if rank == 0:
+                    print(json.dumps(line), flush=True)
+    else:
+        cfg = I.CONFIGS[args.config]
+        if args.batch:
+            cfg = cfg.with_batch(args.batch)
+        line = bench_config(cfg, args, mode, rank, world, local, with_cpu=not args.no_cpu)
+        if rank == 0:
+            print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

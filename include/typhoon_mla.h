@@ -212,6 +212,28 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
  * elements each (device memory), on `stream`. */
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_dst, void* v_t_dst, void* stream);
 
+/* Kernel kinds of the decode step, in launch order (Algorithm 1 lines 4-8). */
+enum {
+    TYPHOON_MLA_KERNEL_NAIVE_ATTN = 0,  /* line 4 */
+    TYPHOON_MLA_KERNEL_Q_ABSORB = 1,    /* line 5 */
+    TYPHOON_MLA_KERNEL_ABSORB_ATTN = 2, /* line 6 */
+    TYPHOON_MLA_KERNEL_MERGE = 3,       /* merge of line 6's KV splits */
+    TYPHOON_MLA_KERNEL_W_UV = 4,        /* line 7 */
+    TYPHOON_MLA_KERNEL_COMBINE = 5,     /* line 8 */
+    TYPHOON_MLA_NUM_KERNELS = 6
+};
+
+/*
+ * Measurement aid: between profile_begin and profile_end every decode call of
+ * the process records a pair of CUDA events around the launch of the chosen
+ * kernel kind, on the stream the kernel is launched on (up to max_launches
+ * launches).  profile_end waits for the recorded events and returns the summed
+ * device time in milliseconds and the number of launches timed.  Host, not
+ * thread-safe; begin allocates events, decode itself still allocates nothing.
+ */
+int typhoon_mla_profile_begin(int32_t kernel_id, int32_t max_launches);
+int typhoon_mla_profile_end(double* total_ms /* host */, int32_t* launches /* host */);
+
 /* Number of kernels the last typhoon_mla_decode call of this thread launched. */
 int typhoon_mla_last_launch_count(void);
 

@@ -76,6 +76,10 @@ def _load():
                                             C.POINTER(i64)]
     lib.typhoon_mla_shared_export.restype = C.c_int
     lib.typhoon_mla_shared_export.argtypes = [vp, vp, vp, vp]
+    lib.typhoon_mla_profile_begin.restype = C.c_int
+    lib.typhoon_mla_profile_begin.argtypes = [i32, i32]
+    lib.typhoon_mla_profile_end.restype = C.c_int
+    lib.typhoon_mla_profile_end.argtypes = [C.POINTER(f64), C.POINTER(i32)]
     lib.typhoon_mla_last_launch_count.restype = C.c_int
     lib.typhoon_mla_last_cuda_error.restype = C.c_int
     return lib
@@ -221,3 +225,16 @@ def typhoon_mla_shared_export(shared: SharedPrefix):
 
 def typhoon_mla_last_launch_count() -> int:
     return int(_lib.typhoon_mla_last_launch_count())
+
+
+KERNEL_NAMES = ("naive_attn", "q_absorb", "absorb_attn", "merge", "w_uv", "combine")
+
+
+def typhoon_mla_profile_begin(kernel_id: int, max_launches: int) -> None:
+    _check(_lib.typhoon_mla_profile_begin(kernel_id, max_launches), "typhoon_mla_profile_begin")
+
+
+def typhoon_mla_profile_end():
+    ms, n = C.c_double(), C.c_int32()
+    _check(_lib.typhoon_mla_profile_end(C.byref(ms), C.byref(n)), "typhoon_mla_profile_end")
+    return ms.value, n.value

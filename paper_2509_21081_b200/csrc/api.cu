@@ -31,6 +31,24 @@ namespace {
 thread_local int g_last_launches = 0;
 thread_local int g_last_cuda_error = 0;
 
+// Optional CUDA-event timing of one kernel kind inside decode calls.
+struct Profile {
+    int kernel_id = -1;
+    int capacity = 0, used = 0;
+    cudaEvent_t* ev = nullptr;  // 2 per recorded launch
+};
+Profile g_prof;
+
+inline void prof_before(int id, cudaStream_t s) {
+    if (id == g_prof.kernel_id && g_prof.used < g_prof.capacity) cudaEventRecord(g_prof.ev[2 * g_prof.used], s);
+}
+inline void prof_after(int id, cudaStream_t s) {
+    if (id == g_prof.kernel_id && g_prof.used < g_prof.capacity) {
+        cudaEventRecord(g_prof.ev[2 * g_prof.used + 1], s);
+        ++g_prof.used;
+    }
+}
+
 // Hardware model of the crossover rule (defaults: measured on B200).
 double g_tensor_flops = 1.0e15;      // sustained rate the attention kernels reach, FLOP/s
 double g_hbm_bytes = 6.0e12;         // bytes/s
@@ -346,7 +364,9 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     if (pl.n_split_naive > 0) {
         NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad,
                      pl.n_split_naive, softmax_scale, o_part_n, lse_part_n};
+        prof_before(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
         e = launch_naive_attn_mma(na, s);
+        prof_after(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
     }
@@ -357,7 +377,9 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         void* q_abs = ws + pl.off_qabs;
         GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,
                   B, 512, 128, H, false};
+        prof_before(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         e = launch_gemm_tn(g1, s);
+        prof_after(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
         // --- absorb attention over latent tokens (Algorithm 1 line 6)
@@ -367,27 +389,74 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
                       ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
                       seq_lens, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
                       o_part_a, lse_part_a};
+        prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         e = launch_absorb_attn_mma(ab, s);
+        prof_after(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
         void* o_lat = ws + pl.off_olat;
+        prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
         e = launch_merge_latent(o_part_a, lse_part_a, n_chunks, B, H, o_lat, lse_a, s);
+        prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
         // --- output projection O_A W_UV^T (Algorithm 1 line 7)
         GemmTN g2{o_lat, (int64_t)H * 512, 512, sh->w_uv, 512, 128 * 512, o_abs, (int64_t)H * 128, 128,
                   B, 128, 512, H, true};
+        prof_before(TYPHOON_MLA_KERNEL_W_UV, s);
         e = launch_gemm_tn(g2, s);
+        prof_after(TYPHOON_MLA_KERNEL_W_UV, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
     }
     // --- LSE combine (Algorithm 1 line 8)
+    prof_before(TYPHOON_MLA_KERNEL_COMBINE, s);
     e = launch_combine(o_part_n, lse_part_n, pl.n_split_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
                        lse_out, s);
+    prof_after(TYPHOON_MLA_KERNEL_COMBINE, s);
     if (e != cudaSuccess) return cuda_fail(e);
     ++launches;
     g_last_launches = launches;
     return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_profile_begin(int32_t kernel_id, int32_t max_launches) {
+    if (kernel_id < 0 || kernel_id >= TYPHOON_MLA_NUM_KERNELS || max_launches < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (g_prof.ev) return TYPHOON_MLA_ERR_INVALID_ARG;
+    g_prof.ev = new (std::nothrow) cudaEvent_t[2 * (size_t)max_launches];
+    if (!g_prof.ev) return TYPHOON_MLA_ERR_ALLOC;
+    for (int i = 0; i < 2 * max_launches; ++i) {
+        cudaError_t e = cudaEventCreate(&g_prof.ev[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(g_prof.ev[j]);
+            delete[] g_prof.ev;
+            g_prof.ev = nullptr;
+            return cuda_fail(e);
+        }
+    }
+    g_prof.capacity = max_launches;
+    g_prof.used = 0;
+    g_prof.kernel_id = kernel_id;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_profile_end(double* total_ms, int32_t* launches) {
+    if (!g_prof.ev) return TYPHOON_MLA_ERR_INVALID_ARG;
+    double tot = 0.0;
+    int st = TYPHOON_MLA_OK;
+    for (int i = 0; i < g_prof.used; ++i) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(g_prof.ev[2 * i + 1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, g_prof.ev[2 * i], g_prof.ev[2 * i + 1]);
+        if (e != cudaSuccess) { st = cuda_fail(e); break; }
+        tot += ms;
+    }
+    if (total_ms) *total_ms = tot;
+    if (launches) *launches = g_prof.used;
+    for (int i = 0; i < 2 * g_prof.capacity; ++i) cudaEventDestroy(g_prof.ev[i]);
+    delete[] g_prof.ev;
+    g_prof = Profile();
+    return st;
 }
 
 size_t typhoon_mla_host_staging_bytes(const typhoon_mla_shared_t* sh, int32_t B, int32_t max_pages) {
