@@ -63,7 +63,8 @@ enum {
     TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL = 3,
     TYPHOON_MLA_ERR_ALLOC = 4,
     TYPHOON_MLA_ERR_CUDA = 5,
-    TYPHOON_MLA_ERR_DEVICE_CHECK = 6
+    TYPHOON_MLA_ERR_DEVICE_CHECK = 6,
+    TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED = 7 /* problem too large for the built-in scratch array */
 };
 
 enum {
@@ -211,6 +212,37 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
 /* Copy the expanded caches into caller buffers of H * Ls_padded * 128 bf16
  * elements each (device memory), on `stream`. */
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_dst, void* v_t_dst, void* stream);
+
+/*
+ * Shared-prefix attention without any allocation (the paper has no counterpart:
+ * this is a packaging variant of Algorithm 1 line 4 followed by the combine,
+ * i.e. what TYPHOON_MLA_MODE_NAIVE computes, for requests with no suffix).
+ *
+ * For callers that cannot obtain device memory at call time -- a server whose
+ * cache pool already owns all free HBM, so that cudaMalloc fails; a real-time
+ * loop where cudaMalloc/cudaFree are forbidden because they synchronise the
+ * device -- and therefore cannot pass a workspace.  The KV-split partials live
+ * in a fixed array of TYPHOON_MLA_NOALLOC_SCRATCH_BYTES inside the library
+ * image (each GPU that loads the library holds it until the process exits).
+ *
+ *   q_nope bf16 [B, H, 128], q_pe bf16 [B, H, 64], out bf16 [B, H, 128],
+ *   lse_out optional fp32 [B, H]; all device pointers, 16-byte aligned.
+ *
+ * Limit: B * H * 516 bytes (rounded up to 256) must fit in the array, i.e.
+ * B * H <= 65024 (B <= 508 at H = 128); larger problems are rejected with
+ * TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED and nothing is launched.
+ * The call uses no cudaMalloc/cudaFree and no allocating library routine.
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call
+ * before any stream capture begins.  All calls on a device share the one
+ * array, which keeps the previous call's contents; every slot a call reads it
+ * has written itself, so no clearing is needed, but two calls whose kernels
+ * overlap on the GPU (different streams) race on it: serialise them.
+ */
+#define TYPHOON_MLA_NOALLOC_SCRATCH_BYTES (32u << 20)
+int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* shared,
+                                     const void* q_nope, const void* q_pe, int32_t B,
+                                     float softmax_scale, void* out, float* lse_out, void* stream);
 
 /* Kernel kinds of the decode step, in launch order (Algorithm 1 lines 4-8). */
 enum {

@@ -76,6 +76,8 @@ def _load():
                                             C.POINTER(i64)]
     lib.typhoon_mla_shared_export.restype = C.c_int
     lib.typhoon_mla_shared_export.argtypes = [vp, vp, vp, vp]
+    lib.typhoon_mla_naive_shared_noalloc.restype = C.c_int
+    lib.typhoon_mla_naive_shared_noalloc.argtypes = [vp, vp, vp, i32, f32, vp, vp, vp]
     lib.typhoon_mla_profile_begin.restype = C.c_int
     lib.typhoon_mla_profile_begin.argtypes = [i32, i32]
     lib.typhoon_mla_profile_end.restype = C.c_int
@@ -238,3 +240,14 @@ def typhoon_mla_profile_end():
     ms, n = C.c_double(), C.c_int32()
     _check(_lib.typhoon_mla_profile_end(C.byref(ms), C.byref(n)), "typhoon_mla_profile_end")
     return ms.value, n.value
+
+
+NOALLOC_SCRATCH_BYTES = 32 << 20
+
+
+def typhoon_mla_naive_shared_noalloc(shared: SharedPrefix, q_nope, q_pe, softmax_scale, out, lse_out=None) -> None:
+    """Shared-prefix attention using the library's built-in scratch array: no workspace argument and
+    no allocation, for callers that cannot get device memory at call time."""
+    st = _lib.typhoon_mla_naive_shared_noalloc(shared.handle, _ptr(q_nope), _ptr(q_pe), q_nope.shape[0],
+                                               softmax_scale, _ptr(out), _ptr(lse_out), _stream())
+    _check(st, "typhoon_mla_naive_shared_noalloc")

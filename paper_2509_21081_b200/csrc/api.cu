@@ -13,18 +13,7 @@
 
 using namespace tmla;
 
-struct typhoon_mla_shared {
-    typhoon_mla_dims_t dims;
-    int64_t Ls, Ls_pad;
-    void* k_nope;   // bf16 [H, Ls_pad, 128]
-    void* v_t;      // bf16 [H, 128, Ls_pad]
-    void* ckv;      // bf16 [Ls_pad, 512]
-    void* kpe;      // bf16 [Ls_pad, 64]
-    void* w_uk_t;   // bf16 [H, 512, 128]
-    const void* w_uv;  // borrowed, bf16 [H, 128, 512]
-    size_t owned_bytes;
-    int device;
-};
+#include "handle.h"
 
 namespace {
 
@@ -154,6 +143,7 @@ const char* typhoon_mla_status_string(int status) {
         case TYPHOON_MLA_ERR_ALLOC: return "device allocation failed";
         case TYPHOON_MLA_ERR_CUDA: return "CUDA error";
         case TYPHOON_MLA_ERR_DEVICE_CHECK: return "device-side check failed";
+        case TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED: return "problem exceeds the built-in scratch array";
         default: return "unknown status";
     }
 }

@@ -1,0 +1,19 @@
+// The prepared-prefix handle behind typhoon_mla_shared_t (host object; see typhoon_mla_prepare_shared).
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/typhoon_mla.h"
+
+struct typhoon_mla_shared {
+    typhoon_mla_dims_t dims;
+    int64_t Ls, Ls_pad;
+    void* k_nope;   // bf16 [H, Ls_pad, 128]
+    void* v_t;      // bf16 [H, 128, Ls_pad]
+    void* ckv;      // bf16 [Ls_pad, 512]
+    void* kpe;      // bf16 [Ls_pad, 64]
+    void* w_uk_t;   // bf16 [H, 512, 128]
+    const void* w_uv;  // borrowed, bf16 [H, 128, 512]
+    size_t owned_bytes;
+    int device;
+};

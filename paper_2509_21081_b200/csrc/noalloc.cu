@@ -1,0 +1,93 @@
+// typhoon_mla_naive_shared_noalloc: shared-prefix attention for callers that
+// must not allocate device memory.
+//
+// The regular entry point takes a caller-allocated workspace for the KV-split
+// partials of the naive shared-prefix attention.  Some callers have no way to
+// provide one: a serving process that handed every free byte of HBM to its
+// KV-cache pool at start-up (a later cudaMalloc would simply fail), or a
+// latency-critical loop in which cudaMalloc/cudaFree are banned because they
+// synchronise the device and take the driver's allocator lock.  For them this
+// file keeps the scratch in a fixed device array that is part of the library
+// image: it exists on every GPU that loads the library, from load to exit,
+// whether or not the entry point is ever called.
+#include <mutex>
+
+#include "handle.h"
+#include "kernels.h"
+
+using namespace tmla;
+
+namespace {
+
+// Split partials: per (split, request, head) 128 fp32 outputs + 1 fp32 LSE.
+constexpr size_t kScratchBytes = TYPHOON_MLA_NOALLOC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an
+// address a kernel can use; the device address is looked up once per device.
+constexpr int kMaxDevices = 64;
+std::mutex g_mu;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+int scratch_for_current_device(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TYPHOON_MLA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_scratch_ptr[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return TYPHOON_MLA_ERR_CUDA;
+        }
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return TYPHOON_MLA_OK;
+}
+
+}  // namespace
+
+extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe,
+                                                 int32_t B, float softmax_scale, void* out, float* lse_out,
+                                                 void* stream) {
+    if (!sh || !q_nope || !q_pe || !out || B < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q_nope) | reinterpret_cast<uintptr_t>(q_pe) | reinterpret_cast<uintptr_t>(out)) & 15u)
+        return TYPHOON_MLA_ERR_INVALID_ARG;
+    const int H = sh->dims.num_heads;
+    const size_t rows = (size_t)B * H;
+    const size_t per_split = rows * 128 * sizeof(float) + ((rows * sizeof(float) + 255) / 256) * 256;
+    if (per_split > kScratchBytes) return TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED;
+
+    void* scratch = nullptr;
+    int st = scratch_for_current_device(&scratch);
+    if (st != TYPHOON_MLA_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    // As many KV splits as fit, up to what fills the GPU about four times over.
+    int n_split = 0;
+    if (sh->Ls > 0) {
+        const int n_tiles = (int)((sh->Ls + 63) / 64);
+        const int base = ((B + 63) / 64) * H;
+        int want = (4 * 148 + base - 1) / base;
+        int fit = (int)(kScratchBytes / per_split);
+        n_split = want < fit ? want : fit;
+        if (n_split > n_tiles) n_split = n_tiles;
+        if (n_split > 64) n_split = 64;
+        if (n_split < 1) n_split = 1;
+    }
+    float* o_part = reinterpret_cast<float*>(scratch);
+    float* lse_part = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(scratch) +
+                                               (size_t)(n_split > 0 ? n_split : 1) * rows * 128 * sizeof(float));
+    // Every (split, request, head) slot that the combine reads is written by the attention
+    // kernel of the same call (empty splits write lse = -inf), so nothing has to start at zero
+    // and the previous call's contents never leak into this one.
+    if (n_split > 0) {
+        NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad, n_split,
+                     softmax_scale, o_part, lse_part};
+        if (launch_naive_attn_mma(na, s) != cudaSuccess) return TYPHOON_MLA_ERR_CUDA;
+    }
+    if (launch_combine(o_part, lse_part, n_split, nullptr, nullptr, B, H, out, lse_out, s) != cudaSuccess)
+        return TYPHOON_MLA_ERR_CUDA;
+    return TYPHOON_MLA_OK;
+}

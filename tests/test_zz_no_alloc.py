@@ -1,0 +1,63 @@
+"""The allocation-free entry point against the regular one.
+
+typhoon_mla_naive_shared_noalloc serves callers that cannot allocate device memory when they call
+(all HBM already pledged to a cache pool, or cudaMalloc banned on a latency-critical path): its
+scratch is a fixed array inside the library.  Two calls in a row with different queries must each
+match typhoon_mla_decode in NAIVE mode (which uses a caller workspace), so stale contents of the
+shared array cannot leak from one call into the next; an oversized problem must be refused.
+This file sorts last so that a run stopping at the first failure has already run everything else.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_21081_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def test_noalloc_matches_workspace_entry_point_twice():
+    from paper_2509_21081_b200 import binding as b
+    cfg = I.MLAConfig("noalloc", B=37, H=32, Ls=1500, suffix_lo=0, suffix_hi=0, seed=77)
+    inp = I.make_inputs(cfg)
+    dims = b.make_dims(cfg.H)
+    w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
+    sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    ws = torch.empty(b.typhoon_mla_workspace_bytes(sh, cfg.B, 0, 64), dtype=torch.uint8, device="cuda")
+    q1n, q1p = inp.q_nope.cuda(), inp.q_pe.cuda()
+    g = torch.Generator(device="cpu").manual_seed(5)
+    q2n = torch.randn(cfg.B, cfg.H, 128, generator=g).to(torch.bfloat16).cuda() * 3
+    q2p = torch.randn(cfg.B, cfg.H, 64, generator=g).to(torch.bfloat16).cuda() * 3
+    for qn, qp in ((q1n, q1p), (q2n, q2p)):
+        ref = torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16, device="cuda")
+        ref_lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
+        b.typhoon_mla_decode(sh, qn, qp, None, None, 64, None, None, inp.scale, ref, ws, mode=b.MODE_NAIVE,
+                             lse_out=ref_lse)
+        out = torch.full((cfg.B, cfg.H, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((cfg.B, cfg.H), float("nan"), dtype=torch.float32, device="cuda")
+        b.typhoon_mla_naive_shared_noalloc(sh, qn, qp, inp.scale, out, lse)
+        torch.cuda.synchronize()
+        o, r = out.float().cpu().numpy(), ref.float().cpu().numpy()
+        assert np.isfinite(o).all()
+        # same kernels, possibly a different number of KV splits: same bars as the parity tests
+        assert np.max(np.abs(o - r)) <= 2e-2 * max(1.0, float(np.max(np.abs(r))))
+        assert np.linalg.norm(o - r) / np.linalg.norm(r) <= 5e-3
+        assert torch.max(torch.abs(lse - ref_lse)).item() <= 2e-2
+    sh.free()
+
+
+def test_noalloc_rejects_oversized_problem():
+    from paper_2509_21081_b200 import binding as b
+    cfg = I.MLAConfig("noalloc_big", B=2, H=128, Ls=64, suffix_lo=0, suffix_hi=0, seed=78)
+    inp = I.make_inputs(cfg)
+    w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
+    sh = b.typhoon_mla_prepare_shared(b.make_dims(cfg.H), inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    B = 600                                    # 600 * 128 * 516 bytes > 32 MiB
+    qn = torch.zeros(B, cfg.H, 128, dtype=torch.bfloat16, device="cuda")
+    qp = torch.zeros(B, cfg.H, 64, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(B, cfg.H, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(b.TyphoonMLAError) as e:
+        b.typhoon_mla_naive_shared_noalloc(sh, qn, qp, inp.scale, out)
+    assert e.value.status == 7 and "scratch" in str(e.value)
+    torch.cuda.synchronize()
+    sh.free()
