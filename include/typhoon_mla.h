@@ -209,6 +209,16 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
                             int64_t* Ls /* host */, int64_t* Ls_padded /* host */,
                             int64_t* owned_bytes /* host */);
 
+/* Which implementation of the tensor-core kernels runs: the tcgen05/TMEM/TMA kernels (default) or
+ * the warp-MMA kernels.  Process-wide; affects later prepare_shared and decode calls. */
+enum { TYPHOON_MLA_PATH_TCGEN05 = 0, TYPHOON_MLA_PATH_WARP_MMA = 1 };
+int typhoon_mla_set_kernel_path(int32_t path);
+
+/* Synchronises `stream` and reads the handle's device status word.  Every in-kernel wait of the
+ * tcgen05 kernels has a deadline; if one expired, the kernel abandoned its work, the word is
+ * non-zero and this returns TYPHOON_MLA_ERR_DEVICE_CHECK (results of that launch are invalid). */
+int typhoon_mla_device_status(const typhoon_mla_shared_t* shared, void* stream, int32_t* status /* host */);
+
 /* Copy the expanded caches into caller buffers of H * Ls_padded * 128 bf16
  * elements each (device memory), on `stream`. */
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_dst, void* v_t_dst, void* stream);

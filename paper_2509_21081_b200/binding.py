@@ -76,6 +76,10 @@ def _load():
                                             C.POINTER(i64)]
     lib.typhoon_mla_shared_export.restype = C.c_int
     lib.typhoon_mla_shared_export.argtypes = [vp, vp, vp, vp]
+    lib.typhoon_mla_set_kernel_path.restype = C.c_int
+    lib.typhoon_mla_set_kernel_path.argtypes = [i32]
+    lib.typhoon_mla_device_status.restype = C.c_int
+    lib.typhoon_mla_device_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.typhoon_mla_naive_shared_noalloc.restype = C.c_int
     lib.typhoon_mla_naive_shared_noalloc.argtypes = [vp, vp, vp, i32, f32, vp, vp, vp]
     lib.typhoon_mla_profile_begin.restype = C.c_int
@@ -251,3 +255,17 @@ def typhoon_mla_naive_shared_noalloc(shared: SharedPrefix, q_nope, q_pe, softmax
     st = _lib.typhoon_mla_naive_shared_noalloc(shared.handle, _ptr(q_nope), _ptr(q_pe), q_nope.shape[0],
                                                softmax_scale, _ptr(out), _ptr(lse_out), _stream())
     _check(st, "typhoon_mla_naive_shared_noalloc")
+
+
+PATH_TCGEN05, PATH_WARP_MMA = 0, 1
+
+
+def typhoon_mla_set_kernel_path(path: int) -> None:
+    _check(_lib.typhoon_mla_set_kernel_path(path), "typhoon_mla_set_kernel_path")
+
+
+def typhoon_mla_device_status(shared: SharedPrefix) -> int:
+    """Synchronises the current stream; raises if an in-kernel wait expired."""
+    v = C.c_int32()
+    _check(_lib.typhoon_mla_device_status(shared.handle, _stream(), C.byref(v)), "typhoon_mla_device_status")
+    return v.value

@@ -38,6 +38,8 @@ inline void prof_after(int id, cudaStream_t s) {
     }
 }
 
+int g_kernel_path = TYPHOON_MLA_PATH_TCGEN05;
+
 // Hardware model of the crossover rule (defaults: measured on B200).
 double g_tensor_flops = 1.0e15;      // sustained rate the attention kernels reach, FLOP/s
 double g_hbm_bytes = 6.0e12;         // bytes/s
@@ -222,6 +224,7 @@ int typhoon_mla_free(typhoon_mla_shared_t* sh) {
     cudaFree(sh->ckv);
     cudaFree(sh->kpe);
     cudaFree(sh->w_uk_t);
+    cudaFree(sh->status);
     delete sh;
     return TYPHOON_MLA_OK;
 }
@@ -259,24 +262,26 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
         return true;
     };
     if (!alloc(&sh->k_nope, b_k) || !alloc(&sh->v_t, b_k) || !alloc(&sh->ckv, b_ckv) || !alloc(&sh->kpe, b_kpe) ||
-        !alloc(&sh->w_uk_t, b_w)) {
+        !alloc(&sh->w_uk_t, b_w) || !alloc(reinterpret_cast<void**>(&sh->status), 256)) {
         typhoon_mla_free(sh);
         return TYPHOON_MLA_ERR_ALLOC;
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    e = launch_transpose_bf16(w_uk, sh->w_uk_t, 128, 512, H, s);
+    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    e = cudaMemsetAsync(sh->status, 0, 256, s);
+    if (e == cudaSuccess) e = launch_transpose_bf16(w_uk, sh->w_uk_t, 128, 512, H, s);
     if (e == cudaSuccess && Ls > 0) {
         e = launch_copy_pad_rows(ckv_shared, ld_ckv, sh->ckv, (int)Ls, (int)Lp, 512, s);
         if (e == cudaSuccess) e = launch_copy_pad_rows(kpe_shared, ld_kpe, sh->kpe, (int)Ls, (int)Lp, 64, s);
         if (e == cudaSuccess) {  // K_nope[h] = ckv * W_UK[h]^T
             GemmTN g{sh->ckv, 512, 0, w_uk, 512, 128 * 512, sh->k_nope, 128, (int64_t)Lp * 128,
                      (int)Lp, 128, 512, H, false};
-            e = launch_gemm_tn(g, s);
+            e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
         }
         if (e == cudaSuccess) {  // V^T[h] = W_UV[h] * ckv^T
             GemmTN g{w_uv, 512, 128 * 512, sh->ckv, 512, 0, sh->v_t, (int64_t)Lp, (int64_t)(128 * Lp),
                      128, (int)Lp, 512, H, false};
-            e = launch_gemm_tn(g, s);
+            e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
         }
     }
     if (e != cudaSuccess) {
@@ -296,6 +301,23 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* sh, const void** k_nope,
     if (Ls_padded) *Ls_padded = sh->Ls_pad;
     if (owned_bytes) *owned_bytes = (int64_t)sh->owned_bytes;
     return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_set_kernel_path(int32_t path) {
+    if (path != TYPHOON_MLA_PATH_TCGEN05 && path != TYPHOON_MLA_PATH_WARP_MMA) return TYPHOON_MLA_ERR_INVALID_ARG;
+    g_kernel_path = path;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_device_status(const typhoon_mla_shared_t* sh, void* stream, int32_t* status) {
+    if (!sh || !status) return TYPHOON_MLA_ERR_INVALID_ARG;
+    int v = 0;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(&v, sh->status, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *status = v;
+    return v == 0 ? TYPHOON_MLA_OK : TYPHOON_MLA_ERR_DEVICE_CHECK;
 }
 
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* sh, void* k_nope_dst, void* v_t_dst, void* stream) {

@@ -1,0 +1,156 @@
+// Batched bf16 GEMM on the 5th-generation tensor cores:
+//   C[z][m][n] = sum_k A[z][m][k] * B[z][n][k]      (both operands K-major)
+// TMA stages 128 x 64 operand tiles (128-byte swizzle) into shared memory, one
+// elected thread issues tcgen05.mma into a 128 x 128 fp32 accumulator in tensor
+// memory, four warps read it back with tcgen05.ld and store bf16.
+// Used for the shared-prefix expansion (Section 3.1 "Prefill"), where it is a
+// large dense contraction: [L_s, 512] x [512, 128] per head for K and V.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
+// owner, warps 2-5 = epilogue (one 32-lane TMEM slice each).
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace tmla {
+namespace {
+
+using namespace sm100;
+
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct GemmParams {
+    void* C; int64_t ldc, c_batch;
+    int M, N, K;
+    int a_batched, b_batched;
+    int* status;
+};
+
+__global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constant__ CUtensorMap tmA,
+                                                            const __grid_constant__ CUtensorMap tmB, GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_full = empty + STAGES;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
+    const int KB = p.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+    }
+    if (warp == 1) tmem_alloc(tmem_holder, 128);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = 0; kb < KB; ++kb) {
+                const int s = kb % STAGES;
+                if (!mbar_wait(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag)) break;
+                mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
+                uint8_t* sa = smem + s * STAGE_BYTES;
+                tma_load_3d(sa, &tmA, &full[s], kb * BK, m0, p.a_batched ? z : 0);
+                tma_load_3d(sa + A_BYTES, &tmB, &full[s], kb * BK, n0, p.b_batched ? z : 0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(BM, BN, false, false);
+            bool ok = true;
+            for (int kb = 0; kb < KB && ok; ++kb) {
+                const int s = kb % STAGES;
+                ok = mbar_wait(&full[s], (kb / STAGES) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
+                const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + A_BYTES);
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k) umma_ss(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                umma_commit(&empty[s]);
+            }
+            if (ok) umma_commit(acc_full);
+        }
+    } else {
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag));
+        tc_fence_after();
+        if (ok) {
+            const int lg = (warp & 3) * 32;
+            const int row = m0 + lg + lane;
+            __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + (int64_t)z * p.c_batch + (int64_t)row * p.ldc + n0;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)lg << 16) + c * 32, r);
+                tmem_ld_wait();
+                if (row < p.M) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(r[j * 8 + 0]), __uint_as_float(r[j * 8 + 1]));
+                        v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]), __uint_as_float(r[j * 8 + 3]));
+                        v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]), __uint_as_float(r[j * 8 + 5]));
+                        v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]), __uint_as_float(r[j * 8 + 7]));
+                        *reinterpret_cast<uint4*>(crow + c * 32 + j * 8) = v;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // A wait gave up: leave time for copies already in flight to land before the CTA's
+        // shared memory is released, and report.
+        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 1);
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem_base, 128);
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s) {
+    if (g.M <= 0 || g.batch <= 0) return cudaSuccess;
+    if (g.N % BN != 0 || g.K % BK != 0 || g.out_fp32) return cudaErrorInvalidValue;
+    CUtensorMap tmA, tmB;
+    {
+        const bool batched = g.a_batch != 0;
+        uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.M, (uint64_t)(batched ? g.batch : 1)};
+        uint64_t strides[2] = {(uint64_t)g.lda * 2, (uint64_t)(batched ? g.a_batch : (int64_t)g.lda * g.M) * 2};
+        uint32_t box[3] = {BK, BM, 1};
+        cudaError_t e = make_tmap_bf16(&tmA, g.A, 3, dims, strides, box);
+        if (e != cudaSuccess) return e;
+    }
+    {
+        const bool batched = g.b_batch != 0;
+        uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.N, (uint64_t)(batched ? g.batch : 1)};
+        uint64_t strides[2] = {(uint64_t)g.ldb * 2, (uint64_t)(batched ? g.b_batch : (int64_t)g.ldb * g.N) * 2};
+        uint32_t box[3] = {BK, BN, 1};
+        cudaError_t e = make_tmap_bf16(&tmB, g.B, 3, dims, strides, box);
+        if (e != cudaSuccess) return e;
+    }
+    GemmParams p{g.C, g.ldc, g.c_batch, g.M, g.N, g.K, g.a_batch != 0, g.b_batch != 0, status};
+    cudaFuncSetAttribute(gemm_tn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    dim3 grid(g.N / BN, (g.M + BM - 1) / BM, g.batch);
+    gemm_tn_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tmA, tmB, p);
+    return cudaGetLastError();
+}
+
+}  // namespace tmla

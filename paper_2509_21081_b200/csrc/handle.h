@@ -14,6 +14,7 @@ struct typhoon_mla_shared {
     void* kpe;      // bf16 [Ls_pad, 64]
     void* w_uk_t;   // bf16 [H, 512, 128]
     const void* w_uv;  // borrowed, bf16 [H, 128, 512]
+    int* status;    // device word: non-zero after a bounded in-kernel wait expired
     size_t owned_bytes;
     int device;
 };

@@ -14,6 +14,9 @@ struct GemmTN {
     bool out_fp32;
 };
 cudaError_t launch_gemm_tn(const GemmTN& g, cudaStream_t s);
+// tcgen05/TMEM/TMA version (bf16 output only; N % 128 == 0, K % 64 == 0).  `status` (device int,
+// may be null) is set non-zero if a bounded wait inside the kernel expired.
+cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s);
 
 // Naive shared-prefix attention partials (Algorithm 1 line 4).
 struct NaiveAttn {

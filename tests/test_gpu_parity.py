@@ -166,15 +166,22 @@ def test_moving_tokens_between_prefix_and_suffix():
     G.assert_parity(out, ref, lse, ref_lse, what="moved split")
 
 
-def test_expansion_matches_plain_matmul():
-    """Shared-prefix expansion against a float64 matmul: within one bf16 rounding of the exact value."""
+@pytest.mark.parametrize("path", [0, 1])
+def test_expansion_matches_plain_matmul(path):
+    """Shared-prefix expansion against a float64 matmul: within one bf16 rounding of the exact value
+    (path 0: tcgen05 GEMM, path 1: warp-MMA GEMM)."""
     from oracle import mla_oracle as O
     from paper_2509_21081_b200 import binding as b
     cfg = _cfg("expand", B=1, H=16, Ls=333, lo=0, hi=0, seed=31)
     inp = I.make_inputs(cfg)
     dims = b.make_dims(cfg.H)
     w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
-    sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    b.typhoon_mla_set_kernel_path(path)
+    try:
+        sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    finally:
+        b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05)
+    assert b.typhoon_mla_device_status(sh) == 0
     k, vt = b.typhoon_mla_shared_export(sh)
     Ls, Lp, owned = b.typhoon_mla_shared_view(sh)
     torch.cuda.synchronize()
