@@ -63,6 +63,7 @@ int cuda_fail(cudaError_t e) {
 struct Plan {
     int mode;
     int n_split_naive;       // KV splits of the naive kernel
+    int n_slots_naive;       // partial slots the naive kernel writes (>= n_split_naive)
     int chunk;               // tokens per absorb chunk
     int n_shared_chunks;     // absorb chunks over the shared prefix (ABSORB mode)
     int n_suffix_chunks;
@@ -71,6 +72,29 @@ struct Plan {
 };
 
 constexpr int kNumSM = 148;
+
+// KV splits of the tcgen05 naive kernel: minimise waves x (tiles per CTA + fixed cost) over the
+// candidate split counts (one CTA per SM; the fixed cost is the Q load and pipeline fill).
+int naive_splits_sm100(int B, int H, int64_t Ls) {
+    if (Ls <= 0) return 0;
+    const int n_tiles = (int)((Ls + 63) / 64);
+    const int base = (B <= 128 ? 1 : (B + 255) / 256) * H;
+    const double fixed = 6.0;
+    int best = 1;
+    double best_cost = 1e30;
+    for (int ns = 1; ns <= std::min(n_tiles, 32); ++ns) {
+        const int per = (n_tiles + ns - 1) / ns;
+        const int real = (n_tiles + per - 1) / per;
+        if (real != ns) continue;
+        const int waves = (real * base + kNumSM - 1) / kNumSM;
+        const double cost = waves * (per + fixed);
+        if (cost < best_cost - 1e-9) {
+            best_cost = cost;
+            best = ns;
+        }
+    }
+    return best;
+}
 
 int naive_splits(int B, int H, int64_t Ls) {
     if (Ls <= 0) return 0;
@@ -98,7 +122,9 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
     const int64_t cap = (int64_t)max_pages * page_size;
     const bool use_naive = (mode != TYPHOON_MLA_MODE_ABSORB) && sh->Ls > 0;
     const bool use_absorb = (mode != TYPHOON_MLA_MODE_NAIVE);
-    p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls) : 0;
+    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    p.n_split_naive = use_naive ? (tc ? naive_splits_sm100(B, H, sh->Ls) : naive_splits(B, H, sh->Ls)) : 0;
+    p.n_slots_naive = tc ? naive_sm100_slots(B, p.n_split_naive) : p.n_split_naive;
     if (use_absorb) {
         absorb_chunks(B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
                       &p.n_suffix_chunks);
@@ -117,8 +143,8 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
     p.off_olat = take(BH * 512 * 2);
     p.off_lse_a = take(BH * 4);
     p.off_oabs = take(BH * 128 * 4);
-    p.off_opart_n = take((size_t)p.n_split_naive * BH * 128 * 4);
-    p.off_lsepart_n = take((size_t)p.n_split_naive * BH * 4);
+    p.off_opart_n = take((size_t)p.n_slots_naive * BH * 128 * 4);
+    p.off_lsepart_n = take((size_t)p.n_slots_naive * BH * 4);
     p.total = off;
     return p;
 }
@@ -284,6 +310,8 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
         }
     }
+    if (e == cudaSuccess && Ls > 0)
+        e = make_naive_sm100_tmaps(sh->k_nope, sh->kpe, sh->v_t, H, sh->Ls_pad, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt);
     if (e != cudaSuccess) {
         typhoon_mla_free(sh);
         return cuda_fail(e);
@@ -332,9 +360,16 @@ int typhoon_mla_shared_export(const typhoon_mla_shared_t* sh, void* k_nope_dst, 
 
 size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* sh, int32_t B, int32_t max_pages, int32_t page_size) {
     if (!sh || B < 1 || max_pages < 0 || (page_size != 64 && page_size != 128)) return 0;
-    size_t a = make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_ABSORB).total;
-    size_t h = make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID).total;
-    return std::max(a, h) + 256;
+    // worst case over modes and kernel paths
+    const int saved = g_kernel_path;
+    size_t worst = 0;
+    for (int path : {TYPHOON_MLA_PATH_TCGEN05, TYPHOON_MLA_PATH_WARP_MMA}) {
+        g_kernel_path = path;
+        worst = std::max(worst, make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_ABSORB).total);
+        worst = std::max(worst, make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID).total);
+    }
+    g_kernel_path = saved;
+    return worst + 256;
 }
 
 int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
@@ -374,10 +409,16 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
 
     // --- naive shared-prefix attention (Algorithm 1 line 4)
     if (pl.n_split_naive > 0) {
-        NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad,
-                     pl.n_split_naive, softmax_scale, o_part_n, lse_part_n};
         prof_before(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
-        e = launch_naive_attn_mma(na, s);
+        if (g_kernel_path == TYPHOON_MLA_PATH_TCGEN05) {
+            NaiveAttnSm100 na{q_nope, q_pe, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt, B, H, (int)sh->Ls,
+                              pl.n_split_naive, softmax_scale, o_part_n, lse_part_n, sh->status};
+            e = launch_naive_attn_sm100(na, s);
+        } else {
+            NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad,
+                         pl.n_split_naive, softmax_scale, o_part_n, lse_part_n};
+            e = launch_naive_attn_mma(na, s);
+        }
         prof_after(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
@@ -423,7 +464,7 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     }
     // --- LSE combine (Algorithm 1 line 8)
     prof_before(TYPHOON_MLA_KERNEL_COMBINE, s);
-    e = launch_combine(o_part_n, lse_part_n, pl.n_split_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
+    e = launch_combine(o_part_n, lse_part_n, pl.n_slots_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
                        lse_out, s);
     prof_after(TYPHOON_MLA_KERNEL_COMBINE, s);
     if (e != cudaSuccess) return cuda_fail(e);

@@ -1,5 +1,6 @@
 // The prepared-prefix handle behind typhoon_mla_shared_t (host object; see typhoon_mla_prepare_shared).
 #pragma once
+#include <cuda.h>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -14,6 +15,7 @@ struct typhoon_mla_shared {
     void* kpe;      // bf16 [Ls_pad, 64]
     void* w_uk_t;   // bf16 [H, 512, 128]
     const void* w_uv;  // borrowed, bf16 [H, 128, 512]
+    CUtensorMap tm_kn, tm_kp, tm_vt;   // TMA descriptors of k_nope, kpe, v_t (valid if Ls > 0)
     int* status;    // device word: non-zero after a bounded in-kernel wait expired
     size_t owned_bytes;
     int device;

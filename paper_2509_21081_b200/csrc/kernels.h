@@ -1,5 +1,6 @@
 // Internal launch interfaces between the C ABI (api.cu) and the kernels.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -28,6 +29,22 @@ struct NaiveAttn {
     float* lse_part; // [n_split][B][H], natural log
 };
 cudaError_t launch_naive_attn_mma(const NaiveAttn& p, cudaStream_t s);
+
+// tcgen05/TMEM/TMA version.  The tensor maps of the expanded cache are built once per prefix
+// (make_naive_sm100_tmaps); partial slots = naive_sm100_slots(B, n_split).
+struct NaiveAttnSm100 {
+    const void* q_nope; const void* q_pe;
+    const CUtensorMap* tm_kn; const CUtensorMap* tm_kp; const CUtensorMap* tm_vt;   // host pointers
+    int B, H; int Ls; int n_split;
+    float scale;
+    float* o_part;   // [slots][B][H][128]
+    float* lse_part; // [slots][B][H]
+    int* status;     // device word, set non-zero if a bounded wait expired
+};
+int naive_sm100_slots(int B, int n_split);
+cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s);
+cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const void* v_t, int H, int64_t Ls_pad,
+                                   CUtensorMap* tm_kn, CUtensorMap* tm_kp, CUtensorMap* tm_vt);
 
 // Absorb attention partials over latent tokens (Algorithm 1 line 6).
 struct AbsorbAttn {

@@ -16,6 +16,15 @@ pytestmark = pytest.mark.gpu
 ABSORB, HYBRID, AUTO, NAIVE = 1, 2, 0, 3
 
 
+@pytest.fixture(autouse=True, params=["tcgen05", "warp_mma"])
+def kernel_path(request):
+    """Every test runs on both implementations of the tensor-core kernels."""
+    from paper_2509_21081_b200 import binding as b
+    b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05 if request.param == "tcgen05" else b.PATH_WARP_MMA)
+    yield request.param
+    b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05)
+
+
 def _cfg(name, B, H, Ls, lo, hi, seed, page_size=64):
     return I.MLAConfig(name, B=B, H=H, Ls=Ls, suffix_lo=lo, suffix_hi=hi, seed=seed, page_size=page_size)
 
@@ -166,21 +175,15 @@ def test_moving_tokens_between_prefix_and_suffix():
     G.assert_parity(out, ref, lse, ref_lse, what="moved split")
 
 
-@pytest.mark.parametrize("path", [0, 1])
-def test_expansion_matches_plain_matmul(path):
-    """Shared-prefix expansion against a float64 matmul: within one bf16 rounding of the exact value
-    (path 0: tcgen05 GEMM, path 1: warp-MMA GEMM)."""
+def test_expansion_matches_plain_matmul():
+    """Shared-prefix expansion against a float64 matmul: within one bf16 rounding of the exact value."""
     from oracle import mla_oracle as O
     from paper_2509_21081_b200 import binding as b
     cfg = _cfg("expand", B=1, H=16, Ls=333, lo=0, hi=0, seed=31)
     inp = I.make_inputs(cfg)
     dims = b.make_dims(cfg.H)
     w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
-    b.typhoon_mla_set_kernel_path(path)
-    try:
-        sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
-    finally:
-        b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05)
+    sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
     assert b.typhoon_mla_device_status(sh) == 0
     k, vt = b.typhoon_mla_shared_export(sh)
     Ls, Lp, owned = b.typhoon_mla_shared_view(sh)
