@@ -335,6 +335,7 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="config 4 fan-out sweep over batch sizes and modes")
     ap.add_argument("--ref-heads", type=int, default=64, help="heads the CPU checker is timed on (scaled up)")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -365,7 +366,8 @@ def main():
         cfg = I.CONFIGS[args.config]
         if args.batch:
             cfg = cfg.with_batch(args.batch)
-        line = bench_config(cfg, args, mode, rank, world, local, with_cpu=not args.no_cpu)
+        line = bench_config(cfg, args, mode, rank, world, local, with_cpu=not args.no_cpu,
+                            with_e2e=not args.no_e2e)
         if rank == 0:
             print(json.dumps(line), flush=True)
     if world > 1:

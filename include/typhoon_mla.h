@@ -86,8 +86,10 @@ enum { TYPHOON_MLA_COST_NAIVE = 0, TYPHOON_MLA_COST_ABSORB = 1, TYPHOON_MLA_COST
  *   w_uk        bf16 [H, 128, 512] contiguous   (W_KVb1)
  *   w_uv        bf16 [H, 128, 512] contiguous   (W_KVb2)
  *
- * The handle OWNS (cudaMalloc) the expanded per-head keys K_nope [H, Ls', 128],
- * the expanded values stored transposed V^T [H, 128, Ls'], a copy of the shared
+ * The handle OWNS (cudaMalloc) the expanded per-head keys K_nope, stored as
+ * contiguous 64-token x 64-dim tiles [H, Ls'/64, 2, 64, 64],
+ * the expanded values stored transposed in 64-token blocks V^T [H, Ls'/64, 128, 64]
+ * (each block contiguous, so one KV tile is one contiguous 16 KB read), a copy of the shared
  * latent cache and rope keys, and a transposed copy of W_UK; Ls' is Ls rounded
  * up to a multiple of 128, the padding is zero.  It BORROWS w_uv: the caller
  * keeps w_uv alive and unchanged until typhoon_mla_free.  Ls may be 0.
@@ -203,7 +205,7 @@ int typhoon_mla_cost_model(const typhoon_mla_dims_t* dims /* host */, int32_t ki
                            int64_t* macs /* host */, int64_t* hbm_words /* host */);
 
 /* Read-only views of what the handle owns (for tests and accounting):
- * k_nope bf16 [H, Ls_padded, 128]; v_t bf16 [H, 128, Ls_padded]. */
+ * k_nope bf16 [H, Ls_padded/64, 2, 64, 64]; v_t bf16 [H, Ls_padded/64, 128, 64]. */
 int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
                             const void** k_nope, const void** v_t,
                             int64_t* Ls /* host */, int64_t* Ls_padded /* host */,

@@ -220,11 +220,11 @@ def typhoon_mla_shared_view(shared: SharedPrefix):
 
 
 def typhoon_mla_shared_export(shared: SharedPrefix):
-    """Copies of the expanded caches: k_nope [H, Ls_pad, 128], v_t [H, 128, Ls_pad]."""
+    """Copies of the expanded caches: k_nope [H, Ls_pad/64, 2, 64, 64], v_t [H, Ls_pad/64, 128, 64]."""
     _, Lp, _ = typhoon_mla_shared_view(shared)
     H = shared.dims.num_heads
-    kt = torch.empty(H, Lp, 128, dtype=torch.bfloat16, device="cuda")
-    vt = torch.empty(H, 128, Lp, dtype=torch.bfloat16, device="cuda")
+    kt = torch.empty(H, Lp // 64, 2, 64, 64, dtype=torch.bfloat16, device="cuda")
+    vt = torch.empty(H, Lp // 64, 128, 64, dtype=torch.bfloat16, device="cuda")
     _check(_lib.typhoon_mla_shared_export(shared.handle, _ptr(kt), _ptr(vt), _stream()), "typhoon_mla_shared_export")
     return kt, vt
 

@@ -40,7 +40,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         o = os.path.join(OBJ_DIR, src[:-3] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr_m):
-            cmd = [NVCC, *FLAGS, "-c", s, "-o", o]
+            cmd = [NVCC, *FLAGS, *os.environ.get("TMLA_NVCC_EXTRA", "").split(), "-c", s, "-o", o]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)

@@ -78,6 +78,13 @@ constexpr int kNumSM = 148;
 int naive_splits_sm100(int B, int H, int64_t Ls) {
     if (Ls <= 0) return 0;
     const int n_tiles = (int)((Ls + 63) / 64);
+    if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_SPLITS")) {   // tuning aid
+        const int v = std::atoi(ov);
+        if (v >= 1) {
+            const int per = (n_tiles + std::min(v, n_tiles) - 1) / std::min(v, n_tiles);
+            return (n_tiles + per - 1) / per;
+        }
+    }
     const int base = (B <= 128 ? 1 : (B + 255) / 256) * H;
     const double fixed = 6.0;
     int best = 1;
@@ -301,12 +308,12 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
         if (e == cudaSuccess) e = launch_copy_pad_rows(kpe_shared, ld_kpe, sh->kpe, (int)Ls, (int)Lp, 64, s);
         if (e == cudaSuccess) {  // K_nope[h] = ckv * W_UK[h]^T
             GemmTN g{sh->ckv, 512, 0, w_uk, 512, 128 * 512, sh->k_nope, 128, (int64_t)Lp * 128,
-                     (int)Lp, 128, 512, H, false};
+                     (int)Lp, 128, 512, H, false, 0, true};
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
         }
         if (e == cudaSuccess) {  // V^T[h] = W_UV[h] * ckv^T
             GemmTN g{w_uv, 512, 128 * 512, sh->ckv, 512, 0, sh->v_t, (int64_t)Lp, (int64_t)(128 * Lp),
-                     128, (int)Lp, 512, H, false};
+                     128, (int)Lp, 512, H, false, 64};
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
         }
     }

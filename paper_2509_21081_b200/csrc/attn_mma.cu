@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(128) naive_attn_mma_kernel(NaiveAttn p) {
     const __nv_bfloat16* qn = reinterpret_cast<const __nv_bfloat16*>(p.q_nope);
     const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(p.q_pe);
     const __nv_bfloat16* kn = reinterpret_cast<const __nv_bfloat16*>(p.k_nope) + (int64_t)h * p.Ls_pad * 128;
-    const __nv_bfloat16* vt = reinterpret_cast<const __nv_bfloat16*>(p.v_t) + (int64_t)h * 128 * p.Ls_pad;
+    const __nv_bfloat16* vt = reinterpret_cast<const __nv_bfloat16*>(p.v_t) + (int64_t)h * 128 * p.Ls_pad;  // [Lp/64][128][64]
     const __nv_bfloat16* kr = reinterpret_cast<const __nv_bfloat16*>(p.kpe);
 
     const int r_lo = lane >> 2;  // this thread's rows within the warp's 16: r_lo and r_lo + 8
@@ -76,13 +76,13 @@ __global__ void __launch_bounds__(128) naive_attn_mma_kernel(NaiveAttn p) {
         const int t0 = tile * NA_TOK;
         for (int idx = tid; idx < NA_TOK * 24; idx += 128) {
             int row = idx / 24, ch = idx % 24;
-            const __nv_bfloat16* src = ch < 16 ? kn + (int64_t)(t0 + row) * 128 + ch * 8
+            const __nv_bfloat16* src = ch < 16 ? kn + (((int64_t)tile * 2 + (ch >> 3)) << 12) + (row << 6) + (ch & 7) * 8
                                                : kr + (int64_t)(t0 + row) * 64 + (ch - 16) * 8;
             cp_async16(smem_u32(sK + swz<24>(row, ch)), src, true);
         }
         for (int idx = tid; idx < 128 * 8; idx += 128) {
             int row = idx >> 3, ch = idx & 7;
-            cp_async16(smem_u32(sV + swz<8>(row, ch)), vt + (int64_t)row * p.Ls_pad + t0 + ch * 8, true);
+            cp_async16(smem_u32(sV + swz<8>(row, ch)), vt + ((int64_t)tile * 128 + row) * 64 + ch * 8, true);
         }
     };
 

@@ -53,7 +53,7 @@ __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(_
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
-    asm volatile("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
     return y;
 }
 

@@ -22,7 +22,7 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256
 
 struct GemmParams {
     void* C; int64_t ldc, c_batch;
-    int M, N, K;
+    int M, N, K, c_block_n, c_tile64;
     int a_batched, b_batched;
     int* status;
 };
@@ -92,13 +92,18 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
         if (ok) {
             const int lg = (warp & 3) * 32;
             const int row = m0 + lg + lane;
-            __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(p.C) + (int64_t)z * p.c_batch + (int64_t)row * p.ldc + n0;
+            __nv_bfloat16* cbase = reinterpret_cast<__nv_bfloat16*>(p.C) + (int64_t)z * p.c_batch;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)lg << 16) + c * 32, r);
                 tmem_ld_wait();
                 if (row < p.M) {
+                    const int gn = n0 + c * 32;
+                    __nv_bfloat16* crow =
+                        cbase + (p.c_tile64 ? (((int64_t)(row >> 6) * (p.N >> 6) + (gn >> 6)) << 12) + ((row & 63) << 6) + (gn & 63)
+                                 : p.c_block_n ? ((int64_t)(gn >> 6) * p.M + row) * 64 + (gn & 63)
+                                               : (int64_t)row * p.ldc + gn);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 v;
@@ -106,7 +111,7 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
                         v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]), __uint_as_float(r[j * 8 + 3]));
                         v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]), __uint_as_float(r[j * 8 + 5]));
                         v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]), __uint_as_float(r[j * 8 + 7]));
-                        *reinterpret_cast<uint4*>(crow + c * 32 + j * 8) = v;
+                        *reinterpret_cast<uint4*>(crow + j * 8) = v;
                     }
                 }
             }
@@ -146,7 +151,7 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s) {
         cudaError_t e = make_tmap_bf16(&tmB, g.B, 3, dims, strides, box);
         if (e != cudaSuccess) return e;
     }
-    GemmParams p{g.C, g.ldc, g.c_batch, g.M, g.N, g.K, g.a_batch != 0, g.b_batch != 0, status};
+    GemmParams p{g.C, g.ldc, g.c_batch, g.M, g.N, g.K, g.c_block_n, g.c_tile64 ? 1 : 0, g.a_batch != 0, g.b_batch != 0, status};
     cudaFuncSetAttribute(gemm_tn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid(g.N / BN, (g.M + BM - 1) / BM, g.batch);
     gemm_tn_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tmA, tmB, p);

@@ -109,11 +109,14 @@ __global__ void __launch_bounds__(256) gemm_tn_kernel(GemmTN g) {
             for (int j = 0; j < 4; ++j) {
                 int gn = n0 + wn * 32 + j * 8 + (lane & 3) * 2;
                 float v0 = acc[i][j][half * 2], v1 = acc[i][j][half * 2 + 1];
+                const int64_t off = g.c_tile64 ? (((int64_t)(gm >> 6) * (g.N >> 6) + (gn >> 6)) << 12) + ((gm & 63) << 6) + (gn & 63)
+                                    : g.c_block_n ? ((int64_t)(gn >> 6) * g.M + gm) * 64 + (gn & 63)
+                                                  : (int64_t)gm * g.ldc + gn;
                 if (OUT_FP32) {
-                    float* C = reinterpret_cast<float*>(g.C) + (int64_t)z * g.c_batch + (int64_t)gm * g.ldc + gn;
+                    float* C = reinterpret_cast<float*>(g.C) + (int64_t)z * g.c_batch + off;
                     *reinterpret_cast<float2*>(C) = make_float2(v0, v1);
                 } else {
-                    __nv_bfloat16* C = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)z * g.c_batch + (int64_t)gm * g.ldc + gn;
+                    __nv_bfloat16* C = reinterpret_cast<__nv_bfloat16*>(g.C) + (int64_t)z * g.c_batch + off;
                     *reinterpret_cast<uint32_t*>(C) = pack_bf16(v0, v1);
                 }
             }

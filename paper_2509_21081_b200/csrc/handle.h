@@ -9,8 +9,8 @@
 struct typhoon_mla_shared {
     typhoon_mla_dims_t dims;
     int64_t Ls, Ls_pad;
-    void* k_nope;   // bf16 [H, Ls_pad, 128]
-    void* v_t;      // bf16 [H, 128, Ls_pad]
+    void* k_nope;   // bf16 [H, Ls_pad/64, 2, 64, 64]: 64-token x 64-dim tiles, each contiguous
+    void* v_t;      // bf16 [H, Ls_pad/64, 128, 64]: V^T in contiguous 64-token blocks
     void* ckv;      // bf16 [Ls_pad, 512]
     void* kpe;      // bf16 [Ls_pad, 64]
     void* w_uk_t;   // bf16 [H, 512, 128]

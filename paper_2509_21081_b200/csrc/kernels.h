@@ -13,6 +13,12 @@ struct GemmTN {
     void* C; int64_t ldc; int64_t c_batch;
     int M, N, K, batch;
     bool out_fp32;
+    // 0: C[m][n] at m*ldc + n.  64: N is stored in blocks of 64 columns, each block a contiguous
+    // [M][64] matrix: C[m][n] at (n/64)*M*64 + m*64 + n%64 (ldc ignored).
+    int c_block_n = 0;
+    // true: C is stored as 64 x 64 tiles, tile (m/64, n/64) contiguous and row-major inside,
+    // tiles ordered by m/64 then n/64: C[m][n] at ((m/64)*(N/64) + n/64)*4096 + (m%64)*64 + n%64.
+    bool c_tile64 = false;
 };
 cudaError_t launch_gemm_tn(const GemmTN& g, cudaStream_t s);
 // tcgen05/TMEM/TMA version (bf16 output only; N % 128 == 0, K % 64 == 0).  `status` (device int,
@@ -22,7 +28,7 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s);
 // Naive shared-prefix attention partials (Algorithm 1 line 4).
 struct NaiveAttn {
     const void* q_nope; const void* q_pe;          // [B,H,128], [B,H,64]
-    const void* k_nope; const void* v_t; const void* kpe;  // [H,Lp,128], [H,128,Lp], [Lp,64]
+    const void* k_nope; const void* v_t; const void* kpe;  // [H,Lp/64,2,64,64], [H,Lp/64,128,64], [Lp,64]
     int B, H; int Ls, Ls_pad; int n_split;
     float scale;
     float* o_part;   // [n_split][B][H][128], each normalised

@@ -13,8 +13,10 @@
 // merges all partials of a (request, head).
 //
 // Warp roles (384 threads): warp 0 = TMA producer for Q and the K ring, warp 2 =
-// TMA producer for the V ring, warp 1 = MMA issuer and TMEM owner, warps 4-7 /
-// 8-11 = softmax warpgroup of stream 0 / 1 (thread = one query row).
+// TMA producer for the V ring, warp 1 = issuer of the S = Q K^T MMAs and TMEM
+// owner, warp 3 = issuer of the O += P V MMAs, warps 4-7 / 8-11 = softmax
+// warpgroup of stream 0 / 1 (thread = one query row).  Two issuing warps keep the
+// K-side and V-side barrier waits from serialising behind each other.
 //
 // Tensor memory (512 columns): S[i][buf] (64 fp32 columns, P in bf16 overwrites
 // the first 32) at (2i+buf)*64, O[i] (128 fp32 columns) at 256 + 128 i.
@@ -35,8 +37,16 @@ constexpr int K_TILE_BYTES = TOK * 192 * 2;   // 3 slabs [64][64]
 constexpr int V_TILE_BYTES = 128 * TOK * 2;   // [128 dims][64 tokens]
 constexpr int MAX_STAGES = 4;
 
+#ifdef TMLA_TRACE
+// Debug build only: clock64 stamps of CTA (0,0): [step][slot].
+__device__ long long g_trace[64 * 32];
+#define TRACE(step, slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (step) >= 0 && (step) < 64 && (threadIdx.x & 31) == 0) g_trace[(step) * 32 + (slot)] = clock64(); } while (0)
+#else
+#define TRACE(step, slot) do {} while (0)
+#endif
+
 struct NaiveSm100Params {
-    int B, H, Ls;
+    int B, H, Ls, Ls_pad;
     int n_split, m_groups, mode_y;
     int k_stages, v_stages;
     float scale_log2;
@@ -49,7 +59,7 @@ struct Barriers {
     uint64_t q_full;
     uint64_t k_full[MAX_STAGES], k_empty[MAX_STAGES];
     uint64_t v_full[MAX_STAGES], v_empty[MAX_STAGES];
-    uint64_t s_ready[2][2], p_ready[2][2], o_done[2];
+    uint64_t s_ready[2][2], p_ready[2][2], sbuf_free[2][2], o_done[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -67,7 +77,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     Barriers* bar = reinterpret_cast<Barriers*>(sV + p.v_stages * V_TILE_BYTES);
     volatile int* abort_flag = &bar->abort_flag;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE(0, 28);
     const int split = blockIdx.x / p.m_groups, mg = blockIdx.x % p.m_groups, h = blockIdx.y;
     const int row0 = mg * (p.mode_y ? 128 : 256);
 
@@ -87,6 +98,11 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         n_str[1] = (row0 + 128 < p.B) ? n_tiles : 0;   // second row tile entirely past B: skip it
     }
     const int n_steps = n_str[0];
+    // Softmax attention does not depend on the order in which KV tiles are visited.  CTAs of
+    // different heads start at different tiles and wrap around, so that the CTAs resident at any
+    // moment do not all read the same offset of their (power-of-two strided) per-head arrays.
+    const int rot = n_tiles > 0 ? (int)(((unsigned)h * 37u + (unsigned)split * 11u) % (unsigned)n_tiles) : 0;
+    auto tile_of = [&](int e) { int t = e + rot; return t_begin + (t >= n_tiles ? t - n_tiles : t); };
 
     if (threadIdx.x == 0) {
         mbar_init(&bar->q_full, 1);
@@ -100,6 +116,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             for (int b = 0; b < 2; ++b) {
                 mbar_init(&bar->s_ready[i][b], 1);
                 mbar_init(&bar->p_ready[i][b], 128);
+                mbar_init(&bar->sbuf_free[i][b], 1);
             }
             mbar_init(&bar->o_done[i], 1);
         }
@@ -111,100 +128,120 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = bar->tmem_base;
+    // broadcast through a shuffle so that the compiler knows the value is warp-uniform
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
+    if (threadIdx.x == 0) TRACE(0, 30);
 
     if (n_tiles > 0) {
         if (warp == 0) {
-            // ---------------- Q + K producer
-            if (lane == 0) {
-                const int nq = (n_str[1] > 0 && !p.mode_y) ? 2 : 1;
-                mbar_arrive_expect_tx(&bar->q_full, nq * Q_TILE_BYTES);
-                for (int t = 0; t < nq; ++t) {
-                    uint8_t* dst = sQ + t * Q_TILE_BYTES;
-                    tma_load_3d(dst, &tm_qn, &bar->q_full, 0, h, row0 + t * 128);
-                    tma_load_3d(dst + 16384, &tm_qn, &bar->q_full, 64, h, row0 + t * 128);
-                    tma_load_3d(dst + 32768, &tm_qp, &bar->q_full, 0, h, row0 + t * 128);
-                }
-                for (int e = 0; e < n_tiles; ++e) {
-                    const int s = e % p.k_stages;
-                    if (!mbar_wait(&bar->k_empty[s], ((e / p.k_stages) & 1) ^ 1, abort_flag)) break;
-                    mbar_arrive_expect_tx(&bar->k_full[s], K_TILE_BYTES);
-                    uint8_t* dst = sK + s * K_TILE_BYTES;
-                    const int tok = (t_begin + e) * TOK;
-                    tma_load_3d(dst, &tm_kn, &bar->k_full[s], 0, tok, h);
-                    tma_load_3d(dst + 8192, &tm_kn, &bar->k_full[s], 64, tok, h);
-                    tma_load_2d(dst + 16384, &tm_kp, &bar->k_full[s], 0, tok);
-                }
+            // ---------------- Q + K producer (whole warp runs the loop, the elected lane issues)
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            const int nq = (n_str[1] > 0 && !p.mode_y) ? 2 : 1;
+            mbar_arrive_expect_tx_if(ld, &bar->q_full, nq * Q_TILE_BYTES);
+            for (int t = 0; t < nq; ++t) {
+                uint8_t* dst = sQ + t * Q_TILE_BYTES;
+                tma_load_3d_if(ld, dst, &tm_qn, &bar->q_full, 0, h, row0 + t * 128);
+                tma_load_3d_if(ld, dst + 16384, &tm_qn, &bar->q_full, 64, h, row0 + t * 128);
+                tma_load_3d_if(ld, dst + 32768, &tm_qp, &bar->q_full, 0, h, row0 + t * 128);
+            }
+            for (int e = 0; e < n_tiles; ++e) {
+                const int s = e % p.k_stages;
+                if (!mbar_wait_warp(&bar->k_empty[s], ((e / p.k_stages) & 1) ^ 1, abort_flag)) break;
+                uint8_t* dst = sK + s * K_TILE_BYTES;
+                const int tok = tile_of(e) * TOK;
+                TRACE(e >> 1, 24 + (e & 1));
+                mbar_arrive_expect_tx_if(ld, &bar->k_full[s], K_TILE_BYTES);
+                tma_load_3d_if(ld, dst, &tm_kn, &bar->k_full[s], 0, 0, h * (p.Ls_pad / TOK) + tile_of(e));
+                tma_load_2d_if(ld, dst + 16384, &tm_kp, &bar->k_full[s], 0, tok);
             }
         } else if (warp == 2) {
             // ---------------- V producer
-            if (lane == 0) {
-                for (int e = 0; e < n_tiles; ++e) {
-                    const int s = e % p.v_stages;
-                    if (!mbar_wait(&bar->v_empty[s], ((e / p.v_stages) & 1) ^ 1, abort_flag)) break;
-                    mbar_arrive_expect_tx(&bar->v_full[s], V_TILE_BYTES);
-                    tma_load_3d(sV + s * V_TILE_BYTES, &tm_vt, &bar->v_full[s], (t_begin + e) * TOK, 0, h);
-                }
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            for (int e = 0; e < n_tiles; ++e) {
+                const int s = e % p.v_stages;
+                if (!mbar_wait_warp(&bar->v_empty[s], ((e / p.v_stages) & 1) ^ 1, abort_flag)) break;
+                TRACE(e >> 1, 26 + (e & 1));
+                mbar_arrive_expect_tx_if(ld, &bar->v_full[s], V_TILE_BYTES);
+                tma_load_4d_if(ld, sV + s * V_TILE_BYTES, &tm_vt, &bar->v_full[s], 0, 0, tile_of(e), h);
             }
+#ifdef TMLA_NOCOMPUTE
         } else if (warp == 1) {
-            // ---------------- MMA issuer
-            if (lane == 0) {
-                constexpr uint32_t idesc_s = idesc_bf16(128, TOK, false, false);
-                constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, false);
-                bool ok = mbar_wait(&bar->q_full, 0, abort_flag);
-                tc_fence_after();
-                // entry (ring position) of the KV tile used by stream i at step j
-                auto entry_of = [&](int j, int i) { return p.mode_y ? 2 * j + i : j; };
-                auto issue_s = [&](int j, int i) {
-                    const int e = entry_of(j, i);
+            // debug: consume the rings without any tensor-core or softmax work
+            for (int e = 0; e < n_tiles; ++e) {
+                if (!mbar_wait_warp(&bar->k_full[e % p.k_stages], (e / p.k_stages) & 1, abort_flag)) break;
+                if (lane == 0) mbar_arrive(&bar->k_empty[e % p.k_stages]);
+                if (!mbar_wait_warp(&bar->v_full[e % p.v_stages], (e / p.v_stages) & 1, abort_flag)) break;
+                if (lane == 0) mbar_arrive(&bar->v_empty[e % p.v_stages]);
+            }
+        }
+#else
+        } else if (warp == 1) {
+            // ---------------- S = Q K^T issuer (whole warp runs the loop, the elected lane issues).
+            // Runs ahead of the softmax by up to two steps (S is double-buffered per stream).
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            constexpr uint32_t idesc_s = idesc_bf16(128, TOK, false, false);
+            bool ok = mbar_wait_warp(&bar->q_full, 0, abort_flag);
+            for (int j = 0; j < n_steps && ok; ++j) {
+                TRACE(j, 0);
+                for (int i = 0; i < 2 && ok; ++i) {
+                    if (j >= n_str[i]) continue;
+                    const int e = p.mode_y ? 2 * j + i : j;      // ring position of this stream's KV tile
                     const int s = e % p.k_stages;
-                    // in mode X stream 1 reuses the tile stream 0 already waited for
-                    if (p.mode_y || i == 0) {
-                        if (!mbar_wait(&bar->k_full[s], (e / p.k_stages) & 1, abort_flag)) return false;
-                        tc_fence_after();
+                    if (p.mode_y || i == 0) {                     // mode X: stream 1 reuses stream 0's tile
+                        ok = mbar_wait_warp(&bar->k_full[s], (e / p.k_stages) & 1, abort_flag);
+                        if (!ok) break;
                     }
+                    if (j >= 2) {   // the PV product that read P from this S buffer two steps ago must be done
+                        ok = mbar_wait_warp(&bar->sbuf_free[i][j & 1], ((j >> 1) - 1) & 1, abort_flag);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    TRACE(j, 6 + i);
                     const uint32_t qa = smem_u32(sQ + (p.mode_y ? 0 : i) * Q_TILE_BYTES);
                     const uint32_t ka = smem_u32(sK + s * K_TILE_BYTES);
                     const uint32_t d = tmem_base + (uint32_t)((2 * i + (j & 1)) * 64);
+                    const bool last_user = p.mode_y || i == 1 || n_str[1] == 0;
 #pragma unroll
                     for (int slab = 0; slab < 3; ++slab) {
                         const uint64_t da = smem_desc_k_sw128(qa + slab * 16384);
                         const uint64_t db = smem_desc_k_sw128(ka + slab * 8192);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_ss(d, da + 2 * k, db + 2 * k, idesc_s, (slab | k) != 0);
+                        for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (slab | k) != 0);
                     }
-                    umma_commit(&bar->s_ready[i][j & 1]);
-                    // last user of this K tile releases the ring slot
-                    const bool last_user = p.mode_y || i == 1 || n_str[1] == 0;
-                    if (last_user) umma_commit(&bar->k_empty[s]);
-                    return true;
-                };
-                for (int i = 0; i < 2 && ok; ++i)
-                    if (n_str[i] > 0) ok = issue_s(0, i);
-                for (int j = 0; j < n_steps && ok; ++j) {
-                    for (int i = 0; i < 2 && ok; ++i)
-                        if (j + 1 < n_str[i]) ok = issue_s(j + 1, i);
-                    for (int i = 0; i < 2 && ok; ++i) {
-                        if (j >= n_str[i]) continue;
-                        const int e = entry_of(j, i);
-                        const int s = e % p.v_stages;
-                        if (p.mode_y || i == 0) {
-                            ok = mbar_wait(&bar->v_full[s], (e / p.v_stages) & 1, abort_flag);
-                            if (!ok) break;
-                        }
-                        ok = mbar_wait(&bar->p_ready[i][j & 1], (j >> 1) & 1, abort_flag);
+                    umma_commit_if(ld, &bar->s_ready[i][j & 1]);
+                    if (last_user) umma_commit_if(ld, &bar->k_empty[s]);   // last user releases the ring slot
+                }
+                TRACE(j, 1);
+            }
+        } else if (warp == 3) {
+            // ---------------- O += P V issuer
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, false);
+            bool ok = true;
+            for (int j = 0; j < n_steps && ok; ++j) {
+                for (int i = 0; i < 2 && ok; ++i) {
+                    if (j >= n_str[i]) continue;
+                    const int e = p.mode_y ? 2 * j + i : j;
+                    const int s = e % p.v_stages;
+                    if (p.mode_y || i == 0) {
+                        ok = mbar_wait_warp(&bar->v_full[s], (e / p.v_stages) & 1, abort_flag);
                         if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t va = smem_u32(sV + s * V_TILE_BYTES);
-                        const uint32_t pa = tmem_base + (uint32_t)((2 * i + (j & 1)) * 64);
-                        const uint32_t d = tmem_base + 256u + (uint32_t)i * 128u;
-                        const uint64_t db = smem_desc_k_sw128(va);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_ts(d, pa + 8 * k, db + 2 * k, idesc_o, (j | k) != 0);
-                        umma_commit(&bar->o_done[i]);
-                        const bool last_user = p.mode_y || i == 1 || n_str[1] == 0;
-                        if (last_user) umma_commit(&bar->v_empty[s]);
                     }
+                    TRACE(j, 2 + 2 * i);
+                    ok = mbar_wait_warp(&bar->p_ready[i][j & 1], (j >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    TRACE(j, 3 + 2 * i);
+                    tc_fence_after();
+                    const uint32_t va = smem_u32(sV + s * V_TILE_BYTES);
+                    const uint32_t pa = tmem_base + (uint32_t)((2 * i + (j & 1)) * 64);
+                    const uint32_t d = tmem_base + 256u + (uint32_t)i * 128u;
+                    const uint64_t db = smem_desc_k_sw128(va);
+                    const bool last_user = p.mode_y || i == 1 || n_str[1] == 0;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_ts_if(ld, d, pa + 8 * k, db + 2 * k, idesc_o, (j | k) != 0);
+                    umma_commit_if(ld, &bar->o_done[i]);
+                    umma_commit_if(ld, &bar->sbuf_free[i][j & 1]);
+                    if (last_user) umma_commit_if(ld, &bar->v_empty[s]);
                 }
             }
         } else if (warp >= 4) {
@@ -218,16 +255,19 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             bool ok = true;
             for (int j = 0; j < nt && ok; ++j) {
                 const int buf = j & 1;
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 8 + 8 * i);
                 ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_ready[i][buf], (j >> 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 9 + 8 * i);
                 const uint32_t s_addr = tmem_base + ((uint32_t)lg << 16) + (uint32_t)((2 * i + buf) * 64);
                 uint32_t sr[2][32];
                 tmem_ld32(s_addr, sr[0]);
                 tmem_ld32(s_addr + 32, sr[1]);
                 tmem_ld_wait();
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 10 + 8 * i);
                 // logits in base-2 units, ragged tail masked
-                const int tile = t_begin + (p.mode_y ? 2 * j + i : j);
+                const int tile = tile_of(p.mode_y ? 2 * j + i : j);
                 const int valid = min(TOK, p.Ls - tile * TOK);
                 float mx = -INFINITY;
 #pragma unroll
@@ -239,11 +279,13 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 }
                 // previous PV of this stream must be complete before O may be rescaled, and
                 // waiting every step keeps the barrier's phase in lockstep
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 11 + 8 * i);
                 if (j > 0) {
                     ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i], (j - 1) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                 }
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 12 + 8 * i);
                 // lazy rescale: only when some row's maximum grew by more than 2^8
                 const bool grow = mx > m_ref + 8.f;
                 if (j == 0) {
@@ -274,10 +316,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     pk[c] = w;
                     l_sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
                 }
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 13 + 8 * i);
                 tmem_st32(s_addr, pk);
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(&bar->p_ready[i][buf]);
+                if ((warp & 3) == 0 && lane == 0) TRACE(j, 14 + 8 * i);
             }
             // epilogue: normalised partial + LSE
             const int slot = p.mode_y ? split * 2 + i : split;
@@ -308,6 +352,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 p.lse_part[((int64_t)slot * p.B + b) * p.H + h] = -INFINITY;
             }
         }
+#endif
     } else if (warp >= 4) {
         // empty split: every slot this CTA owns gets weight zero in the combine
         const int i = (warp - 4) >> 2;
@@ -318,6 +363,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) TRACE(0, 29);
     if (*abort_flag) {
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, 2);
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
@@ -327,6 +373,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 }
 
 }  // namespace
+
+#ifdef TMLA_TRACE
+extern "C" int typhoon_mla_debug_read_trace(long long* dst) {
+    return (int)cudaMemcpyFromSymbol(dst, g_trace, sizeof(long long) * 64 * 32);
+}
+#endif
 
 int naive_sm100_slots(int B, int n_split) { return B <= 128 ? 2 * n_split : n_split; }
 
@@ -348,7 +400,7 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
     }
     NaiveSm100Params p{};
-    p.B = a.B; p.H = a.H; p.Ls = a.Ls;
+    p.B = a.B; p.H = a.H; p.Ls = a.Ls; p.Ls_pad = (a.Ls + 127) / 128 * 128;
     p.n_split = a.n_split;
     p.mode_y = a.B <= 128 ? 1 : 0;
     p.m_groups = p.mode_y ? 1 : (a.B + 255) / 256;
@@ -367,9 +419,10 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
 cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const void* v_t, int H, int64_t Ls_pad,
                                    CUtensorMap* tm_kn, CUtensorMap* tm_kp, CUtensorMap* tm_vt) {
     {
-        uint64_t dims[3] = {128, (uint64_t)Ls_pad, (uint64_t)H};
-        uint64_t str[2] = {128 * 2, (uint64_t)Ls_pad * 128 * 2};
-        uint32_t box[3] = {64, TOK, 1};
+        // K_nope is stored as contiguous 16 KB tiles: [H * Ls_pad/64][2 slabs * 64 tokens][64 dims]
+        uint64_t dims[3] = {64, 2 * TOK, (uint64_t)H * (uint64_t)(Ls_pad / TOK)};
+        uint64_t str[2] = {64 * 2, 2 * TOK * 64 * 2};
+        uint32_t box[3] = {64, 2 * TOK, 1};
         cudaError_t e = make_tmap_bf16(tm_kn, k_nope, 3, dims, str, box);
         if (e != cudaSuccess) return e;
     }
@@ -381,10 +434,11 @@ cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const vo
         if (e != cudaSuccess) return e;
     }
     {
-        uint64_t dims[3] = {(uint64_t)Ls_pad, 128, (uint64_t)H};
-        uint64_t str[2] = {(uint64_t)Ls_pad * 2, (uint64_t)Ls_pad * 128 * 2};
-        uint32_t box[3] = {TOK, 128, 1};
-        cudaError_t e = make_tmap_bf16(tm_vt, v_t, 3, dims, str, box);
+        // V^T is stored in 64-token blocks, each a contiguous [128 dims][64 tokens] matrix
+        uint64_t dims[4] = {TOK, 128, (uint64_t)(Ls_pad / TOK), (uint64_t)H};
+        uint64_t str[3] = {TOK * 2, 128 * TOK * 2, (uint64_t)Ls_pad * 128 * 2};
+        uint32_t box[4] = {TOK, 128, 1, 1};
+        cudaError_t e = make_tmap_bf16(tm_vt, v_t, 4, dims, str, box);
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;

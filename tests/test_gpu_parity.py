@@ -189,7 +189,7 @@ def test_expansion_matches_plain_matmul():
     Ls, Lp, owned = b.typhoon_mla_shared_view(sh)
     torch.cuda.synchronize()
     assert (Ls, Lp) == (333, 384) and owned >= 2 * cfg.H * Lp * 128 * 2
-    k = k.float().cpu().double().numpy(); v = vt.float().cpu().double().numpy().transpose(0, 2, 1)
+    k = k.float().cpu().double().numpy().transpose(0, 1, 3, 2, 4).reshape(cfg.H, Lp, 128); v = vt.float().cpu().double().numpy().transpose(0, 1, 3, 2).reshape(cfg.H, Lp, 128)
     sh.free()
     kr = O.expand_shared(I.to_f64(inp.ckv_shared), I.to_f64(inp.w_uk))
     vr = O.expand_shared(I.to_f64(inp.ckv_shared), I.to_f64(inp.w_uv))
