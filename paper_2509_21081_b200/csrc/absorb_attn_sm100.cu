@@ -1,0 +1,447 @@
+// Absorb attention over latent tokens (Algorithm 1 line 6) on tcgen05 / TMEM / TMA.
+//
+// Work item (CTA) = (request b, group of 64 heads, KV chunk).  The problem is run
+// transposed so that the 64 x 512 latent accumulator fits tensor memory:
+//     S^T [64 tokens, 64 heads] = KV_tile [64, 576] * Q_g^T [576, 64]
+//     O^T [512 latent, 64 heads] += C_tile^T [512, 64 tokens] * P^T [64 tokens, 64 heads]
+// with KV_tile = [latent 512 | rope 64] of one 64-token tile of the (paged) cache and
+// Q_g = [Q_A | q_pe] of the head group.  The latent part of the tile is used twice
+// from shared memory: K-major as the A operand of S^T, MN-major (transposed view)
+// as the A operand of O^T.  P^T (bf16) is written by the softmax threads into the
+// tile's rope slab, which is dead once S^T has been computed.
+//
+// Softmax runs over tokens, i.e. across TMEM lanes.  To avoid a cross-lane
+// reduction per tile, every head column keeps a reference exponent m_ref that is
+// only raised when some logit exceeds it by more than 2^8 (a rare, collective
+// "rescale" event that also rescales O^T); row sums are accumulated per thread
+// and reduced across lanes once, at the end of the chunk.
+//
+// Warp roles (384 threads): warp 0 = TMA producer (Q once, KV ring), warp 1 =
+// S^T issuer and TMEM owner, warp 3 = O^T issuer, warps 4-7 / 8-11 = softmax
+// warpgroup for head columns 0-31 / 32-63.  S^T uses M = 64: token row r lives in
+// TMEM lane 32 (r / 16) + r % 16, so lanes 0-15 of every softmax warp own a token.
+//
+// Tensor memory (512 columns allocated): S^T[buf] at 64 buf (2 buffers), O^T block
+// m (128 latent rows x 64 heads) at 128 + 64 m.
+#include "kernels.h"
+#include "sm100.cuh"
+
+namespace tmla {
+namespace {
+
+using namespace sm100;
+
+constexpr int TOK = 64;
+constexpr int SLAB_BYTES = 64 * 64 * 2;          // [64 rows][64 bf16], 128-byte swizzled rows
+constexpr int TILE_BYTES = 9 * SLAB_BYTES;       // 8 latent slabs + 1 rope slab = 72 KB
+constexpr int STAGES = 2;
+constexpr float kRescaleThreshold = 8.f;         // log2 units
+
+struct AbsorbSm100Params {
+    int B, H;
+    int chunk, n_shared_chunks, n_suffix_chunks;
+    int Ls_absorb;
+    int page_size, max_pages;
+    const int32_t* block_table;
+    const int32_t* seq_lens;
+    float scale_log2;
+    float* o_part;     // [n_chunks][B][H][512]
+    float* lse_part;   // [n_chunks][B][H]
+    int* status;
+};
+
+struct Shared {
+    uint64_t q_full;
+    uint64_t kv_full[STAGES], kv_empty[STAGES];
+    uint64_t s_ready[2], p_ready[2], o_done;
+    uint32_t tmem_base;
+    int abort_flag;
+    float red[2][4][32];   // [warpgroup][warp][column]: cross-warp reductions
+};
+
+__device__ __forceinline__ bool wg_vote_or(int bar_id, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\nsetp.ne.b32 q, %2, 0;\n"
+        "bar.red.or.pred p, %1, 128, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(r) : "r"(bar_id), "r"(pred ? 1u : 0u) : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ void wg_sync(int bar_id) { asm volatile("bar.sync %0, 128;\n" ::"r"(bar_id) : "memory"); }
+
+__global__ void __launch_bounds__(384, 1)
+absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ CUtensorMap tm_qp,
+                         const __grid_constant__ CUtensorMap tm_ckv_sh, const __grid_constant__ CUtensorMap tm_kpe_sh,
+                         const __grid_constant__ CUtensorMap tm_ckv_pg, const __grid_constant__ CUtensorMap tm_kpe_pg,
+                         AbsorbSm100Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sKV = smem;                                  // STAGES tiles
+    uint8_t* sQ = smem + STAGES * TILE_BYTES;             // 9 slabs [64 heads][64]
+    Shared* sh = reinterpret_cast<Shared*>(sQ + TILE_BYTES);
+    volatile int* abort_flag = &sh->abort_flag;
+
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
+    const int chunk = blockIdx.x, h0 = blockIdx.y * 64, b = blockIdx.z;
+
+    // token range of this chunk
+    const bool shared_seg = chunk < p.n_shared_chunks;
+    int seg_len, tok_begin;
+    if (shared_seg) {
+        seg_len = p.Ls_absorb;
+        tok_begin = chunk * p.chunk;
+    } else {
+        seg_len = min(max(p.seq_lens[b], 0), p.max_pages * p.page_size);
+        tok_begin = (chunk - p.n_shared_chunks) * p.chunk;
+    }
+    const int tok_end = min(seg_len, tok_begin + p.chunk);
+    const int n_tiles = tok_end > tok_begin ? (tok_end - tok_begin + TOK - 1) / TOK : 0;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sh->q_full, 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&sh->kv_full[s], 1);
+            mbar_init(&sh->kv_empty[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sh->s_ready[i], 1);
+            mbar_init(&sh->p_ready[i], 256);
+        }
+        mbar_init(&sh->o_done, 1);
+        sh->abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tmap(&tm_qa); prefetch_tmap(&tm_qp);
+        prefetch_tmap(shared_seg ? &tm_ckv_sh : &tm_ckv_pg);
+        prefetch_tmap(shared_seg ? &tm_kpe_sh : &tm_kpe_pg);
+    }
+    if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, sh->tmem_base, 0);
+
+    if (n_tiles > 0) {
+        if (warp == 0) {
+            // ---------------- producer: Q once, then the KV ring
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            mbar_arrive_expect_tx_if(ld, &sh->q_full, TILE_BYTES);
+#pragma unroll 1
+            for (int s = 0; s < 8; ++s) tma_load_3d_if(ld, sQ + s * SLAB_BYTES, &tm_qa, &sh->q_full, s * 64, h0, b);
+            tma_load_3d_if(ld, sQ + 8 * SLAB_BYTES, &tm_qp, &sh->q_full, 0, h0, b);
+            const CUtensorMap* tc = shared_seg ? &tm_ckv_sh : &tm_ckv_pg;
+            const CUtensorMap* tk = shared_seg ? &tm_kpe_sh : &tm_kpe_pg;
+            const int32_t* bt = p.block_table + (int64_t)b * p.max_pages;
+            for (int j = 0; j < n_tiles; ++j) {
+                const int s = j & 1;
+                if (!mbar_wait_warp(&sh->kv_empty[s], ((j >> 1) & 1) ^ 1, abort_flag)) break;
+                const int t0 = tok_begin + j * TOK;
+                int page, slot;
+                if (shared_seg) {
+                    page = t0 / TOK;
+                    slot = 0;
+                } else {
+                    page = __shfl_sync(0xffffffffu, bt[t0 / p.page_size], 0);
+                    slot = t0 % p.page_size;
+                }
+                uint8_t* dst = sKV + s * TILE_BYTES;
+                mbar_arrive_expect_tx_if(ld, &sh->kv_full[s], TILE_BYTES);
+#pragma unroll 1
+                for (int sl = 0; sl < 8; ++sl) tma_load_3d_if(ld, dst + sl * SLAB_BYTES, tc, &sh->kv_full[s], sl * 64, slot, page);
+                tma_load_3d_if(ld, dst + 8 * SLAB_BYTES, tk, &sh->kv_full[s], 0, slot, page);
+            }
+        } else if (warp == 1) {
+            // ---------------- S^T = KV_tile * Q^T issuer (M = 64 tokens, N = 64 heads, K = 576)
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            constexpr uint32_t idesc_s = idesc_bf16(64, 64, false, false);
+            bool ok = mbar_wait_warp(&sh->q_full, 0, abort_flag);
+            const uint32_t qa = smem_u32(sQ);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int s = j & 1;
+                ok = mbar_wait_warp(&sh->kv_full[s], (j >> 1) & 1, abort_flag);
+                if (!ok) break;
+                if (j >= 2) {   // the softmax of tile j-2 has finished reading this S^T buffer
+                    ok = mbar_wait_warp(&sh->p_ready[s], ((j >> 1) - 1) & 1, abort_flag);
+                    if (!ok) break;
+                }
+                tc_fence_after();
+                const uint32_t ka = smem_u32(sKV + s * TILE_BYTES);
+                const uint32_t d = tmem_base + (uint32_t)(s * 64);
+#pragma unroll
+                for (int sl = 0; sl < 9; ++sl) {
+                    const uint64_t da = smem_desc_k_sw128(ka + sl * SLAB_BYTES);
+                    const uint64_t db = smem_desc_k_sw128(qa + sl * SLAB_BYTES);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (sl | k) != 0);
+                }
+                umma_commit_if(ld, &sh->s_ready[s]);
+            }
+        } else if (warp == 3) {
+            // ---------------- O^T += C^T * P^T issuer (4 blocks of M = 128 latent rows, N = 64 heads, K = 64 tokens)
+            const uint32_t ld = elect_one() ? 1u : 0u;
+            constexpr uint32_t idesc_o = idesc_bf16(128, 64, true, true);
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int s = j & 1;
+                ok = mbar_wait_warp(&sh->p_ready[s], (j >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t ca = smem_u32(sKV + s * TILE_BYTES);
+                const uint32_t pa = ca + 8 * SLAB_BYTES;     // P^T lives in the rope slab
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    const uint32_t d = tmem_base + 128u + (uint32_t)m * 64u;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t da = smem_desc_mn_sw128(ca + (2 * m) * SLAB_BYTES + k * 2048, SLAB_BYTES, 1024);
+                        const uint64_t db = smem_desc_mn_sw128(pa + k * 2048, SLAB_BYTES, 1024);
+                        umma_ss_if(ld, d, da, db, idesc_o, (j | k) != 0);
+                    }
+                }
+                umma_commit_if(ld, &sh->o_done);
+                umma_commit_if(ld, &sh->kv_empty[s]);
+            }
+        } else if (warp >= 4) {
+            // ---------------- softmax warpgroups
+            const int cg = (warp - 4) >> 2;                 // column group: heads h0 + 32 cg .. + 31
+            const int q = warp & 3;                         // TMEM lane quadrant of this warp
+            const int bar_id = 1 + cg;
+            const bool has_token = lane < 16;               // M = 64 layout: 16 token rows per quadrant
+            const int r = 16 * q + lane;                    // token row within the tile (valid when has_token)
+            const uint32_t lane_base = (uint32_t)(32 * q) << 16;
+            float m_ref[32], l_part[32];
+#pragma unroll
+            for (int c = 0; c < 32; ++c) { m_ref[c] = -INFINITY; l_part[c] = 0.f; }
+
+            for (int j = 0; j < n_tiles; ++j) {
+                const int s = j & 1;
+                bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->s_ready[s], (j >> 1) & 1, abort_flag));
+                const int t0 = tok_begin + j * TOK;
+                const int n_valid = min(TOK, tok_end - t0);
+                const bool valid = has_token && r < n_valid;
+                uint32_t sr[32];
+                bool exceed = false;
+                if (ok) {
+                    tc_fence_after();
+                    tmem_ld32(tmem_base + lane_base + (uint32_t)(s * 64 + cg * 32), sr);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float v = valid ? __uint_as_float(sr[c]) * p.scale_log2 : -INFINITY;
+                        sr[c] = __float_as_uint(v);
+                        exceed |= v > m_ref[c] + kRescaleThreshold;
+                    }
+                    if (j > 0) {   // O^T of the previous tile complete (needed by a rescale; keeps the phase in step)
+                        ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done, (j - 1) & 1, abort_flag));
+                        tc_fence_after();
+                    }
+                }
+                const bool rescale = wg_vote_or(bar_id, exceed);
+                if (*abort_flag) break;                      // uniform across the warpgroup after the barrier
+                if (rescale) {
+                    // exact column maxima of this tile across the 64 token lanes
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        float v = __uint_as_float(sr[c]);
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 8));
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 4));
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+                        if (lane == c) sh->red[cg][q][c] = v;
+                    }
+                    wg_sync(bar_id);
+                    float f[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float cm = fmaxf(fmaxf(sh->red[cg][0][c], sh->red[cg][1][c]), fmaxf(sh->red[cg][2][c], sh->red[cg][3][c]));
+                        const float m_new = fmaxf(m_ref[c], cm);
+                        f[c] = (m_new == -INFINITY) ? 1.f : fast_exp2(m_ref[c] - m_new);
+                        m_ref[c] = m_new;
+                        l_part[c] *= f[c];
+                    }
+                    wg_sync(bar_id);                         // red[] may be reused by the next event
+                    if (j > 0) {
+                        // rescale this column group's 32 columns of all four O^T blocks (all 128 lanes)
+#pragma unroll 1
+                        for (int m = 0; m < 4; ++m) {
+                            uint32_t orr[32];
+                            const uint32_t o_addr = tmem_base + lane_base + 128u + (uint32_t)(m * 64 + cg * 32);
+                            tmem_ld32(o_addr, orr);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * f[c]);
+                            tmem_st32(o_addr, orr);
+                        }
+                        tmem_st_wait();
+                    }
+                }
+                // probabilities (bf16), per-thread partial row sums, P^T row into the rope slab
+                uint8_t* tile = sKV + s * TILE_BYTES;
+                if (has_token) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float p0 = valid ? fast_exp2(__uint_as_float(sr[2 * c]) - m_ref[2 * c]) : 0.f;
+                        const float p1 = valid ? fast_exp2(__uint_as_float(sr[2 * c + 1]) - m_ref[2 * c + 1]) : 0.f;
+                        const uint32_t w = pack_bf16(p0, p1);
+                        pk[c] = w;
+                        l_part[2 * c] += __uint_as_float(w << 16);
+                        l_part[2 * c + 1] += __uint_as_float(w & 0xffff0000u);
+                    }
+                    // MN-major P^T: row r (token) = 64 heads = 128 bytes, 16-byte chunks swizzled by r & 7
+                    uint8_t* prow = tile + 8 * SLAB_BYTES + r * 128;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int ch = (cg * 4 + i) ^ (r & 7);
+                        *reinterpret_cast<uint4*>(prow + ch * 16) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+                    }
+                }
+                if (n_valid < TOK) {
+                    // ragged tail: latent rows of tokens past the end may hold anything (even NaN);
+                    // zero them so that 0 * garbage cannot reach the accumulator
+                    const int tid_sm = threadIdx.x - 128;
+                    const int n_chunks16 = (TOK - n_valid) * 64;             // 8 slabs x 8 chunks per row
+                    for (int idx = tid_sm; idx < n_chunks16; idx += 256) {
+                        const int row = n_valid + idx / 64, rem = idx % 64;
+                        *reinterpret_cast<uint4*>(tile + (rem >> 3) * SLAB_BYTES + row * 128 + (rem & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                fence_proxy_async();
+                tc_fence_before();
+                mbar_arrive(&sh->p_ready[s]);
+            }
+
+            // ---------------- epilogue: row sums across lanes, normalised partial, LSE
+            // (the decision to run it is taken by a warpgroup vote so that every thread of the
+            // warpgroup reaches the same named barriers)
+            if (!wg_vote_or(bar_id, *abort_flag != 0)) {
+                bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done, (n_tiles - 1) & 1, abort_flag));
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    float v = l_part[c];
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    if (lane == c) sh->red[cg][q][c] = v;
+                }
+                wg_sync(bar_id);
+                if (ok && !*abort_flag) {
+                    float inv[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float l = sh->red[cg][0][c] + sh->red[cg][1][c] + sh->red[cg][2][c] + sh->red[cg][3][c];
+                        inv[c] = 1.f / l;
+                        if (q == 0 && lane == c) {
+                            const int h = h0 + cg * 32 + c;
+                            if (h < p.H) p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = (m_ref[c] + log2f(l)) * kLn2;
+                        }
+                    }
+                    const int64_t row_base = ((int64_t)chunk * p.B + b) * p.H;
+#pragma unroll 1
+                    for (int m = 0; m < 4; ++m) {
+                        uint32_t orr[32];
+                        tmem_ld32(tmem_base + lane_base + 128u + (uint32_t)(m * 64 + cg * 32), orr);
+                        tmem_ld_wait();
+                        const int lat = m * 128 + 32 * q + lane;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const int h = h0 + cg * 32 + c;
+                            if (h < p.H) p.o_part[(row_base + h) * 512 + lat] = __uint_as_float(orr[c]) * inv[c];
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp >= 4) {
+        // empty chunk: weight zero in the merge
+        const int i = threadIdx.x - 128;
+        if (i < 64 && h0 + i < p.H) p.lse_part[((int64_t)chunk * p.B + b) * p.H + h0 + i] = -INFINITY;
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 3);
+        for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
+        __syncthreads();
+    }
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+cudaError_t make_kv_tmaps(const void* ckv, const void* kpe, int64_t ckv_stride, int64_t kpe_stride, int page_size,
+                          uint64_t n_pages, CUtensorMap* tm_ckv, CUtensorMap* tm_kpe) {
+    {
+        uint64_t dims[3] = {512, (uint64_t)page_size, n_pages};
+        uint64_t str[2] = {(uint64_t)ckv_stride * 2, (uint64_t)page_size * ckv_stride * 2};
+        uint32_t box[3] = {64, TOK, 1};
+        cudaError_t e = make_tmap_bf16(tm_ckv, ckv, 3, dims, str, box);
+        if (e != cudaSuccess) return e;
+    }
+    {
+        uint64_t dims[3] = {64, (uint64_t)page_size, n_pages};
+        uint64_t str[2] = {(uint64_t)kpe_stride * 2, (uint64_t)page_size * kpe_stride * 2};
+        uint32_t box[3] = {64, TOK, 1};
+        cudaError_t e = make_tmap_bf16(tm_kpe, kpe, 3, dims, str, box);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t Ls_pad, CUtensorMap* tm_ckv,
+                                     CUtensorMap* tm_kpe) {
+    return make_kv_tmaps(ckv, kpe, 512, 64, TOK, (uint64_t)(Ls_pad / TOK), tm_ckv, tm_kpe);
+}
+
+cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_ckv_sh, const CUtensorMap* tm_kpe_sh,
+                                     int* status, cudaStream_t s) {
+    const int n_chunks = a.n_shared_chunks + a.n_suffix_chunks;
+    if (a.B <= 0 || n_chunks <= 0) return cudaSuccess;
+    if (a.chunk % TOK != 0) return cudaErrorInvalidValue;
+    CUtensorMap tm_qa, tm_qp, tm_ckv_pg, tm_kpe_pg;
+    {
+        uint64_t dims[3] = {512, (uint64_t)a.H, (uint64_t)a.B};
+        uint64_t str[2] = {512 * 2, (uint64_t)a.H * 512 * 2};
+        uint32_t box[3] = {64, 64, 1};
+        cudaError_t e = make_tmap_bf16(&tm_qa, a.q_abs, 3, dims, str, box);
+        if (e != cudaSuccess) return e;
+    }
+    {
+        uint64_t dims[3] = {64, (uint64_t)a.H, (uint64_t)a.B};
+        uint64_t str[2] = {64 * 2, (uint64_t)a.H * 64 * 2};
+        uint32_t box[3] = {64, 64, 1};
+        cudaError_t e = make_tmap_bf16(&tm_qp, a.q_pe, 3, dims, str, box);
+        if (e != cudaSuccess) return e;
+    }
+    if (a.n_suffix_chunks > 0) {
+        // the number of physical pages is not part of the interface: the caller's block table is trusted
+        cudaError_t e = make_kv_tmaps(a.ckv_pages, a.kpe_pages, a.ckv_stride, a.kpe_stride, a.page_size,
+                                      (uint64_t)1 << 24, &tm_ckv_pg, &tm_kpe_pg);
+        if (e != cudaSuccess) return e;
+    } else {
+        tm_ckv_pg = *tm_ckv_sh;
+        tm_kpe_pg = *tm_kpe_sh;
+    }
+    AbsorbSm100Params p{};
+    p.B = a.B; p.H = a.H;
+    p.chunk = a.chunk; p.n_shared_chunks = a.n_shared_chunks; p.n_suffix_chunks = a.n_suffix_chunks;
+    p.Ls_absorb = a.Ls_absorb;
+    p.page_size = a.page_size; p.max_pages = a.max_pages;
+    p.block_table = a.block_table; p.seq_lens = a.seq_lens;
+    p.scale_log2 = a.scale * kLog2e;
+    p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = status;
+    const int smem = (STAGES + 1) * TILE_BYTES + 1024 + (int)sizeof(Shared) + 64;
+    cudaFuncSetAttribute(absorb_attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    dim3 grid(n_chunks, (a.H + 63) / 64, a.B);
+    const CUtensorMap* sh_c = a.n_shared_chunks > 0 ? tm_ckv_sh : &tm_ckv_pg;
+    const CUtensorMap* sh_k = a.n_shared_chunks > 0 ? tm_kpe_sh : &tm_kpe_pg;
+    absorb_attn_sm100_kernel<<<grid, 384, smem, s>>>(tm_qa, tm_qp, *sh_c, *sh_k, tm_ckv_pg, tm_kpe_pg, p);
+    return cudaGetLastError();
+}
+
+}  // namespace tmla

@@ -319,6 +319,7 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
     }
     if (e == cudaSuccess && Ls > 0)
         e = make_naive_sm100_tmaps(sh->k_nope, sh->kpe, sh->v_t, H, sh->Ls_pad, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt);
+    if (e == cudaSuccess && Ls > 0) e = make_absorb_shared_tmaps(sh->ckv, sh->kpe, sh->Ls_pad, &sh->tm_ckv, &sh->tm_kpe_tok);
     if (e != cudaSuccess) {
         typhoon_mla_free(sh);
         return cuda_fail(e);
@@ -450,7 +451,9 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
                       seq_lens, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
                       o_part_a, lse_part_a};
         prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
-        e = launch_absorb_attn_mma(ab, s);
+        e = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05
+                ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, sh->status, s)
+                : launch_absorb_attn_mma(ab, s);
         prof_after(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;

@@ -67,6 +67,13 @@ struct AbsorbAttn {
 };
 cudaError_t launch_absorb_attn_mma(const AbsorbAttn& p, cudaStream_t s);
 
+// tcgen05/TMEM/TMA version (chunk must be a multiple of 64).  The tensor maps of the handle's copy of the
+// shared latent cache come from make_absorb_shared_tmaps (used when n_shared_chunks > 0).
+cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_ckv_sh, const CUtensorMap* tm_kpe_sh,
+                                     int* status, cudaStream_t s);
+cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t Ls_pad, CUtensorMap* tm_ckv,
+                                     CUtensorMap* tm_kpe);
+
 // Merge absorb chunk partials -> bf16 latent output [B,H,512] + lse [B,H].
 cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,
                                 void* o_lat_bf16, float* lse, cudaStream_t s);
