@@ -37,6 +37,13 @@ constexpr int TILE_BYTES = 9 * SLAB_BYTES;       // 8 latent slabs + 1 rope slab
 constexpr int STAGES = 2;
 constexpr float kRescaleThreshold = 8.f;         // log2 units
 
+#ifdef TMLA_TRACE
+__device__ long long g_trace_ab[64 * 32];
+#define TRACE(step, slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (step) >= 0 && (step) < 64 && (threadIdx.x & 31) == 0) g_trace_ab[(step) * 32 + (slot)] = clock64(); } while (0)
+#else
+#define TRACE(step, slot) do {} while (0)
+#endif
+
 struct AbsorbSm100Params {
     int B, H;
     int chunk, n_shared_chunks, n_suffix_chunks;
@@ -57,6 +64,7 @@ struct Shared {
     uint32_t tmem_base;
     int abort_flag;
     float red[2][4][32];   // [warpgroup][warp][column]: cross-warp reductions
+    float mref[2][32];     // [warpgroup][column]: reference exponent (log2 units) of each head column
 };
 
 __device__ __forceinline__ bool wg_vote_or(int bar_id, bool pred) {
@@ -83,6 +91,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     volatile int* abort_flag = &sh->abort_flag;
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE(0, 28);
     const int chunk = blockIdx.x, h0 = blockIdx.y * 64, b = blockIdx.z;
 
     // token range of this chunk
@@ -98,22 +107,53 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     const int tok_end = min(seg_len, tok_begin + p.chunk);
     const int n_tiles = tok_end > tok_begin ? (tok_end - tok_begin + TOK - 1) / TOK : 0;
 
-    if (threadIdx.x == 0) {
-        mbar_init(&sh->q_full, 1);
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&sh->kv_full[s], 1);
-            mbar_init(&sh->kv_empty[s], 1);
+    // Warp 0 initialises the barriers and at once issues the Q load and the first tiles, so that the
+    // first copies are in flight while the rest of the CTA sets up (tensor-memory allocation, barrier).
+    const CUtensorMap* tc = shared_seg ? &tm_ckv_sh : &tm_ckv_pg;
+    const CUtensorMap* tk = shared_seg ? &tm_kpe_sh : &tm_kpe_pg;
+    const int32_t* bt = p.block_table + (int64_t)b * p.max_pages;
+    const uint32_t ld0 = (warp == 0 && elect_one()) ? 1u : 0u;
+    auto issue_tile = [&](int j) {
+        const int s = j & 1;
+        const int t0 = tok_begin + j * TOK;
+        int page, slot;
+        if (shared_seg) {
+            page = t0 / TOK;
+            slot = 0;
+        } else {
+            page = __shfl_sync(0xffffffffu, bt[t0 / p.page_size], 0);
+            slot = t0 % p.page_size;
         }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(&sh->s_ready[i], 1);
-            mbar_init(&sh->p_ready[i], 256);
+        uint8_t* dst = sKV + s * TILE_BYTES;
+        TRACE(j, 0);
+        mbar_arrive_expect_tx_if(ld0, &sh->kv_full[s], TILE_BYTES);
+#pragma unroll 1
+        for (int sl = 0; sl < 8; ++sl) tma_load_3d_if(ld0, dst + sl * SLAB_BYTES, tc, &sh->kv_full[s], sl * 64, slot, page);
+        tma_load_3d_if(ld0, dst + 8 * SLAB_BYTES, tk, &sh->kv_full[s], 0, slot, page);
+    };
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_init(&sh->q_full, 1);
+            for (int s = 0; s < STAGES; ++s) {
+                mbar_init(&sh->kv_full[s], 1);
+                mbar_init(&sh->kv_empty[s], 1);
+            }
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(&sh->s_ready[i], 1);
+                mbar_init(&sh->p_ready[i], 256);
+            }
+            mbar_init(&sh->o_done, 1);
+            sh->abort_flag = 0;
+            fence_mbar_init();
         }
-        mbar_init(&sh->o_done, 1);
-        sh->abort_flag = 0;
-        fence_mbar_init();
-        prefetch_tmap(&tm_qa); prefetch_tmap(&tm_qp);
-        prefetch_tmap(shared_seg ? &tm_ckv_sh : &tm_ckv_pg);
-        prefetch_tmap(shared_seg ? &tm_kpe_sh : &tm_kpe_pg);
+        __syncwarp();
+        if (n_tiles > 0) {
+            mbar_arrive_expect_tx_if(ld0, &sh->q_full, TILE_BYTES);
+#pragma unroll 1
+            for (int s = 0; s < 8; ++s) tma_load_3d_if(ld0, sQ + s * SLAB_BYTES, &tm_qa, &sh->q_full, s * 64, h0, b);
+            tma_load_3d_if(ld0, sQ + 8 * SLAB_BYTES, &tm_qp, &sh->q_full, 0, h0, b);
+            for (int j = 0; j < min(n_tiles, STAGES); ++j) issue_tile(j);
+        }
     }
     if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
     tc_fence_before();
@@ -123,32 +163,10 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 
     if (n_tiles > 0) {
         if (warp == 0) {
-            // ---------------- producer: Q once, then the KV ring
-            const uint32_t ld = elect_one() ? 1u : 0u;
-            mbar_arrive_expect_tx_if(ld, &sh->q_full, TILE_BYTES);
-#pragma unroll 1
-            for (int s = 0; s < 8; ++s) tma_load_3d_if(ld, sQ + s * SLAB_BYTES, &tm_qa, &sh->q_full, s * 64, h0, b);
-            tma_load_3d_if(ld, sQ + 8 * SLAB_BYTES, &tm_qp, &sh->q_full, 0, h0, b);
-            const CUtensorMap* tc = shared_seg ? &tm_ckv_sh : &tm_ckv_pg;
-            const CUtensorMap* tk = shared_seg ? &tm_kpe_sh : &tm_kpe_pg;
-            const int32_t* bt = p.block_table + (int64_t)b * p.max_pages;
-            for (int j = 0; j < n_tiles; ++j) {
-                const int s = j & 1;
-                if (!mbar_wait_warp(&sh->kv_empty[s], ((j >> 1) & 1) ^ 1, abort_flag)) break;
-                const int t0 = tok_begin + j * TOK;
-                int page, slot;
-                if (shared_seg) {
-                    page = t0 / TOK;
-                    slot = 0;
-                } else {
-                    page = __shfl_sync(0xffffffffu, bt[t0 / p.page_size], 0);
-                    slot = t0 % p.page_size;
-                }
-                uint8_t* dst = sKV + s * TILE_BYTES;
-                mbar_arrive_expect_tx_if(ld, &sh->kv_full[s], TILE_BYTES);
-#pragma unroll 1
-                for (int sl = 0; sl < 8; ++sl) tma_load_3d_if(ld, dst + sl * SLAB_BYTES, tc, &sh->kv_full[s], sl * 64, slot, page);
-                tma_load_3d_if(ld, dst + 8 * SLAB_BYTES, tk, &sh->kv_full[s], 0, slot, page);
+            // ---------------- producer: the rest of the KV ring (Q and the first tiles are already in flight)
+            for (int j = STAGES; j < n_tiles; ++j) {
+                if (!mbar_wait_warp(&sh->kv_empty[j & 1], ((j >> 1) & 1) ^ 1, abort_flag)) break;
+                issue_tile(j);
             }
         } else if (warp == 1) {
             // ---------------- S^T = KV_tile * Q^T issuer (M = 64 tokens, N = 64 heads, K = 576)
@@ -160,6 +178,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 const int s = j & 1;
                 ok = mbar_wait_warp(&sh->kv_full[s], (j >> 1) & 1, abort_flag);
                 if (!ok) break;
+                TRACE(j, 1);
                 if (j >= 2) {   // the softmax of tile j-2 has finished reading this S^T buffer
                     ok = mbar_wait_warp(&sh->p_ready[s], ((j >> 1) - 1) & 1, abort_flag);
                     if (!ok) break;
@@ -175,6 +194,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (sl | k) != 0);
                 }
                 umma_commit_if(ld, &sh->s_ready[s]);
+                TRACE(j, 2);
             }
         } else if (warp == 3) {
             // ---------------- O^T += C^T * P^T issuer (4 blocks of M = 128 latent rows, N = 64 heads, K = 64 tokens)
@@ -185,6 +205,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 const int s = j & 1;
                 ok = mbar_wait_warp(&sh->p_ready[s], (j >> 1) & 1, abort_flag);
                 if (!ok) break;
+                TRACE(j, 3);
                 tc_fence_after();
                 const uint32_t ca = smem_u32(sKV + s * TILE_BYTES);
                 const uint32_t pa = ca + 8 * SLAB_BYTES;     // P^T lives in the rope slab
@@ -200,6 +221,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 }
                 umma_commit_if(ld, &sh->o_done);
                 umma_commit_if(ld, &sh->kv_empty[s]);
+                TRACE(j, 4);
             }
         } else if (warp >= 4) {
             // ---------------- softmax warpgroups
@@ -209,60 +231,71 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             const bool has_token = lane < 16;               // M = 64 layout: 16 token rows per quadrant
             const int r = 16 * q + lane;                    // token row within the tile (valid when has_token)
             const uint32_t lane_base = (uint32_t)(32 * q) << 16;
-            float m_ref[32], l_part[32];
+            // Per-thread state: partial row sums of this thread's token slot.  The reference exponents
+            // are the same for every thread of the warpgroup and live in shared memory.
+            float l_part[32];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) { m_ref[c] = -INFINITY; l_part[c] = 0.f; }
+            for (int c = 0; c < 32; ++c) l_part[c] = 0.f;
+            volatile float* mref = sh->mref[cg];
+            if (q == 0) mref[lane] = -INFINITY;
+            wg_sync(bar_id);
 
             for (int j = 0; j < n_tiles; ++j) {
                 const int s = j & 1;
                 bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->s_ready[s], (j >> 1) & 1, abort_flag));
+                if (warp == 4) TRACE(j, 8);
                 const int t0 = tok_begin + j * TOK;
                 const int n_valid = min(TOK, tok_end - t0);
                 const bool valid = has_token && r < n_valid;
-                uint32_t sr[32];
+                uint32_t sr[32], pk[16];
                 bool exceed = false;
                 if (ok) {
                     tc_fence_after();
                     tmem_ld32(tmem_base + lane_base + (uint32_t)(s * 64 + cg * 32), sr);
                     tmem_ld_wait();
+                    // one pass: scaled logit, distance to the reference, probability (speculative: final
+                    // unless the warpgroup votes for a rescale)
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float v = valid ? __uint_as_float(sr[c]) * p.scale_log2 : -INFINITY;
-                        sr[c] = __float_as_uint(v);
-                        exceed |= v > m_ref[c] + kRescaleThreshold;
-                    }
-                    if (j > 0) {   // O^T of the previous tile complete (needed by a rescale; keeps the phase in step)
-                        ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done, (j - 1) & 1, abort_flag));
-                        tc_fence_after();
+                    for (int c = 0; c < 16; ++c) {
+                        const float v0 = valid ? __uint_as_float(sr[2 * c]) * p.scale_log2 : -INFINITY;
+                        const float v1 = valid ? __uint_as_float(sr[2 * c + 1]) * p.scale_log2 : -INFINITY;
+                        sr[2 * c] = __float_as_uint(v0);
+                        sr[2 * c + 1] = __float_as_uint(v1);
+                        const float d0 = v0 - mref[2 * c], d1 = v1 - mref[2 * c + 1];
+                        exceed |= (d0 > kRescaleThreshold) | (d1 > kRescaleThreshold);
+                        pk[c] = pack_bf16(fast_exp2(d0), fast_exp2(d1));
                     }
                 }
+                if (warp == 4) TRACE(j, 9);
                 const bool rescale = wg_vote_or(bar_id, exceed);
+                if (warp == 4) TRACE(j, 10);
                 if (*abort_flag) break;                      // uniform across the warpgroup after the barrier
                 if (rescale) {
-                    // exact column maxima of this tile across the 64 token lanes
+                    // exact column maxima of this tile across the 64 token lanes: warp-wide integer max of
+                    // order-preserving keys, then across the four warps through shared memory
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        float v = __uint_as_float(sr[c]);
-                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
-                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 8));
-                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 4));
-                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
-                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
-                        if (lane == c) sh->red[cg][q][c] = v;
+                        const int bits = (int)sr[c];
+                        const int key = bits >= 0 ? bits : bits ^ 0x7fffffff;
+                        const int mk = __reduce_max_sync(0xffffffffu, key);
+                        if (lane == c) sh->red[cg][q][c] = __int_as_float(mk >= 0 ? mk : mk ^ 0x7fffffff);
                     }
                     wg_sync(bar_id);
-                    float f[32];
+                    const float cm = fmaxf(fmaxf(sh->red[cg][0][lane], sh->red[cg][1][lane]), fmaxf(sh->red[cg][2][lane], sh->red[cg][3][lane]));
+                    const float m_old = mref[lane];
+                    const float m_new = fmaxf(m_old, cm);
+                    const float f_lane = (m_new == -INFINITY) ? 1.f : fast_exp2(m_old - m_new);   // factor of column `lane`
+                    wg_sync(bar_id);                         // everyone has read the old references
+                    if (q == 0) mref[lane] = m_new;
+                    wg_sync(bar_id);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float cm = fmaxf(fmaxf(sh->red[cg][0][c], sh->red[cg][1][c]), fmaxf(sh->red[cg][2][c], sh->red[cg][3][c]));
-                        const float m_new = fmaxf(m_ref[c], cm);
-                        f[c] = (m_new == -INFINITY) ? 1.f : fast_exp2(m_ref[c] - m_new);
-                        m_ref[c] = m_new;
-                        l_part[c] *= f[c];
-                    }
-                    wg_sync(bar_id);                         // red[] may be reused by the next event
+                    for (int c = 0; c < 32; ++c) l_part[c] *= __shfl_sync(0xffffffffu, f_lane, c);
                     if (j > 0) {
-                        // rescale this column group's 32 columns of all four O^T blocks (all 128 lanes)
+                        // rescale this column group's 32 columns of all four O^T blocks (all 128 lanes), once
+                        // the previous tile's accumulation has landed
+                        mbar_wait(&sh->o_done, (j - 1) & 1, abort_flag);
+                        __syncwarp();
+                        tc_fence_after();
 #pragma unroll 1
                         for (int m = 0; m < 4; ++m) {
                             uint32_t orr[32];
@@ -270,24 +303,26 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                             tmem_ld32(o_addr, orr);
                             tmem_ld_wait();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * f[c]);
+                            for (int c = 0; c < 32; ++c)
+                                orr[c] = __float_as_uint(__uint_as_float(orr[c]) * __shfl_sync(0xffffffffu, f_lane, c));
                             tmem_st32(o_addr, orr);
                         }
                         tmem_st_wait();
                     }
+                    // probabilities again, against the new references
+#pragma unroll
+                    for (int c = 0; c < 16; ++c)
+                        pk[c] = pack_bf16(fast_exp2(__uint_as_float(sr[2 * c]) - mref[2 * c]),
+                                          fast_exp2(__uint_as_float(sr[2 * c + 1]) - mref[2 * c + 1]));
                 }
-                // probabilities (bf16), per-thread partial row sums, P^T row into the rope slab
+                if (warp == 4) TRACE(j, 11);
+                // per-thread partial row sums (of the bf16-rounded values), P^T row into the rope slab
                 uint8_t* tile = sKV + s * TILE_BYTES;
                 if (has_token) {
-                    uint32_t pk[16];
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        const float p0 = valid ? fast_exp2(__uint_as_float(sr[2 * c]) - m_ref[2 * c]) : 0.f;
-                        const float p1 = valid ? fast_exp2(__uint_as_float(sr[2 * c + 1]) - m_ref[2 * c + 1]) : 0.f;
-                        const uint32_t w = pack_bf16(p0, p1);
-                        pk[c] = w;
-                        l_part[2 * c] += __uint_as_float(w << 16);
-                        l_part[2 * c + 1] += __uint_as_float(w & 0xffff0000u);
+                        l_part[2 * c] += __uint_as_float(pk[c] << 16);
+                        l_part[2 * c + 1] += __uint_as_float(pk[c] & 0xffff0000u);
                     }
                     // MN-major P^T: row r (token) = 64 heads = 128 bytes, 16-byte chunks swizzled by r & 7
                     uint8_t* prow = tile + 8 * SLAB_BYTES + r * 128;
@@ -310,6 +345,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(&sh->p_ready[s]);
+                if (warp == 4) TRACE(j, 12);
             }
 
             // ---------------- epilogue: row sums across lanes, normalised partial, LSE
@@ -337,7 +373,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                         inv[c] = 1.f / l;
                         if (q == 0 && lane == c) {
                             const int h = h0 + cg * 32 + c;
-                            if (h < p.H) p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = (m_ref[c] + log2f(l)) * kLn2;
+                            if (h < p.H) p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = (mref[c] + log2f(l)) * kLn2;
                         }
                     }
                     const int64_t row_base = ((int64_t)chunk * p.B + b) * p.H;
@@ -364,6 +400,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) TRACE(0, 29);
     if (*abort_flag) {
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, 3);
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
@@ -392,6 +429,12 @@ cudaError_t make_kv_tmaps(const void* ckv, const void* kpe, int64_t ckv_stride, 
 }
 
 }  // namespace
+
+#ifdef TMLA_TRACE
+extern "C" int typhoon_mla_debug_read_trace_absorb(long long* dst) {
+    return (int)cudaMemcpyFromSymbol(dst, g_trace_ab, sizeof(long long) * 64 * 32);
+}
+#endif
 
 cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t Ls_pad, CUtensorMap* tm_ckv,
                                      CUtensorMap* tm_kpe) {

@@ -112,11 +112,30 @@ int naive_splits(int B, int H, int64_t Ls) {
 }
 
 void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chunk, int* n_sh, int* n_sf) {
-    int units = B * ((H + 63) / 64);
-    int target = std::max(1, (2 * kNumSM + units - 1) / units);
-    int64_t longest = std::max<int64_t>(std::max(Ls_absorb, cap_suffix), 1);
-    int64_t c = round_up((longest + target - 1) / target, 64);
-    c = std::max<int64_t>(c, 256);
+    const int units = B * ((H + 63) / 64);
+    const int64_t longest = std::max<int64_t>(std::max(Ls_absorb, cap_suffix), 1);
+    int64_t c;
+    if (g_kernel_path == TYPHOON_MLA_PATH_TCGEN05) {
+        // One CTA per SM: minimise waves x (tiles per chunk + fixed cost in tile units) over the number of
+        // chunks the longest segment is cut into.
+        const double fixed = 3.0;
+        double best_cost = 1e30;
+        c = round_up(longest, 64);
+        for (int parts = 1; parts <= 32; ++parts) {
+            const int64_t ch = round_up((longest + parts - 1) / parts, 64);
+            const int64_t ctas = (int64_t)units * ((Ls_absorb + ch - 1) / ch + (cap_suffix + ch - 1) / ch);
+            const int64_t waves = (ctas + kNumSM - 1) / kNumSM;
+            const double cost = (double)waves * ((double)ch / 64.0 + fixed);
+            if (cost < best_cost - 1e-9) {
+                best_cost = cost;
+                c = ch;
+            }
+            if (ch <= 64) break;
+        }
+    } else {
+        const int target = std::max(1, (2 * kNumSM + units - 1) / units);
+        c = std::max<int64_t>(round_up((longest + target - 1) / target, 64), 256);
+    }
     *chunk = (int)c;
     *n_sh = (int)((Ls_absorb + c - 1) / c);
     *n_sf = (int)((cap_suffix + c - 1) / c);

@@ -277,20 +277,15 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     sr[c >> 5][c & 31] = __float_as_uint(v);
                     mx = fmaxf(mx, v);
                 }
-                // previous PV of this stream must be complete before O may be rescaled, and
-                // waiting every step keeps the barrier's phase in lockstep
-                if ((warp & 3) == 0 && lane == 0) TRACE(j, 11 + 8 * i);
-                if (j > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i], (j - 1) & 1, abort_flag));
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-                if ((warp & 3) == 0 && lane == 0) TRACE(j, 12 + 8 * i);
                 // lazy rescale: only when some row's maximum grew by more than 2^8
                 const bool grow = mx > m_ref + 8.f;
                 if (j == 0) {
                     m_ref = mx;
                 } else if (__any_sync(0xffffffffu, grow)) {
+                    // the previous PV of this stream must have landed before O is touched
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i], (j - 1) & 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
                     const float m_new = grow ? mx : m_ref;
                     const float f = fast_exp2(m_ref - m_new);
                     m_ref = m_new;
