@@ -54,6 +54,9 @@ struct AbsorbSm100Params {
     float scale_log2;
     float* o_part;     // [n_chunks][B][H][512]
     float* lse_part;   // [n_chunks][B][H]
+    // single-chunk launches write the merged result directly and skip the merge step
+    __nv_bfloat16* o_lat_direct;   // bf16 [B][H][512] or null
+    float* lse_direct;             // [B][H]
     int* status;
 };
 
@@ -373,7 +376,11 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                         inv[c] = 1.f / l;
                         if (q == 0 && lane == c) {
                             const int h = h0 + cg * 32 + c;
-                            if (h < p.H) p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = (mref[c] + log2f(l)) * kLn2;
+                            if (h < p.H) {
+                                const float lse = (mref[c] + log2f(l)) * kLn2;
+                                if (p.o_lat_direct) p.lse_direct[(int64_t)b * p.H + h] = lse;
+                                else p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = lse;
+                            }
                         }
                     }
                     const int64_t row_base = ((int64_t)chunk * p.B + b) * p.H;
@@ -386,7 +393,11 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 #pragma unroll
                         for (int c = 0; c < 32; ++c) {
                             const int h = h0 + cg * 32 + c;
-                            if (h < p.H) p.o_part[(row_base + h) * 512 + lat] = __uint_as_float(orr[c]) * inv[c];
+                            if (h < p.H) {
+                                const float v = __uint_as_float(orr[c]) * inv[c];
+                                if (p.o_lat_direct) p.o_lat_direct[((int64_t)b * p.H + h) * 512 + lat] = __float2bfloat16_rn(v);
+                                else p.o_part[(row_base + h) * 512 + lat] = v;
+                            }
                         }
                     }
                 }
@@ -395,7 +406,16 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     } else if (warp >= 4) {
         // empty chunk: weight zero in the merge
         const int i = threadIdx.x - 128;
-        if (i < 64 && h0 + i < p.H) p.lse_part[((int64_t)chunk * p.B + b) * p.H + h0 + i] = -INFINITY;
+        if (i < 64 && h0 + i < p.H) {
+            if (p.o_lat_direct) {
+                // a request without any latent token: zero latent output, weight zero in the combine
+                p.lse_direct[(int64_t)b * p.H + h0 + i] = -INFINITY;
+                for (int l = 0; l < 512; l += 8)
+                    *reinterpret_cast<uint4*>(p.o_lat_direct + ((int64_t)b * p.H + h0 + i) * 512 + l) = make_uint4(0, 0, 0, 0);
+            } else {
+                p.lse_part[((int64_t)chunk * p.B + b) * p.H + h0 + i] = -INFINITY;
+            }
+        }
     }
 
     tc_fence_before();
@@ -442,7 +462,7 @@ cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t L
 }
 
 cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_ckv_sh, const CUtensorMap* tm_kpe_sh,
-                                     int* status, cudaStream_t s) {
+                                     void* o_lat_direct, float* lse_direct, int* status, cudaStream_t s) {
     const int n_chunks = a.n_shared_chunks + a.n_suffix_chunks;
     if (a.B <= 0 || n_chunks <= 0) return cudaSuccess;
     if (a.chunk % TOK != 0) return cudaErrorInvalidValue;
@@ -478,6 +498,8 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     p.block_table = a.block_table; p.seq_lens = a.seq_lens;
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = status;
+    p.o_lat_direct = n_chunks == 1 ? reinterpret_cast<__nv_bfloat16*>(o_lat_direct) : nullptr;
+    p.lse_direct = lse_direct;
     const int smem = (STAGES + 1) * TILE_BYTES + 1024 + (int)sizeof(Shared) + 64;
     cudaFuncSetAttribute(absorb_attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     dim3 grid(n_chunks, (a.H + 63) / 64, a.B);

@@ -338,6 +338,7 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
     }
     if (e == cudaSuccess && Ls > 0)
         e = make_naive_sm100_tmaps(sh->k_nope, sh->kpe, sh->v_t, H, sh->Ls_pad, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt);
+    if (e == cudaSuccess) e = make_q_absorb_tmap(sh->w_uk_t, H, &sh->tm_wuk_t);
     if (e == cudaSuccess && Ls > 0) e = make_absorb_shared_tmaps(sh->ckv, sh->kpe, sh->Ls_pad, &sh->tm_ckv, &sh->tm_kpe_tok);
     if (e != cudaSuccess) {
         typhoon_mla_free(sh);
@@ -452,52 +453,71 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     }
     const int n_chunks = pl.n_shared_chunks + pl.n_suffix_chunks;
     const bool have_absorb = use_absorb && n_chunks > 0;
+    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    bool combined = false;
     if (have_absorb) {
         // --- query absorption Q_A = Q_N W_UK (Algorithm 1 line 5)
         void* q_abs = ws + pl.off_qabs;
-        GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,
-                  B, 512, 128, H, false};
         prof_before(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
-        e = launch_gemm_tn(g1, s);
+        if (tc) {
+            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->status, s);
+        } else {
+            GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,
+                      B, 512, 128, H, false};
+            e = launch_gemm_tn(g1, s);
+        }
         prof_after(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
         // --- absorb attention over latent tokens (Algorithm 1 line 6)
         float* o_part_a = reinterpret_cast<float*>(ws + pl.off_opart_a);
         float* lse_part_a = reinterpret_cast<float*>(ws + pl.off_lsepart_a);
+        void* o_lat = ws + pl.off_olat;
         AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
                       ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
                       seq_lens, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
                       o_part_a, lse_part_a};
         prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
-        e = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05
-                ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, sh->status, s)
-                : launch_absorb_attn_mma(ab, s);
+        e = tc ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, o_lat, lse_a, sh->status, s)
+               : launch_absorb_attn_mma(ab, s);
         prof_after(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
-        void* o_lat = ws + pl.off_olat;
-        prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
-        e = launch_merge_latent(o_part_a, lse_part_a, n_chunks, B, H, o_lat, lse_a, s);
-        prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
-        if (e != cudaSuccess) return cuda_fail(e);
-        ++launches;
-        // --- output projection O_A W_UV^T (Algorithm 1 line 7)
-        GemmTN g2{o_lat, (int64_t)H * 512, 512, sh->w_uv, 512, 128 * 512, o_abs, (int64_t)H * 128, 128,
-                  B, 128, 512, H, true};
+        if (!(tc && n_chunks == 1)) {   // a single-chunk tcgen05 launch has already written the merged result
+            prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
+            e = launch_merge_latent(o_part_a, lse_part_a, n_chunks, B, H, o_lat, lse_a, s);
+            prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
+            if (e != cudaSuccess) return cuda_fail(e);
+            ++launches;
+        }
+        // --- output projection O_A W_UV^T (Algorithm 1 line 7); on the tcgen05 path its epilogue also does the
+        //     LSE combine (line 8)
         prof_before(TYPHOON_MLA_KERNEL_W_UV, s);
-        e = launch_gemm_tn(g2, s);
+        if (tc) {
+            GemmTN g2{o_lat, (int64_t)H * 512, 512, sh->w_uv, 512, 128 * 512, nullptr, 0, 0, B, 128, 512, H, false};
+            CombineEpilogue ce;
+            ce.o_naive = o_part_n; ce.lse_naive = lse_part_n; ce.n_naive = pl.n_slots_naive;
+            ce.lse_abs = lse_a; ce.out = out; ce.lse_out = lse_out; ce.H = H;
+            e = launch_gemm_tn_sm100(g2, sh->status, s, &ce);
+            combined = true;
+        } else {
+            GemmTN g2{o_lat, (int64_t)H * 512, 512, sh->w_uv, 512, 128 * 512, o_abs, (int64_t)H * 128, 128,
+                      B, 128, 512, H, true};
+            e = launch_gemm_tn(g2, s);
+        }
         prof_after(TYPHOON_MLA_KERNEL_W_UV, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
     }
     // --- LSE combine (Algorithm 1 line 8)
-    prof_before(TYPHOON_MLA_KERNEL_COMBINE, s);
-    e = launch_combine(o_part_n, lse_part_n, pl.n_slots_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
-                       lse_out, s);
-    prof_after(TYPHOON_MLA_KERNEL_COMBINE, s);
-    if (e != cudaSuccess) return cuda_fail(e);
-    ++launches;
+    if (!combined) {
+        prof_before(TYPHOON_MLA_KERNEL_COMBINE, s);
+        e = launch_combine(o_part_n, lse_part_n, pl.n_slots_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
+                           lse_out, s);
+        prof_after(TYPHOON_MLA_KERNEL_COMBINE, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+    }
     g_last_launches = launches;
     return TYPHOON_MLA_OK;
 }

@@ -23,8 +23,10 @@ constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256
 struct GemmParams {
     void* C; int64_t ldc, c_batch;
     int M, N, K, c_block_n, c_tile64;
-    int a_batched, b_batched;
+    int a_batched, b_batched, a_swap;
     int* status;
+    int out_mode;          // 0: bf16 C, 1: fp32 C, 2: LSE combine epilogue (N == 128, row = request, batch = head)
+    CombineEpilogue ce;
 };
 
 __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constant__ CUtensorMap tmA,
@@ -37,7 +39,7 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
     const int KB = p.K / BK;
 
@@ -56,62 +58,127 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_holder;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_holder, 0);
 
     if (warp == 0) {
-        if (lane == 0) {
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % STAGES;
-                if (!mbar_wait(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag)) break;
-                mbar_arrive_expect_tx(&full[s], STAGE_BYTES);
-                uint8_t* sa = smem + s * STAGE_BYTES;
-                tma_load_3d(sa, &tmA, &full[s], kb * BK, m0, p.a_batched ? z : 0);
-                tma_load_3d(sa + A_BYTES, &tmB, &full[s], kb * BK, n0, p.b_batched ? z : 0);
-            }
+        // producer: the whole warp runs the loop, the elected lane issues
+        const uint32_t ld = elect_one() ? 1u : 0u;
+        for (int kb = 0; kb < KB; ++kb) {
+            const int s = kb % STAGES;
+            if (!mbar_wait_warp(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag)) break;
+            mbar_arrive_expect_tx_if(ld, &full[s], STAGE_BYTES);
+            uint8_t* sa = smem + s * STAGE_BYTES;
+            if (p.a_swap) tma_load_3d_if(ld, sa, &tmA, &full[s], kb * BK, z, m0);
+            else tma_load_3d_if(ld, sa, &tmA, &full[s], kb * BK, m0, p.a_batched ? z : 0);
+            tma_load_3d_if(ld, sa + A_BYTES, &tmB, &full[s], kb * BK, n0, p.b_batched ? z : 0);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(BM, BN, false, false);
-            bool ok = true;
-            for (int kb = 0; kb < KB && ok; ++kb) {
-                const int s = kb % STAGES;
-                ok = mbar_wait(&full[s], (kb / STAGES) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
-                const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + A_BYTES);
+        const uint32_t ld = elect_one() ? 1u : 0u;
+        constexpr uint32_t idesc = idesc_bf16(BM, BN, false, false);
+        bool ok = true;
+        for (int kb = 0; kb < KB && ok; ++kb) {
+            const int s = kb % STAGES;
+            ok = mbar_wait_warp(&full[s], (kb / STAGES) & 1, abort_flag);
+            if (!ok) break;
+            const uint32_t sa = smem_u32(smem + s * STAGE_BYTES);
+            const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + A_BYTES);
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k) umma_ss(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-                umma_commit(&empty[s]);
-            }
-            if (ok) umma_commit(acc_full);
+            for (int k = 0; k < BK / 16; ++k) umma_ss_if(ld, tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            umma_commit_if(ld, &empty[s]);
         }
+        if (ok) umma_commit_if(ld, acc_full);
     } else {
         const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag));
         tc_fence_after();
         if (ok) {
             const int lg = (warp & 3) * 32;
             const int row = m0 + lg + lane;
-            __nv_bfloat16* cbase = reinterpret_cast<__nv_bfloat16*>(p.C) + (int64_t)z * p.c_batch;
+            if (p.out_mode == 2) {
+                // The accumulator row is the absorb-side output O_A[b, h, :] (already normalised).  Merge it
+                // with the naive-side partials of the same (request, head) by their log-sum-exps
+                // (Algorithm 1 line 8) and write the final bf16 row.
+                const CombineEpilogue& ce = p.ce;
+                const int64_t BH = (int64_t)p.M * ce.H;
+                const int64_t bh = (int64_t)row * ce.H + z;
+                const bool live = row < p.M;
+                float m = -INFINITY, la = -INFINITY;
+                if (live) {
+                    la = ce.lse_abs[bh];
+                    m = la;
+                    for (int i = 0; i < ce.n_naive; ++i) m = fmaxf(m, ce.lse_naive[i * BH + bh]);
+                }
+                float wa = 0.f, zsum = 0.f;
+                if (m != -INFINITY) {
+                    wa = (la == -INFINITY) ? 0.f : __expf(la - m);
+                    zsum = wa;
+                    for (int i = 0; i < ce.n_naive; ++i) {
+                        const float l = ce.lse_naive[i * BH + bh];
+                        if (l != -INFINITY) zsum += __expf(l - m);
+                    }
+                }
+                const float inv = zsum > 0.f ? 1.f / zsum : 0.f;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)lg << 16) + c * 32, r);
-                tmem_ld_wait();
-                if (row < p.M) {
-                    const int gn = n0 + c * 32;
-                    __nv_bfloat16* crow =
-                        cbase + (p.c_tile64 ? (((int64_t)(row >> 6) * (p.N >> 6) + (gn >> 6)) << 12) + ((row & 63) << 6) + (gn & 63)
-                                 : p.c_block_n ? ((int64_t)(gn >> 6) * p.M + row) * 64 + (gn & 63)
-                                               : (int64_t)row * p.ldc + gn);
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)lg << 16) + c * 32, r);
+                    tmem_ld_wait();
+                    if (!live) continue;
+                    float acc[32];
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) acc[q] = wa > 0.f ? wa * __uint_as_float(r[q]) : 0.f;
+                    for (int i = 0; i < ce.n_naive; ++i) {
+                        const float l = ce.lse_naive[i * BH + bh];
+                        if (l == -INFINITY) continue;          // empty partial: its O slot was never written
+                        const float w = __expf(l - m);
+                        const float4* src = reinterpret_cast<const float4*>(ce.o_naive + (i * BH + bh) * 128 + c * 32);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 v = src[q];
+                            acc[4 * q] += w * v.x; acc[4 * q + 1] += w * v.y; acc[4 * q + 2] += w * v.z; acc[4 * q + 3] += w * v.w;
+                        }
+                    }
+                    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(ce.out) + bh * 128 + c * 32;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         uint4 v;
-                        v.x = pack_bf16(__uint_as_float(r[j * 8 + 0]), __uint_as_float(r[j * 8 + 1]));
-                        v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]), __uint_as_float(r[j * 8 + 3]));
-                        v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]), __uint_as_float(r[j * 8 + 5]));
-                        v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]), __uint_as_float(r[j * 8 + 7]));
-                        *reinterpret_cast<uint4*>(crow + j * 8) = v;
+                        v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
+                        v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
+                        v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
+                        v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + j * 8) = v;
+                    }
+                }
+                if (live && ce.lse_out) ce.lse_out[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(zsum);
+            } else {
+                uint8_t* cbase = reinterpret_cast<uint8_t*>(p.C) + (int64_t)z * p.c_batch * (p.out_mode == 1 ? 4 : 2);
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)lg << 16) + c * 32, r);
+                    tmem_ld_wait();
+                    if (row < p.M) {
+                        const int gn = n0 + c * 32;
+                        const int64_t off = p.c_tile64 ? (((int64_t)(row >> 6) * (p.N >> 6) + (gn >> 6)) << 12) + ((row & 63) << 6) + (gn & 63)
+                                            : p.c_block_n ? ((int64_t)(gn >> 6) * p.M + row) * 64 + (gn & 63)
+                                                          : (int64_t)row * p.ldc + gn;
+                        if (p.out_mode == 1) {
+                            float4* crow = reinterpret_cast<float4*>(cbase + off * 4);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                crow[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                                      __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                        } else {
+                            __nv_bfloat16* crow = reinterpret_cast<__nv_bfloat16*>(cbase + off * 2);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(r[j * 8 + 0]), __uint_as_float(r[j * 8 + 1]));
+                                v.y = pack_bf16(__uint_as_float(r[j * 8 + 2]), __uint_as_float(r[j * 8 + 3]));
+                                v.z = pack_bf16(__uint_as_float(r[j * 8 + 4]), __uint_as_float(r[j * 8 + 5]));
+                                v.w = pack_bf16(__uint_as_float(r[j * 8 + 6]), __uint_as_float(r[j * 8 + 7]));
+                                *reinterpret_cast<uint4*>(crow + j * 8) = v;
+                            }
+                        }
                     }
                 }
             }
@@ -131,11 +198,21 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
 
 }  // namespace
 
-cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s) {
+cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, const CombineEpilogue* ce) {
     if (g.M <= 0 || g.batch <= 0) return cudaSuccess;
-    if (g.N % BN != 0 || g.K % BK != 0 || g.out_fp32) return cudaErrorInvalidValue;
+    if (g.N % BN != 0 || g.K % BK != 0) return cudaErrorInvalidValue;
+    if (ce && g.N != BN) return cudaErrorInvalidValue;
     CUtensorMap tmA, tmB;
-    {
+    // When the batch stride of A is smaller than its row stride (activations laid out [M, batch, K]) the
+    // tensor map is built with the batch dimension in the middle so that strides stay increasing.
+    const bool a_swap = g.a_batch != 0 && g.a_batch < g.lda;
+    if (a_swap) {
+        uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.batch, (uint64_t)g.M};
+        uint64_t strides[2] = {(uint64_t)g.a_batch * 2, (uint64_t)g.lda * 2};
+        uint32_t box[3] = {BK, 1, BM};
+        cudaError_t e = make_tmap_bf16(&tmA, g.A, 3, dims, strides, box);
+        if (e != cudaSuccess) return e;
+    } else {
         const bool batched = g.a_batch != 0;
         uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.M, (uint64_t)(batched ? g.batch : 1)};
         uint64_t strides[2] = {(uint64_t)g.lda * 2, (uint64_t)(batched ? g.a_batch : (int64_t)g.lda * g.M) * 2};
@@ -151,7 +228,8 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s) {
         cudaError_t e = make_tmap_bf16(&tmB, g.B, 3, dims, strides, box);
         if (e != cudaSuccess) return e;
     }
-    GemmParams p{g.C, g.ldc, g.c_batch, g.M, g.N, g.K, g.c_block_n, g.c_tile64 ? 1 : 0, g.a_batch != 0, g.b_batch != 0, status};
+    GemmParams p{g.C, g.ldc, g.c_batch, g.M, g.N, g.K, g.c_block_n, g.c_tile64 ? 1 : 0, g.a_batch != 0, g.b_batch != 0, a_swap ? 1 : 0, status,
+                 ce ? 2 : (g.out_fp32 ? 1 : 0), ce ? *ce : CombineEpilogue{}};
     cudaFuncSetAttribute(gemm_tn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid(g.N / BN, (g.M + BM - 1) / BM, g.batch);
     gemm_tn_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tmA, tmB, p);

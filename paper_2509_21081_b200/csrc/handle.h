@@ -16,6 +16,7 @@ struct typhoon_mla_shared {
     void* w_uk_t;   // bf16 [H, 512, 128]
     const void* w_uv;  // borrowed, bf16 [H, 128, 512]
     CUtensorMap tm_kn, tm_kp, tm_vt;   // TMA descriptors of k_nope, kpe, v_t (valid if Ls > 0)
+    CUtensorMap tm_wuk_t;              // TMA descriptor of w_uk_t
     CUtensorMap tm_ckv, tm_kpe_tok;    // TMA descriptors of ckv, kpe as 64-token pages (valid if Ls > 0)
     int* status;    // device word: non-zero after a bounded in-kernel wait expired
     size_t owned_bytes;

@@ -23,7 +23,23 @@ struct GemmTN {
 cudaError_t launch_gemm_tn(const GemmTN& g, cudaStream_t s);
 // tcgen05/TMEM/TMA version (bf16 output only; N % 128 == 0, K % 64 == 0).  `status` (device int,
 // may be null) is set non-zero if a bounded wait inside the kernel expired.
-cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s);
+// Optional fused epilogue (N must be 128): the accumulator row of (request m, head z) is taken as the
+// normalised absorb-side output and merged with n_naive naive-side partials by their LSEs.
+struct CombineEpilogue {
+    const float* o_naive = nullptr;    // [n_naive][B][H][128]
+    const float* lse_naive = nullptr;  // [n_naive][B][H]
+    int n_naive = 0;
+    const float* lse_abs = nullptr;    // [B][H]
+    void* out = nullptr;               // bf16 [B][H][128]
+    float* lse_out = nullptr;          // optional [B][H]
+    int H = 0;
+};
+cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, const CombineEpilogue* ce = nullptr);
+
+// Query absorption on tcgen05 (one CTA per head and 128 requests); tm_w from make_q_absorb_tmap.
+cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w);
+cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int* status,
+                                  cudaStream_t s);
 
 // Naive shared-prefix attention partials (Algorithm 1 line 4).
 struct NaiveAttn {
@@ -69,8 +85,10 @@ cudaError_t launch_absorb_attn_mma(const AbsorbAttn& p, cudaStream_t s);
 
 // tcgen05/TMEM/TMA version (chunk must be a multiple of 64).  The tensor maps of the handle's copy of the
 // shared latent cache come from make_absorb_shared_tmaps (used when n_shared_chunks > 0).
+// With a single chunk in total the kernel writes the merged bf16 latent output [B,H,512] and its LSE [B,H]
+// directly to o_lat_direct / lse_direct (no merge step needed); otherwise it writes the partials.
 cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_ckv_sh, const CUtensorMap* tm_kpe_sh,
-                                     int* status, cudaStream_t s);
+                                     void* o_lat_direct, float* lse_direct, int* status, cudaStream_t s);
 cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t Ls_pad, CUtensorMap* tm_ckv,
                                      CUtensorMap* tm_kpe);
 
