@@ -39,6 +39,12 @@ inline void prof_after(int id, cudaStream_t s) {
 }
 
 int g_kernel_path = TYPHOON_MLA_PATH_TCGEN05;
+// Run the absorb branch of a hybrid step on a side stream next to the naive kernel (tuning aid:
+// TYPHOON_MLA_OVERLAP=0 in the environment keeps everything on the caller's stream).
+const bool g_overlap = [] {
+    const char* v = std::getenv("TYPHOON_MLA_OVERLAP");
+    return !(v && v[0] == '0');
+}();
 
 // Hardware model of the crossover rule (defaults: measured on B200).
 double g_tensor_flops = 1.0e15;      // sustained rate the attention kernels reach, FLOP/s
@@ -277,6 +283,9 @@ int typhoon_mla_free(typhoon_mla_shared_t* sh) {
     cudaFree(sh->kpe);
     cudaFree(sh->w_uk_t);
     cudaFree(sh->status);
+    if (sh->side_stream) cudaStreamDestroy(sh->side_stream);
+    if (sh->ev_fork) cudaEventDestroy(sh->ev_fork);
+    if (sh->ev_join) cudaEventDestroy(sh->ev_join);
     delete sh;
     return TYPHOON_MLA_OK;
 }
@@ -320,6 +329,17 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    {
+        int lo = 0, hi = 0;
+        cudaDeviceGetStreamPriorityRange(&lo, &hi);   // hi is the numerically lowest = highest priority
+        e = cudaStreamCreateWithPriority(&sh->side_stream, cudaStreamNonBlocking, hi);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sh->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sh->ev_join, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+        typhoon_mla_free(sh);
+        return cuda_fail(e);
+    }
     e = cudaMemsetAsync(sh->status, 0, 256, s);
     if (e == cudaSuccess) e = launch_transpose_bf16(w_uk, sh->w_uk_t, 128, 512, H, s);
     if (e == cudaSuccess && Ls > 0) {
@@ -435,6 +455,20 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     float* o_abs = reinterpret_cast<float*>(ws + pl.off_oabs);
     float* lse_a = reinterpret_cast<float*>(ws + pl.off_lse_a);
 
+    const int n_chunks = pl.n_shared_chunks + pl.n_suffix_chunks;
+    const bool have_absorb = use_absorb && n_chunks > 0;
+    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    // In a hybrid step the absorb branch (lines 5-6) does not depend on the naive kernel (line 4): it runs
+    // on the handle's (high-priority) side stream, forked behind the caller's stream here and joined
+    // before the projection.
+    cudaStream_t s_main = s;
+    const bool forked = g_overlap && have_absorb && pl.n_split_naive > 0 && sh->side_stream != nullptr;
+    if (forked) {
+        e = cudaEventRecord(sh->ev_fork, s_main);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(sh->side_stream, sh->ev_fork, 0);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+
     // --- naive shared-prefix attention (Algorithm 1 line 4)
     if (pl.n_split_naive > 0) {
         prof_before(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
@@ -451,10 +485,8 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
     }
-    const int n_chunks = pl.n_shared_chunks + pl.n_suffix_chunks;
-    const bool have_absorb = use_absorb && n_chunks > 0;
-    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
     bool combined = false;
+    if (forked) s = sh->side_stream;
     if (have_absorb) {
         // --- query absorption Q_A = Q_N W_UK (Algorithm 1 line 5)
         void* q_abs = ws + pl.off_qabs;
@@ -489,6 +521,12 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
             prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
             if (e != cudaSuccess) return cuda_fail(e);
             ++launches;
+        }
+        if (forked) {
+            e = cudaEventRecord(sh->ev_join, sh->side_stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(s_main, sh->ev_join, 0);
+            if (e != cudaSuccess) return cuda_fail(e);
+            s = s_main;
         }
         // --- output projection O_A W_UV^T (Algorithm 1 line 7); on the tcgen05 path its epilogue also does the
         //     LSE combine (line 8)

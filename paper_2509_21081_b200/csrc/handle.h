@@ -1,6 +1,7 @@
 // The prepared-prefix handle behind typhoon_mla_shared_t (host object; see typhoon_mla_prepare_shared).
 #pragma once
 #include <cuda.h>
+#include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -18,6 +19,8 @@ struct typhoon_mla_shared {
     CUtensorMap tm_kn, tm_kp, tm_vt;   // TMA descriptors of k_nope, kpe, v_t (valid if Ls > 0)
     CUtensorMap tm_wuk_t;              // TMA descriptor of w_uk_t
     CUtensorMap tm_ckv, tm_kpe_tok;    // TMA descriptors of ckv, kpe as 64-token pages (valid if Ls > 0)
+    cudaStream_t side_stream;          // absorb branch of a hybrid step runs here, beside the naive kernel
+    cudaEvent_t ev_fork, ev_join;
     int* status;    // device word: non-zero after a bounded in-kernel wait expired
     size_t owned_bytes;
     int device;
