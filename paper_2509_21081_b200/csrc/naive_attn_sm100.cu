@@ -104,25 +104,58 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     const int rot = n_tiles > 0 ? (int)(((unsigned)h * 37u + (unsigned)split * 11u) % (unsigned)n_tiles) : 0;
     auto tile_of = [&](int e) { int t = e + rot; return t_begin + (t >= n_tiles ? t - n_tiles : t); };
 
-    if (threadIdx.x == 0) {
-        mbar_init(&bar->q_full, 1);
-        for (int s = 0; s < MAX_STAGES; ++s) {
-            mbar_init(&bar->k_full[s], 1);
-            mbar_init(&bar->k_empty[s], 1);
-            mbar_init(&bar->v_full[s], 1);
-            mbar_init(&bar->v_empty[s], 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            for (int b = 0; b < 2; ++b) {
-                mbar_init(&bar->s_ready[i][b], 1);
-                mbar_init(&bar->p_ready[i][b], 128);
-                mbar_init(&bar->sbuf_free[i][b], 1);
+    // Warp 0 initialises the barriers and at once issues Q and the first K and V tiles, so that the
+    // first copies are in flight while the rest of the CTA sets up (tensor-memory allocation, barrier).
+    const uint32_t ld0 = (warp == 0 && elect_one()) ? 1u : 0u;
+    auto issue_k = [&](int e) {
+        const int s = e % p.k_stages;
+        uint8_t* dst = sK + s * K_TILE_BYTES;
+        TRACE(e >> 1, 24 + (e & 1));
+        mbar_arrive_expect_tx_if(ld0, &bar->k_full[s], K_TILE_BYTES);
+        tma_load_3d_if(ld0, dst, &tm_kn, &bar->k_full[s], 0, 0, h * (p.Ls_pad / TOK) + tile_of(e));
+        tma_load_2d_if(ld0, dst + 16384, &tm_kp, &bar->k_full[s], 0, tile_of(e) * TOK);
+    };
+    auto issue_v = [&](int e, uint32_t ld) {
+        const int s = e % p.v_stages;
+        mbar_arrive_expect_tx_if(ld, &bar->v_full[s], V_TILE_BYTES);
+        tma_load_4d_if(ld, sV + s * V_TILE_BYTES, &tm_vt, &bar->v_full[s], 0, 0, tile_of(e), h);
+    };
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_init(&bar->q_full, 1);
+            for (int s = 0; s < MAX_STAGES; ++s) {
+                mbar_init(&bar->k_full[s], 1);
+                mbar_init(&bar->k_empty[s], 1);
+                mbar_init(&bar->v_full[s], 1);
+                mbar_init(&bar->v_empty[s], 1);
             }
-            mbar_init(&bar->o_done[i], 1);
+            for (int i = 0; i < 2; ++i) {
+                for (int b = 0; b < 2; ++b) {
+                    mbar_init(&bar->s_ready[i][b], 1);
+                    mbar_init(&bar->p_ready[i][b], 128);
+                    mbar_init(&bar->sbuf_free[i][b], 1);
+                }
+                mbar_init(&bar->o_done[i], 1);
+            }
+            bar->abort_flag = 0;
+            fence_mbar_init();
         }
-        bar->abort_flag = 0;
-        fence_mbar_init();
-        prefetch_tmap(&tm_qn); prefetch_tmap(&tm_qp); prefetch_tmap(&tm_kn); prefetch_tmap(&tm_kp); prefetch_tmap(&tm_vt);
+        __syncwarp();
+        if (n_tiles > 0) {
+            const int nq = (n_str[1] > 0 && !p.mode_y) ? 2 : 1;
+            mbar_arrive_expect_tx_if(ld0, &bar->q_full, nq * Q_TILE_BYTES);
+            for (int t = 0; t < nq; ++t) {
+                uint8_t* dst = sQ + t * Q_TILE_BYTES;
+                tma_load_3d_if(ld0, dst, &tm_qn, &bar->q_full, 0, h, row0 + t * 128);
+                tma_load_3d_if(ld0, dst + 16384, &tm_qn, &bar->q_full, 64, h, row0 + t * 128);
+                tma_load_3d_if(ld0, dst + 32768, &tm_qp, &bar->q_full, 0, h, row0 + t * 128);
+            }
+            // interleave K and V so that the tiles of the first steps arrive first
+            for (int e = 0; e < max(p.k_stages, p.v_stages); ++e) {
+                if (e < p.k_stages && e < n_tiles) issue_k(e);
+                if (e < p.v_stages && e < n_tiles) issue_v(e, ld0);
+            }
+        }
     }
     if (warp == 1) tmem_alloc(&bar->tmem_base, 512);
     tc_fence_before();
@@ -134,47 +167,18 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     if (n_tiles > 0) {
         if (warp == 0) {
-            // ---------------- Q + K producer (whole warp runs the loop, the elected lane issues)
-            const uint32_t ld = elect_one() ? 1u : 0u;
-            const int nq = (n_str[1] > 0 && !p.mode_y) ? 2 : 1;
-            mbar_arrive_expect_tx_if(ld, &bar->q_full, nq * Q_TILE_BYTES);
-            for (int t = 0; t < nq; ++t) {
-                uint8_t* dst = sQ + t * Q_TILE_BYTES;
-                tma_load_3d_if(ld, dst, &tm_qn, &bar->q_full, 0, h, row0 + t * 128);
-                tma_load_3d_if(ld, dst + 16384, &tm_qn, &bar->q_full, 64, h, row0 + t * 128);
-                tma_load_3d_if(ld, dst + 32768, &tm_qp, &bar->q_full, 0, h, row0 + t * 128);
-            }
-            for (int e = 0; e < n_tiles; ++e) {
-                const int s = e % p.k_stages;
-                if (!mbar_wait_warp(&bar->k_empty[s], ((e / p.k_stages) & 1) ^ 1, abort_flag)) break;
-                uint8_t* dst = sK + s * K_TILE_BYTES;
-                const int tok = tile_of(e) * TOK;
-                TRACE(e >> 1, 24 + (e & 1));
-                mbar_arrive_expect_tx_if(ld, &bar->k_full[s], K_TILE_BYTES);
-                tma_load_3d_if(ld, dst, &tm_kn, &bar->k_full[s], 0, 0, h * (p.Ls_pad / TOK) + tile_of(e));
-                tma_load_2d_if(ld, dst + 16384, &tm_kp, &bar->k_full[s], 0, tok);
+            // ---------------- K producer: the rest of the ring (Q and the first tiles are already in flight)
+            for (int e = p.k_stages; e < n_tiles; ++e) {
+                if (!mbar_wait_warp(&bar->k_empty[e % p.k_stages], ((e / p.k_stages) & 1) ^ 1, abort_flag)) break;
+                issue_k(e);
             }
         } else if (warp == 2) {
             // ---------------- V producer
             const uint32_t ld = elect_one() ? 1u : 0u;
-            for (int e = 0; e < n_tiles; ++e) {
-                const int s = e % p.v_stages;
-                if (!mbar_wait_warp(&bar->v_empty[s], ((e / p.v_stages) & 1) ^ 1, abort_flag)) break;
-                TRACE(e >> 1, 26 + (e & 1));
-                mbar_arrive_expect_tx_if(ld, &bar->v_full[s], V_TILE_BYTES);
-                tma_load_4d_if(ld, sV + s * V_TILE_BYTES, &tm_vt, &bar->v_full[s], 0, 0, tile_of(e), h);
+            for (int e = p.v_stages; e < n_tiles; ++e) {
+                if (!mbar_wait_warp(&bar->v_empty[e % p.v_stages], ((e / p.v_stages) & 1) ^ 1, abort_flag)) break;
+                issue_v(e, ld);
             }
-#ifdef TMLA_NOCOMPUTE
-        } else if (warp == 1) {
-            // debug: consume the rings without any tensor-core or softmax work
-            for (int e = 0; e < n_tiles; ++e) {
-                if (!mbar_wait_warp(&bar->k_full[e % p.k_stages], (e / p.k_stages) & 1, abort_flag)) break;
-                if (lane == 0) mbar_arrive(&bar->k_empty[e % p.k_stages]);
-                if (!mbar_wait_warp(&bar->v_full[e % p.v_stages], (e / p.v_stages) & 1, abort_flag)) break;
-                if (lane == 0) mbar_arrive(&bar->v_empty[e % p.v_stages]);
-            }
-        }
-#else
         } else if (warp == 1) {
             // ---------------- S = Q K^T issuer (whole warp runs the loop, the elected lane issues).
             // Runs ahead of the softmax by up to two steps (S is double-buffered per stream).
@@ -251,6 +255,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const int r = lg + lane;                  // row within the 128-row tile
             const int b = row0 + (p.mode_y ? 0 : i * 128) + r;
             const int nt = n_str[i];
+            const bool warp_has_rows = (b - lane) < p.B;   // warp-uniform: first row of this warp is a real request
             float m_ref = -INFINITY, l_sum = 0.f;
             bool ok = true;
             for (int j = 0; j < nt && ok; ++j) {
@@ -260,6 +265,13 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 if (!ok) break;
                 tc_fence_after();
                 if ((warp & 3) == 0 && lane == 0) TRACE(j, 9 + 8 * i);
+                if (!warp_has_rows) {
+                    // all 32 rows of this warp are padding past B: their P rows may hold anything (rows of
+                    // the MMA are independent and these output rows are never stored); just keep in step
+                    tc_fence_before();
+                    mbar_arrive(&bar->p_ready[i][buf]);
+                    continue;
+                }
                 const uint32_t s_addr = tmem_base + ((uint32_t)lg << 16) + (uint32_t)((2 * i + buf) * 64);
                 uint32_t sr[2][32];
                 tmem_ld32(s_addr, sr[0]);
@@ -347,7 +359,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 p.lse_part[((int64_t)slot * p.B + b) * p.H + h] = -INFINITY;
             }
         }
-#endif
     } else if (warp >= 4) {
         // empty split: every slot this CTA owns gets weight zero in the combine
         const int i = (warp - 4) >> 2;
