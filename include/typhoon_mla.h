@@ -22,7 +22,8 @@
  *   - Tensors are bf16 (raw uint16 storage) unless stated; accumulation,
  *     softmax statistics, split partials and the combine are fp32.
  *   - q_pe and all cached rope keys arrive already rotated: no RoPE is applied.
- *   - softmax_scale multiplies the sum of the nope and the rope logits.
+ *   - softmax_scale multiplies the sum of the nope and the rope logits; it must be
+ *     positive and finite.
  *   - Log-sum-exps are natural logarithms of sum(exp(scaled logit)).
  *   - A single decode query attends to every cached token (no mask).
  *   - Every call returns a status (0 = OK); nothing throws, aborts or traps.

@@ -83,7 +83,8 @@ constexpr int kNumSM = 148;
 // candidate split counts (one CTA per SM; the fixed cost is the Q load and pipeline fill).
 int naive_splits_sm100(int B, int H, int64_t Ls) {
     if (Ls <= 0) return 0;
-    const int n_tiles = (int)((Ls + 63) / 64);
+    const int tile_tok = naive_sm100_tile_tokens(B);
+    const int n_tiles = (int)((Ls + tile_tok - 1) / tile_tok);
     if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_SPLITS")) {   // tuning aid
         const int v = std::atoi(ov);
         if (v >= 1) {
@@ -430,7 +431,7 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (mode < TYPHOON_MLA_MODE_AUTO || mode > TYPHOON_MLA_MODE_NAIVE) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (!(softmax_scale == softmax_scale)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return TYPHOON_MLA_ERR_INVALID_ARG;   // positive, finite
     mode = resolve_mode(sh, B, max_pages, mode);
     const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
     if (use_absorb && max_pages > 0) {

@@ -64,6 +64,7 @@ struct NaiveAttnSm100 {
     int* status;     // device word, set non-zero if a bounded wait expired
 };
 int naive_sm100_slots(int B, int n_split);
+int naive_sm100_tile_tokens(int B);   // KV tile width the kernel uses for this batch size (64 or 128)
 cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s);
 cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const void* v_t, int H, int64_t Ls_pad,
                                    CUtensorMap* tm_kn, CUtensorMap* tm_kp, CUtensorMap* tm_vt);
