@@ -51,6 +51,7 @@ struct AbsorbSm100Params {
     int page_size, max_pages;
     const int32_t* block_table;
     const int32_t* seq_lens;
+    const int32_t* order;
     float scale_log2;
     float* o_part;     // [n_chunks][B][H][512]
     float* lse_part;   // [n_chunks][B][H]
@@ -95,7 +96,8 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     if (threadIdx.x == 0) TRACE(0, 28);
-    const int chunk = blockIdx.x, h0 = blockIdx.y * 64, b = blockIdx.z;
+    const int chunk = blockIdx.x, h0 = blockIdx.y * 64;
+    const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
 
     // token range of this chunk
     const bool shared_seg = chunk < p.n_shared_chunks;
@@ -116,10 +118,10 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     const CUtensorMap* tk = shared_seg ? &tm_kpe_sh : &tm_kpe_pg;
     const int32_t* bt = p.block_table + (int64_t)b * p.max_pages;
     const uint32_t ld0 = (warp == 0 && elect_one()) ? 1u : 0u;
-    auto issue_tile = [&](int j) {
-        const int s = j & 1;
+    // physical page and slot of tile j (the block-table read is issued ahead of the wait for a free
+    // ring slot so that its latency is off the critical path)
+    auto page_of = [&](int j, int& page, int& slot) {
         const int t0 = tok_begin + j * TOK;
-        int page, slot;
         if (shared_seg) {
             page = t0 / TOK;
             slot = 0;
@@ -127,6 +129,9 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             page = __shfl_sync(0xffffffffu, bt[t0 / p.page_size], 0);
             slot = t0 % p.page_size;
         }
+    };
+    auto issue_tile = [&](int j, int page, int slot) {
+        const int s = j & 1;
         uint8_t* dst = sKV + s * TILE_BYTES;
         TRACE(j, 0);
         mbar_arrive_expect_tx_if(ld0, &sh->kv_full[s], TILE_BYTES);
@@ -155,7 +160,11 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 #pragma unroll 1
             for (int s = 0; s < 8; ++s) tma_load_3d_if(ld0, sQ + s * SLAB_BYTES, &tm_qa, &sh->q_full, s * 64, h0, b);
             tma_load_3d_if(ld0, sQ + 8 * SLAB_BYTES, &tm_qp, &sh->q_full, 0, h0, b);
-            for (int j = 0; j < min(n_tiles, STAGES); ++j) issue_tile(j);
+            for (int j = 0; j < min(n_tiles, STAGES); ++j) {
+                int page, slot;
+                page_of(j, page, slot);
+                issue_tile(j, page, slot);
+            }
         }
     }
     if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
@@ -168,8 +177,10 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
         if (warp == 0) {
             // ---------------- producer: the rest of the KV ring (Q and the first tiles are already in flight)
             for (int j = STAGES; j < n_tiles; ++j) {
+                int page, slot;
+                page_of(j, page, slot);
                 if (!mbar_wait_warp(&sh->kv_empty[j & 1], ((j >> 1) & 1) ^ 1, abort_flag)) break;
-                issue_tile(j);
+                issue_tile(j, page, slot);
             }
         } else if (warp == 1) {
             // ---------------- S^T = KV_tile * Q^T issuer (M = 64 tokens, N = 64 heads, K = 576)
@@ -242,6 +253,9 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             volatile float* mref = sh->mref[cg];
             if (q == 0) mref[lane] = -INFINITY;
             wg_sync(bar_id);
+            float neg_mr[32];      // register copy of -m_ref, refreshed after every rescale event
+#pragma unroll
+            for (int c = 0; c < 32; ++c) neg_mr[c] = INFINITY;
 
             for (int j = 0; j < n_tiles; ++j) {
                 const int s = j & 1;
@@ -256,15 +270,17 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     tc_fence_after();
                     tmem_ld32(tmem_base + lane_base + (uint32_t)(s * 64 + cg * 32), sr);
                     tmem_ld_wait();
-                    // one pass: scaled logit, distance to the reference, probability (speculative: final
-                    // unless the warpgroup votes for a rescale)
+                    // one pass: distance of the scaled logit to the reference (one FMA), probability
+                    // (speculative: final unless the warpgroup votes for a rescale).  Lanes without a valid
+                    // token carry -inf.
+                    if (!valid) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) sr[c] = 0xff800000u;
+                    }
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        const float v0 = valid ? __uint_as_float(sr[2 * c]) * p.scale_log2 : -INFINITY;
-                        const float v1 = valid ? __uint_as_float(sr[2 * c + 1]) * p.scale_log2 : -INFINITY;
-                        sr[2 * c] = __float_as_uint(v0);
-                        sr[2 * c + 1] = __float_as_uint(v1);
-                        const float d0 = v0 - mref[2 * c], d1 = v1 - mref[2 * c + 1];
+                        const float d0 = fmaf(__uint_as_float(sr[2 * c]), p.scale_log2, neg_mr[2 * c]);
+                        const float d1 = fmaf(__uint_as_float(sr[2 * c + 1]), p.scale_log2, neg_mr[2 * c + 1]);
                         exceed |= (d0 > kRescaleThreshold) | (d1 > kRescaleThreshold);
                         pk[c] = pack_bf16(fast_exp2(d0), fast_exp2(d1));
                     }
@@ -278,7 +294,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     // order-preserving keys, then across the four warps through shared memory
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        const int bits = (int)sr[c];
+                        const int bits = __float_as_int(__uint_as_float(sr[c]) * p.scale_log2);
                         const int key = bits >= 0 ? bits : bits ^ 0x7fffffff;
                         const int mk = __reduce_max_sync(0xffffffffu, key);
                         if (lane == c) sh->red[cg][q][c] = __int_as_float(mk >= 0 ? mk : mk ^ 0x7fffffff);
@@ -314,9 +330,11 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     }
                     // probabilities again, against the new references
 #pragma unroll
+                    for (int c = 0; c < 32; ++c) neg_mr[c] = -mref[c];
+#pragma unroll
                     for (int c = 0; c < 16; ++c)
-                        pk[c] = pack_bf16(fast_exp2(__uint_as_float(sr[2 * c]) - mref[2 * c]),
-                                          fast_exp2(__uint_as_float(sr[2 * c + 1]) - mref[2 * c + 1]));
+                        pk[c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(sr[2 * c]), p.scale_log2, neg_mr[2 * c])),
+                                          fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), p.scale_log2, neg_mr[2 * c + 1])));
                 }
                 if (warp == 4) TRACE(j, 11);
                 // per-thread partial row sums (of the bf16-rounded values), P^T row into the rope slab
@@ -495,7 +513,7 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     p.chunk = a.chunk; p.n_shared_chunks = a.n_shared_chunks; p.n_suffix_chunks = a.n_suffix_chunks;
     p.Ls_absorb = a.Ls_absorb;
     p.page_size = a.page_size; p.max_pages = a.max_pages;
-    p.block_table = a.block_table; p.seq_lens = a.seq_lens;
+    p.block_table = a.block_table; p.seq_lens = a.seq_lens; p.order = a.order;
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = status;
     p.o_lat_direct = n_chunks == 1 ? reinterpret_cast<__nv_bfloat16*>(o_lat_direct) : nullptr;

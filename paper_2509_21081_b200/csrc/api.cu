@@ -74,7 +74,7 @@ struct Plan {
     int n_shared_chunks;     // absorb chunks over the shared prefix (ABSORB mode)
     int n_suffix_chunks;
     // byte offsets into the workspace
-    size_t off_qabs, off_opart_a, off_lsepart_a, off_olat, off_lse_a, off_oabs, off_opart_n, off_lsepart_n, total;
+    size_t off_order, off_qabs, off_opart_a, off_lsepart_a, off_olat, off_lse_a, off_oabs, off_opart_n, off_lsepart_n, total;
 };
 
 constexpr int kNumSM = 148;
@@ -132,7 +132,10 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
             const int64_t ch = round_up((longest + parts - 1) / parts, 64);
             const int64_t ctas = (int64_t)units * ((Ls_absorb + ch - 1) / ch + (cap_suffix + ch - 1) / ch);
             const int64_t waves = (ctas + kNumSM - 1) / kNumSM;
-            const double cost = (double)waves * ((double)ch / 64.0 + fixed);
+            // a split segment writes and re-reads fp32 partials (64 heads x 2 KB, both ways): about 3.5 tiles
+            // worth of traffic per chunk
+            const double split_cost = (ctas > units) ? 3.5 : 0.0;
+            const double cost = (double)waves * ((double)ch / 64.0 + fixed + split_cost);
             if (cost < best_cost - 1e-9) {
                 best_cost = cost;
                 c = ch;
@@ -170,6 +173,7 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
         off += round_up((int64_t)bytes, 256);
         return o;
     };
+    p.off_order = take((size_t)B * 4);
     p.off_qabs = take(BH * 512 * 2);
     p.off_opart_a = take((size_t)n_chunks * BH * 512 * 4);
     p.off_lsepart_a = take((size_t)n_chunks * BH * 4);
@@ -506,9 +510,17 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         float* o_part_a = reinterpret_cast<float*>(ws + pl.off_opart_a);
         float* lse_part_a = reinterpret_cast<float*>(ws + pl.off_lsepart_a);
         void* o_lat = ws + pl.off_olat;
+        // ragged suffixes: launch the longest requests first (order computed on the device, no host sync)
+        int32_t* order = nullptr;
+        if (pl.n_suffix_chunks > 0 && B > 1 && B <= 4096) {
+            order = reinterpret_cast<int32_t*>(ws + pl.off_order);
+            e = launch_order_by_length(seq_lens, B, order, s);
+            if (e != cudaSuccess) return cuda_fail(e);
+            ++launches;
+        }
         AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
                       ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
-                      seq_lens, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
+                      seq_lens, order, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
                       o_part_a, lse_part_a};
         prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         e = tc ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, o_lat, lse_a, sh->status, s)

@@ -219,7 +219,8 @@ __global__ void __launch_bounds__(256) absorb_attn_mma_kernel(AbsorbAttn p) {
     __nv_bfloat16* sQ = smem;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = warp & 3, chalf = warp >> 2;
-    const int chunk = blockIdx.x, h0 = blockIdx.y * AB_ROWS, b = blockIdx.z;
+    const int chunk = blockIdx.x, h0 = blockIdx.y * AB_ROWS;
+    const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
     const int n_chunks = p.n_shared_chunks + p.n_suffix_chunks;
 
     // token range of this chunk

@@ -76,6 +76,7 @@ struct AbsorbAttn {
     const void* ckv_pages; const void* kpe_pages;
     int64_t ckv_stride, kpe_stride; int page_size;
     const int32_t* block_table; int max_pages; const int32_t* seq_lens;
+    const int32_t* order;                          // optional [B]: request handled by block z (longest first)
     int B, H; int chunk;                           // tokens per chunk
     int n_shared_chunks, n_suffix_chunks;
     float scale;
@@ -92,6 +93,9 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
                                      void* o_lat_direct, float* lse_direct, int* status, cudaStream_t s);
 cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t Ls_pad, CUtensorMap* tm_ckv,
                                      CUtensorMap* tm_kpe);
+
+// perm[0..B) = request indices by descending suffix length (B <= 4096).
+cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm, cudaStream_t s);
 
 // Merge absorb chunk partials -> bf16 latent output [B,H,512] + lse [B,H].
 cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,
