@@ -31,7 +31,11 @@ UNIT = "queries/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (key: (config, kernel)); None where no capture exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("cfg1", "naive_attn"): 276_514_816,     # profiles/naive_attn_sm100_cfg1_and_cfg4_b512.md
+    ("cfg3", "absorb_attn"): 652_168_192,    # profiles/absorb_attn_sm100_cfg3.md
+    ("cfg4_B512", "naive_attn"): 1_226_916_040,
+}
 
 
 def _peaks():
@@ -276,6 +280,20 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     flops, bytes_ = algorithmic_work(cfg, inp.suffix_lens, mode_name)
     t_lb = max(flops / (pk["bf16_tflops"] * 1e12), bytes_ / (pk["hbm_gbs"] * 1e9))
     roof["step_frac_of_combined_roofline"] = t_lb / (ms_per_step * 1e-3)
+    # The same kernel with the side stream switched off (every kernel alone on the GPU), outside the
+    # timed region: what the kernel reaches when it does not share the machine.
+    b.typhoon_mla_set_overlap(False)
+    n_alone = max(5, min(K, 50))
+    for i in range(3):
+        step(i)
+    b.typhoon_mla_profile_begin(kid, n_alone)
+    for i in range(n_alone):
+        step(i)
+    a_ms, a_n = b.typhoon_mla_profile_end()
+    b.typhoon_mla_set_overlap(True)
+    a_s = (a_ms / max(a_n, 1)) * 1e-3
+    alone = (k_bytes / a_s / 1e9) if roof["bound"] == "hbm" else (k_flops / a_s / 1e12)
+    roof.update({"kernel_ms_alone": a_s * 1e3, "achieved_alone": alone, "frac_alone": alone / roof["peak"]})
 
     # ---- end to end: per-step tensors from pinned host memory, result read back, every step
     e2e = None

@@ -217,6 +217,11 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
 enum { TYPHOON_MLA_PATH_TCGEN05 = 0, TYPHOON_MLA_PATH_WARP_MMA = 1 };
 int typhoon_mla_set_kernel_path(int32_t path);
 
+/* In a hybrid step the absorb branch (Algorithm 1 lines 5-6) runs on a stream owned by the handle,
+ * beside the naive kernel (line 4), and is joined before the projection (default).  0 keeps every
+ * kernel on the caller's stream, one after the other (measurement aid).  Process-wide. */
+int typhoon_mla_set_overlap(int32_t enable);
+
 /* Synchronises `stream` and reads the handle's device status word.  Every in-kernel wait of the
  * tcgen05 kernels has a deadline; if one expired, the kernel abandoned its work, the word is
  * non-zero and this returns TYPHOON_MLA_ERR_DEVICE_CHECK (results of that launch are invalid). */

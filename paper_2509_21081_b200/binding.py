@@ -78,6 +78,8 @@ def _load():
     lib.typhoon_mla_shared_export.argtypes = [vp, vp, vp, vp]
     lib.typhoon_mla_set_kernel_path.restype = C.c_int
     lib.typhoon_mla_set_kernel_path.argtypes = [i32]
+    lib.typhoon_mla_set_overlap.restype = C.c_int
+    lib.typhoon_mla_set_overlap.argtypes = [i32]
     lib.typhoon_mla_device_status.restype = C.c_int
     lib.typhoon_mla_device_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.typhoon_mla_naive_shared_noalloc.restype = C.c_int
@@ -269,3 +271,7 @@ def typhoon_mla_device_status(shared: SharedPrefix) -> int:
     v = C.c_int32()
     _check(_lib.typhoon_mla_device_status(shared.handle, _stream(), C.byref(v)), "typhoon_mla_device_status")
     return v.value
+
+
+def typhoon_mla_set_overlap(enable: bool) -> None:
+    _check(_lib.typhoon_mla_set_overlap(1 if enable else 0), "typhoon_mla_set_overlap")

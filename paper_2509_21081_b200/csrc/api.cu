@@ -41,7 +41,7 @@ inline void prof_after(int id, cudaStream_t s) {
 int g_kernel_path = TYPHOON_MLA_PATH_TCGEN05;
 // Run the absorb branch of a hybrid step on a side stream next to the naive kernel (tuning aid:
 // TYPHOON_MLA_OVERLAP=0 in the environment keeps everything on the caller's stream).
-const bool g_overlap = [] {
+bool g_overlap = [] {
     const char* v = std::getenv("TYPHOON_MLA_OVERLAP");
     return !(v && v[0] == '0');
 }();
@@ -381,6 +381,11 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* sh, const void** k_nope,
     if (Ls) *Ls = sh->Ls;
     if (Ls_padded) *Ls_padded = sh->Ls_pad;
     if (owned_bytes) *owned_bytes = (int64_t)sh->owned_bytes;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_set_overlap(int32_t enable) {
+    g_overlap = enable != 0;
     return TYPHOON_MLA_OK;
 }
 
