@@ -85,6 +85,27 @@ def dominant_kernel(cfg, suffix_lens, mode_name):
     return 2, "absorb_attn", absorb_bytes, absorb_flops
 
 
+# ------------------------------------------------------------------ multi-rank helpers (no data-path collective)
+def rank_config(cfg, rank):
+    """Each rank serves its own requests: same prefix and weights (same seed for the shared draws would need
+    the same generator, so the whole problem is re-drawn with a rank-shifted seed); rank 0 keeps the config."""
+    return cfg if rank == 0 else dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+
+
+def max_over_ranks(ms, world, device):
+    """Timing of a multi-rank run is the slowest rank's (MAX all-reduce); the only collective in the bench."""
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(per_rank_batch, world, ms_per_step):
+    """queries/s of the whole job: every rank processes `per_rank_batch` queries per step (weak scaling)."""
+    return world * per_rank_batch / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
@@ -209,7 +230,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
 
     dev = "cuda"
     # Each rank draws its own requests (seed shifted by rank); the prefix and weights are replicated.
-    rcfg = cfg if rank == 0 else dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+    rcfg = rank_config(cfg, rank)
     inp = I.make_inputs(rcfg)
     pc = I.build_pages(inp, poison=False)
     max_pages = pc.block_table.shape[1]
@@ -254,12 +275,9 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         barrier()
     total_ms = ev0.elapsed_time(ev1)
     k_ms, k_n = b.typhoon_mla_profile_end()
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / K
-    value = world * cfg.B / (ms_per_step * 1e-3)
+    value = whole_job_value(cfg.B, world, ms_per_step)
 
     # ---- roofline of the dominant kernel
     pk = _peaks()
@@ -301,26 +319,43 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         hq = [(inp.q_nope.pin_memory(), inp.q_pe.pin_memory(), pc.block_table.pin_memory(), pc.seq_lens.pin_memory(),
                torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16).pin_memory()) for _ in range(n_sets)]
 
-        def step_host(i):
-            s, h = sets[i % n_sets], hq[i % n_sets]
-            s["dec"].decode_host(h[0], h[1], s["ckv"], s["kpe"], h[2], h[3], h[4], mode=mode)
+        # Two steps are kept in flight, each on its own stream with its own decoder (workspace, staging,
+        # pinned buffers), so that the copies of one step overlap the kernels of the other, as a serving
+        # loop would do.  Every step still copies its inputs in and its result out.
+        streams = [torch.cuda.Stream() for _ in range(n_sets)]
 
+        def step_host(i):
+            k = i % n_sets
+            s, h = sets[k], hq[k]
+            with torch.cuda.stream(streams[k]):
+                s["dec"].decode_host(h[0], h[1], s["ckv"], s["kpe"], h[2], h[3], h[4], mode=mode)
+
+        def fork():
+            for st in streams:
+                st.wait_stream(torch.cuda.current_stream())
+
+        def join():
+            for st in streams:
+                torch.cuda.current_stream().wait_stream(st)
+
+        fork()
         for i in range(W):
             step_host(i)
+        join()
         barrier()
         ev0.record()
+        fork()
         for i in range(K):
             step_host(i)
+        join()
         ev1.record()
         barrier()
-        t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e_ms = float(t.item()) / K
+        e_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / K
         h2d = inp.q_nope.numel() * 2 + inp.q_pe.numel() * 2 + pc.block_table.numel() * 4 + pc.seq_lens.numel() * 4
         d2h = cfg.B * cfg.H * 128 * 2
-        e2e = {"value": world * cfg.B / (e_ms * 1e-3), "unit": UNIT, "ms_per_step": e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        e2e = {"value": whole_job_value(cfg.B, world, e_ms), "unit": UNIT, "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "pipelining": f"{n_sets} steps in flight on {n_sets} streams (own workspace, staging and pinned buffers each)"}
 
     cpu = None
     if with_cpu and rank == 0 and world == 1:

@@ -262,6 +262,10 @@ int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* shared,
                                      const void* q_nope, const void* q_pe, int32_t B,
                                      float softmax_scale, void* out, float* lse_out, void* stream);
 
+/* Longest-first order used for ragged suffixes: perm[0..B) (device, int32) = request indices sorted
+ * by descending seq_lens (device, int32), ties by ascending index.  B <= 4096.  Exposed for tests. */
+int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* perm, void* stream);
+
 /* Kernel kinds of the decode step, in launch order (Algorithm 1 lines 4-8). */
 enum {
     TYPHOON_MLA_KERNEL_NAIVE_ATTN = 0,  /* line 4 */

@@ -78,6 +78,8 @@ def _load():
     lib.typhoon_mla_shared_export.argtypes = [vp, vp, vp, vp]
     lib.typhoon_mla_set_kernel_path.restype = C.c_int
     lib.typhoon_mla_set_kernel_path.argtypes = [i32]
+    lib.typhoon_mla_order_by_length.restype = C.c_int
+    lib.typhoon_mla_order_by_length.argtypes = [vp, i32, vp, vp]
     lib.typhoon_mla_set_overlap.restype = C.c_int
     lib.typhoon_mla_set_overlap.argtypes = [i32]
     lib.typhoon_mla_device_status.restype = C.c_int
@@ -275,3 +277,10 @@ def typhoon_mla_device_status(shared: SharedPrefix) -> int:
 
 def typhoon_mla_set_overlap(enable: bool) -> None:
     _check(_lib.typhoon_mla_set_overlap(1 if enable else 0), "typhoon_mla_set_overlap")
+
+
+def typhoon_mla_order_by_length(seq_lens: torch.Tensor) -> torch.Tensor:
+    perm = torch.empty_like(seq_lens)
+    _check(_lib.typhoon_mla_order_by_length(_ptr(seq_lens), seq_lens.numel(), _ptr(perm), _stream()),
+           "typhoon_mla_order_by_length")
+    return perm

@@ -384,6 +384,12 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* sh, const void** k_nope,
     return TYPHOON_MLA_OK;
 }
 
+int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* perm, void* stream) {
+    if (!seq_lens || !perm || B < 1 || B > 4096) return TYPHOON_MLA_ERR_INVALID_ARG;
+    cudaError_t e = launch_order_by_length(seq_lens, B, perm, reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
+}
+
 int typhoon_mla_set_overlap(int32_t enable) {
     g_overlap = enable != 0;
     return TYPHOON_MLA_OK;

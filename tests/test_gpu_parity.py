@@ -242,6 +242,17 @@ def test_invalid_arguments():
     sh.free()
 
 
+def test_order_by_length_is_a_stable_descending_sort():
+    """Index work: bit-exact against numpy (descending length, ties by ascending index)."""
+    from paper_2509_21081_b200 import binding as b
+    rng = np.random.default_rng(3)
+    for B in (1, 2, 5, 64, 257, 1000, 4096):
+        lens = rng.integers(0, 40, size=B).astype(np.int32)        # many ties
+        perm = b.typhoon_mla_order_by_length(torch.from_numpy(lens).cuda()).cpu().numpy()
+        ref = np.lexsort((np.arange(B), -lens.astype(np.int64)))
+        assert np.array_equal(perm, ref), f"B={B}"
+
+
 # ------------------------------------------------------------ full-size configs
 def _sampled_pairs(cfg, n, seed):
     r = np.random.default_rng(seed)
