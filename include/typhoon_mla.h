@@ -195,6 +195,11 @@ int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims /* host */, int64
  * Process-wide; not thread-safe against concurrent decode calls. */
 int typhoon_mla_set_hw_model(double tensor_flops, double hbm_bytes_per_s, double hybrid_fixed_s);
 
+/* Fraction of `tensor_flops` the absorb formulation reaches over the shared prefix in this
+ * implementation (default 0.5, calibrated on B200; 1.0 gives the paper's zero-overhead rule of Eq. 1).
+ * Values outside (0, 1] restore the default. */
+int typhoon_mla_set_absorb_efficiency(double fraction);
+
 /* Eq. 1: B_theta = (D_qk + D_v) / (S_q (2 D_l + D_r)) * T / M.  Host, pure. */
 double typhoon_mla_batch_threshold(const typhoon_mla_dims_t* dims /* host */, int32_t S_q, double T, double M);
 

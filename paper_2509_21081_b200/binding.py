@@ -67,6 +67,8 @@ def _load():
     lib.typhoon_mla_choose_mode_for.argtypes = [C.POINTER(Dims), i64, i32, i64]
     lib.typhoon_mla_set_hw_model.restype = C.c_int
     lib.typhoon_mla_set_hw_model.argtypes = [f64, f64, f64]
+    lib.typhoon_mla_set_absorb_efficiency.restype = C.c_int
+    lib.typhoon_mla_set_absorb_efficiency.argtypes = [f64]
     lib.typhoon_mla_batch_threshold.restype = f64
     lib.typhoon_mla_batch_threshold.argtypes = [C.POINTER(Dims), i32, f64, f64]
     lib.typhoon_mla_cost_model.restype = C.c_int
@@ -284,3 +286,7 @@ def typhoon_mla_order_by_length(seq_lens: torch.Tensor) -> torch.Tensor:
     _check(_lib.typhoon_mla_order_by_length(_ptr(seq_lens), seq_lens.numel(), _ptr(perm), _stream()),
            "typhoon_mla_order_by_length")
     return perm
+
+
+def typhoon_mla_set_absorb_efficiency(fraction: float) -> None:
+    _check(_lib.typhoon_mla_set_absorb_efficiency(fraction), "typhoon_mla_set_absorb_efficiency")

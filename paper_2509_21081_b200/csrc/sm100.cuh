@@ -55,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
-// Warp-collective form: all 32 lanes poll, the verdict is made warp-uniform.  Role warps run
+// Warp-collective form: all 32 lanes poll, the result is made warp-uniform.  Role warps run
 // their loops with all lanes (uniform control flow lets the compiler keep descriptors, addresses
 // and coordinates in uniform registers) and elect one lane only for the issuing instruction.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {

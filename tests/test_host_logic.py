@@ -79,6 +79,7 @@ def test_crossover_rule(b):
     # zero fixed cost and the paper's NPU numbers: the switch happens where Eq. 1 says, up to the
     # rope keys being read once per token instead of once per head (256.5 vs 320 words per head-token)
     b.typhoon_mla_set_hw_model(376e12, 1.8e12, 0.0)
+    b.typhoon_mla_set_absorb_efficiency(1.0)
     modes = [b.typhoon_mla_choose_mode_for(d, 4096, B) for B in range(1, 200)]
     first_hybrid = modes.index(b.MODE_HYBRID) + 1
     assert all(m == b.MODE_ABSORB for m in modes[: first_hybrid - 1])
@@ -92,10 +93,17 @@ def test_crossover_rule(b):
     # empty suffixes -> naive only; no prefix -> absorb
     assert b.typhoon_mla_choose_mode_for(d, 4096, 8, 0) == b.MODE_NAIVE
     assert b.typhoon_mla_choose_mode_for(d, 0, 512) == b.MODE_ABSORB
+    # a less efficient absorb kernel lowers the threshold in proportion
+    b.typhoon_mla_set_hw_model(376e12, 1.8e12, 0.0)
+    b.typhoon_mla_set_absorb_efficiency(0.5)
+    modes = [b.typhoon_mla_choose_mode_for(d, 4096, B) for B in range(1, 200)]
+    assert abs((modes.index(b.MODE_HYBRID) + 1) - first_hybrid / 2) <= 1
     b.typhoon_mla_set_hw_model(0, 0, -1)   # restore defaults
+    b.typhoon_mla_set_absorb_efficiency(0)
     # defaults (B200): tiny batches fall back, large batches go hybrid
     assert b.typhoon_mla_choose_mode_for(d, 16384, 1) == b.MODE_ABSORB
     assert b.typhoon_mla_choose_mode_for(d, 16384, 8) == b.MODE_ABSORB
+    assert b.typhoon_mla_choose_mode_for(d, 16384, 32) == b.MODE_HYBRID
     assert b.typhoon_mla_choose_mode_for(d, 16384, 512) == b.MODE_HYBRID
 
 
