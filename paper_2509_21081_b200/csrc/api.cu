@@ -512,15 +512,23 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     bool combined = false;
     if (forked) s = sh->side_stream;
     if (have_absorb) {
+        // ragged suffixes: the longest requests are launched first (order computed on the device, no host
+        // sync): by an extra block of the query-absorption kernel on the tcgen05 path, by its own kernel otherwise
+        int32_t* order = nullptr;
+        if (pl.n_suffix_chunks > 0 && B > 1 && B <= 4096) order = reinterpret_cast<int32_t*>(ws + pl.off_order);
         // --- query absorption Q_A = Q_N W_UK (Algorithm 1 line 5)
         void* q_abs = ws + pl.off_qabs;
         prof_before(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (tc) {
-            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->status, s);
+            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->status, order ? seq_lens : nullptr, order, s);
         } else {
             GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,
                       B, 512, 128, H, false};
             e = launch_gemm_tn(g1, s);
+            if (e == cudaSuccess && order) {
+                e = launch_order_by_length(seq_lens, B, order, s);
+                ++launches;
+            }
         }
         prof_after(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (e != cudaSuccess) return cuda_fail(e);
@@ -529,14 +537,6 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         float* o_part_a = reinterpret_cast<float*>(ws + pl.off_opart_a);
         float* lse_part_a = reinterpret_cast<float*>(ws + pl.off_lsepart_a);
         void* o_lat = ws + pl.off_olat;
-        // ragged suffixes: launch the longest requests first (order computed on the device, no host sync)
-        int32_t* order = nullptr;
-        if (pl.n_suffix_chunks > 0 && B > 1 && B <= 4096) {
-            order = reinterpret_cast<int32_t*>(ws + pl.off_order);
-            e = launch_order_by_length(seq_lens, B, order, s);
-            if (e != cudaSuccess) return cuda_fail(e);
-            ++launches;
-        }
         AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
                       ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
                       seq_lens, order, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,

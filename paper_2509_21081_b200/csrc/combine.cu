@@ -109,27 +109,7 @@ __global__ void __launch_bounds__(256) copy_pad_rows_kernel(const __nv_bfloat16*
 __global__ void __launch_bounds__(1024) order_by_length_kernel(const int32_t* __restrict__ seq_lens, int B,
                                                                int32_t* __restrict__ perm) {
     __shared__ unsigned long long keys[4096];
-    int n = 1;
-    while (n < B) n <<= 1;
-    for (int i = threadIdx.x; i < n; i += 1024) {
-        // descending length, ascending index: sort ascending on (~len, index)
-        unsigned long long k = ~0ull;
-        if (i < B) k = ((unsigned long long)(0x7fffffffu - (unsigned)max(seq_lens[i], 0)) << 32) | (unsigned)i;
-        keys[i] = k;
-    }
-    __syncthreads();
-    for (int size = 2; size <= n; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int i = threadIdx.x; i < n / 2; i += 1024) {
-                const int lo = (i / stride) * 2 * stride + (i % stride), hi = lo + stride;
-                const bool up = ((lo & size) == 0);
-                const unsigned long long a = keys[lo], b = keys[hi];
-                if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
-            }
-            __syncthreads();
-        }
-    }
-    for (int i = threadIdx.x; i < B; i += 1024) perm[i] = (int32_t)(keys[i] & 0xffffffffu);
+    block_order_by_length(seq_lens, B, perm, keys);
 }
 
 }  // namespace

@@ -57,4 +57,32 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Block-wide sort used for the longest-first launch order of ragged suffixes: perm[] = request
+// indices by descending length, ties by ascending index.  `keys` is shared memory for the next
+// power of two >= B (<= 4096) 64-bit keys.  Called by every thread of the block.
+__device__ __forceinline__ void block_order_by_length(const int32_t* __restrict__ seq_lens, int B,
+                                                      int32_t* __restrict__ perm, unsigned long long* keys) {
+    const int nt = blockDim.x, tid = threadIdx.x;
+    int n = 1;
+    while (n < B) n <<= 1;
+    for (int i = tid; i < n; i += nt) {
+        unsigned long long k = ~0ull;   // padding sorts last
+        if (i < B) k = ((unsigned long long)(0x7fffffffu - (unsigned)max(seq_lens[i], 0)) << 32) | (unsigned)i;
+        keys[i] = k;
+    }
+    __syncthreads();
+    for (int size = 2; size <= n; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = tid; i < n / 2; i += nt) {
+                const int lo = (i / stride) * 2 * stride + (i % stride), hi = lo + stride;
+                const bool up = ((lo & size) == 0);
+                const unsigned long long a = keys[lo], b = keys[hi];
+                if ((a > b) == up) { keys[lo] = b; keys[hi] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = tid; i < B; i += nt) perm[i] = (int32_t)(keys[i] & 0xffffffffu);
+}
+
 }  // namespace tmla

@@ -38,8 +38,9 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, c
 
 // Query absorption on tcgen05 (one CTA per head and 128 requests); tm_w from make_q_absorb_tmap.
 cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w);
+// With seq_lens and order given (B <= 4096) one extra block also writes the longest-first request order.
 cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int* status,
-                                  cudaStream_t s);
+                                  const int32_t* seq_lens, int32_t* order, cudaStream_t s);
 
 // Naive shared-prefix attention partials (Algorithm 1 line 4).
 struct NaiveAttn {

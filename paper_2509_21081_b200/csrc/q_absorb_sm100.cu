@@ -24,12 +24,20 @@ struct QAbsorbParams {
     void* q_abs;   // bf16 [B, H, 512]
     int B, H;
     int* status;
+    // optional: one extra block (blockIdx.y == H) computes the longest-first request order that the
+    // absorb attention kernel launched next uses, saving a launch on the absorb branch
+    const int32_t* seq_lens;
+    int32_t* order;
 };
 
 __global__ void __launch_bounds__(192, 1)
 q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w, QAbsorbParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    if ((int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
+        if (blockIdx.x == 0) block_order_by_length(p.seq_lens, p.B, p.order, reinterpret_cast<unsigned long long*>(smem));
+        return;
+    }
     uint8_t* sA = smem;
     uint8_t* sW = smem + A_BYTES;
     uint64_t* full = reinterpret_cast<uint64_t*>(sW + W_BYTES);   // [0..3]: q + weight tile n ; [4]: accumulators done
@@ -126,7 +134,7 @@ cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w) {
 }
 
 cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int* status,
-                                  cudaStream_t s) {
+                                  const int32_t* seq_lens, int32_t* order, cudaStream_t s) {
     if (B <= 0) return cudaSuccess;
     CUtensorMap tm_q;
     uint64_t dims[3] = {128, (uint64_t)H, (uint64_t)B};
@@ -134,9 +142,10 @@ cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, v
     uint32_t box[3] = {64, 1, 128};
     cudaError_t e = make_tmap_bf16(&tm_q, q_nope, 3, dims, str, box);
     if (e != cudaSuccess) return e;
-    QAbsorbParams p{q_abs, B, H, status};
+    const bool with_order = seq_lens != nullptr && order != nullptr && B <= 4096;
+    QAbsorbParams p{q_abs, B, H, status, seq_lens, order};
     cudaFuncSetAttribute(q_absorb_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    dim3 grid((B + 127) / 128, H, 1);
+    dim3 grid((B + 127) / 128, H + (with_order ? 1 : 0), 1);
     q_absorb_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tm_q, *tm_w, p);
     return cudaGetLastError();
 }

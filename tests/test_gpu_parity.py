@@ -242,6 +242,29 @@ def test_invalid_arguments():
     sh.free()
 
 
+def test_fused_page_layout_and_strides():
+    """Latent and rope keys interleaved in one 576-wide page array, passed through the token strides."""
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    cfg = _cfg("fused", B=5, H=32, Ls=200, lo=1, hi=300, seed=34)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    pc = I.build_pages(inp)
+    fused = torch.cat([pc.ckv_pages, pc.kpe_pages], dim=-1).contiguous().cuda()     # [P, 64, 576]
+    ckv_view, kpe_view = fused[..., :512], fused[..., 512:]
+    assert ckv_view.stride(-2) == 576 and kpe_view.data_ptr() == fused.data_ptr() + 1024
+    dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(),
+                            inp.scale, cfg.B, pc.block_table.shape[1])
+    for mode in (HYBRID, ABSORB):
+        lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
+        out = dec.decode(inp.q_nope.cuda(), inp.q_pe.cuda(), ckv_view, kpe_view, pc.block_table.cuda(),
+                         pc.seq_lens.cuda(), mode=mode, lse_out=lse)
+        assert b.typhoon_mla_device_status(dec.shared) == 0
+        G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse,
+                        what=f"fused layout mode {mode}")
+    dec.close()
+
+
 def test_order_by_length_is_a_stable_descending_sort():
     """Index work: bit-exact against numpy (descending length, ties by ascending index)."""
     from paper_2509_21081_b200 import binding as b
