@@ -88,63 +88,69 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
         }
         if (ok) umma_commit_if(ld, acc_full);
     } else {
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag));
-        tc_fence_after();
-        if (ok) {
-            const int lg = (warp & 3) * 32;
-            const int row = m0 + lg + lane;
-            if (p.out_mode == 2) {
-                // The accumulator row is the absorb-side output O_A[b, h, :] (already normalised).  Merge it
-                // with the naive-side partials of the same (request, head) by their log-sum-exps
-                // (Algorithm 1 line 8) and write the final bf16 row.
-                const CombineEpilogue& ce = p.ce;
-                const int64_t BH = (int64_t)p.M * ce.H;
-                const int64_t bh = (int64_t)row * ce.H + z;
-                const bool live = row < p.M;
-                float m = -INFINITY, la = -INFINITY;
-                if (live) {
-                    la = ce.lse_abs[bh];
-                    m = la;
-                    for (int i = 0; i < ce.n_naive; ++i) m = fmaxf(m, ce.lse_naive[i * BH + bh]);
-                }
-                float wa = 0.f, zsum = 0.f;
+        const int lg = (warp & 3) * 32;
+        const int row = m0 + lg + lane;
+        // Combine epilogue, first half: while the main loop runs, this thread (one request row) reads the
+        // LSEs of its (request, head), derives the merge weights and accumulates the weighted naive-side
+        // partials in registers, so that their memory latency is hidden behind the GEMM.
+        float accn[128];
+        float wa = 0.f, inv = 0.f, m = -INFINITY, zsum = 0.f;
+        int64_t bh = 0;
+        const bool live = p.out_mode == 2 && row < p.M;
+        if (p.out_mode == 2) {
+            const CombineEpilogue& ce = p.ce;
+            const int64_t BH = (int64_t)p.M * ce.H;
+            bh = (int64_t)row * ce.H + z;
+#pragma unroll
+            for (int q = 0; q < 128; ++q) accn[q] = 0.f;
+            if (live) {
+                const float la = ce.lse_abs[bh];
+                m = la;
+                for (int i = 0; i < ce.n_naive; ++i) m = fmaxf(m, ce.lse_naive[i * BH + bh]);
                 if (m != -INFINITY) {
                     wa = (la == -INFINITY) ? 0.f : __expf(la - m);
                     zsum = wa;
                     for (int i = 0; i < ce.n_naive; ++i) {
                         const float l = ce.lse_naive[i * BH + bh];
-                        if (l != -INFINITY) zsum += __expf(l - m);
+                        if (l == -INFINITY) continue;          // empty partial: its O slot was never written
+                        const float w = __expf(l - m);
+                        zsum += w;
+                        const float4* src = reinterpret_cast<const float4*>(ce.o_naive + (i * BH + bh) * 128);
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) {
+                            const float4 v = src[q];
+                            accn[4 * q] += w * v.x; accn[4 * q + 1] += w * v.y; accn[4 * q + 2] += w * v.z; accn[4 * q + 3] += w * v.w;
+                        }
                     }
                 }
-                const float inv = zsum > 0.f ? 1.f / zsum : 0.f;
-#pragma unroll 1
+                inv = zsum > 0.f ? 1.f / zsum : 0.f;
+            }
+        }
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, abort_flag));
+        tc_fence_after();
+        if (ok) {
+            if (p.out_mode == 2) {
+                // second half: add the absorb-side row (the accumulator, already normalised) with its weight,
+                // normalise (Algorithm 1 line 8) and write the final bf16 row
+                const CombineEpilogue& ce = p.ce;
+#pragma unroll
                 for (int c = 0; c < BN / 32; ++c) {
                     uint32_t r[32];
                     tmem_ld32(tmem_base + ((uint32_t)lg << 16) + c * 32, r);
                     tmem_ld_wait();
                     if (!live) continue;
-                    float acc[32];
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) acc[q] = wa > 0.f ? wa * __uint_as_float(r[q]) : 0.f;
-                    for (int i = 0; i < ce.n_naive; ++i) {
-                        const float l = ce.lse_naive[i * BH + bh];
-                        if (l == -INFINITY) continue;          // empty partial: its O slot was never written
-                        const float w = __expf(l - m);
-                        const float4* src = reinterpret_cast<const float4*>(ce.o_naive + (i * BH + bh) * 128 + c * 32);
-#pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const float4 v = src[q];
-                            acc[4 * q] += w * v.x; acc[4 * q + 1] += w * v.y; acc[4 * q + 2] += w * v.z; acc[4 * q + 3] += w * v.w;
-                        }
-                    }
                     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(ce.out) + bh * 128 + c * 32;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
+                        float o[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float oa = wa > 0.f ? wa * __uint_as_float(r[j * 8 + e]) : 0.f;
+                            o[e] = (accn[c * 32 + j * 8 + e] + oa) * inv;
+                        }
                         uint4 v;
-                        v.x = pack_bf16(acc[j * 8 + 0] * inv, acc[j * 8 + 1] * inv);
-                        v.y = pack_bf16(acc[j * 8 + 2] * inv, acc[j * 8 + 3] * inv);
-                        v.z = pack_bf16(acc[j * 8 + 4] * inv, acc[j * 8 + 5] * inv);
-                        v.w = pack_bf16(acc[j * 8 + 6] * inv, acc[j * 8 + 7] * inv);
+                        v.x = pack_bf16(o[0], o[1]); v.y = pack_bf16(o[2], o[3]);
+                        v.z = pack_bf16(o[4], o[5]); v.w = pack_bf16(o[6], o[7]);
                         *reinterpret_cast<uint4*>(dst + j * 8) = v;
                     }
                 }
