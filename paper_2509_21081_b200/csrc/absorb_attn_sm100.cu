@@ -64,7 +64,11 @@ struct AbsorbSm100Params {
 struct Shared {
     uint64_t q_full;
     uint64_t kv_full[STAGES], kv_empty[STAGES];
-    uint64_t s_ready[2], p_ready[2], o_done;
+    uint64_t s_ready[2], p_ready[2];
+    // completion of the accumulation of tile j goes to o_done[j & 1]: a waiter that knows tile j-2 has
+    // landed (every wait below does) then sees a barrier at most one completion from the awaited one,
+    // which is what a parity wait can tell apart
+    uint64_t o_done[2];
     uint32_t tmem_base;
     int abort_flag;
     float red[2][4][32];   // [warpgroup][warp][column]: cross-warp reductions
@@ -150,7 +154,8 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 mbar_init(&sh->s_ready[i], 1);
                 mbar_init(&sh->p_ready[i], 256);
             }
-            mbar_init(&sh->o_done, 1);
+            mbar_init(&sh->o_done[0], 1);
+            mbar_init(&sh->o_done[1], 1);
             sh->abort_flag = 0;
             fence_mbar_init();
         }
@@ -233,7 +238,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                         umma_ss_if(ld, d, da, db, idesc_o, (j | k) != 0);
                     }
                 }
-                umma_commit_if(ld, &sh->o_done);
+                umma_commit_if(ld, &sh->o_done[s]);
                 umma_commit_if(ld, &sh->kv_empty[s]);
                 TRACE(j, 4);
             }
@@ -312,7 +317,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     if (j > 0) {
                         // rescale this column group's 32 columns of all four O^T blocks (all 128 lanes), once
                         // the previous tile's accumulation has landed
-                        mbar_wait(&sh->o_done, (j - 1) & 1, abort_flag);
+                        mbar_wait(&sh->o_done[(j - 1) & 1], ((j - 1) >> 1) & 1, abort_flag);
                         __syncwarp();
                         tc_fence_after();
 #pragma unroll 1
@@ -373,7 +378,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             // (the decision to run it is taken by a warpgroup vote so that every thread of the
             // warpgroup reaches the same named barriers)
             if (!wg_vote_or(bar_id, *abort_flag != 0)) {
-                bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done, (n_tiles - 1) & 1, abort_flag));
+                bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag));
                 tc_fence_after();
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {

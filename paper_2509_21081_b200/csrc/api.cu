@@ -69,7 +69,7 @@ int cuda_fail(cudaError_t e) {
 // ---- workspace plan --------------------------------------------------------
 struct Plan {
     int mode;
-    int n_split_naive;       // KV splits of the naive kernel
+    int n_split_naive;       // KV splits of the warp-MMA naive kernel / tile ranges of the tcgen05 one
     int n_slots_naive;       // partial slots the naive kernel writes (>= n_split_naive)
     int chunk;               // tokens per absorb chunk
     int n_shared_chunks;     // absorb chunks over the shared prefix (ABSORB mode)
@@ -80,35 +80,21 @@ struct Plan {
 
 constexpr int kNumSM = 148;
 
-// KV splits of the tcgen05 naive kernel: minimise waves x (tiles per CTA + fixed cost) over the
-// candidate split counts (one CTA per SM; the fixed cost is the Q load and pipeline fill).
-int naive_splits_sm100(int B, int H, int64_t Ls) {
-    if (Ls <= 0) return 0;
-    const int tile_tok = naive_sm100_tile_tokens(B);
-    const int n_tiles = (int)((Ls + tile_tok - 1) / tile_tok);
-    if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_SPLITS")) {   // tuning aid
+// Tuning aids for the tcgen05 naive kernel: TYPHOON_MLA_NAIVE_CTAS overrides the SM count the plan
+// fills, TYPHOON_MLA_NAIVE_SCHEDULE forces "split" (column split) or "streamk".
+int naive_sm_budget() {
+    if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_CTAS")) {
         const int v = std::atoi(ov);
-        if (v >= 1) {
-            const int per = (n_tiles + std::min(v, n_tiles) - 1) / std::min(v, n_tiles);
-            return (n_tiles + per - 1) / per;
-        }
+        if (v >= 1 && v <= kNumSM) return v;
     }
-    const int base = (B <= 128 ? 1 : (B + 255) / 256) * H;
-    const double fixed = 6.0;
-    int best = 1;
-    double best_cost = 1e30;
-    for (int ns = 1; ns <= std::min(n_tiles, 32); ++ns) {
-        const int per = (n_tiles + ns - 1) / ns;
-        const int real = (n_tiles + per - 1) / per;
-        if (real != ns) continue;
-        const int waves = (real * base + kNumSM - 1) / kNumSM;
-        const double cost = waves * (per + fixed);
-        if (cost < best_cost - 1e-9) {
-            best_cost = cost;
-            best = ns;
-        }
+    return kNumSM;
+}
+int naive_schedule() {
+    if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_SCHEDULE")) {
+        if (std::strcmp(ov, "split") == 0) return 1;
+        if (std::strcmp(ov, "streamk") == 0) return 2;
     }
-    return best;
+    return 0;
 }
 
 int naive_splits(int B, int H, int64_t Ls) {
@@ -160,8 +146,12 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
     const bool use_naive = (mode != TYPHOON_MLA_MODE_ABSORB) && sh->Ls > 0;
     const bool use_absorb = (mode != TYPHOON_MLA_MODE_NAIVE);
     const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
-    p.n_split_naive = use_naive ? (tc ? naive_splits_sm100(B, H, sh->Ls) : naive_splits(B, H, sh->Ls)) : 0;
-    p.n_slots_naive = tc ? naive_sm100_slots(B, p.n_split_naive) : p.n_split_naive;
+    if (use_naive && tc) {
+        naive_sm100_plan(B, H, sh->Ls, naive_sm_budget(), naive_schedule(), &p.n_split_naive, &p.n_slots_naive);   // n_split_naive = tile ranges
+    } else {
+        p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls) : 0;
+        p.n_slots_naive = p.n_split_naive;
+    }
     if (use_absorb) {
         absorb_chunks(B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
                       &p.n_suffix_chunks);
@@ -498,7 +488,7 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         prof_before(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
         if (g_kernel_path == TYPHOON_MLA_PATH_TCGEN05) {
             NaiveAttnSm100 na{q_nope, q_pe, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt, B, H, (int)sh->Ls,
-                              pl.n_split_naive, softmax_scale, o_part_n, lse_part_n, sh->status};
+                              pl.n_split_naive, pl.n_slots_naive, softmax_scale, o_part_n, lse_part_n, sh->status};
             e = launch_naive_attn_sm100(na, s);
         } else {
             NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad,

@@ -54,18 +54,21 @@ struct NaiveAttn {
 cudaError_t launch_naive_attn_mma(const NaiveAttn& p, cudaStream_t s);
 
 // tcgen05/TMEM/TMA version.  The tensor maps of the expanded cache are built once per prefix
-// (make_naive_sm100_tmaps); partial slots = naive_sm100_slots(B, n_split).
+// (make_naive_sm100_tmaps); number of tile ranges and partial slots come from naive_sm100_plan.
 struct NaiveAttnSm100 {
     const void* q_nope; const void* q_pe;
     const CUtensorMap* tm_kn; const CUtensorMap* tm_kp; const CUtensorMap* tm_vt;   // host pointers
-    int B, H; int Ls; int n_split;
+    int B, H; int Ls; int n_ranges, n_slots;
     float scale;
     float* o_part;   // [slots][B][H][128]
     float* lse_part; // [slots][B][H]
     int* status;     // device word, set non-zero if a bounded wait expired
 };
-int naive_sm100_slots(int B, int n_split);
 int naive_sm100_tile_tokens(int B);   // KV tile width the kernel uses for this batch size (64 or 128)
+// CTAs (at most n_sm, each with an equal contiguous share of all (head, row group, tile) work) and
+// partial slots for a problem size; a pure function of its arguments.
+// schedule: 0 = chosen by the plan, 1 = column split, 2 = stream-K
+void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots);
 cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s);
 cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const void* v_t, int H, int64_t Ls_pad,
                                    CUtensorMap* tm_kn, CUtensorMap* tm_kp, CUtensorMap* tm_vt);

@@ -2,35 +2,42 @@
 //
 // Per head h the step is a dense contraction over all B query rows:
 //     S = Q_h [B,192] * [K_nope_h | k_pe]^T [192, L_s],  O = softmax(S) * V_h [L_s,128].
-// A CTA owns one head, one group of query rows and one KV split, and runs two
-// independent attention "streams" that share the TMA/MMA machinery:
-//   * B > 128  (mode X, 128-token KV tiles): stream i = query rows [256g + 128i, +128);
-//     both streams consume every KV tile of the split (tiles are loaded once).  This
-//     is the compute-bound regime: N = 128 per S MMA halves the re-reads of Q from
-//     shared memory, the two streams ping-pong between tensor core and softmax.
-//   * B <= 128 (mode Y, 64-token KV tiles): both streams use the same 128 query rows;
-//     stream i takes every second KV tile (tile k -> stream k & 1) with its own softmax
-//     state.  This is the HBM-bound regime: small tiles give a four-deep ring per operand.
-// Each stream writes a normalised fp32 partial and its LSE; the combine step merges all
-// partials of a (request, head).
 //
-// Warp roles (384 threads): warp 0 = TMA producer for Q and the K ring, warp 2 = TMA
-// producer for the V ring, warp 1 = issuer of the S = Q K^T MMAs and TMEM owner, warp 3
-// = issuer of the O += P V MMAs, warps 4-7 / 8-11 = softmax warpgroup of stream 0 / 1
-// (thread = one query row).  Two issuing warps keep the K-side and V-side barrier waits
-// from serialising behind each other; role warps run their loops with all lanes and
-// predicate the issuing instruction on one elected lane.
+// Work decomposition.  The KV tiles of all heads form one sequence of T = H * n_tiles tiles, which
+// is cut into R equal contiguous ranges.  A CTA owns one range and one group of query rows (128
+// rows for B <= 128, else 256; CTAs of the same range are adjacent in the grid, so the row groups
+// of a head walk the same KV tiles at about the same time and share them through L2).  A CTA works
+// through its range as a few "segments" (head, tile range), each a complete flash-attention pass
+// with its own Q tile that ends in a normalised fp32 partial plus LSE; the combine step merges the
+// partials of a (request, head).  The host picks R: a multiple of H (every range inside one head,
+// "column split") or the number of SMs over the number of row groups ("stream-K": one resident CTA
+// per SM, every SM gets the same number of tiles whatever H and L_s are).
 //
-// Tensor memory (512 columns).  64-token tiles: S[i][buf] (64 fp32 columns, double
-// buffered; P in bf16 overwrites the first 32) at (2i+buf)*64, O[i] at 256 + 128 i.
-// 128-token tiles: S[i] (128 columns, P overwrites the first 64) at 128 i, O[i] at
-// 256 + 128 i.
+// Inside a segment two independent attention "streams" share the TMA/MMA machinery:
+//   * B > 128  (mode X, 128-token KV tiles): stream i = query rows [256g + 128i, +128); both
+//     streams consume every KV tile (tiles are loaded once).  Compute-bound regime: N = 128 per
+//     S MMA halves the re-reads of Q from shared memory, the streams ping-pong between tensor
+//     core and softmax.
+//   * B <= 128 (mode Y, 64-token KV tiles): both streams use the same 128 query rows; stream i
+//     takes every second KV tile with its own softmax state.  HBM-bound regime: small tiles give
+//     deep K and V rings.
+//
+// Warp roles (384 threads): warp 0 = TMA producer for Q and the K ring, warp 2 = TMA producer
+// for the V ring, warp 1 = issuer of the S = Q K^T MMAs and TMEM owner, warp 3 = issuer of the
+// O += P V MMAs, warps 4-7 / 8-11 = softmax warpgroup of stream 0 / 1 (thread = one query row).
+// Role warps run their loops with all lanes and predicate the issuing instruction on one
+// elected lane.  Ring positions, S-buffer uses and accumulator completions are counted across
+// segments, so the pipeline never drains inside a CTA except for the Q tile of a new segment.
+//
+// Tensor memory (512 columns).  64-token tiles: S[i][buf] (64 fp32 columns, double buffered; P
+// in bf16 overwrites the first 32) at (2i+buf)*64, O[i] at 256 + 128 i.  128-token tiles: S[i]
+// (128 columns, P overwrites the first 64) at 128 i, O[i] at 256 + 128 i.
 //
 // The expanded cache is stored in 64-token blocks: K_nope [H, L/64, 2 slabs, 64, 64],
 // V^T [H, L/64, 128, 64], rope keys [L, 64]; every TMA box is a contiguous 8 or 16 KB.
 //
-// Every mbarrier wait has a deadline; on expiry all roles fall through to the common
-// teardown and the status word is set.
+// Every mbarrier wait has a deadline; on expiry all roles fall through to the common teardown
+// and the status word is set.
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -44,7 +51,11 @@ constexpr int MAX_STAGES = 4;
 
 struct NaiveSm100Params {
     int B, H, Ls, Ls_pad;
-    int n_split, m_groups;
+    int m_groups;          // query-row groups per head
+    int n_tiles;           // KV tiles per head
+    int n_ranges;          // R (grid = R * m_groups CTAs)
+    int per, rem;          // T = R * per + rem: ranges [0, rem) hold per + 1 tiles, the others per
+    int n_seg_max;         // partial slots per head (x2 streams in mode Y)
     int k_stages, v_stages;
     float scale_log2;
     float* o_part;     // [n_slots][B][H][128]
@@ -53,12 +64,25 @@ struct NaiveSm100Params {
 };
 
 struct Barriers {
-    uint64_t q_full;
+    uint64_t q_full, q_free;
     uint64_t k_full[MAX_STAGES], k_empty[MAX_STAGES];
     uint64_t v_full[MAX_STAGES], v_empty[MAX_STAGES];
-    uint64_t s_ready[2][2], p_ready[2][2], sbuf_free[2][2], o_done[2];
+    uint64_t s_ready[2][2], p_ready[2][2], sbuf_free[2][2], o_free[2];
+    // completion of PV product u of stream i goes to o_done[i][u & 1]: a waiter that knows product
+    // u-2 has landed (every wait below does) then sees a barrier at most one completion from the
+    // awaited one, which is what a parity wait can tell apart
+    uint64_t o_done[2][2];
     uint32_t tmem_base;
     int abort_flag;
+};
+
+// One segment of a CTA's tile range.
+struct Segment {
+    int t0, cnt;           // first tile, number of tiles
+    int h, row0;           // head, first query row
+    int slot_seg;          // index of this segment among the head's segments
+    bool last_of_col;      // this segment ends the head
+    int n_str0, n_str1;    // tiles per stream
 };
 
 // TOK = tokens per KV tile: 64 (mode Y, B <= 128) or 128 (mode X, B > 128).
@@ -73,6 +97,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     constexpr int K_SLAB = TOK * 128;                   // bytes of one [TOK][64] K slab
     constexpr int K_TILE_BYTES = 3 * K_SLAB;
     constexpr int V_TILE_BYTES = BLK * 16384;           // BLK slabs [128 dims][64 tokens]
+    constexpr int ROWS = MODE_Y ? 128 : 256;            // query rows per column
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -84,94 +109,119 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     volatile int* abort_flag = &bar->abort_flag;
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
-    const int split = blockIdx.x / p.m_groups, mg = blockIdx.x % p.m_groups, h = blockIdx.y;
-    const int row0 = mg * (MODE_Y ? 128 : 256);
+    const int rng = blockIdx.x / p.m_groups, grp = blockIdx.x % p.m_groups;
 
-    // KV tiles of this split
-    const int n_tiles_total = (p.Ls + TOK - 1) / TOK;
-    const int per = (n_tiles_total + p.n_split - 1) / p.n_split;
-    const int t_begin = split * per;
-    const int t_end = min(n_tiles_total, t_begin + per);
-    const int n_tiles = max(t_end - t_begin, 0);
-    // tiles per stream and number of steps
-    int n_str[2];
-    if (MODE_Y) {
-        n_str[0] = (n_tiles + 1) >> 1;
-        n_str[1] = n_tiles >> 1;
-    } else {
-        n_str[0] = n_tiles;
-        n_str[1] = (row0 + 128 < p.B) ? n_tiles : 0;   // second row tile entirely past B: skip it
-    }
-    const int n_steps = n_str[0];
-    // Softmax attention does not depend on the order in which KV tiles are visited.  CTAs of
+    // this CTA's contiguous range of the global tile sequence (T < 2^31: 32-bit arithmetic)
+    const int g_begin = rng * p.per + min(rng, p.rem);
+    const int g_end = g_begin + p.per + (rng < p.rem ? 1 : 0);
+
+    // Segment starting at global tile g (g_begin <= g < g_end).
+    auto segment_at = [&](int g) {
+        Segment s;
+        s.h = g / p.n_tiles;
+        s.t0 = g - s.h * p.n_tiles;
+        s.cnt = min(p.n_tiles - s.t0, g_end - g);
+        s.row0 = grp * ROWS;
+        // first range that reaches into this head: the one containing the head's first tile
+        const int first_tile = s.h * p.n_tiles, big = p.rem * (p.per + 1);
+        const int r_first = first_tile < big ? first_tile / (p.per + 1) : p.rem + (first_tile - big) / p.per;
+        s.slot_seg = rng - r_first;
+        s.last_of_col = (s.t0 + s.cnt == p.n_tiles);
+        if (MODE_Y) {
+            s.n_str0 = (s.cnt + 1) >> 1;
+            s.n_str1 = s.cnt >> 1;
+        } else {
+            s.n_str0 = s.cnt;
+            s.n_str1 = (s.row0 + 128 < p.B) ? s.cnt : 0;   // second row tile entirely past B: skip it
+        }
+        return s;
+    };
+    // Softmax attention does not depend on the order in which KV tiles are visited.  Segments of
     // different heads start at different tiles and wrap around, so that the CTAs resident at any
-    // moment do not all read the same offset of their (power-of-two strided) per-head arrays.
-    const int rot = n_tiles > 0 ? (int)(((unsigned)h * 37u + (unsigned)split * 11u) % (unsigned)n_tiles) : 0;
-    auto tile_of = [&](int e) { int t = e + rot; return t_begin + (t >= n_tiles ? t - n_tiles : t); };
-    // ring position of the KV tile used by stream i at step j, S buffer and its use count
+    // moment do not all read the same offset of their (power-of-two strided) per-head arrays
+    // (the row groups of one range use the same order).
+    auto tile_of = [&](const Segment& s, int e) {
+        const int rot = (int)(((unsigned)s.h * 37u + (unsigned)s.slot_seg * 11u) % (unsigned)s.cnt);
+        const int t = e + rot;
+        return s.t0 + (t >= s.cnt ? t - s.cnt : t);
+    };
+    // ring position (within the segment) of the KV tile used by stream i at step j; S columns of use u
     auto entry_of = [&](int j, int i) { return MODE_Y ? 2 * j + i : j; };
-    auto s_col = [&](int i, int j) { return (uint32_t)(MODE_Y ? (2 * i + (j & 1)) * 64 : i * 128); };
+    auto s_col = [&](int i, int u) { return (uint32_t)(MODE_Y ? (2 * i + (u & 1)) * 64 : i * 128); };
 
-    // Warp 0 initialises the barriers and at once issues Q and the first K and V tiles, so that the
-    // first copies are in flight while the rest of the CTA sets up (tensor-memory allocation, barrier).
     const uint32_t ld0 = (warp == 0 && elect_one()) ? 1u : 0u;
-    auto issue_k = [&](int e) {
-        const int s = e % p.k_stages;
-        uint8_t* dst = sK + s * K_TILE_BYTES;
-        const int blk0 = tile_of(e) * BLK;
-        mbar_arrive_expect_tx_if(ld0, &bar->k_full[s], K_TILE_BYTES);
+    auto issue_q = [&](const Segment& s) {
+        const int nq = (s.n_str1 > 0 && !MODE_Y) ? 2 : 1;
+        mbar_arrive_expect_tx_if(ld0, &bar->q_full, nq * Q_TILE_BYTES);
+        for (int t = 0; t < nq; ++t) {
+            uint8_t* dst = sQ + t * Q_TILE_BYTES;
+            tma_load_3d_if(ld0, dst, &tm_qn, &bar->q_full, 0, s.h, s.row0 + t * 128);
+            tma_load_3d_if(ld0, dst + 16384, &tm_qn, &bar->q_full, 64, s.h, s.row0 + t * 128);
+            tma_load_3d_if(ld0, dst + 32768, &tm_qp, &bar->q_full, 0, s.h, s.row0 + t * 128);
+        }
+    };
+    auto issue_k = [&](const Segment& s, int e, int ring_pos) {
+        const int st = ring_pos % p.k_stages;
+        uint8_t* dst = sK + st * K_TILE_BYTES;
+        const int blk0 = tile_of(s, e) * BLK;
+        mbar_arrive_expect_tx_if(ld0, &bar->k_full[st], K_TILE_BYTES);
 #pragma unroll
         for (int bi = 0; bi < BLK; ++bi) {
-            const int gb = h * (p.Ls_pad / 64) + blk0 + bi;
-            tma_load_3d_if(ld0, dst + bi * 8192, &tm_kn, &bar->k_full[s], 0, 0, gb);
-            tma_load_3d_if(ld0, dst + K_SLAB + bi * 8192, &tm_kn, &bar->k_full[s], 0, 64, gb);
-            tma_load_2d_if(ld0, dst + 2 * K_SLAB + bi * 8192, &tm_kp, &bar->k_full[s], 0, (blk0 + bi) * 64);
+            const int gb = s.h * (p.Ls_pad / 64) + blk0 + bi;
+            tma_load_3d_if(ld0, dst + bi * 8192, &tm_kn, &bar->k_full[st], 0, 0, gb);
+            tma_load_3d_if(ld0, dst + K_SLAB + bi * 8192, &tm_kn, &bar->k_full[st], 0, 64, gb);
+            tma_load_2d_if(ld0, dst + 2 * K_SLAB + bi * 8192, &tm_kp, &bar->k_full[st], 0, (blk0 + bi) * 64);
         }
     };
-    auto issue_v = [&](int e, uint32_t ld) {
-        const int s = e % p.v_stages;
-        const int blk0 = tile_of(e) * BLK;
-        mbar_arrive_expect_tx_if(ld, &bar->v_full[s], V_TILE_BYTES);
+    auto issue_v = [&](const Segment& s, int e, int ring_pos, uint32_t ld) {
+        const int st = ring_pos % p.v_stages;
+        const int blk0 = tile_of(s, e) * BLK;
+        mbar_arrive_expect_tx_if(ld, &bar->v_full[st], V_TILE_BYTES);
 #pragma unroll
         for (int bi = 0; bi < BLK; ++bi)
-            tma_load_4d_if(ld, sV + s * V_TILE_BYTES + bi * 16384, &tm_vt, &bar->v_full[s], 0, 0, blk0 + bi, h);
+            tma_load_4d_if(ld, sV + st * V_TILE_BYTES + bi * 16384, &tm_vt, &bar->v_full[st], 0, 0, blk0 + bi, s.h);
     };
-    if (warp == 0) {
-        if (lane == 0) {
-            mbar_init(&bar->q_full, 1);
-            for (int s = 0; s < MAX_STAGES; ++s) {
-                mbar_init(&bar->k_full[s], 1);
-                mbar_init(&bar->k_empty[s], 1);
-                mbar_init(&bar->v_full[s], 1);
-                mbar_init(&bar->v_empty[s], 1);
-            }
-            for (int i = 0; i < 2; ++i) {
-                for (int b = 0; b < 2; ++b) {
-                    mbar_init(&bar->s_ready[i][b], 1);
-                    mbar_init(&bar->p_ready[i][b], 128);
-                    mbar_init(&bar->sbuf_free[i][b], 1);
+
+    // Warp 0 initialises the barriers and at once issues the first segment's Q and first K and V
+    // tiles, so that the first copies are in flight while the rest of the CTA sets up.
+    int n_pre_k = 0, n_pre_v = 0;
+    if (g_begin < g_end) {
+        const Segment s0 = segment_at(g_begin);
+        n_pre_k = min(p.k_stages, s0.cnt);
+        n_pre_v = min(p.v_stages, s0.cnt);
+        if (warp == 0) {
+            if (lane == 0) {
+                mbar_init(&bar->q_full, 1);
+                mbar_init(&bar->q_free, 1);
+                for (int s = 0; s < MAX_STAGES; ++s) {
+                    mbar_init(&bar->k_full[s], 1);
+                    mbar_init(&bar->k_empty[s], 1);
+                    mbar_init(&bar->v_full[s], 1);
+                    mbar_init(&bar->v_empty[s], 1);
                 }
-                mbar_init(&bar->o_done[i], 1);
+                for (int i = 0; i < 2; ++i) {
+                    for (int b = 0; b < 2; ++b) {
+                        mbar_init(&bar->s_ready[i][b], 1);
+                        mbar_init(&bar->p_ready[i][b], 128);
+                        mbar_init(&bar->sbuf_free[i][b], 1);
+                    }
+                    mbar_init(&bar->o_done[i][0], 1);
+                    mbar_init(&bar->o_done[i][1], 1);
+                    mbar_init(&bar->o_free[i], 128);
+                }
+                bar->abort_flag = 0;
+                fence_mbar_init();
             }
-            bar->abort_flag = 0;
-            fence_mbar_init();
-        }
-        __syncwarp();
-        if (n_tiles > 0) {
-            const int nq = (n_str[1] > 0 && !MODE_Y) ? 2 : 1;
-            mbar_arrive_expect_tx_if(ld0, &bar->q_full, nq * Q_TILE_BYTES);
-            for (int t = 0; t < nq; ++t) {
-                uint8_t* dst = sQ + t * Q_TILE_BYTES;
-                tma_load_3d_if(ld0, dst, &tm_qn, &bar->q_full, 0, h, row0 + t * 128);
-                tma_load_3d_if(ld0, dst + 16384, &tm_qn, &bar->q_full, 64, h, row0 + t * 128);
-                tma_load_3d_if(ld0, dst + 32768, &tm_qp, &bar->q_full, 0, h, row0 + t * 128);
-            }
+            __syncwarp();
+            issue_q(s0);
             // interleave K and V so that the tiles of the first steps arrive first
-            for (int e = 0; e < max(p.k_stages, p.v_stages); ++e) {
-                if (e < p.k_stages && e < n_tiles) issue_k(e);
-                if (e < p.v_stages && e < n_tiles) issue_v(e, ld0);
+            for (int e = 0; e < max(n_pre_k, n_pre_v); ++e) {
+                if (e < n_pre_k) issue_k(s0, e, e);
+                if (e < n_pre_v) issue_v(s0, e, e, ld0);
             }
         }
+    } else if (threadIdx.x == 0) {
+        bar->abort_flag = 0;
     }
     if (warp == 1) tmem_alloc(&bar->tmem_base, 512);
     tc_fence_before();
@@ -180,44 +230,75 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     // broadcast through a shuffle so that the compiler knows the value is warp-uniform
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
 
-    if (n_tiles > 0) {
-        if (warp == 0) {
-            // ---------------- K producer: the rest of the ring (Q and the first tiles are already in flight)
-            for (int e = p.k_stages; e < n_tiles; ++e) {
-                if (!mbar_wait_warp(&bar->k_empty[e % p.k_stages], ((e / p.k_stages) & 1) ^ 1, abort_flag)) break;
-                issue_k(e);
+    if (warp == 0) {
+        // ---------------- Q + K producer
+        int ring = 0, seg = 0;
+        bool ok = true;
+        for (int g = g_begin; g < g_end && ok; ++seg) {
+            const Segment s = segment_at(g);
+            // K tiles first (they only need free ring slots), so that they are in flight while the
+            // previous segment's last S products still hold the Q tile
+            const int head_k = min(s.cnt, p.k_stages);
+            int e = 0;
+            for (; e < head_k && ok; ++e, ++ring) {
+                if (ring < n_pre_k) continue;                 // issued before the setup barrier
+                ok = mbar_wait_warp(&bar->k_empty[ring % p.k_stages], ((ring / p.k_stages) & 1) ^ 1, abort_flag);
+                if (ok) issue_k(s, e, ring);
             }
-        } else if (warp == 2) {
-            // ---------------- V producer
-            const uint32_t ld = elect_one() ? 1u : 0u;
-            for (int e = p.v_stages; e < n_tiles; ++e) {
-                if (!mbar_wait_warp(&bar->v_empty[e % p.v_stages], ((e / p.v_stages) & 1) ^ 1, abort_flag)) break;
-                issue_v(e, ld);
+            if (seg > 0 && ok) {
+                ok = mbar_wait_warp(&bar->q_free, (seg - 1) & 1, abort_flag);   // previous segment's S products done
+                if (ok) issue_q(s);
             }
-        } else if (warp == 1) {
-            // ---------------- S = Q K^T issuer.  With two S buffers per stream it runs ahead of the softmax
-            // by up to two steps; with one it follows the PV product of the previous step.
-            const uint32_t ld = elect_one() ? 1u : 0u;
-            constexpr uint32_t idesc_s = idesc_bf16(128, TOK, false, false);
-            bool ok = mbar_wait_warp(&bar->q_full, 0, abort_flag);
-            for (int j = 0; j < n_steps && ok; ++j) {
+            for (; e < s.cnt && ok; ++e, ++ring) {
+                ok = mbar_wait_warp(&bar->k_empty[ring % p.k_stages], ((ring / p.k_stages) & 1) ^ 1, abort_flag);
+                if (ok) issue_k(s, e, ring);
+            }
+            g += s.cnt;
+        }
+    } else if (warp == 2) {
+        // ---------------- V producer
+        const uint32_t ld = elect_one() ? 1u : 0u;
+        int ring = 0;
+        bool ok = true;
+        for (int g = g_begin; g < g_end && ok;) {
+            const Segment s = segment_at(g);
+            for (int e = 0; e < s.cnt && ok; ++e, ++ring) {
+                if (ring < n_pre_v) continue;
+                ok = mbar_wait_warp(&bar->v_empty[ring % p.v_stages], ((ring / p.v_stages) & 1) ^ 1, abort_flag);
+                if (ok) issue_v(s, e, ring, ld);
+            }
+            g += s.cnt;
+        }
+    } else if (warp == 1) {
+        // ---------------- S = Q K^T issuer.  With two S buffers per stream it runs ahead of the softmax by
+        // up to two steps; with one it follows the PV product of the previous step.
+        const uint32_t ld = elect_one() ? 1u : 0u;
+        constexpr uint32_t idesc_s = idesc_bf16(128, TOK, false, false);
+        int ring_base = 0, seg = 0;
+        int used0 = 0, used1 = 0;                              // S-buffer uses so far, per stream
+        bool ok = true;
+        for (int g = g_begin; g < g_end && ok; ++seg) {
+            const Segment s = segment_at(g);
+            ok = mbar_wait_warp(&bar->q_full, seg & 1, abort_flag);
+            for (int j = 0; j < s.n_str0 && ok; ++j) {
                 for (int i = 0; i < 2 && ok; ++i) {
-                    if (j >= n_str[i]) continue;
-                    const int e = entry_of(j, i);
-                    const int s = e % p.k_stages;
+                    if (j >= (i == 0 ? s.n_str0 : s.n_str1)) continue;
+                    const int ring = ring_base + entry_of(j, i);
+                    const int st = ring % p.k_stages;
                     if (MODE_Y || i == 0) {                       // mode X: stream 1 reuses stream 0's tile
-                        ok = mbar_wait_warp(&bar->k_full[s], (e / p.k_stages) & 1, abort_flag);
+                        ok = mbar_wait_warp(&bar->k_full[st], (ring / p.k_stages) & 1, abort_flag);
                         if (!ok) break;
                     }
-                    if (j >= NB) {   // the PV product that read P from this S buffer NB steps ago must be done
-                        ok = mbar_wait_warp(&bar->sbuf_free[i][j % NB], ((j / NB) - 1) & 1, abort_flag);
+                    const int u = (i == 0 ? used0 : used1) + j;
+                    if (u >= NB) {   // the PV product that read P from this S buffer NB uses ago must be done
+                        ok = mbar_wait_warp(&bar->sbuf_free[i][u % NB], ((u / NB) - 1) & 1, abort_flag);
                         if (!ok) break;
                     }
                     tc_fence_after();
                     const uint32_t qa = smem_u32(sQ + (MODE_Y ? 0 : i) * Q_TILE_BYTES);
-                    const uint32_t ka = smem_u32(sK + s * K_TILE_BYTES);
-                    const uint32_t d = tmem_base + s_col(i, j);
-                    const bool last_user = MODE_Y || i == 1 || n_str[1] == 0;
+                    const uint32_t ka = smem_u32(sK + st * K_TILE_BYTES);
+                    const uint32_t d = tmem_base + s_col(i, u);
+                    const bool last_user = MODE_Y || i == 1 || s.n_str1 == 0;
 #pragma unroll
                     for (int slab = 0; slab < 3; ++slab) {
                         const uint64_t da = smem_desc_k_sw128(qa + slab * 16384);
@@ -225,31 +306,46 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 #pragma unroll
                         for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (slab | k) != 0);
                     }
-                    umma_commit_if(ld, &bar->s_ready[i][j % NB]);
-                    if (last_user) umma_commit_if(ld, &bar->k_empty[s]);   // last user releases the ring slot
+                    umma_commit_if(ld, &bar->s_ready[i][u % NB]);
+                    if (last_user) umma_commit_if(ld, &bar->k_empty[st]);   // last user releases the ring slot
                 }
             }
-        } else if (warp == 3) {
-            // ---------------- O += P V issuer
-            const uint32_t ld = elect_one() ? 1u : 0u;
-            constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, false);
-            bool ok = true;
-            for (int j = 0; j < n_steps && ok; ++j) {
+            umma_commit_if(ld, &bar->q_free);                     // the Q tile may be replaced
+            used0 += s.n_str0;
+            used1 += s.n_str1;
+            ring_base += s.cnt;
+            g += s.cnt;
+        }
+    } else if (warp == 3) {
+        // ---------------- O += P V issuer
+        const uint32_t ld = elect_one() ? 1u : 0u;
+        constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, false);
+        int ring_base = 0, seg = 0;
+        int used0 = 0, used1 = 0;
+        bool ok = true;
+        for (int g = g_begin; g < g_end && ok; ++seg) {
+            const Segment s = segment_at(g);
+            for (int j = 0; j < s.n_str0 && ok; ++j) {
                 for (int i = 0; i < 2 && ok; ++i) {
-                    if (j >= n_str[i]) continue;
-                    const int e = entry_of(j, i);
-                    const int s = e % p.v_stages;
+                    if (j >= (i == 0 ? s.n_str0 : s.n_str1)) continue;
+                    const int ring = ring_base + entry_of(j, i);
+                    const int st = ring % p.v_stages;
                     if (MODE_Y || i == 0) {
-                        ok = mbar_wait_warp(&bar->v_full[s], (e / p.v_stages) & 1, abort_flag);
+                        ok = mbar_wait_warp(&bar->v_full[st], (ring / p.v_stages) & 1, abort_flag);
                         if (!ok) break;
                     }
-                    ok = mbar_wait_warp(&bar->p_ready[i][j % NB], (j / NB) & 1, abort_flag);
+                    const int u = (i == 0 ? used0 : used1) + j;
+                    ok = mbar_wait_warp(&bar->p_ready[i][u % NB], (u / NB) & 1, abort_flag);
                     if (!ok) break;
+                    if (j == 0 && seg > 0) {   // the previous segment's epilogue has read this accumulator
+                        ok = mbar_wait_warp(&bar->o_free[i], (seg - 1) & 1, abort_flag);
+                        if (!ok) break;
+                    }
                     tc_fence_after();
-                    const uint32_t va = smem_u32(sV + s * V_TILE_BYTES);
-                    const uint32_t pa = tmem_base + s_col(i, j);
+                    const uint32_t va = smem_u32(sV + st * V_TILE_BYTES);
+                    const uint32_t pa = tmem_base + s_col(i, u);
                     const uint32_t d = tmem_base + 256u + (uint32_t)i * 128u;
-                    const bool last_user = MODE_Y || i == 1 || n_str[1] == 0;
+                    const bool last_user = MODE_Y || i == 1 || s.n_str1 == 0;
 #pragma unroll
                     for (int bi = 0; bi < BLK; ++bi) {
                         const uint64_t db = smem_desc_k_sw128(va + bi * 16384);
@@ -257,24 +353,33 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         for (int k = 0; k < 4; ++k)
                             umma_ts_if(ld, d, pa + 8 * (bi * 4 + k), db + 2 * k, idesc_o, (j | bi | k) != 0);
                     }
-                    umma_commit_if(ld, &bar->o_done[i]);
-                    umma_commit_if(ld, &bar->sbuf_free[i][j % NB]);
-                    if (last_user) umma_commit_if(ld, &bar->v_empty[s]);
+                    umma_commit_if(ld, &bar->o_done[i][u & 1]);
+                    umma_commit_if(ld, &bar->sbuf_free[i][u % NB]);
+                    if (last_user) umma_commit_if(ld, &bar->v_empty[st]);
                 }
             }
-        } else if (warp >= 4) {
-            // ---------------- softmax warpgroups
-            const int i = (warp - 4) >> 2;            // stream
-            const int lg = (warp & 3) * 32;           // TMEM lane group of this warp
-            const int r = lg + lane;                  // row within the 128-row tile
-            const int b = row0 + (MODE_Y ? 0 : i * 128) + r;
-            const int nt = n_str[i];
+            used0 += s.n_str0;
+            used1 += s.n_str1;
+            ring_base += s.cnt;
+            g += s.cnt;
+        }
+    } else if (warp >= 4) {
+        // ---------------- softmax warpgroups
+        const int i = (warp - 4) >> 2;            // stream
+        const int lg = (warp & 3) * 32;           // TMEM lane group of this warp
+        const int r = lg + lane;                  // row within the 128-row tile
+        int used = 0;                             // S-buffer uses (= PV products) of this stream so far
+        bool ok = true;
+        for (int g = g_begin; g < g_end && ok;) {
+            const Segment s = segment_at(g);
+            const int b = s.row0 + (MODE_Y ? 0 : i * 128) + r;
+            const int nt = i == 0 ? s.n_str0 : s.n_str1;
             const bool warp_has_rows = (b - lane) < p.B;   // warp-uniform: first row of this warp is a real request
             float m_ref = -INFINITY, l_sum = 0.f;
-            bool ok = true;
             for (int j = 0; j < nt && ok; ++j) {
-                const int buf = j % NB;
-                ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_ready[i][buf], (j / NB) & 1, abort_flag));
+                const int u = used + j;
+                const int buf = u % NB;
+                ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_ready[i][buf], (u / NB) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 if (!warp_has_rows) {
@@ -284,8 +389,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     mbar_arrive(&bar->p_ready[i][buf]);
                     continue;
                 }
-                const uint32_t s_addr = tmem_base + ((uint32_t)lg << 16) + s_col(i, j);
-                const int tile = tile_of(entry_of(j, i));
+                const uint32_t s_addr = tmem_base + ((uint32_t)lg << 16) + s_col(i, u);
+                const int tile = tile_of(s, entry_of(j, i));
                 const int valid = min(TOK, p.Ls - tile * TOK);
                 // pass 1: row maximum of the raw logits (the scale is positive, so it commutes with the
                 // maximum); the ragged tail is masked with -inf in place
@@ -311,7 +416,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     m_ref = mx;
                 } else if (__any_sync(0xffffffffu, grow)) {
                     // the previous PV of this stream must have landed before O is touched
-                    ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i], (j - 1) & 1, abort_flag));
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i][(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     const float m_new = grow ? mx : m_ref;
@@ -363,41 +468,52 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 tc_fence_before();
                 mbar_arrive(&bar->p_ready[i][buf]);
             }
-            // epilogue: normalised partial + LSE
-            const int slot = MODE_Y ? split * 2 + i : split;
-            if (nt > 0 && ok) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i], (nt - 1) & 1, abort_flag));
+            if (!ok) break;
+            // ---- segment epilogue: normalised partial + LSE into this segment's slot
+            const int n_sub = MODE_Y ? 2 : 1;
+            const int slot = s.slot_seg * n_sub + (MODE_Y ? i : 0);
+            const bool owns_rows = MODE_Y || i == 0 || s.row0 + 128 < p.B;
+            if (nt > 0) {
+                const int u_last = used + nt - 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i][u_last & 1], (u_last >> 1) & 1, abort_flag));
+                if (!ok) break;
                 tc_fence_after();
-            }
-            if (nt > 0 && ok && warp_has_rows) {
-                const float inv = 1.f / l_sum;
-                const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)i * 128u;
-                float* dst = p.o_part + (((int64_t)slot * p.B + b) * p.H + h) * 128;
+                if (warp_has_rows) {
+                    const float inv = 1.f / l_sum;
+                    const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)i * 128u;
+                    float* dst = p.o_part + (((int64_t)slot * p.B + b) * p.H + s.h) * 128;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t orr[32];
-                    tmem_ld32(o_addr + c * 32, orr);
-                    tmem_ld_wait();
-                    if (b < p.B) {
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t orr[32];
+                        tmem_ld32(o_addr + c * 32, orr);
+                        tmem_ld_wait();
+                        if (b < p.B) {
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            float4 v = make_float4(__uint_as_float(orr[4 * q]) * inv, __uint_as_float(orr[4 * q + 1]) * inv,
-                                                   __uint_as_float(orr[4 * q + 2]) * inv, __uint_as_float(orr[4 * q + 3]) * inv);
-                            *reinterpret_cast<float4*>(dst + c * 32 + 4 * q) = v;
+                            for (int q = 0; q < 8; ++q) {
+                                float4 v = make_float4(__uint_as_float(orr[4 * q]) * inv, __uint_as_float(orr[4 * q + 1]) * inv,
+                                                       __uint_as_float(orr[4 * q + 2]) * inv, __uint_as_float(orr[4 * q + 3]) * inv);
+                                *reinterpret_cast<float4*>(dst + c * 32 + 4 * q) = v;
+                            }
                         }
                     }
+                    if (b < p.B) p.lse_part[((int64_t)slot * p.B + b) * p.H + s.h] = (m_ref + log2f(l_sum)) * kLn2;
                 }
-                if (b < p.B) p.lse_part[((int64_t)slot * p.B + b) * p.H + h] = (m_ref + log2f(l_sum)) * kLn2;
-            } else if (nt == 0 && b < p.B && (MODE_Y || i == 0 || row0 + 128 < p.B)) {
-                p.lse_part[((int64_t)slot * p.B + b) * p.H + h] = -INFINITY;
+            } else if (owns_rows && b < p.B) {
+                p.lse_part[((int64_t)slot * p.B + b) * p.H + s.h] = -INFINITY;   // this stream had no tile
             }
+            // the segment that ends a column marks the column's unused slots as empty
+            if (s.last_of_col && owns_rows && b < p.B) {
+                for (int ss = s.slot_seg + 1; ss < p.n_seg_max; ++ss) {
+                    const int sl = ss * n_sub + (MODE_Y ? i : 0);
+                    p.lse_part[((int64_t)sl * p.B + b) * p.H + s.h] = -INFINITY;
+                }
+            }
+            // the accumulator of this stream may be overwritten by the next segment
+            tc_fence_before();
+            mbar_arrive(&bar->o_free[i]);
+            used += nt;
+            g += s.cnt;
         }
-    } else if (warp >= 4) {
-        // empty split: every slot this CTA owns gets weight zero in the combine
-        const int i = (warp - 4) >> 2;
-        const int b = row0 + (MODE_Y ? 0 : i * 128) + (warp & 3) * 32 + lane;
-        const int slot = MODE_Y ? split * 2 + i : split;
-        if (b < p.B) p.lse_part[((int64_t)slot * p.B + b) * p.H + h] = -INFINITY;
     }
 
     tc_fence_before();
@@ -412,11 +528,74 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
 }  // namespace
 
-int naive_sm100_slots(int B, int n_split) { return B <= 128 ? 2 * n_split : n_split; }
 int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 
+// Host-side plan (pure function of the sizes): number of tile ranges R and of partial slots.
+//
+// Two schedules are weighed.  "Column split" cuts every head into ns equal parts (R = H * ns, CTAs
+// may run in several waves); ns minimises waves x (tiles per CTA + a fixed cost of about six tile
+// times for the Q load and the pipeline fill).  "Stream-K" uses R = SMs / row groups resident
+// CTAs and gives every SM the same number of tiles at the price of a few more segments (each
+// pays the fixed cost and a pair of partial slots).  Stream-K is taken when its modelled cost is
+// at least 5% lower: column split often leaves SMs to the concurrent absorb branch and writes
+// fewer partials.
+void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots) {
+    const bool mode_y = B <= 128;
+    const int tok = mode_y ? 64 : 128;
+    const int m_groups = mode_y ? 1 : (B + 255) / 256;
+    const int n_tiles = (int)((Ls + tok - 1) / tok);
+    const long long T = (long long)H * n_tiles;
+    if (T <= 0) {
+        *n_ranges = 0;
+        *n_slots = 0;
+        return;
+    }
+    // column split
+    const long long base = (long long)H * m_groups;
+    const double fixed = 6.0;
+    int ns_best = 1;
+    double cost_best = 1e30, eff_best = 0.0;
+    for (int ns = 1; ns <= std::min(n_tiles, 32); ++ns) {
+        const int per = (n_tiles + ns - 1) / ns;
+        if (n_tiles % ns != 0) continue;   // equal parts only: every range stays inside one head
+        const long long waves = (ns * base + n_sm - 1) / n_sm;
+        const double cost = (double)waves * (per + fixed);
+        if (cost < cost_best - 1e-9) {
+            cost_best = cost;
+            ns_best = ns;
+            eff_best = (double)(T * m_groups) / ((double)waves * per * n_sm);
+        }
+    }
+    // stream-K: equal ranges; a CTA meets at most (tiles per range / tiles per head) + 2 segments
+    const int r_stream = (int)std::min<long long>(std::max(1, n_sm / m_groups), T);
+    const long long per_stream = (T + r_stream - 1) / r_stream;
+    const long long waves_stream = ((long long)r_stream * m_groups + n_sm - 1) / n_sm;
+    const double segs_stream = (per_stream >= n_tiles) ? (double)per_stream / n_tiles + 1.0 : 2.0;
+    const double cost_stream = (double)waves_stream * (per_stream + segs_stream * fixed);
+    bool stream_k;
+    if (schedule == 1) stream_k = false;
+    else if (schedule == 2) stream_k = true;
+    else {
+        // With at most 64 query rows a CTA keeps up with its share of HBM: more resident CTAs do not
+        // help as long as most SMs are busy, and spare SMs go to the concurrent absorb branch.
+        const bool hbm_bound_small = mode_y && B <= 64 && eff_best >= 0.8;
+        stream_k = !hbm_bound_small && cost_stream < 0.95 * cost_best;
+    }
+    const int R = stream_k ? r_stream : H * ns_best;
+    // ranges [0, rem) hold per + 1 tiles, the others per (the kernel uses the same partition)
+    const long long per = T / R, rem = T % R, big = rem * (per + 1);
+    auto range_of = [&](long long t) { return t < big ? t / (per + 1) : rem + (t - big) / per; };
+    int seg_max = 1;
+    for (long long h = 0; h < H; ++h) {
+        const long long first = h * n_tiles, last = first + n_tiles - 1;
+        seg_max = std::max(seg_max, (int)(range_of(last) - range_of(first)) + 1);
+    }
+    *n_ranges = R;
+    *n_slots = seg_max * (mode_y ? 2 : 1);
+}
+
 cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
-    if (a.B <= 0 || a.Ls <= 0 || a.n_split <= 0) return cudaSuccess;
+    if (a.B <= 0 || a.Ls <= 0 || a.n_ranges <= 0) return cudaSuccess;
     CUtensorMap tm_qn, tm_qp;
     {
         uint64_t dims[3] = {128, (uint64_t)a.H, (uint64_t)a.B};
@@ -433,17 +612,26 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
     }
     const bool mode_y = a.B <= 128;
+    const int tok = mode_y ? 64 : 128;
     NaiveSm100Params p{};
     p.B = a.B; p.H = a.H; p.Ls = a.Ls; p.Ls_pad = (a.Ls + 127) / 128 * 128;
-    p.n_split = a.n_split;
     p.m_groups = mode_y ? 1 : (a.B + 255) / 256;
+    p.n_tiles = (a.Ls + tok - 1) / tok;
+    p.n_ranges = a.n_ranges;
+    {
+        const long long T = (long long)a.H * p.n_tiles;
+        if (T >= (1LL << 31) || a.n_ranges > T) return cudaErrorInvalidValue;
+        p.per = (int)(T / a.n_ranges);
+        p.rem = (int)(T % a.n_ranges);
+    }
+    p.n_seg_max = a.n_slots / (mode_y ? 2 : 1);
     p.k_stages = mode_y ? 4 : 2;
     p.v_stages = mode_y ? 4 : 1;
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = a.status;
-    const int k_tile = mode_y ? 64 * 384 : 128 * 384, v_tile = mode_y ? 16384 : 32768;
+    const int k_tile = tok * 384, v_tile = mode_y ? 16384 : 32768;
     const int smem = (mode_y ? 1 : 2) * Q_TILE_BYTES + p.k_stages * k_tile + p.v_stages * v_tile + 1024 + (int)sizeof(Barriers) + 64;
-    dim3 grid(p.n_split * p.m_groups, a.H, 1);
+    dim3 grid(p.n_ranges * p.m_groups, 1, 1);
     if (mode_y) {
         cudaFuncSetAttribute(naive_attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         naive_attn_sm100_kernel<64><<<grid, 384, smem, s>>>(tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);

@@ -61,6 +61,20 @@ def test_head_counts_and_batch_tail(H):
         G.assert_parity(out, ref, lse, ref_lse, what=f"H={H} mode {mode}")
 
 
+@pytest.mark.parametrize("schedule", ["split", "streamk"])
+@pytest.mark.parametrize("B,H,Ls", [(70, 64, 520), (5, 32, 1000), (150, 16, 1100), (300, 16, 700), (400, 32, 450)])
+def test_naive_schedules(schedule, B, H, Ls, monkeypatch):
+    """Both work decompositions of the shared-prefix kernel (every tile range inside one head; equal
+    ranges that cross heads), for 64- and 128-token tiles, one and two query-row groups, a last
+    row group with and without a second row tile."""
+    monkeypatch.setenv("TYPHOON_MLA_NAIVE_SCHEDULE", schedule)
+    cfg = _cfg("sched", B=B, H=H, Ls=Ls, lo=0, hi=90, seed=40 + B)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, HYBRID)
+    G.assert_parity(out, ref, lse, ref_lse, what=f"schedule {schedule} B={B} H={H} Ls={Ls}")
+
+
 def test_no_prefix():
     """Ls = 0: absorb path alone (Algorithm 1 lines 5-7)."""
     cfg = _cfg("noprefix", B=6, H=32, Ls=0, lo=1, hi=400, seed=23)
