@@ -39,9 +39,13 @@ constexpr float kRescaleThreshold = 8.f;         // log2 units
 
 #ifdef TMLA_TRACE
 __device__ long long g_trace_ab[64 * 32];
+__device__ long long g_trace_cta[4096 * 2];
+__device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TRACE_CTA(which) do { if (threadIdx.x == 0) { int lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); if (lin < 4096) g_trace_cta[lin * 2 + (which)] = gtimer(); } } while (0)
 #define TRACE(step, slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (step) >= 0 && (step) < 64 && (threadIdx.x & 31) == 0) g_trace_ab[(step) * 32 + (slot)] = clock64(); } while (0)
 #else
 #define TRACE(step, slot) do {} while (0)
+#define TRACE_CTA(which) do {} while (0)
 #endif
 
 struct AbsorbSm100Params {
@@ -52,6 +56,7 @@ struct AbsorbSm100Params {
     const int32_t* block_table;
     const int32_t* seq_lens;
     const int32_t* order;
+    const int4* desc;      // optional, per launch position: {request, clamped suffix length, page 0, page 1}
     float scale_log2;
     float* o_part;     // [n_chunks][B][H][512]
     float* lse_part;   // [n_chunks][B][H]
@@ -63,7 +68,11 @@ struct AbsorbSm100Params {
 
 struct Shared {
     uint64_t q_full;
-    uint64_t kv_full[STAGES], kv_empty[STAGES];
+    // A KV tile is loaded, consumed and released in four slab groups: group g = latent slabs 2g and
+    // 2g+1 (the latent rows of accumulator block g), group 3 also holds the rope slab (which becomes
+    // P^T).  The logits product starts on the first group while the others are still in flight, and a
+    // group is refilled as soon as its accumulator block has read it.
+    uint64_t kv_full[STAGES][4], kv_empty[STAGES][4];
     uint64_t s_ready[2], p_ready[2];
     // completion of the accumulation of tile j goes to o_done[j & 1]: a waiter that knows tile j-2 has
     // landed (every wait below does) then sees a barrier at most one completion from the awaited one,
@@ -73,6 +82,7 @@ struct Shared {
     int abort_flag;
     float red[2][4][32];   // [warpgroup][warp][column]: cross-warp reductions
     float mref[2][32];     // [warpgroup][column]: reference exponent (log2 units) of each head column
+    alignas(16) float inv[2][32];   // [warpgroup][column]: inverse row sums for the epilogue
 };
 
 __device__ __forceinline__ bool wg_vote_or(int bar_id, bool pred) {
@@ -100,8 +110,17 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     if (threadIdx.x == 0) TRACE(0, 28);
+    TRACE_CTA(0);
     const int chunk = blockIdx.x, h0 = blockIdx.y * 64;
-    const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
+    // one 16-byte load gives the request, its suffix length and its first two pages (else three
+    // dependent loads stand between the kernel's start and its first copy)
+    int b, len_b = -1, pg0 = -1, pg1 = -1;
+    if (p.desc != nullptr) {
+        const int4 d = p.desc[blockIdx.z];
+        b = d.x; len_b = d.y; pg0 = d.z; pg1 = d.w;
+    } else {
+        b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
+    }
 
     // token range of this chunk
     const bool shared_seg = chunk < p.n_shared_chunks;
@@ -110,7 +129,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
         seg_len = p.Ls_absorb;
         tok_begin = chunk * p.chunk;
     } else {
-        seg_len = min(max(p.seq_lens[b], 0), p.max_pages * p.page_size);
+        seg_len = len_b >= 0 ? len_b : min(max(p.seq_lens[b], 0), p.max_pages * p.page_size);
         tok_begin = (chunk - p.n_shared_chunks) * p.chunk;
     }
     const int tok_end = min(seg_len, tok_begin + p.chunk);
@@ -130,25 +149,28 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             page = t0 / TOK;
             slot = 0;
         } else {
-            page = __shfl_sync(0xffffffffu, bt[t0 / p.page_size], 0);
+            const int idx = t0 / p.page_size;
+            page = (p.desc != nullptr && idx < 2) ? (idx == 0 ? pg0 : pg1) : __shfl_sync(0xffffffffu, bt[idx], 0);
             slot = t0 % p.page_size;
         }
     };
-    auto issue_tile = [&](int j, int page, int slot) {
+    auto issue_group = [&](int j, int g, int page, int slot) {
         const int s = j & 1;
         uint8_t* dst = sKV + s * TILE_BYTES;
-        TRACE(j, 0);
-        mbar_arrive_expect_tx_if(ld0, &sh->kv_full[s], TILE_BYTES);
-#pragma unroll 1
-        for (int sl = 0; sl < 8; ++sl) tma_load_3d_if(ld0, dst + sl * SLAB_BYTES, tc, &sh->kv_full[s], sl * 64, slot, page);
-        tma_load_3d_if(ld0, dst + 8 * SLAB_BYTES, tk, &sh->kv_full[s], 0, slot, page);
+        if (g == 0) TRACE(j, 0);
+        mbar_arrive_expect_tx_if(ld0, &sh->kv_full[s][g], (g == 3 ? 3 : 2) * SLAB_BYTES);
+        tma_load_3d_if(ld0, dst + (2 * g) * SLAB_BYTES, tc, &sh->kv_full[s][g], (2 * g) * 64, slot, page);
+        tma_load_3d_if(ld0, dst + (2 * g + 1) * SLAB_BYTES, tc, &sh->kv_full[s][g], (2 * g + 1) * 64, slot, page);
+        if (g == 3) tma_load_3d_if(ld0, dst + 8 * SLAB_BYTES, tk, &sh->kv_full[s][g], 0, slot, page);
     };
     if (warp == 0) {
         if (lane == 0) {
             mbar_init(&sh->q_full, 1);
             for (int s = 0; s < STAGES; ++s) {
-                mbar_init(&sh->kv_full[s], 1);
-                mbar_init(&sh->kv_empty[s], 1);
+                for (int g = 0; g < 4; ++g) {
+                    mbar_init(&sh->kv_full[s][g], 1);
+                    mbar_init(&sh->kv_empty[s][g], 1);
+                }
             }
             for (int i = 0; i < 2; ++i) {
                 mbar_init(&sh->s_ready[i], 1);
@@ -168,7 +190,8 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             for (int j = 0; j < min(n_tiles, STAGES); ++j) {
                 int page, slot;
                 page_of(j, page, slot);
-                issue_tile(j, page, slot);
+#pragma unroll 1
+                for (int g = 0; g < 4; ++g) issue_group(j, g, page, slot);
             }
         }
     }
@@ -184,8 +207,13 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             for (int j = STAGES; j < n_tiles; ++j) {
                 int page, slot;
                 page_of(j, page, slot);
-                if (!mbar_wait_warp(&sh->kv_empty[j & 1], ((j >> 1) & 1) ^ 1, abort_flag)) break;
-                issue_tile(j, page, slot);
+                bool ok = true;
+#pragma unroll 1
+                for (int g = 0; g < 4 && ok; ++g) {
+                    ok = mbar_wait_warp(&sh->kv_empty[j & 1][g], ((j >> 1) & 1) ^ 1, abort_flag);
+                    if (ok) issue_group(j, g, page, slot);
+                }
+                if (!ok) break;
             }
         } else if (warp == 1) {
             // ---------------- S^T = KV_tile * Q^T issuer (M = 64 tokens, N = 64 heads, K = 576)
@@ -195,23 +223,30 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             const uint32_t qa = smem_u32(sQ);
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int s = j & 1;
-                ok = mbar_wait_warp(&sh->kv_full[s], (j >> 1) & 1, abort_flag);
-                if (!ok) break;
-                TRACE(j, 1);
                 if (j >= 2) {   // the softmax of tile j-2 has finished reading this S^T buffer
                     ok = mbar_wait_warp(&sh->p_ready[s], ((j >> 1) - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
-                tc_fence_after();
                 const uint32_t ka = smem_u32(sKV + s * TILE_BYTES);
                 const uint32_t d = tmem_base + (uint32_t)(s * 64);
+                // the contraction over the 576 dims runs group by group as the slabs land
 #pragma unroll
-                for (int sl = 0; sl < 9; ++sl) {
-                    const uint64_t da = smem_desc_k_sw128(ka + sl * SLAB_BYTES);
-                    const uint64_t db = smem_desc_k_sw128(qa + sl * SLAB_BYTES);
+                for (int g = 0; g < 4; ++g) {
+                    ok = mbar_wait_warp(&sh->kv_full[s][g], (j >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (sl | k) != 0);
+                    for (int i = 0; i < 3; ++i) {
+                        if (i == 2 && g != 3) continue;
+                        const int sl = (i == 2) ? 8 : 2 * g + i;
+                        const uint64_t da = smem_desc_k_sw128(ka + sl * SLAB_BYTES);
+                        const uint64_t db = smem_desc_k_sw128(qa + sl * SLAB_BYTES);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (g | i | k) != 0);
+                    }
                 }
+                if (!ok) break;
+                TRACE(j, 1);
                 umma_commit_if(ld, &sh->s_ready[s]);
                 TRACE(j, 2);
             }
@@ -237,9 +272,10 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                         const uint64_t db = smem_desc_mn_sw128(pa + k * 2048, SLAB_BYTES, 1024);
                         umma_ss_if(ld, d, da, db, idesc_o, (j | k) != 0);
                     }
+                    // accumulator block m was the last reader of latent slabs 2m, 2m+1 (and, for m = 3, of P^T)
+                    umma_commit_if(ld, &sh->kv_empty[s][m]);
                 }
                 umma_commit_if(ld, &sh->o_done[s]);
-                umma_commit_if(ld, &sh->kv_empty[s]);
                 TRACE(j, 4);
             }
         } else if (warp >= 4) {
@@ -377,53 +413,105 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             // ---------------- epilogue: row sums across lanes, normalised partial, LSE
             // (the decision to run it is taken by a warpgroup vote so that every thread of the
             // warpgroup reaches the same named barriers)
+            bool staged = false;
             if (!wg_vote_or(bar_id, *abort_flag != 0)) {
-                bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag));
-                tc_fence_after();
+                // Row sums first (they do not depend on the accumulator, whose last product is still
+                // running): a transposing butterfly over the 32 lanes leaves lane c with column c's sum
+                // over this warp's token rows (31 shuffles), then the four warps add up through shared memory.
+                float a16[16], a8[8], a4[4], a2[2];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    float v = l_part[c];
-                    v += __shfl_xor_sync(0xffffffffu, v, 16);
-                    v += __shfl_xor_sync(0xffffffffu, v, 8);
-                    v += __shfl_xor_sync(0xffffffffu, v, 4);
-                    v += __shfl_xor_sync(0xffffffffu, v, 2);
-                    v += __shfl_xor_sync(0xffffffffu, v, 1);
-                    if (lane == c) sh->red[cg][q][c] = v;
+                for (int c = 0; c < 16; ++c) {
+                    const bool up = (lane & 16) != 0;
+                    const float keep = up ? l_part[c + 16] : l_part[c], send = up ? l_part[c] : l_part[c + 16];
+                    a16[c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+                }
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const bool up = (lane & 8) != 0;
+                    const float keep = up ? a16[c + 8] : a16[c], send = up ? a16[c] : a16[c + 8];
+                    a8[c] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const bool up = (lane & 4) != 0;
+                    const float keep = up ? a8[c + 4] : a8[c], send = up ? a8[c] : a8[c + 4];
+                    a4[c] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const bool up = (lane & 2) != 0;
+                    const float keep = up ? a4[c + 2] : a4[c], send = up ? a4[c] : a4[c + 2];
+                    a2[c] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+                }
+                {
+                    const bool up = (lane & 1) != 0;
+                    const float keep = up ? a2[1] : a2[0], send = up ? a2[0] : a2[1];
+                    sh->red[cg][q][lane] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
                 }
                 wg_sync(bar_id);
-                if (ok && !*abort_flag) {
-                    float inv[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float l = sh->red[cg][0][c] + sh->red[cg][1][c] + sh->red[cg][2][c] + sh->red[cg][3][c];
-                        inv[c] = 1.f / l;
-                        if (q == 0 && lane == c) {
-                            const int h = h0 + cg * 32 + c;
-                            if (h < p.H) {
-                                const float lse = (mref[c] + log2f(l)) * kLn2;
-                                if (p.o_lat_direct) p.lse_direct[(int64_t)b * p.H + h] = lse;
-                                else p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = lse;
-                            }
-                        }
+                if (q == 0) {   // lane = head column: its inverse row sum and LSE
+                    const float l = sh->red[cg][0][lane] + sh->red[cg][1][lane] + sh->red[cg][2][lane] + sh->red[cg][3][lane];
+                    sh->inv[cg][lane] = 1.f / l;
+                    const int h = h0 + cg * 32 + lane;
+                    if (h < p.H) {
+                        const float lse = (mref[lane] + log2f(l)) * kLn2;
+                        if (p.o_lat_direct) p.lse_direct[(int64_t)b * p.H + h] = lse;
+                        else p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = lse;
                     }
-                    const int64_t row_base = ((int64_t)chunk * p.B + b) * p.H;
+                }
+                wg_sync(bar_id);
+                float inv[32];
+#pragma unroll
+                for (int c = 0; c < 32; c += 4) {
+                    const float4 v = *reinterpret_cast<const float4*>(&sh->inv[cg][c]);
+                    inv[c] = v.x; inv[c + 1] = v.y; inv[c + 2] = v.z; inv[c + 3] = v.w;
+                }
+                if (warp == 4) TRACE(0, 13);
+                const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag));
+                tc_fence_after();
+                if (warp == 4) TRACE(0, 14);
+                if (ok && !*abort_flag) {
+                    // The normalised O (head-major rows of 512 latent values) is staged in the KV ring, which
+                    // no product reads any more, as the contiguous block of up to 64 head rows it forms in
+                    // global memory, and leaves with one bulk copy.
+                    const bool direct = p.o_lat_direct != nullptr;
+                    if (warp == 4) TRACE(0, 15);
 #pragma unroll 1
                     for (int m = 0; m < 4; ++m) {
                         uint32_t orr[32];
                         tmem_ld32(tmem_base + lane_base + 128u + (uint32_t)(m * 64 + cg * 32), orr);
                         tmem_ld_wait();
                         const int lat = m * 128 + 32 * q + lane;
+                        if (direct) {
+                            __nv_bfloat16* st = reinterpret_cast<__nv_bfloat16*>(sKV) + (cg * 32) * 512 + lat;
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const int h = h0 + cg * 32 + c;
-                            if (h < p.H) {
-                                const float v = __uint_as_float(orr[c]) * inv[c];
-                                if (p.o_lat_direct) p.o_lat_direct[((int64_t)b * p.H + h) * 512 + lat] = __float2bfloat16_rn(v);
-                                else p.o_part[(row_base + h) * 512 + lat] = v;
-                            }
+                            for (int c = 0; c < 32; ++c) st[c * 512] = __float2bfloat16_rn(__uint_as_float(orr[c]) * inv[c]);
+                        } else {
+                            float* st = reinterpret_cast<float*>(sKV) + (cg * 32) * 512 + lat;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) st[c * 512] = __uint_as_float(orr[c]) * inv[c];
                         }
                     }
+                    fence_proxy_async();
+                    staged = true;
                 }
+            }
+            // Both warpgroups have staged their heads, or at least one has set the abort flag (every
+            // thread of the two warpgroups gets here: named barrier 3, 256 threads).
+            if (warp == 4) TRACE(0, 16);
+            asm volatile("bar.sync 3, 256;\n" ::: "memory");
+            if (warp == 4) TRACE(0, 17);
+            if (threadIdx.x == 128 && staged && !*abort_flag) {
+                const int n_heads = min(64, p.H - h0);
+                if (p.o_lat_direct) {
+                    bulk_store(p.o_lat_direct + ((int64_t)b * p.H + h0) * 512, sKV, (uint32_t)n_heads * 1024u);
+                } else {
+                    const int64_t row_base = ((int64_t)chunk * p.B + b) * p.H;
+                    bulk_store(p.o_part + (row_base + h0) * 512, sKV, (uint32_t)n_heads * 2048u);
+                }
+                bulk_commit();
+                bulk_wait_read();   // the staging buffer must outlive the copy; the kernel end publishes the writes
+                TRACE(0, 18);
             }
         }
     } else if (warp >= 4) {
@@ -444,6 +532,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) TRACE(0, 29);
+    TRACE_CTA(1);
     if (*abort_flag) {
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, 3);
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
@@ -474,6 +563,9 @@ cudaError_t make_kv_tmaps(const void* ckv, const void* kpe, int64_t ckv_stride, 
 }  // namespace
 
 #ifdef TMLA_TRACE
+extern "C" int typhoon_mla_debug_read_trace_absorb_cta(long long* dst) {
+    return (int)cudaMemcpyFromSymbol(dst, g_trace_cta, sizeof(long long) * 4096 * 2);
+}
 extern "C" int typhoon_mla_debug_read_trace_absorb(long long* dst) {
     return (int)cudaMemcpyFromSymbol(dst, g_trace_ab, sizeof(long long) * 64 * 32);
 }
@@ -519,6 +611,7 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     p.Ls_absorb = a.Ls_absorb;
     p.page_size = a.page_size; p.max_pages = a.max_pages;
     p.block_table = a.block_table; p.seq_lens = a.seq_lens; p.order = a.order;
+    p.desc = reinterpret_cast<const int4*>(a.desc);
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = status;
     p.o_lat_direct = n_chunks == 1 ? reinterpret_cast<__nv_bfloat16*>(o_lat_direct) : nullptr;

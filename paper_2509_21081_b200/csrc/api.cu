@@ -75,7 +75,7 @@ struct Plan {
     int n_shared_chunks;     // absorb chunks over the shared prefix (ABSORB mode)
     int n_suffix_chunks;
     // byte offsets into the workspace
-    size_t off_order, off_qabs, off_opart_a, off_lsepart_a, off_olat, off_lse_a, off_oabs, off_opart_n, off_lsepart_n, total;
+    size_t off_order, off_desc, off_qabs, off_opart_a, off_lsepart_a, off_olat, off_lse_a, off_oabs, off_opart_n, off_lsepart_n, total;
 };
 
 constexpr int kNumSM = 148;
@@ -165,6 +165,7 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
         return o;
     };
     p.off_order = take((size_t)B * 4);
+    p.off_desc = take((size_t)B * 16);
     p.off_qabs = take(BH * 512 * 2);
     p.off_opart_a = take((size_t)n_chunks * BH * 512 * 4);
     p.off_lsepart_a = take((size_t)n_chunks * BH * 4);
@@ -505,12 +506,15 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         // ragged suffixes: the longest requests are launched first (order computed on the device, no host
         // sync): by an extra block of the query-absorption kernel on the tcgen05 path, by its own kernel otherwise
         int32_t* order = nullptr;
+        int32_t* desc = nullptr;   // per-position descriptors, written next to the order on the tcgen05 path
         if (pl.n_suffix_chunks > 0 && B > 1 && B <= 4096) order = reinterpret_cast<int32_t*>(ws + pl.off_order);
         // --- query absorption Q_A = Q_N W_UK (Algorithm 1 line 5)
         void* q_abs = ws + pl.off_qabs;
         prof_before(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (tc) {
-            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->status, order ? seq_lens : nullptr, order, s);
+            if (order) desc = reinterpret_cast<int32_t*>(ws + pl.off_desc);
+            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->status, order ? seq_lens : nullptr, order,
+                                      block_table, max_pages, page_size, desc, s);
         } else {
             GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,
                       B, 512, 128, H, false};
@@ -529,7 +533,7 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
         void* o_lat = ws + pl.off_olat;
         AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
                       ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
-                      seq_lens, order, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
+                      seq_lens, order, desc, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
                       o_part_a, lse_part_a};
         prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         e = tc ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, o_lat, lse_a, sh->status, s)

@@ -38,9 +38,12 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, c
 
 // Query absorption on tcgen05 (one CTA per head and 128 requests); tm_w from make_q_absorb_tmap.
 cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w);
-// With seq_lens and order given (B <= 4096) one extra block also writes the longest-first request order.
+// With seq_lens and order given (B <= 4096) one extra block also writes the longest-first request order and,
+// with desc given, one int4 per launch position {request, clamped suffix length, first page, second page}
+// (-1 where the block table has no such column) that saves the absorb kernel three dependent loads.
 cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int* status,
-                                  const int32_t* seq_lens, int32_t* order, cudaStream_t s);
+                                  const int32_t* seq_lens, int32_t* order, const int32_t* block_table, int max_pages,
+                                  int page_size, int32_t* desc, cudaStream_t s);
 
 // Naive shared-prefix attention partials (Algorithm 1 line 4).
 struct NaiveAttn {
@@ -81,6 +84,7 @@ struct AbsorbAttn {
     int64_t ckv_stride, kpe_stride; int page_size;
     const int32_t* block_table; int max_pages; const int32_t* seq_lens;
     const int32_t* order;                          // optional [B]: request handled by block z (longest first)
+    const int32_t* desc;                           // optional [B][4]: per launch position, see launch_q_absorb_sm100
     int B, H; int chunk;                           // tokens per chunk
     int n_shared_chunks, n_suffix_chunks;
     float scale;

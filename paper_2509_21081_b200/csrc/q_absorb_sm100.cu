@@ -28,6 +28,10 @@ struct QAbsorbParams {
     // absorb attention kernel launched next uses, saving a launch on the absorb branch
     const int32_t* seq_lens;
     int32_t* order;
+    // optional per-position descriptors for the absorb kernel
+    const int32_t* block_table;
+    int max_pages, page_size;
+    int4* desc;
 };
 
 __global__ void __launch_bounds__(192, 1)
@@ -35,7 +39,18 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     if ((int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
-        if (blockIdx.x == 0) block_order_by_length(p.seq_lens, p.B, p.order, reinterpret_cast<unsigned long long*>(smem));
+        if (blockIdx.x == 0) {
+            block_order_by_length(p.seq_lens, p.B, p.order, reinterpret_cast<unsigned long long*>(smem));
+            if (p.desc != nullptr) {
+                __syncthreads();   // perm[] written by this block is read back below
+                for (int i = threadIdx.x; i < p.B; i += blockDim.x) {
+                    const int b = p.order[i];
+                    const int len = min(max(p.seq_lens[b], 0), p.max_pages * p.page_size);
+                    const int32_t* bt = p.block_table + (int64_t)b * p.max_pages;
+                    p.desc[i] = make_int4(b, len, p.max_pages > 0 ? bt[0] : -1, p.max_pages > 1 ? bt[1] : -1);
+                }
+            }
+        }
         return;
     }
     uint8_t* sA = smem;
@@ -134,7 +149,8 @@ cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w) {
 }
 
 cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int* status,
-                                  const int32_t* seq_lens, int32_t* order, cudaStream_t s) {
+                                  const int32_t* seq_lens, int32_t* order, const int32_t* block_table, int max_pages,
+                                  int page_size, int32_t* desc, cudaStream_t s) {
     if (B <= 0) return cudaSuccess;
     CUtensorMap tm_q;
     uint64_t dims[3] = {128, (uint64_t)H, (uint64_t)B};
@@ -143,7 +159,8 @@ cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, v
     cudaError_t e = make_tmap_bf16(&tm_q, q_nope, 3, dims, str, box);
     if (e != cudaSuccess) return e;
     const bool with_order = seq_lens != nullptr && order != nullptr && B <= 4096;
-    QAbsorbParams p{q_abs, B, H, status, seq_lens, order};
+    QAbsorbParams p{q_abs, B, H, status, seq_lens, order, block_table, max_pages, page_size,
+                    (with_order && block_table != nullptr) ? reinterpret_cast<int4*>(desc) : nullptr};
     cudaFuncSetAttribute(q_absorb_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid((B + 127) / 128, H + (with_order ? 1 : 0), 1);
     q_absorb_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tm_q, *tm_w, p);
