@@ -23,6 +23,8 @@
 //
 // Tensor memory (512 columns allocated): S^T[buf] at 64 buf (2 buffers), O^T block
 // m (128 latent rows x 64 heads) at 128 + 64 m.
+#include <cstddef>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -163,24 +165,23 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
         tma_load_3d_if(ld0, dst + (2 * g + 1) * SLAB_BYTES, tc, &sh->kv_full[s][g], (2 * g + 1) * 64, slot, page);
         if (g == 3) tma_load_3d_if(ld0, dst + 8 * SLAB_BYTES, tk, &sh->kv_full[s][g], 0, slot, page);
     };
+    if (warp == 2) {   // otherwise idle: fetch the tensor maps while warp 0 sets up the barriers
+        if (lane == 0) prefetch_tmap(&tm_qa);
+        if (lane == 1) prefetch_tmap(&tm_qp);
+        if (lane == 2) prefetch_tmap(tc);
+        if (lane == 3) prefetch_tmap(tk);
+    }
     if (warp == 0) {
-        if (lane == 0) {
-            mbar_init(&sh->q_full, 1);
-            for (int s = 0; s < STAGES; ++s) {
-                for (int g = 0; g < 4; ++g) {
-                    mbar_init(&sh->kv_full[s][g], 1);
-                    mbar_init(&sh->kv_empty[s][g], 1);
-                }
-            }
-            for (int i = 0; i < 2; ++i) {
-                mbar_init(&sh->s_ready[i], 1);
-                mbar_init(&sh->p_ready[i], 256);
-            }
-            mbar_init(&sh->o_done[0], 1);
-            mbar_init(&sh->o_done[1], 1);
-            sh->abort_flag = 0;
-            fence_mbar_init();
+        // the mbarriers are the leading uint64_t members of the struct, one lane each; p_ready counts the
+        // 256 softmax threads, all others one arrival
+        uint64_t* all = &sh->q_full;
+        constexpr int n_bars = (int)(offsetof(Shared, tmem_base) / sizeof(uint64_t));
+        for (int i = lane; i < n_bars; i += 32) {
+            uint64_t* m = all + i;
+            mbar_init(m, (m >= &sh->p_ready[0] && m < &sh->o_done[0]) ? 256 : 1);
         }
+        if (lane == 0) sh->abort_flag = 0;
+        fence_mbar_init();
         __syncwarp();
         if (n_tiles > 0) {
             mbar_arrive_expect_tx_if(ld0, &sh->q_full, TILE_BYTES);

@@ -38,6 +38,8 @@
 //
 // Every mbarrier wait has a deadline; on expiry all roles fall through to the common teardown
 // and the status word is set.
+#include <cstddef>
+
 #include "kernels.h"
 #include "sm100.cuh"
 
@@ -47,6 +49,14 @@ namespace {
 using namespace sm100;
 
 constexpr int Q_TILE_BYTES = 128 * 192 * 2;   // 3 slabs [128][64] bf16
+
+#ifdef TMLA_TRACE
+__device__ long long g_trace_ncta[4096 * 8];
+__device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TRACE_CTA(tid, which) do { if ((int)threadIdx.x == (tid) && blockIdx.x < 4096) g_trace_ncta[blockIdx.x * 8 + (which)] = gtimer(); } while (0)
+#else
+#define TRACE_CTA(tid, which) do {} while (0)
+#endif
 constexpr int MAX_STAGES = 4;
 
 struct NaiveSm100Params {
@@ -110,6 +120,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const int rng = blockIdx.x / p.m_groups, grp = blockIdx.x % p.m_groups;
+    TRACE_CTA(0, 0);
 
     // this CTA's contiguous range of the global tile sequence (T < 2^31: 32-bit arithmetic)
     const int g_begin = rng * p.per + min(rng, p.rem);
@@ -182,53 +193,57 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             tma_load_4d_if(ld, sV + st * V_TILE_BYTES + bi * 16384, &tm_vt, &bar->v_full[st], 0, 0, blk0 + bi, s.h);
     };
 
-    // Warp 0 initialises the barriers and at once issues the first segment's Q and first K and V
-    // tiles, so that the first copies are in flight while the rest of the CTA sets up.
+    // Warp 0 initialises the barriers (one per lane) and at once issues the first segment's Q and
+    // first K tiles; warp 2 fetches the tensor maps while the barriers are set up and then issues the
+    // first V tiles.  The first copies are thus in flight while the rest of the CTA sets up.
+    const uint32_t ld2 = (warp == 2 && elect_one()) ? 1u : 0u;
     int n_pre_k = 0, n_pre_v = 0;
     if (g_begin < g_end) {
         const Segment s0 = segment_at(g_begin);
         n_pre_k = min(p.k_stages, s0.cnt);
         n_pre_v = min(p.v_stages, s0.cnt);
+        if (warp == 2) {
+            if (lane == 0) prefetch_tmap(&tm_qn);
+            if (lane == 1) prefetch_tmap(&tm_qp);
+            if (lane == 2) prefetch_tmap(&tm_kn);
+            if (lane == 3) prefetch_tmap(&tm_kp);
+            if (lane == 4) prefetch_tmap(&tm_vt);
+            asm volatile("bar.sync 1, 64;\n" ::: "memory");   // warp 0 has initialised the barriers
+            asm volatile("bar.sync 2, 64;\n" ::: "memory");   // ... and issued Q and the first K tile (needed first)
+            for (int e = 0; e < n_pre_v; ++e) issue_v(s0, e, e, ld2);
+        }
         if (warp == 0) {
-            if (lane == 0) {
-                mbar_init(&bar->q_full, 1);
-                mbar_init(&bar->q_free, 1);
-                for (int s = 0; s < MAX_STAGES; ++s) {
-                    mbar_init(&bar->k_full[s], 1);
-                    mbar_init(&bar->k_empty[s], 1);
-                    mbar_init(&bar->v_full[s], 1);
-                    mbar_init(&bar->v_empty[s], 1);
-                }
-                for (int i = 0; i < 2; ++i) {
-                    for (int b = 0; b < 2; ++b) {
-                        mbar_init(&bar->s_ready[i][b], 1);
-                        mbar_init(&bar->p_ready[i][b], 128);
-                        mbar_init(&bar->sbuf_free[i][b], 1);
-                    }
-                    mbar_init(&bar->o_done[i][0], 1);
-                    mbar_init(&bar->o_done[i][1], 1);
-                    mbar_init(&bar->o_free[i], 128);
-                }
-                bar->abort_flag = 0;
-                fence_mbar_init();
+            // the mbarriers are the leading uint64_t members of the struct; p_ready and o_free count the
+            // 128 threads of a softmax warpgroup, all others one arrival
+            uint64_t* all = &bar->q_full;
+            constexpr int n_bars = (int)(offsetof(Barriers, tmem_base) / sizeof(uint64_t));
+            for (int i = lane; i < n_bars; i += 32) {
+                uint64_t* m = all + i;
+                const bool wg = (m >= &bar->p_ready[0][0] && m < &bar->sbuf_free[0][0]) || (m >= &bar->o_free[0] && m < &bar->o_done[0][0]);
+                mbar_init(m, wg ? 128 : 1);
             }
+            if (lane == 0) bar->abort_flag = 0;
+            fence_mbar_init();
             __syncwarp();
+            asm volatile("bar.sync 1, 64;\n" ::: "memory");
+            TRACE_CTA(0, 6);
             issue_q(s0);
-            // interleave K and V so that the tiles of the first steps arrive first
-            for (int e = 0; e < max(n_pre_k, n_pre_v); ++e) {
-                if (e < n_pre_k) issue_k(s0, e, e);
-                if (e < n_pre_v) issue_v(s0, e, e, ld0);
-            }
+            issue_k(s0, 0, 0);
+            asm volatile("bar.sync 2, 64;\n" ::: "memory");
+            for (int e = 1; e < n_pre_k; ++e) issue_k(s0, e, e);
         }
     } else if (threadIdx.x == 0) {
         bar->abort_flag = 0;
     }
+    TRACE_CTA(0, 7);
     if (warp == 1) tmem_alloc(&bar->tmem_base, 512);
+    TRACE_CTA(32, 3);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     // broadcast through a shuffle so that the compiler knows the value is warp-uniform
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
+    TRACE_CTA(0, 1);
 
     if (warp == 0) {
         // ---------------- Q + K producer
@@ -257,13 +272,13 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         }
     } else if (warp == 2) {
         // ---------------- V producer
-        const uint32_t ld = elect_one() ? 1u : 0u;
+        const uint32_t ld = ld2;
         int ring = 0;
         bool ok = true;
         for (int g = g_begin; g < g_end && ok;) {
             const Segment s = segment_at(g);
             for (int e = 0; e < s.cnt && ok; ++e, ++ring) {
-                if (ring < n_pre_v) continue;
+                if (ring < n_pre_v) continue;                 // issued before the setup barrier
                 ok = mbar_wait_warp(&bar->v_empty[ring % p.v_stages], ((ring / p.v_stages) & 1) ^ 1, abort_flag);
                 if (ok) issue_v(s, e, ring, ld);
             }
@@ -382,6 +397,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_ready[i][buf], (u / NB) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
+                if (used + j == 0) TRACE_CTA(128, 2);
                 if (!warp_has_rows) {
                     // all 32 rows of this warp are padding past B: their P rows may hold anything (rows of
                     // the MMA are independent and these output rows are never stored); just keep in step
@@ -469,6 +485,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 mbar_arrive(&bar->p_ready[i][buf]);
             }
             if (!ok) break;
+            TRACE_CTA(128, 3);
             // ---- segment epilogue: normalised partial + LSE into this segment's slot
             const int n_sub = MODE_Y ? 2 : 1;
             const int slot = s.slot_seg * n_sub + (MODE_Y ? i : 0);
@@ -509,6 +526,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 }
             }
             // the accumulator of this stream may be overwritten by the next segment
+            TRACE_CTA(128, 4);
             tc_fence_before();
             mbar_arrive(&bar->o_free[i]);
             used += nt;
@@ -518,6 +536,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     tc_fence_before();
     __syncthreads();
+    TRACE_CTA(0, 5);
     if (*abort_flag) {
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, 2);
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
@@ -527,6 +546,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 }
 
 }  // namespace
+
+#ifdef TMLA_TRACE
+extern "C" int typhoon_mla_debug_read_trace_naive_cta(long long* dst) {
+    return (int)cudaMemcpyFromSymbol(dst, g_trace_ncta, sizeof(long long) * 4096 * 8);
+}
+#endif
 
 int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 
