@@ -562,8 +562,7 @@ int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 // times for the Q load and the pipeline fill).  "Stream-K" uses R = SMs / row groups resident
 // CTAs and gives every SM the same number of tiles at the price of a few more segments (each
 // pays the fixed cost and a pair of partial slots).  Stream-K is taken when its modelled cost is
-// at least 5% lower: column split often leaves SMs to the concurrent absorb branch and writes
-// fewer partials.
+// lower (by at least 5% in the HBM-bound regime of 64-token tiles).
 void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots) {
     const bool mode_y = B <= 128;
     const int tok = mode_y ? 64 : 128;
@@ -604,7 +603,9 @@ void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_r
         // With at most 64 query rows a CTA keeps up with its share of HBM: more resident CTAs do not
         // help as long as most SMs are busy, and spare SMs go to the concurrent absorb branch.
         const bool hbm_bound_small = mode_y && B <= 64 && eff_best >= 0.8;
-        stream_k = !hbm_bound_small && cost_stream < 0.95 * cost_best;
+        // 64-token tiles (HBM-bound regime): column split must lose by 5%, since it often leaves SMs to
+        // the concurrent absorb branch and writes fewer partials
+        stream_k = !hbm_bound_small && cost_stream < (mode_y ? 0.95 : 1.0) * cost_best;
     }
     const int R = stream_k ? r_stream : H * ns_best;
     // ranges [0, rem) hold per + 1 tiles, the others per (the kernel uses the same partition)
