@@ -210,6 +210,17 @@ int typhoon_mla_cost_model(const typhoon_mla_dims_t* dims /* host */, int32_t ki
                            int64_t B, int64_t S_q, int64_t L_s, int64_t L_n,
                            int64_t* macs /* host */, int64_t* hbm_words /* host */);
 
+/* Work decomposition the tcgen05 shared-prefix kernel (Algorithm 1 line 4) would use for a problem
+ * size: tokens per KV tile (64 for B <= 128, else 128), number of contiguous tile ranges the H * n_tiles
+ * tiles are cut into, query-row groups per range (CTAs = ranges * row_groups) and partial slots written
+ * per (request, head).  schedule: 0 = the library's choice, 1 = every range inside one head ("column
+ * split"), 2 = ranges of equal size over all heads ("stream-K").  Host, pure (a function of the sizes
+ * only, so the decomposition and with it the summation order are reproducible).  INVALID_ARG for
+ * B < 1, L_s < 1, unsupported H or schedule outside 0..2; no output is written then. */
+int typhoon_mla_naive_plan(int32_t num_heads, int32_t B, int64_t L_s, int32_t schedule,
+                           int32_t* tile_tokens /* host */, int32_t* n_ranges /* host */,
+                           int32_t* row_groups /* host */, int32_t* n_slots /* host */);
+
 /* Read-only views of what the handle owns (for tests and accounting):
  * k_nope bf16 [H, Ls_padded/64, 2, 64, 64]; v_t bf16 [H, Ls_padded/64, 128, 64]. */
 int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,

@@ -73,6 +73,8 @@ def _load():
     lib.typhoon_mla_batch_threshold.argtypes = [C.POINTER(Dims), i32, f64, f64]
     lib.typhoon_mla_cost_model.restype = C.c_int
     lib.typhoon_mla_cost_model.argtypes = [C.POINTER(Dims), i32, i64, i64, i64, i64, C.POINTER(i64), C.POINTER(i64)]
+    lib.typhoon_mla_naive_plan.restype = C.c_int
+    lib.typhoon_mla_naive_plan.argtypes = [i32, i32, i64, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     lib.typhoon_mla_shared_view.restype = C.c_int
     lib.typhoon_mla_shared_view.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), C.POINTER(i64),
                                             C.POINTER(i64)]
@@ -214,6 +216,14 @@ def typhoon_mla_cost_model(dims: Dims, kind: int, B: int, S_q: int, L_s: int, L_
     _check(_lib.typhoon_mla_cost_model(C.byref(dims), kind, B, S_q, L_s, L_n, C.byref(m), C.byref(w)),
            "typhoon_mla_cost_model")
     return m.value, w.value
+
+
+def typhoon_mla_naive_plan(num_heads: int, B: int, L_s: int, schedule: int = 0):
+    """(tile_tokens, n_ranges, row_groups, n_slots) of the shared-prefix kernel's work decomposition."""
+    t, r, g, sl = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+    _check(_lib.typhoon_mla_naive_plan(num_heads, B, L_s, schedule, C.byref(t), C.byref(r), C.byref(g), C.byref(sl)),
+           "typhoon_mla_naive_plan")
+    return t.value, r.value, g.value, sl.value
 
 
 def typhoon_mla_shared_view(shared: SharedPrefix):

@@ -214,6 +214,20 @@ double typhoon_mla_batch_threshold(const typhoon_mla_dims_t* d, int32_t S_q, dou
     return (d_qk + d->d_v) / ((double)S_q * (2.0 * d->kv_lora_rank + d->d_rope)) * (T / M);
 }
 
+int typhoon_mla_naive_plan(int32_t num_heads, int32_t B, int64_t L_s, int32_t schedule, int32_t* tile_tokens,
+                           int32_t* n_ranges, int32_t* row_groups, int32_t* n_slots) {
+    if (B < 1 || L_s < 1 || L_s > (int64_t)1 << 30 || schedule < 0 || schedule > 2) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (num_heads < 16 || num_heads > 128 || num_heads % 16) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!tile_tokens || !n_ranges || !row_groups || !n_slots) return TYPHOON_MLA_ERR_INVALID_ARG;
+    int r = 0, sl = 0;
+    naive_sm100_plan(B, num_heads, L_s, kNumSM, schedule, &r, &sl);
+    *tile_tokens = naive_sm100_tile_tokens(B);
+    *n_ranges = r;
+    *row_groups = B <= 128 ? 1 : (B + 255) / 256;
+    *n_slots = sl;
+    return TYPHOON_MLA_OK;
+}
+
 int typhoon_mla_cost_model(const typhoon_mla_dims_t* d, int32_t kind, int64_t B, int64_t S_q, int64_t L_s,
                            int64_t L_n, int64_t* macs, int64_t* hbm_words) {
     if (!d || B < 0 || S_q < 1 || L_s < 0 || L_n < 0) return TYPHOON_MLA_ERR_INVALID_ARG;

@@ -75,6 +75,26 @@ def test_naive_schedules(schedule, B, H, Ls, monkeypatch):
     G.assert_parity(out, ref, lse, ref_lse, what=f"schedule {schedule} B={B} H={H} Ls={Ls}")
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes(seed, monkeypatch):
+    """Seeded random problem sizes, modes, page sizes and work decompositions: pipeline phase logic
+    (ring wrap-around, segments per CTA, odd tile counts, partial row groups) against the checker."""
+    import random
+    rnd = random.Random(1000 + seed)
+    H = rnd.choice([16, 32, 48, 64, 128])
+    B = rnd.choice([rnd.randint(1, 8), rnd.randint(9, 128), rnd.randint(129, 300)])
+    Ls = rnd.choice([rnd.randint(1, 200), rnd.randint(200, 1500), rnd.randint(1500, 2600) if H <= 32 else rnd.randint(64, 900)])
+    hi = rnd.choice([0, 5, 70, 200])
+    page_size = rnd.choice([64, 128])
+    mode = rnd.choice([HYBRID, HYBRID, ABSORB, AUTO])
+    monkeypatch.setenv("TYPHOON_MLA_NAIVE_SCHEDULE", rnd.choice(["split", "streamk", "auto"]))
+    cfg = _cfg("rand", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=500 + seed, page_size=page_size)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, mode, page_size=page_size)
+    G.assert_parity(out, ref, lse, ref_lse, what=f"random {seed}: B={B} H={H} Ls={Ls} hi={hi} ps={page_size} mode={mode}")
+
+
 def test_no_prefix():
     """Ls = 0: absorb path alone (Algorithm 1 lines 5-7)."""
     cfg = _cfg("noprefix", B=6, H=32, Ls=0, lo=1, hi=400, seed=23)

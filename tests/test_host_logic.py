@@ -113,3 +113,38 @@ def test_pure_entry_points_reject_bad_arguments(b):
     assert b.typhoon_mla_batch_threshold(b.make_dims(128), 0, 1.0, 1.0) < 0
     with pytest.raises(b.TyphoonMLAError):
         b.typhoon_mla_cost_model(b.make_dims(128), 9, 1, 1, 1, 1)
+
+
+def test_naive_plan_invariants(b):
+    """Work decomposition of the shared-prefix kernel: every schedule covers all tiles with at most
+    `n_slots` segments per head; the benchmark sizes get the decompositions the design states."""
+    import random
+    rnd = random.Random(5)
+    for _ in range(400):
+        H = rnd.choice([16, 32, 48, 64, 128])
+        B = rnd.choice([1, 7, 64, 65, 128, 129, 256, 300, 512, 1024])
+        Ls = rnd.randint(1, 40000)
+        for schedule in (0, 1, 2):
+            tok, R, groups, slots = b.typhoon_mla_naive_plan(H, B, Ls, schedule)
+            assert tok == (64 if B <= 128 else 128)
+            assert groups == (1 if B <= 128 else (B + 255) // 256)
+            n_tiles = (Ls + tok - 1) // tok
+            T = H * n_tiles
+            assert 1 <= R <= T
+            # same partition as the kernel: ranges [0, rem) hold per + 1 tiles
+            per, rem = divmod(T, R)
+            big = rem * (per + 1)
+            rng = lambda t: t // (per + 1) if t < big else rem + (t - big) // per
+            seg_max = max(rng(h * n_tiles + n_tiles - 1) - rng(h * n_tiles) + 1 for h in range(H))
+            assert slots == seg_max * (2 if B <= 128 else 1)
+            if schedule == 1:
+                assert R % H == 0 and n_tiles % (R // H) == 0 and seg_max == R // H
+            if schedule == 2:
+                assert R == min(max(1, 148 // groups), T)
+    # benchmark configs: config 1 one range per head; config 2 and config 4 at B = 512 one CTA per SM
+    assert b.typhoon_mla_naive_plan(128, 64, 4096)[1:] == (128, 1, 2)
+    assert b.typhoon_mla_naive_plan(128, 128, 26624)[1] == 148
+    assert b.typhoon_mla_naive_plan(128, 512, 16384)[1:3] == (74, 2)
+    for bad in ((8, 1, 10, 0), (128, 0, 10, 0), (128, 1, 0, 0), (128, 1, 10, 3)):
+        with pytest.raises(Exception):
+            b.typhoon_mla_naive_plan(*bad)
