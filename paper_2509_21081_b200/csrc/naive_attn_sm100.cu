@@ -54,8 +54,11 @@ constexpr int Q_TILE_BYTES = 128 * 192 * 2;   // 3 slabs [128][64] bf16
 __device__ long long g_trace_ncta[4096 * 8];
 __device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define TRACE_CTA(tid, which) do { if ((int)threadIdx.x == (tid) && blockIdx.x < 4096) g_trace_ncta[blockIdx.x * 8 + (which)] = gtimer(); } while (0)
+__device__ long long g_trace_nstep[64 * 32];
+#define TRACE(step, slot) do { if (blockIdx.x == 3 && (step) >= 0 && (step) < 64 && (threadIdx.x & 31) == 0) g_trace_nstep[(step) * 32 + (slot)] = clock64(); } while (0)
 #else
 #define TRACE_CTA(tid, which) do {} while (0)
+#define TRACE(step, slot) do {} while (0)
 #endif
 constexpr int MAX_STAGES = 4;
 
@@ -310,6 +313,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         if (!ok) break;
                     }
                     tc_fence_after();
+                    TRACE(j, 0 + i);
                     const uint32_t qa = smem_u32(sQ + (MODE_Y ? 0 : i) * Q_TILE_BYTES);
                     const uint32_t ka = smem_u32(sK + st * K_TILE_BYTES);
                     const uint32_t d = tmem_base + s_col(i, u);
@@ -322,6 +326,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (slab | k) != 0);
                     }
                     umma_commit_if(ld, &bar->s_ready[i][u % NB]);
+                    TRACE(j, 2 + i);
                     if (last_user) umma_commit_if(ld, &bar->k_empty[st]);   // last user releases the ring slot
                 }
             }
@@ -357,6 +362,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         if (!ok) break;
                     }
                     tc_fence_after();
+                    TRACE(j, 4 + i);
                     const uint32_t va = smem_u32(sV + st * V_TILE_BYTES);
                     const uint32_t pa = tmem_base + s_col(i, u);
                     const uint32_t d = tmem_base + 256u + (uint32_t)i * 128u;
@@ -369,6 +375,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                             umma_ts_if(ld, d, pa + 8 * (bi * 4 + k), db + 2 * k, idesc_o, (j | bi | k) != 0);
                     }
                     umma_commit_if(ld, &bar->o_done[i][u & 1]);
+                    TRACE(j, 6 + i);
                     umma_commit_if(ld, &bar->sbuf_free[i][u % NB]);
                     if (last_user) umma_commit_if(ld, &bar->v_empty[st]);
                 }
@@ -394,7 +401,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             for (int j = 0; j < nt && ok; ++j) {
                 const int u = used + j;
                 const int buf = u % NB;
+                if ((warp & 3) == 0) TRACE(j, 8 + 8 * i);
                 ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_ready[i][buf], (u / NB) & 1, abort_flag));
+                if ((warp & 3) == 0) TRACE(j, 9 + 8 * i);
                 if (!ok) break;
                 tc_fence_after();
                 if (used + j == 0) TRACE_CTA(128, 2);
@@ -426,6 +435,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     for (int c = 0; c < 64; ++c) mx_raw = fmaxf(mx_raw, __uint_as_float(sr[c >> 5][c & 31]));
                 }
                 const float mx = mx_raw * p.scale_log2;
+                if ((warp & 3) == 0) TRACE(j, 10 + 8 * i);
                 // lazy rescale: only when some row's maximum grew by more than 2^8
                 const bool grow = mx > m_ref + 8.f;
                 if (j == 0) {
@@ -481,8 +491,10 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     tmem_st32(s_addr + half * 32, pk);
                 }
                 tmem_st_wait();
+                if ((warp & 3) == 0) TRACE(j, 11 + 8 * i);
                 tc_fence_before();
                 mbar_arrive(&bar->p_ready[i][buf]);
+                if ((warp & 3) == 0) TRACE(j, 12 + 8 * i);
             }
             if (!ok) break;
             TRACE_CTA(128, 3);
@@ -548,6 +560,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 }  // namespace
 
 #ifdef TMLA_TRACE
+extern "C" int typhoon_mla_debug_read_trace_naive_step(long long* dst) {
+    return (int)cudaMemcpyFromSymbol(dst, g_trace_nstep, sizeof(long long) * 64 * 32);
+}
 extern "C" int typhoon_mla_debug_read_trace_naive_cta(long long* dst) {
     return (int)cudaMemcpyFromSymbol(dst, g_trace_ncta, sizeof(long long) * 4096 * 8);
 }
