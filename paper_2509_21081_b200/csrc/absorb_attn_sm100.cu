@@ -28,6 +28,23 @@
 #include "kernels.h"
 #include "sm100.cuh"
 
+
+#ifdef TMLA_TRACE
+static __device__ unsigned long long g_kt_absorb[2] = {~0ull, 0ull};
+__device__ __forceinline__ unsigned long long kt_now_absorb() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_absorb[0], kt_now_absorb()); } while (0)
+#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_absorb[1], kt_now_absorb()); } while (0)
+extern "C" int typhoon_mla_debug_kt_absorb(unsigned long long* out) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_absorb, 16);
+    unsigned long long init[2] = {~0ull, 0ull};
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_absorb, init, 16);
+    return (int)e;
+}
+#else
+#define KT_BEGIN() do {} while (0)
+#define KT_END() do {} while (0)
+#endif
+
 namespace tmla {
 namespace {
 
@@ -112,6 +129,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     if (threadIdx.x == 0) TRACE(0, 28);
+    KT_BEGIN();
     TRACE_CTA(0);
     const int chunk = blockIdx.x, h0 = blockIdx.y * 64;
     // one 16-byte load gives the request, its suffix length and its first two pages (else three
@@ -539,6 +557,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
         __syncthreads();
     }
+    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 

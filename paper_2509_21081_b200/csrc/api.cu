@@ -79,6 +79,7 @@ struct Plan {
 };
 
 constexpr int kNumSM = 148;
+constexpr int kMaxAbsorbChunks = 1024;   // chunks per request the merge kernel accepts
 
 // Tuning aids for the tcgen05 naive kernel: TYPHOON_MLA_NAIVE_CTAS overrides the SM count the plan
 // fills, TYPHOON_MLA_NAIVE_SCHEDULE forces "split" (column split) or "streamk".
@@ -115,9 +116,10 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
         const double fixed = 3.0;
         double best_cost = 1e30;
         c = round_up(longest, 64);
-        for (int parts = 1; parts <= 32; ++parts) {
+        for (int parts = 1; parts <= 512; ++parts) {
             const int64_t ch = round_up((longest + parts - 1) / parts, 64);
             const int64_t ctas = (int64_t)units * ((Ls_absorb + ch - 1) / ch + (cap_suffix + ch - 1) / ch);
+            if (ctas / units > kMaxAbsorbChunks) continue;   // limit of the merge kernel
             const int64_t waves = (ctas + kNumSM - 1) / kNumSM;
             // a split segment writes and re-reads fp32 partials (64 heads x 2 KB, both ways): about 3.5 tiles
             // worth of traffic per chunk
@@ -132,6 +134,7 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
     } else {
         const int target = std::max(1, (2 * kNumSM + units - 1) / units);
         c = std::max<int64_t>(round_up((longest + target - 1) / target, 64), 256);
+        while ((Ls_absorb + c - 1) / c + (cap_suffix + c - 1) / c > kMaxAbsorbChunks) c *= 2;
     }
     *chunk = (int)c;
     *n_sh = (int)((Ls_absorb + c - 1) / c);

@@ -7,31 +7,109 @@
 namespace tmla {
 namespace {
 
-// One block of 128 threads per (b, h); each thread owns 4 of the 512 latent columns.
-__global__ void __launch_bounds__(128) merge_latent_kernel(const float* __restrict__ o_part,
+// One block of G x 128 threads per (b, h) (G = 1 for a few chunks, else 4): group g takes chunks g, g+G, ...;
+// each thread owns 4 of the 512 latent columns.  The chunk weights are computed once into shared
+// memory, so the partial rows are fetched by independent loads (many chunks of few tokens each are
+// the rule at small batch sizes, where this kernel would otherwise be a chain of dependent loads).
+constexpr int MERGE_MAX_CHUNKS = 1024;
+__global__ void __launch_bounds__(512) merge_latent_kernel(const float* __restrict__ o_part,
                                                            const float* __restrict__ lse_part, int n_chunks,
                                                            int BH, __nv_bfloat16* __restrict__ o_lat,
                                                            float* __restrict__ lse) {
-    const int bh = blockIdx.x;
+    __shared__ float w_s[MERGE_MAX_CHUNKS];
+    __shared__ float red[16];
+    __shared__ float4 acc_s[3][128];
+    const int bh = blockIdx.x, tid = threadIdx.x, grp = tid >> 7, col = tid & 127;
+    const int nthr = blockDim.x, G = nthr >> 7, nwarp = nthr >> 5;
+    // maximum of the chunk LSEs
     float m = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) m = fmaxf(m, lse_part[(int64_t)c * BH + bh]);
+    for (int c = tid; c < n_chunks; c += nthr) {
+        const float l = lse_part[(int64_t)c * BH + bh];
+        w_s[c] = l;
+        m = fmaxf(m, l);
+    }
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((tid & 31) == 0) red[tid >> 5] = m;
+    __syncthreads();
+    m = red[0];
+    for (int i = 1; i < nwarp; ++i) m = fmaxf(m, red[i]);
+    __syncthreads();
+    // weights (0 for an empty chunk, whose O slot was never written) and their sum
+    float z = 0.f;
+    for (int c = tid; c < n_chunks; c += nthr) {
+        const float l = w_s[c];
+        const float w = (l == -INFINITY) ? 0.f : __expf(l - m);
+        w_s[c] = w;
+        z += w;
+    }
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    if ((tid & 31) == 0) red[tid >> 5] = z;
+    __syncthreads();
+    z = 0.f;
+    for (int i = 0; i < nwarp; ++i) z += red[i];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (m != -INFINITY) {
+        const float* src = o_part + (int64_t)bh * 512 + col * 4;
+#pragma unroll 4
+        for (int c = grp; c < n_chunks; c += G) {
+            const float w = w_s[c];
+            if (w != 0.f) {
+                const float4 v = *reinterpret_cast<const float4*>(src + (int64_t)c * BH * 512);
+                acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+            }
+        }
+    }
+    if (grp > 0) acc_s[grp - 1][col] = acc;
+    __syncthreads();
+    if (grp == 0) {
+        for (int g = 0; g < G - 1; ++g) {
+            const float4 v = acc_s[g][col];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (m != -INFINITY) {
+            const float inv = 1.f / z;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        }
+        uint2 pk = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+        *reinterpret_cast<uint2*>(o_lat + (int64_t)bh * 512 + col * 4) = pk;
+        if (col == 0) lse[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(z);
+    }
+}
+
+// Few chunks per request (the common case at larger batch sizes): no shared memory, four (b, h) rows
+// per block of 512 threads, each thread owns 4 of a row's 512 latent columns and recomputes the (at most
+// MERGE_FEW) chunk weights itself.
+constexpr int MERGE_FEW = 16;
+__global__ void __launch_bounds__(512) merge_latent_few_kernel(const float* __restrict__ o_part,
+                                                               const float* __restrict__ lse_part, int n_chunks,
+                                                               int BH, __nv_bfloat16* __restrict__ o_lat,
+                                                               float* __restrict__ lse) {
+    const int bh = blockIdx.x * 4 + (threadIdx.x >> 7), col = threadIdx.x & 127;
+    if (bh >= BH) return;
+    float l[MERGE_FEW];
+    float m = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < MERGE_FEW; ++c) {
+        l[c] = c < n_chunks ? lse_part[(int64_t)c * BH + bh] : -INFINITY;
+        m = fmaxf(m, l[c]);
+    }
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
     if (m != -INFINITY) {
-        for (int c = 0; c < n_chunks; ++c) {
-            float l = lse_part[(int64_t)c * BH + bh];
-            if (l == -INFINITY) continue;  // empty chunk: its O slot was never written
-            float w = __expf(l - m);
-            float4 v = *reinterpret_cast<const float4*>(o_part + ((int64_t)c * BH + bh) * 512 + threadIdx.x * 4);
+#pragma unroll
+        for (int c = 0; c < MERGE_FEW; ++c) {
+            if (l[c] == -INFINITY) continue;   // empty chunk (or none): its O slot was never written
+            const float w = __expf(l[c] - m);
+            const float4 v = *reinterpret_cast<const float4*>(o_part + ((int64_t)c * BH + bh) * 512 + col * 4);
             acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
             z += w;
         }
-        float inv = 1.f / z;
+        const float inv = 1.f / z;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }
     uint2 pk = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-    *reinterpret_cast<uint2*>(o_lat + (int64_t)bh * 512 + threadIdx.x * 4) = pk;
-    if (threadIdx.x == 0) lse[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(z);
+    *reinterpret_cast<uint2*>(o_lat + (int64_t)bh * 512 + col * 4) = pk;
+    if (col == 0) lse[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(z);
 }
 
 // One warp per (b, h); each lane owns 4 of the 128 output columns.
@@ -123,8 +201,14 @@ cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm
 cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,
                                 void* o_lat_bf16, float* lse, cudaStream_t s) {
     if (B * H <= 0) return cudaSuccess;
-    merge_latent_kernel<<<B * H, 128, 0, s>>>(o_part, lse_part, n_chunks, B * H,
-                                              reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
+    if (n_chunks > MERGE_MAX_CHUNKS) return cudaErrorInvalidValue;
+    if (n_chunks <= MERGE_FEW) {
+        merge_latent_few_kernel<<<(B * H + 3) / 4, 512, 0, s>>>(o_part, lse_part, n_chunks, B * H,
+                                                                reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
+    } else {
+        merge_latent_kernel<<<B * H, 512, 0, s>>>(o_part, lse_part, n_chunks, B * H,
+                                                  reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
+    }
     return cudaGetLastError();
 }
 

@@ -11,6 +11,23 @@
 #include "kernels.h"
 #include "sm100.cuh"
 
+
+#ifdef TMLA_TRACE
+static __device__ unsigned long long g_kt_gemm[2] = {~0ull, 0ull};
+__device__ __forceinline__ unsigned long long kt_now_gemm() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_gemm[0], kt_now_gemm()); } while (0)
+#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_gemm[1], kt_now_gemm()); } while (0)
+extern "C" int typhoon_mla_debug_kt_gemm(unsigned long long* out) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_gemm, 16);
+    unsigned long long init[2] = {~0ull, 0ull};
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_gemm, init, 16);
+    return (int)e;
+}
+#else
+#define KT_BEGIN() do {} while (0)
+#define KT_END() do {} while (0)
+#endif
+
 namespace tmla {
 namespace {
 
@@ -41,6 +58,7 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
+    KT_BEGIN();
     const int KB = p.K / BK;
 
     if (threadIdx.x == 0) {
@@ -199,6 +217,7 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
+    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 128);
 }
 

@@ -43,6 +43,23 @@
 #include "kernels.h"
 #include "sm100.cuh"
 
+
+#ifdef TMLA_TRACE
+static __device__ unsigned long long g_kt_naive[2] = {~0ull, 0ull};
+__device__ __forceinline__ unsigned long long kt_now_naive() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_naive[0], kt_now_naive()); } while (0)
+#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_naive[1], kt_now_naive()); } while (0)
+extern "C" int typhoon_mla_debug_kt_naive(unsigned long long* out) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_naive, 16);
+    unsigned long long init[2] = {~0ull, 0ull};
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_naive, init, 16);
+    return (int)e;
+}
+#else
+#define KT_BEGIN() do {} while (0)
+#define KT_END() do {} while (0)
+#endif
+
 namespace tmla {
 namespace {
 
@@ -123,6 +140,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const int rng = blockIdx.x / p.m_groups, grp = blockIdx.x % p.m_groups;
+    KT_BEGIN();
     TRACE_CTA(0, 0);
 
     // this CTA's contiguous range of the global tile sequence (T < 2^31: 32-bit arithmetic)
@@ -554,6 +572,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
         __syncthreads();
     }
+    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 

@@ -11,6 +11,23 @@
 #include "kernels.h"
 #include "sm100.cuh"
 
+
+#ifdef TMLA_TRACE
+static __device__ unsigned long long g_kt_qabs[2] = {~0ull, 0ull};
+__device__ __forceinline__ unsigned long long kt_now_qabs() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_qabs[0], kt_now_qabs()); } while (0)
+#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_qabs[1], kt_now_qabs()); } while (0)
+extern "C" int typhoon_mla_debug_kt_qabs(unsigned long long* out) {
+    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_qabs, 16);
+    unsigned long long init[2] = {~0ull, 0ull};
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_qabs, init, 16);
+    return (int)e;
+}
+#else
+#define KT_BEGIN() do {} while (0)
+#define KT_END() do {} while (0)
+#endif
+
 namespace tmla {
 namespace {
 
@@ -38,6 +55,7 @@ __global__ void __launch_bounds__(192, 1)
 q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w, QAbsorbParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    KT_BEGIN();
     if ((int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
         if (blockIdx.x == 0) {
             block_order_by_length(p.seq_lens, p.B, p.order, reinterpret_cast<unsigned long long*>(smem));
@@ -136,6 +154,7 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
+    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
