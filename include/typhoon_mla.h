@@ -138,7 +138,13 @@ size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* shared, int32_t B
  * Token slots past a request's length and unused block-table entries are never
  * read into the result.  A request with no context at all (Ls = 0 and
  * seq_lens[b] = 0) gets a zero output row and lse = -inf.
- * The call never allocates and never synchronises.
+ * The call never allocates and never synchronises.  It only enqueues kernels on
+ * `stream` and, in HYBRID mode, on the handle's side stream (forked from and
+ * joined back to `stream` with events inside the call), so it may be captured
+ * into a CUDA graph; a replay reads the buffers' contents at replay time and
+ * uses the pointers, sizes and mode given at capture time (AUTO is resolved at
+ * capture).  Calls on the same handle from several host threads at once are not
+ * supported (the side stream and its events belong to the handle).
  * Errors: INVALID_ARG (NULL/misaligned pointers, B < 1, bad mode or page size),
  * WORKSPACE_TOO_SMALL, CUDA (launch failure; see typhoon_mla_last_cuda_error).
  */

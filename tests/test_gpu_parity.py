@@ -252,6 +252,44 @@ def test_decode_host_matches_device_call():
     dec.close()
 
 
+def test_decode_captured_in_a_cuda_graph(kernel_path):
+    """The decode call only enqueues kernels and event record/wait operations (on the given stream and
+    on the handle's side stream), so it can be captured; replays see the buffers' current contents."""
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    cfg = _cfg("graph", B=7, H=32, Ls=300, lo=5, hi=200, seed=36)
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp, poison=False)
+    dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(),
+                            inp.scale, cfg.B, pc.block_table.shape[1])
+    q_nope, q_pe = inp.q_nope.cuda(), inp.q_pe.cuda()
+    args = (q_nope, q_pe, pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), pc.block_table.cuda(), pc.seq_lens.cuda())
+    out = torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16, device="cuda")
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        dec.decode(*args, mode=HYBRID, out=out)      # an ordinary call first
+        st.synchronize()
+        direct = out.clone()
+        with torch.cuda.graph(g, stream=st):
+            dec.decode(*args, mode=HYBRID, out=out)
+    out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, direct)
+    # new queries in the same buffers
+    q_nope.copy_(torch.flip(q_nope, dims=[0]))
+    q_pe.copy_(torch.flip(q_pe, dims=[0]))
+    g.replay()
+    torch.cuda.synchronize()
+    replayed = out.clone()
+    dec.decode(*args, mode=HYBRID, out=out)
+    torch.cuda.synchronize()
+    assert torch.equal(out, replayed) and not torch.equal(out, direct)
+    assert b.typhoon_mla_device_status(dec.shared) == 0
+    dec.close()
+
+
 def test_invalid_arguments():
     from paper_2509_21081_b200 import binding as b
     cfg = _cfg("inval", B=2, H=16, Ls=64, lo=8, hi=8, seed=33)
