@@ -316,19 +316,28 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     # ---- end to end: per-step tensors from pinned host memory, result read back, every step
     e2e = None
     if with_e2e:
-        hq = [(inp.q_nope.pin_memory(), inp.q_pe.pin_memory(), pc.block_table.pin_memory(), pc.seq_lens.pin_memory(),
-               torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16).pin_memory()) for _ in range(n_sets)]
-
-        # Two steps are kept in flight, each on its own stream with its own decoder (workspace, staging,
-        # pinned buffers), so that the copies of one step overlap the kernels of the other, as a serving
-        # loop would do.  Every step still copies its inputs in and its result out.
-        streams = [torch.cuda.Stream() for _ in range(n_sets)]
+        # Four steps are kept in flight ("lanes"), each on its own stream with its own decoder (prepared
+        # prefix, workspace, staging) and pinned buffers, so that the copies of one step overlap the kernels
+        # of the others, as a serving loop with several micro-batches would do.  Every step still copies
+        # its inputs in and its result out.  Lane k reads the device-resident caches of input set k % 2.
+        n_lanes = int(os.environ.get("TYPHOON_MLA_BENCH_LANES", "4"))
+        lanes = []
+        for k in range(n_lanes):
+            s = sets[k % n_sets]
+            dec = s["dec"] if k < n_sets else TyphoonMLADecoder(
+                cfg.H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), s["dec"].w_uk, s["dec"].w_uv, inp.scale,
+                cfg.B, max_pages, pc.page_size)
+            lanes.append(dict(dec=dec, ckv=s["ckv"], kpe=s["kpe"], stream=torch.cuda.Stream(),
+                              h=(inp.q_nope.pin_memory(), inp.q_pe.pin_memory(), pc.block_table.pin_memory(),
+                                 pc.seq_lens.pin_memory(),
+                                 torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16).pin_memory())))
+        streams = [ln["stream"] for ln in lanes]
 
         def step_host(i):
-            k = i % n_sets
-            s, h = sets[k], hq[k]
-            with torch.cuda.stream(streams[k]):
-                s["dec"].decode_host(h[0], h[1], s["ckv"], s["kpe"], h[2], h[3], h[4], mode=mode)
+            ln = lanes[i % n_lanes]
+            h = ln["h"]
+            with torch.cuda.stream(ln["stream"]):
+                ln["dec"].decode_host(h[0], h[1], ln["ckv"], ln["kpe"], h[2], h[3], h[4], mode=mode)
 
         def fork():
             for st in streams:
@@ -355,7 +364,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         d2h = cfg.B * cfg.H * 128 * 2
         e2e = {"value": whole_job_value(cfg.B, world, e_ms), "unit": UNIT, "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "pipelining": f"{n_sets} steps in flight on {n_sets} streams (own workspace, staging and pinned buffers each)"}
+               "pipelining": f"{n_lanes} steps in flight on {n_lanes} streams (own decoder, workspace, staging and pinned buffers each)"}
 
     cpu = None
     if with_cpu and rank == 0 and world == 1:
