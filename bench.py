@@ -143,7 +143,7 @@ class ClockSampler:
                             self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.005)
+            time.sleep(0.001)
 
     def __enter__(self):
         if self.nv:

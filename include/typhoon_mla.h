@@ -244,6 +244,10 @@ int typhoon_mla_set_kernel_path(int32_t path);
  * kernel on the caller's stream, one after the other (measurement aid).  Process-wide. */
 int typhoon_mla_set_overlap(int32_t enable);
 
+/* Work decomposition of the tcgen05 shared-prefix kernel (see typhoon_mla_naive_plan): 0 = the
+ * library's choice (default), 1 = column split, 2 = stream-K.  Measurement and test aid; process-wide. */
+int typhoon_mla_set_naive_schedule(int32_t schedule);
+
 /* Synchronises `stream` and reads the handle's device status word.  Every in-kernel wait of the
  * tcgen05 kernels has a deadline; if one expired, the kernel abandoned its work, the word is
  * non-zero and this returns TYPHOON_MLA_ERR_DEVICE_CHECK (results of that launch are invalid). */

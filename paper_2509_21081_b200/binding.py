@@ -84,6 +84,8 @@ def _load():
     lib.typhoon_mla_set_kernel_path.argtypes = [i32]
     lib.typhoon_mla_order_by_length.restype = C.c_int
     lib.typhoon_mla_order_by_length.argtypes = [vp, i32, vp, vp]
+    lib.typhoon_mla_set_naive_schedule.restype = C.c_int
+    lib.typhoon_mla_set_naive_schedule.argtypes = [i32]
     lib.typhoon_mla_set_overlap.restype = C.c_int
     lib.typhoon_mla_set_overlap.argtypes = [i32]
     lib.typhoon_mla_device_status.restype = C.c_int
@@ -285,6 +287,10 @@ def typhoon_mla_device_status(shared: SharedPrefix) -> int:
     v = C.c_int32()
     _check(_lib.typhoon_mla_device_status(shared.handle, _stream(), C.byref(v)), "typhoon_mla_device_status")
     return v.value
+
+
+def typhoon_mla_set_naive_schedule(schedule: int) -> None:
+    _check(_lib.typhoon_mla_set_naive_schedule(schedule), "typhoon_mla_set_naive_schedule")
 
 
 def typhoon_mla_set_overlap(enable: bool) -> None:

@@ -82,7 +82,7 @@ constexpr int kNumSM = 148;
 constexpr int kMaxAbsorbChunks = 1024;   // chunks per request the merge kernel accepts
 
 // Tuning aids for the tcgen05 naive kernel: TYPHOON_MLA_NAIVE_CTAS overrides the SM count the plan
-// fills, TYPHOON_MLA_NAIVE_SCHEDULE forces "split" (column split) or "streamk".
+// fills, TYPHOON_MLA_NAIVE_SCHEDULE ("split" or "streamk") the initial value of typhoon_mla_set_naive_schedule.
 int naive_sm_budget() {
     if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_CTAS")) {
         const int v = std::atoi(ov);
@@ -90,13 +90,14 @@ int naive_sm_budget() {
     }
     return kNumSM;
 }
-int naive_schedule() {
+int g_naive_schedule = [] {   // process-wide; TYPHOON_MLA_NAIVE_SCHEDULE sets the initial value
     if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_SCHEDULE")) {
         if (std::strcmp(ov, "split") == 0) return 1;
         if (std::strcmp(ov, "streamk") == 0) return 2;
     }
     return 0;
-}
+}();
+int naive_schedule() { return g_naive_schedule; }
 
 int naive_splits(int B, int H, int64_t Ls) {
     if (Ls <= 0) return 0;
@@ -408,6 +409,12 @@ int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* per
 
 int typhoon_mla_set_overlap(int32_t enable) {
     g_overlap = enable != 0;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_set_naive_schedule(int32_t schedule) {
+    if (schedule < 0 || schedule > 2) return TYPHOON_MLA_ERR_INVALID_ARG;
+    g_naive_schedule = schedule;
     return TYPHOON_MLA_OK;
 }
 

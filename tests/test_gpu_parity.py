@@ -25,6 +25,14 @@ def kernel_path(request):
     b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05)
 
 
+@pytest.fixture
+def naive_schedule():
+    """Selects the work decomposition of the shared-prefix kernel for one test."""
+    from paper_2509_21081_b200 import binding as b
+    yield lambda name: b.typhoon_mla_set_naive_schedule({"auto": 0, "split": 1, "streamk": 2}[name])
+    b.typhoon_mla_set_naive_schedule(0)
+
+
 def _cfg(name, B, H, Ls, lo, hi, seed, page_size=64):
     return I.MLAConfig(name, B=B, H=H, Ls=Ls, suffix_lo=lo, suffix_hi=hi, seed=seed, page_size=page_size)
 
@@ -63,11 +71,11 @@ def test_head_counts_and_batch_tail(H):
 
 @pytest.mark.parametrize("schedule", ["split", "streamk"])
 @pytest.mark.parametrize("B,H,Ls", [(70, 64, 520), (5, 32, 1000), (150, 16, 1100), (300, 16, 700), (400, 32, 450)])
-def test_naive_schedules(schedule, B, H, Ls, monkeypatch):
+def test_naive_schedules(schedule, B, H, Ls, naive_schedule):
     """Both work decompositions of the shared-prefix kernel (every tile range inside one head; equal
     ranges that cross heads), for 64- and 128-token tiles, one and two query-row groups, a last
     row group with and without a second row tile."""
-    monkeypatch.setenv("TYPHOON_MLA_NAIVE_SCHEDULE", schedule)
+    naive_schedule(schedule)
     cfg = _cfg("sched", B=B, H=H, Ls=Ls, lo=0, hi=90, seed=40 + B)
     inp = I.make_inputs(cfg)
     ref, ref_lse = G.run_oracle(inp)
@@ -76,7 +84,7 @@ def test_naive_schedules(schedule, B, H, Ls, monkeypatch):
 
 
 @pytest.mark.parametrize("seed", range(10))
-def test_random_shapes(seed, monkeypatch):
+def test_random_shapes(seed, naive_schedule):
     """Seeded random problem sizes, modes, page sizes and work decompositions: pipeline phase logic
     (ring wrap-around, segments per CTA, odd tile counts, partial row groups) against the checker."""
     import random
@@ -87,7 +95,7 @@ def test_random_shapes(seed, monkeypatch):
     hi = rnd.choice([0, 5, 70, 200])
     page_size = rnd.choice([64, 128])
     mode = rnd.choice([HYBRID, HYBRID, ABSORB, AUTO])
-    monkeypatch.setenv("TYPHOON_MLA_NAIVE_SCHEDULE", rnd.choice(["split", "streamk", "auto"]))
+    naive_schedule(rnd.choice(["split", "streamk", "auto"]))
     cfg = _cfg("rand", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=500 + seed, page_size=page_size)
     inp = I.make_inputs(cfg)
     ref, ref_lse = G.run_oracle(inp)
