@@ -216,6 +216,19 @@ int typhoon_mla_cost_model(const typhoon_mla_dims_t* dims /* host */, int32_t ki
                            int64_t B, int64_t S_q, int64_t L_s, int64_t L_n,
                            int64_t* macs /* host */, int64_t* hbm_words /* host */);
 
+/* Several query tokens per request (S_q of Table 1, e.g. the verification step of speculative
+ * decoding): the cache already holds the S_q new tokens of every request and query token j
+ * (0 <= j < S_q) attends to the shared prefix and to the first seq_lens[b] - (S_q - 1 - j) suffix
+ * tokens (causal among the new tokens).  The path treats every (request, query token) pair as a row:
+ * this call writes the page table block_table_rows int32 [B * S_q, max_pages] and the lengths
+ * seq_lens_rows int32 [B * S_q] of the rows (row = b * S_q + j; negative lengths become 0), which
+ * typhoon_mla_decode then takes with B * S_q in place of B and q arrays of B * S_q rows.  All pointers
+ * are device pointers; asynchronous on `stream`; no allocation.  The paper states the cost model for
+ * S_q (Table 1, Eq. 1) and evaluates S_q = 1 only. */
+int typhoon_mla_expand_query_rows(const int32_t* block_table, const int32_t* seq_lens, int32_t B,
+                                  int32_t max_pages, int32_t S_q, int32_t* block_table_rows,
+                                  int32_t* seq_lens_rows, void* stream);
+
 /* Work decomposition the tcgen05 shared-prefix kernel (Algorithm 1 line 4) would use for a problem
  * size: tokens per KV tile (64 for B <= 128, else 128), number of contiguous tile ranges the H * n_tiles
  * tiles are cut into, query-row groups per range (CTAs = ranges * row_groups) and partial slots written

@@ -84,6 +84,8 @@ def _load():
     lib.typhoon_mla_set_kernel_path.argtypes = [i32]
     lib.typhoon_mla_order_by_length.restype = C.c_int
     lib.typhoon_mla_order_by_length.argtypes = [vp, i32, vp, vp]
+    lib.typhoon_mla_expand_query_rows.restype = C.c_int
+    lib.typhoon_mla_expand_query_rows.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.typhoon_mla_set_naive_schedule.restype = C.c_int
     lib.typhoon_mla_set_naive_schedule.argtypes = [i32]
     lib.typhoon_mla_set_overlap.restype = C.c_int
@@ -287,6 +289,16 @@ def typhoon_mla_device_status(shared: SharedPrefix) -> int:
     v = C.c_int32()
     _check(_lib.typhoon_mla_device_status(shared.handle, _stream(), C.byref(v)), "typhoon_mla_device_status")
     return v.value
+
+
+def typhoon_mla_expand_query_rows(block_table: torch.Tensor, seq_lens: torch.Tensor, S_q: int):
+    """(block_table_rows [B*S_q, max_pages], seq_lens_rows [B*S_q]) for S_q query tokens per request."""
+    B, max_pages = block_table.shape
+    bt = torch.empty(B * S_q, max_pages, dtype=torch.int32, device=block_table.device)
+    sl = torch.empty(B * S_q, dtype=torch.int32, device=block_table.device)
+    _check(_lib.typhoon_mla_expand_query_rows(_ptr(block_table), _ptr(seq_lens), B, max_pages, S_q, _ptr(bt), _ptr(sl),
+                                              _stream()), "typhoon_mla_expand_query_rows")
+    return bt, sl
 
 
 def typhoon_mla_set_naive_schedule(schedule: int) -> None:

@@ -401,6 +401,16 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* sh, const void** k_nope,
     return TYPHOON_MLA_OK;
 }
 
+int typhoon_mla_expand_query_rows(const int32_t* block_table, const int32_t* seq_lens, int32_t B, int32_t max_pages,
+                                  int32_t S_q, int32_t* block_table_rows, int32_t* seq_lens_rows, void* stream) {
+    if (!seq_lens || !seq_lens_rows || B < 1 || S_q < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (max_pages > 0 && (!block_table || !block_table_rows)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if ((int64_t)B * S_q > INT32_MAX) return TYPHOON_MLA_ERR_INVALID_ARG;
+    cudaError_t e = launch_expand_query_rows(block_table, seq_lens, B, max_pages, S_q, block_table_rows, seq_lens_rows,
+                                             reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
+}
+
 int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* perm, void* stream) {
     if (!seq_lens || !perm || B < 1 || B > 4096) return TYPHOON_MLA_ERR_INVALID_ARG;
     cudaError_t e = launch_order_by_length(seq_lens, B, perm, reinterpret_cast<cudaStream_t>(stream));

@@ -1,6 +1,8 @@
 // Vector kernels of the path: merge of absorb chunk partials, the final LSE
 // combine (Algorithm 1 line 8; Section 3.2 "CombineLSE") and layout helpers
 // used once per prefix by the expansion step.
+#include <algorithm>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -190,11 +192,36 @@ __global__ void __launch_bounds__(1024) order_by_length_kernel(const int32_t* __
     block_order_by_length(seq_lens, B, perm, keys);
 }
 
+// Row expansion for S_q query tokens per request (Table 1's S_q; causal among the new tokens):
+// row b * S_q + j gets request b's page-table row and the suffix length minus the S_q - 1 - j later tokens.
+__global__ void __launch_bounds__(256) expand_query_rows_kernel(const int32_t* __restrict__ block_table,
+                                                                const int32_t* __restrict__ seq_lens, int B,
+                                                                int max_pages, int S_q,
+                                                                int32_t* __restrict__ bt_rows,
+                                                                int32_t* __restrict__ len_rows) {
+    const int64_t n_bt = (int64_t)B * S_q * max_pages;
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n_bt; i += (int64_t)gridDim.x * 256) {
+        const int64_t row = i / max_pages;
+        bt_rows[i] = block_table[(row / S_q) * max_pages + i % max_pages];
+    }
+    for (int i = blockIdx.x * 256 + threadIdx.x; i < B * S_q; i += gridDim.x * 256)
+        len_rows[i] = max(seq_lens[i / S_q] - (S_q - 1 - i % S_q), 0);
+}
+
 }  // namespace
 
 cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm, cudaStream_t s) {
     if (B <= 0 || B > 4096) return cudaErrorInvalidValue;
     order_by_length_kernel<<<1, 1024, 0, s>>>(seq_lens, B, perm);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_expand_query_rows(const int32_t* block_table, const int32_t* seq_lens, int B, int max_pages, int S_q,
+                                     int32_t* bt_rows, int32_t* len_rows, cudaStream_t s) {
+    if (B <= 0 || S_q <= 0) return cudaSuccess;
+    const int64_t n = std::max<int64_t>((int64_t)B * S_q * max_pages, (int64_t)B * S_q);
+    const unsigned blocks = (unsigned)std::min<int64_t>((n + 255) / 256, 1184);
+    expand_query_rows_kernel<<<blocks, 256, 0, s>>>(block_table, seq_lens, B, max_pages, S_q, bt_rows, len_rows);
     return cudaGetLastError();
 }
 

@@ -103,6 +103,9 @@ cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t L
                                      CUtensorMap* tm_kpe);
 
 // perm[0..B) = request indices by descending suffix length (B <= 4096).
+// Page table and lengths of the (request, query token) rows of a step with S_q query tokens per request.
+cudaError_t launch_expand_query_rows(const int32_t* block_table, const int32_t* seq_lens, int B, int max_pages, int S_q,
+                                     int32_t* bt_rows, int32_t* len_rows, cudaStream_t s);
 cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm, cudaStream_t s);
 
 // Merge absorb chunk partials -> bf16 latent output [B,H,512] + lse [B,H].

@@ -298,6 +298,42 @@ def test_decode_captured_in_a_cuda_graph(kernel_path):
     dec.close()
 
 
+@pytest.mark.parametrize("S_q", [2, 3])
+def test_several_query_tokens_per_request(S_q):
+    """S_q query tokens per request (Table 1's S_q): rows = (request, query token) pairs sharing the
+    request's pages, causal among the new tokens.  The checker sees each row as a request whose suffix is
+    cut after its own token; one request is shorter than S_q (its first query sees the prefix only)."""
+    import dataclasses
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    B, H = 6, 32
+    cfg = _cfg("sq", B=B, H=H, Ls=300, lo=0, hi=0, seed=37)
+    lens = [S_q - 1, 5, 64, 65, 130, 200]
+    inp = I.make_inputs(cfg, suffix_lens=lens)
+    pc = I.build_pages(inp)
+    # queries of the B * S_q rows: a second draw with as many requests (same seed: same prefix and weights)
+    rows = I.make_inputs(dataclasses.replace(cfg, B=B * S_q), suffix_lens=[0] * (B * S_q))
+    row_lens = [max(lens[r // S_q] - (S_q - 1 - r % S_q), 0) for r in range(B * S_q)]
+    rows.suffix_lens = row_lens
+    rows.ckv_suffix = [inp.ckv_suffix[r // S_q][: row_lens[r]] for r in range(B * S_q)]
+    rows.kpe_suffix = [inp.kpe_suffix[r // S_q][: row_lens[r]] for r in range(B * S_q)]
+    assert torch.equal(rows.ckv_shared, inp.ckv_shared) and torch.equal(rows.w_uk, inp.w_uk)
+    ref, ref_lse = G.run_oracle(rows)
+    bt_rows, sl_rows = b.typhoon_mla_expand_query_rows(pc.block_table.cuda(), pc.seq_lens.cuda(), S_q)
+    assert sl_rows.cpu().tolist() == row_lens
+    assert torch.equal(bt_rows.cpu(), pc.block_table.repeat_interleave(S_q, dim=0))
+    dec = TyphoonMLADecoder(H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(),
+                            inp.scale, B * S_q, pc.block_table.shape[1])
+    for mode in (HYBRID, ABSORB):
+        lse = torch.empty(B * S_q, H, dtype=torch.float32, device="cuda")
+        out = dec.decode(rows.q_nope.cuda(), rows.q_pe.cuda(), pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), bt_rows,
+                         sl_rows, mode=mode, lse_out=lse)
+        assert b.typhoon_mla_device_status(dec.shared) == 0
+        G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse,
+                        what=f"S_q={S_q} mode {mode}")
+    dec.close()
+
+
 def test_invalid_arguments():
     from paper_2509_21081_b200 import binding as b
     cfg = _cfg("inval", B=2, H=16, Ls=64, lo=8, hi=8, seed=33)
