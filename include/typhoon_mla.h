@@ -216,6 +216,37 @@ int typhoon_mla_cost_model(const typhoon_mla_dims_t* dims /* host */, int32_t ki
                            int64_t B, int64_t S_q, int64_t L_s, int64_t L_n,
                            int64_t* macs /* host */, int64_t* hbm_words /* host */);
 
+/*
+ * Several shared prefixes in one step (Section 3.1: tree-structured prompts, e.g. a system prompt
+ * shared by all requests and one further prompt per group of requests).  A level partitions the
+ * requests 0..B-1 into consecutive groups; group g = requests [group_begin[g], group_begin[g+1]) shares
+ * prefixes[g] (NULL: that group has no prefix at this level).  A request attends to the prefix of its
+ * group at every level and to its own suffix; all parts are merged by the LSE combine (Algorithm 1
+ * line 8 with more partials).  Line 4 runs once per (level, group) over that group's query rows; lines
+ * 5-7 run once for the whole batch.  All handles must have the same head count and were prepared with
+ * the same weights (the first non-NULL handle's are used for the projections).  Both arrays are host
+ * arrays; at most 8 levels and 256 non-empty (level, group) pairs.  tcgen05 kernel path only
+ * (UNSUPPORTED_DIMS otherwise).  Other arguments, errors and the stream behaviour are those of
+ * typhoon_mla_decode in HYBRID mode.  The paper describes this extension and does not evaluate it.
+ */
+typedef struct {
+    const typhoon_mla_shared_t* const* prefixes; /* host array [n_groups] */
+    const int32_t* group_begin;                  /* host array [n_groups + 1]: 0 = [0] <= ... <= [n_groups] = B */
+    int32_t n_groups;
+} typhoon_mla_prefix_level_t;
+
+size_t typhoon_mla_tree_workspace_bytes(const typhoon_mla_prefix_level_t* levels /* host */, int32_t n_levels,
+                                        int32_t B, int32_t max_pages, int32_t page_size);
+
+int typhoon_mla_decode_tree(const typhoon_mla_prefix_level_t* levels /* host */, int32_t n_levels,
+                            const void* q_nope, const void* q_pe, int32_t B,
+                            const void* ckv_pages, const void* kpe_pages,
+                            int64_t ckv_token_stride, int64_t kpe_token_stride,
+                            int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                            const int32_t* seq_lens, float softmax_scale,
+                            void* out, float* lse_out,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 /* Several query tokens per request (S_q of Table 1, e.g. the verification step of speculative
  * decoding): the cache already holds the S_q new tokens of every request and query token j
  * (0 <= j < S_q) attends to the shared prefix and to the first seq_lens[b] - (S_q - 1 - j) suffix

@@ -56,6 +56,11 @@ def _load():
     lib.typhoon_mla_decode.restype = C.c_int
     lib.typhoon_mla_decode.argtypes = [vp, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, i32, vp, vp,
                                        vp, sz, vp]
+    lib.typhoon_mla_tree_workspace_bytes.restype = sz
+    lib.typhoon_mla_tree_workspace_bytes.argtypes = [vp, i32, i32, i32, i32]
+    lib.typhoon_mla_decode_tree.restype = C.c_int
+    lib.typhoon_mla_decode_tree.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, vp, vp,
+                                            vp, sz, vp]
     lib.typhoon_mla_host_staging_bytes.restype = sz
     lib.typhoon_mla_host_staging_bytes.argtypes = [vp, i32, i32]
     lib.typhoon_mla_decode_host.restype = C.c_int
@@ -179,6 +184,44 @@ def typhoon_mla_decode(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages,
                                  _ptr(seq_lens), softmax_scale, mode, _ptr(out), _ptr(lse_out),
                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check(st, "typhoon_mla_decode")
+
+
+class PrefixLevel(C.Structure):
+    """typhoon_mla_prefix_level_t"""
+    _fields_ = [("prefixes", C.POINTER(C.c_void_p)), ("group_begin", C.POINTER(C.c_int32)), ("n_groups", C.c_int32)]
+
+
+def _marshal_levels(levels):
+    """levels: list of (prefixes, group_begin) with prefixes a list of SharedPrefix or None.
+    Returns (array of PrefixLevel, keepalive)."""
+    arr = (PrefixLevel * len(levels))()
+    keep = []
+    for i, (prefixes, group_begin) in enumerate(levels):
+        if len(group_begin) != len(prefixes) + 1:
+            raise ValueError("group_begin needs one more entry than prefixes")
+        hp = (C.c_void_p * len(prefixes))(*[None if p is None else p.handle.value for p in prefixes])
+        gb = (C.c_int32 * len(group_begin))(*group_begin)
+        keep += [hp, gb]
+        arr[i] = PrefixLevel(C.cast(hp, C.POINTER(C.c_void_p)), C.cast(gb, C.POINTER(C.c_int32)), len(prefixes))
+    return arr, keep
+
+
+def typhoon_mla_tree_workspace_bytes(levels, B: int, max_pages: int, page_size: int) -> int:
+    arr, keep = _marshal_levels(levels)
+    return int(_lib.typhoon_mla_tree_workspace_bytes(C.cast(arr, C.c_void_p), len(levels), B, max_pages, page_size))
+
+
+def typhoon_mla_decode_tree(levels, q_nope, q_pe, ckv_pages, kpe_pages, page_size, block_table, seq_lens,
+                            softmax_scale, out, workspace, lse_out=None) -> None:
+    arr, keep = _marshal_levels(levels)
+    B = q_nope.shape[0]
+    max_pages = 0 if block_table is None else block_table.shape[1]
+    st = _lib.typhoon_mla_decode_tree(
+        C.cast(arr, C.c_void_p), len(levels), _ptr(q_nope), _ptr(q_pe), B, _ptr(ckv_pages), _ptr(kpe_pages),
+        512 if ckv_pages is None else ckv_pages.stride(-2), 64 if kpe_pages is None else kpe_pages.stride(-2),
+        page_size, _ptr(block_table), max_pages, _ptr(seq_lens), softmax_scale, _ptr(out), _ptr(lse_out),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
+    _check(st, "typhoon_mla_decode_tree")
 
 
 def typhoon_mla_host_staging_bytes(shared: SharedPrefix, B: int, max_pages: int) -> int:

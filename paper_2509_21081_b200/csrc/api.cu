@@ -142,7 +142,7 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
     *n_sf = (int)((cap_suffix + c - 1) / c);
 }
 
-Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size, int mode) {
+Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size, int mode, int naive_slots_override = -1) {
     Plan p{};
     const int H = sh->dims.num_heads;
     p.mode = mode;
@@ -150,7 +150,10 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
     const bool use_naive = (mode != TYPHOON_MLA_MODE_ABSORB) && sh->Ls > 0;
     const bool use_absorb = (mode != TYPHOON_MLA_MODE_NAIVE);
     const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
-    if (use_naive && tc) {
+    if (naive_slots_override >= 0) {   // several shared-prefix launches planned by the caller
+        p.n_split_naive = naive_slots_override > 0 ? 1 : 0;
+        p.n_slots_naive = naive_slots_override;
+    } else if (use_naive && tc) {
         naive_sm100_plan(B, H, sh->Ls, naive_sm_budget(), naive_schedule(), &p.n_split_naive, &p.n_slots_naive);   // n_split_naive = tile ranges
     } else {
         p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls) : 0;
@@ -469,30 +472,29 @@ size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* sh, int32_t B, in
     return worst + 256;
 }
 
-int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
-                       const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
-                       int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
-                       const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
-                       void* workspace, size_t workspace_bytes, void* stream) {
-    g_last_launches = 0;
-    if (!sh || !q_nope || !q_pe || !out || B < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (mode < TYPHOON_MLA_MODE_AUTO || mode > TYPHOON_MLA_MODE_NAIVE) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return TYPHOON_MLA_ERR_INVALID_ARG;   // positive, finite
-    mode = resolve_mode(sh, B, max_pages, mode);
-    const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
-    if (use_absorb && max_pages > 0) {
-        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens) return TYPHOON_MLA_ERR_INVALID_ARG;
-        if (!aligned16(ckv_pages) || !aligned16(kpe_pages) || ckv_token_stride < 512 || kpe_token_stride < 64 ||
-            ckv_token_stride % 8 || kpe_token_stride % 8)
-            return TYPHOON_MLA_ERR_INVALID_ARG;
-    }
-    if (mode == TYPHOON_MLA_MODE_NAIVE && sh->Ls == 0) max_pages = 0;
-    const Plan pl = make_plan(sh, B, use_absorb ? max_pages : 0, page_size, mode);
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
+// One launch of the shared-prefix kernel: `rows` requests starting at `row0` against the prefix of
+// `sh`, partial slots [slot0, slot0 + n_slots_level) of the step's partial arrays.
+struct NaiveJob {
+    const typhoon_mla_shared* sh;
+    int row0, rows;
+    int n_ranges;         // tile ranges (tcgen05 path) or KV splits (warp-MMA path)
+    int n_slots_level;    // slots of this job's level (the kernel marks the ones it does not fill as empty)
+    int slot0;
+};
+// Rows of a level that have no prefix: their slots get weight zero in the combine.
+struct EmptySlots {
+    int slot0, n_slots, row0, rows;
+};
 
+// Launch sequence of one step.  `sh` provides the weights, the absorb-side tensor maps, the side stream
+// and the status word; `mode` is resolved (ABSORB, HYBRID or NAIVE); `pl.n_slots_naive` is the total
+// number of naive partial slots.
+static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n_jobs, const EmptySlots* empties, int n_empties,
+                const Plan& pl, const void* q_nope, const void* q_pe, int32_t B, const void* ckv_pages,
+                const void* kpe_pages, int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size,
+                const int32_t* block_table, int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode,
+                void* out, float* lse_out, void* workspace, void* stream) {
+    const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     char* ws = reinterpret_cast<char*>(workspace);
     const int H = sh->dims.num_heads;
@@ -511,26 +513,39 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     // on the handle's (high-priority) side stream, forked behind the caller's stream here and joined
     // before the projection.
     cudaStream_t s_main = s;
-    const bool forked = g_overlap && have_absorb && pl.n_split_naive > 0 && sh->side_stream != nullptr;
+    const bool forked = g_overlap && have_absorb && n_jobs > 0 && sh->side_stream != nullptr;
     if (forked) {
         e = cudaEventRecord(sh->ev_fork, s_main);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(sh->side_stream, sh->ev_fork, 0);
         if (e != cudaSuccess) return cuda_fail(e);
     }
 
-    // --- naive shared-prefix attention (Algorithm 1 line 4)
-    if (pl.n_split_naive > 0) {
+    // --- naive shared-prefix attention (Algorithm 1 line 4), one launch per (prefix, row range)
+    for (int j = 0; j < n_jobs; ++j) {
+        const NaiveJob& jb = jobs[j];
+        const char* qn = reinterpret_cast<const char*>(q_nope) + (size_t)jb.row0 * H * 128 * 2;
+        const char* qp = reinterpret_cast<const char*>(q_pe) + (size_t)jb.row0 * H * 64 * 2;
+        float* op = o_part_n + ((size_t)jb.slot0 * B + jb.row0) * H * 128;
+        float* lp = lse_part_n + ((size_t)jb.slot0 * B + jb.row0) * H;
         prof_before(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
         if (g_kernel_path == TYPHOON_MLA_PATH_TCGEN05) {
-            NaiveAttnSm100 na{q_nope, q_pe, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt, B, H, (int)sh->Ls,
-                              pl.n_split_naive, pl.n_slots_naive, softmax_scale, o_part_n, lse_part_n, sh->status};
+            NaiveAttnSm100 na{qn, qp, &jb.sh->tm_kn, &jb.sh->tm_kp, &jb.sh->tm_vt, jb.rows, H, (int)jb.sh->Ls,
+                              jb.n_ranges, jb.n_slots_level, softmax_scale, op, lp, sh->status, B};
             e = launch_naive_attn_sm100(na, s);
         } else {
-            NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad,
-                         pl.n_split_naive, softmax_scale, o_part_n, lse_part_n};
+            if (jb.rows != B) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;   // row ranges need the tcgen05 kernel
+            NaiveAttn na{qn, qp, jb.sh->k_nope, jb.sh->v_t, jb.sh->kpe, B, H, (int)jb.sh->Ls, (int)jb.sh->Ls_pad,
+                         jb.n_ranges, softmax_scale, op, lp};
             e = launch_naive_attn_mma(na, s);
         }
         prof_after(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++launches;
+    }
+    for (int j = 0; j < n_empties; ++j) {
+        const EmptySlots& es = empties[j];
+        e = launch_fill_neg_inf(lse_part_n + ((size_t)es.slot0 * B + es.row0) * H, es.n_slots, (int64_t)B * H,
+                                (int64_t)es.rows * H, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
     }
@@ -618,6 +633,125 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     }
     g_last_launches = launches;
     return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
+                       const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
+                       int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                       const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    g_last_launches = 0;
+    if (!sh || !q_nope || !q_pe || !out || B < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (mode < TYPHOON_MLA_MODE_AUTO || mode > TYPHOON_MLA_MODE_NAIVE) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return TYPHOON_MLA_ERR_INVALID_ARG;   // positive, finite
+    mode = resolve_mode(sh, B, max_pages, mode);
+    const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
+    if (use_absorb && max_pages > 0) {
+        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens) return TYPHOON_MLA_ERR_INVALID_ARG;
+        if (!aligned16(ckv_pages) || !aligned16(kpe_pages) || ckv_token_stride < 512 || kpe_token_stride < 64 ||
+            ckv_token_stride % 8 || kpe_token_stride % 8)
+            return TYPHOON_MLA_ERR_INVALID_ARG;
+    }
+    if (mode == TYPHOON_MLA_MODE_NAIVE && sh->Ls == 0) max_pages = 0;
+    const Plan pl = make_plan(sh, B, use_absorb ? max_pages : 0, page_size, mode);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
+
+    NaiveJob job{sh, 0, B, pl.n_split_naive, pl.n_slots_naive, 0};
+    return decode_core(sh, &job, pl.n_split_naive > 0 ? 1 : 0, nullptr, 0, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
+                       ckv_token_stride, kpe_token_stride, page_size, block_table, use_absorb ? max_pages : 0, seq_lens,
+                       softmax_scale, mode, out, lse_out, workspace, stream);
+}
+// ---- several shared prefixes per step (tree-structured prompts) ------------------------------------
+namespace {
+constexpr int kMaxLevels = 8, kMaxTreeJobs = 256;
+struct TreePlan {
+    const typhoon_mla_shared* sh0 = nullptr;   // first prefix: weights, absorb-side tensor maps, side stream, status
+    NaiveJob jobs[kMaxTreeJobs];
+    EmptySlots empties[kMaxTreeJobs];
+    int n_jobs = 0, n_empties = 0, total_slots = 0;
+};
+int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, TreePlan* tp) {
+    if (!levels || n_levels < 1 || n_levels > kMaxLevels || B < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
+    for (int l = 0; l < n_levels && !tp->sh0; ++l) {
+        if (!levels[l].prefixes || !levels[l].group_begin || levels[l].n_groups < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
+        for (int g = 0; g < levels[l].n_groups && !tp->sh0; ++g) tp->sh0 = levels[l].prefixes[g];
+    }
+    if (!tp->sh0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const int H = tp->sh0->dims.num_heads;
+    int slot0 = 0;
+    for (int l = 0; l < n_levels; ++l) {
+        const typhoon_mla_prefix_level_t& lv = levels[l];
+        if (!lv.prefixes || !lv.group_begin || lv.n_groups < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
+        if (lv.group_begin[0] != 0 || lv.group_begin[lv.n_groups] != B) return TYPHOON_MLA_ERR_INVALID_ARG;
+        const int first_job = tp->n_jobs;
+        int level_slots = 0;
+        for (int g = 0; g < lv.n_groups; ++g) {
+            const int r0 = lv.group_begin[g], r1 = lv.group_begin[g + 1];
+            if (r1 < r0) return TYPHOON_MLA_ERR_INVALID_ARG;
+            const typhoon_mla_shared* sh = lv.prefixes[g];
+            if (sh && sh->dims.num_heads != H) return TYPHOON_MLA_ERR_INVALID_ARG;
+            if (!sh || sh->Ls == 0 || r1 == r0) continue;
+            if (tp->n_jobs == kMaxTreeJobs) return TYPHOON_MLA_ERR_INVALID_ARG;
+            int ranges = 0, slots = 0;
+            naive_sm100_plan(r1 - r0, H, sh->Ls, naive_sm_budget(), naive_schedule(), &ranges, &slots);
+            tp->jobs[tp->n_jobs++] = NaiveJob{sh, r0, r1 - r0, ranges, 0, slot0};
+            level_slots = std::max(level_slots, slots);
+        }
+        if (level_slots == 0) continue;   // no prefix at this level at all: no slots
+        for (int j = first_job; j < tp->n_jobs; ++j) tp->jobs[j].n_slots_level = level_slots;
+        for (int g = 0; g < lv.n_groups; ++g) {
+            const int r0 = lv.group_begin[g], r1 = lv.group_begin[g + 1];
+            const typhoon_mla_shared* sh = lv.prefixes[g];
+            if ((sh && sh->Ls > 0) || r1 == r0) continue;
+            if (tp->n_empties == kMaxTreeJobs) return TYPHOON_MLA_ERR_INVALID_ARG;
+            tp->empties[tp->n_empties++] = EmptySlots{slot0, level_slots, r0, r1 - r0};
+        }
+        slot0 += level_slots;
+    }
+    tp->total_slots = slot0;
+    return TYPHOON_MLA_OK;
+}
+}  // namespace
+
+size_t typhoon_mla_tree_workspace_bytes(const typhoon_mla_prefix_level_t* levels, int32_t n_levels, int32_t B,
+                                        int32_t max_pages, int32_t page_size) {
+    if (max_pages < 0 || (page_size != 64 && page_size != 128) || g_kernel_path != TYPHOON_MLA_PATH_TCGEN05) return 0;
+    TreePlan tp;
+    if (plan_tree(levels, n_levels, B, &tp) != TYPHOON_MLA_OK) return 0;
+    return make_plan(tp.sh0, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID, tp.total_slots).total + 256;
+}
+
+int typhoon_mla_decode_tree(const typhoon_mla_prefix_level_t* levels, int32_t n_levels, const void* q_nope,
+                            const void* q_pe, int32_t B, const void* ckv_pages, const void* kpe_pages,
+                            int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size,
+                            const int32_t* block_table, int32_t max_pages, const int32_t* seq_lens, float softmax_scale,
+                            void* out, float* lse_out, void* workspace, size_t workspace_bytes, void* stream) {
+    g_last_launches = 0;
+    if (!q_nope || !q_pe || !out || B < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (g_kernel_path != TYPHOON_MLA_PATH_TCGEN05) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;
+    if (max_pages > 0) {
+        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens) return TYPHOON_MLA_ERR_INVALID_ARG;
+        if (!aligned16(ckv_pages) || !aligned16(kpe_pages) || ckv_token_stride < 512 || kpe_token_stride < 64 ||
+            ckv_token_stride % 8 || kpe_token_stride % 8)
+            return TYPHOON_MLA_ERR_INVALID_ARG;
+    }
+    TreePlan tp;
+    const int rc = plan_tree(levels, n_levels, B, &tp);
+    if (rc != TYPHOON_MLA_OK) return rc;
+    // NAIVE when there is no page table (nothing for the absorb branch), else Algorithm 1 with several line-4 launches
+    const int mode = max_pages == 0 ? TYPHOON_MLA_MODE_NAIVE : TYPHOON_MLA_MODE_HYBRID;
+    const Plan pl = make_plan(tp.sh0, B, max_pages, page_size, mode, tp.total_slots);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
+    return decode_core(tp.sh0, tp.jobs, tp.n_jobs, tp.empties, tp.n_empties, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
+                       ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages, seq_lens, softmax_scale,
+                       mode, out, lse_out, workspace, stream);
 }
 
 int typhoon_mla_profile_begin(int32_t kernel_id, int32_t max_launches) {

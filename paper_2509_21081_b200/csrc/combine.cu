@@ -192,6 +192,13 @@ __global__ void __launch_bounds__(1024) order_by_length_kernel(const int32_t* __
     block_order_by_length(seq_lens, B, perm, keys);
 }
 
+// -inf into n_slots segments of `count` floats, `stride` floats apart (LSE of partial slots no kernel fills).
+__global__ void __launch_bounds__(256) fill_neg_inf_kernel(float* __restrict__ dst, int n_slots, int64_t stride, int64_t count) {
+    const int64_t total = (int64_t)n_slots * count;
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (int64_t)gridDim.x * 256)
+        dst[(i / count) * stride + i % count] = -INFINITY;
+}
+
 // Row expansion for S_q query tokens per request (Table 1's S_q; causal among the new tokens):
 // row b * S_q + j gets request b's page-table row and the suffix length minus the S_q - 1 - j later tokens.
 __global__ void __launch_bounds__(256) expand_query_rows_kernel(const int32_t* __restrict__ block_table,
@@ -213,6 +220,13 @@ __global__ void __launch_bounds__(256) expand_query_rows_kernel(const int32_t* _
 cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm, cudaStream_t s) {
     if (B <= 0 || B > 4096) return cudaErrorInvalidValue;
     order_by_length_kernel<<<1, 1024, 0, s>>>(seq_lens, B, perm);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fill_neg_inf(float* dst, int n_slots, int64_t stride, int64_t count, cudaStream_t s) {
+    if (n_slots <= 0 || count <= 0) return cudaSuccess;
+    const int64_t total = (int64_t)n_slots * count;
+    fill_neg_inf_kernel<<<(unsigned)std::min<int64_t>((total + 255) / 256, 1184), 256, 0, s>>>(dst, n_slots, stride, count);
     return cudaGetLastError();
 }
 

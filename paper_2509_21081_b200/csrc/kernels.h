@@ -63,9 +63,10 @@ struct NaiveAttnSm100 {
     const CUtensorMap* tm_kn; const CUtensorMap* tm_kp; const CUtensorMap* tm_vt;   // host pointers
     int B, H; int Ls; int n_ranges, n_slots;
     float scale;
-    float* o_part;   // [slots][B][H][128]
-    float* lse_part; // [slots][B][H]
+    float* o_part;   // [slots][part_rows][H][128], pointing at this launch's first row
+    float* lse_part; // [slots][part_rows][H]
     int* status;     // device word, set non-zero if a bounded wait expired
+    int part_rows = 0;   // rows of the partial arrays; 0 = B (a launch may fill a row range of a larger batch)
 };
 int naive_sm100_tile_tokens(int B);   // KV tile width the kernel uses for this batch size (64 or 128)
 // CTAs (at most n_sm, each with an equal contiguous share of all (head, row group, tile) work) and
@@ -103,6 +104,8 @@ cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t L
                                      CUtensorMap* tm_kpe);
 
 // perm[0..B) = request indices by descending suffix length (B <= 4096).
+// -inf into n_slots segments of `count` floats, `stride` floats apart.
+cudaError_t launch_fill_neg_inf(float* dst, int n_slots, int64_t stride, int64_t count, cudaStream_t s);
 // Page table and lengths of the (request, query token) rows of a step with S_q query tokens per request.
 cudaError_t launch_expand_query_rows(const int32_t* block_table, const int32_t* seq_lens, int B, int max_pages, int S_q,
                                      int32_t* bt_rows, int32_t* len_rows, cudaStream_t s);

@@ -81,6 +81,7 @@ constexpr int MAX_STAGES = 4;
 
 struct NaiveSm100Params {
     int B, H, Ls, Ls_pad;
+    int part_rows;         // rows of the partial arrays (>= B: a launch may fill a row range of a larger batch)
     int m_groups;          // query-row groups per head
     int n_tiles;           // KV tiles per head
     int n_ranges;          // R (grid = R * m_groups CTAs)
@@ -88,8 +89,8 @@ struct NaiveSm100Params {
     int n_seg_max;         // partial slots per head (x2 streams in mode Y)
     int k_stages, v_stages;
     float scale_log2;
-    float* o_part;     // [n_slots][B][H][128]
-    float* lse_part;   // [n_slots][B][H]
+    float* o_part;     // [n_slots][part_rows][H][128]
+    float* lse_part;   // [n_slots][part_rows][H]
     int* status;
 };
 
@@ -528,7 +529,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 if (warp_has_rows) {
                     const float inv = 1.f / l_sum;
                     const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)i * 128u;
-                    float* dst = p.o_part + (((int64_t)slot * p.B + b) * p.H + s.h) * 128;
+                    float* dst = p.o_part + (((int64_t)slot * p.part_rows + b) * p.H + s.h) * 128;
 #pragma unroll 1
                     for (int c = 0; c < 4; ++c) {
                         uint32_t orr[32];
@@ -543,16 +544,16 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                             }
                         }
                     }
-                    if (b < p.B) p.lse_part[((int64_t)slot * p.B + b) * p.H + s.h] = (m_ref + log2f(l_sum)) * kLn2;
+                    if (b < p.B) p.lse_part[((int64_t)slot * p.part_rows + b) * p.H + s.h] = (m_ref + log2f(l_sum)) * kLn2;
                 }
             } else if (owns_rows && b < p.B) {
-                p.lse_part[((int64_t)slot * p.B + b) * p.H + s.h] = -INFINITY;   // this stream had no tile
+                p.lse_part[((int64_t)slot * p.part_rows + b) * p.H + s.h] = -INFINITY;   // this stream had no tile
             }
             // the segment that ends a column marks the column's unused slots as empty
             if (s.last_of_col && owns_rows && b < p.B) {
                 for (int ss = s.slot_seg + 1; ss < p.n_seg_max; ++ss) {
                     const int sl = ss * n_sub + (MODE_Y ? i : 0);
-                    p.lse_part[((int64_t)sl * p.B + b) * p.H + s.h] = -INFINITY;
+                    p.lse_part[((int64_t)sl * p.part_rows + b) * p.H + s.h] = -INFINITY;
                 }
             }
             // the accumulator of this stream may be overwritten by the next segment
@@ -675,6 +676,7 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     const int tok = mode_y ? 64 : 128;
     NaiveSm100Params p{};
     p.B = a.B; p.H = a.H; p.Ls = a.Ls; p.Ls_pad = (a.Ls + 127) / 128 * 128;
+    p.part_rows = a.part_rows > 0 ? a.part_rows : a.B;
     p.m_groups = mode_y ? 1 : (a.B + 255) / 256;
     p.n_tiles = (a.Ls + tok - 1) / tok;
     p.n_ranges = a.n_ranges;

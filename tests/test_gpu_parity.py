@@ -334,6 +334,84 @@ def test_several_query_tokens_per_request(S_q):
     dec.close()
 
 
+def _tree_problem(B, H, root_len, branches, lens, seed):
+    """Requests with a root prefix shared by all (may be 0 tokens = none) and one optional branch prefix per
+    consecutive group.  `branches`: list of (first request, tokens); requests before the first branch and
+    groups with 0 tokens have none.  Returns (rows for the checker, suffix-only inputs, branch latents)."""
+    import dataclasses
+    cfg = _cfg("tree", B=B, H=H, Ls=max(root_len, 1), lo=0, hi=0, seed=seed)
+    inp = I.make_inputs(cfg, suffix_lens=lens)
+    if root_len == 0:
+        inp.ckv_shared, inp.kpe_shared = inp.ckv_shared[:0], inp.kpe_shared[:0]
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * 77 + 1)
+    starts = [b0 for b0, _ in branches] + [B]
+    br = []
+    for k, (b0, n) in enumerate(branches):
+        br.append((b0, starts[k + 1], torch.randn(n, 512, generator=g).to(torch.bfloat16),
+                   torch.randn(n, 64, generator=g).to(torch.bfloat16)))
+    # checker: every request's own context = branch prefix + suffix (dense); the root stays shared
+    rows = dataclasses.replace(inp, ckv_suffix=list(inp.ckv_suffix), kpe_suffix=list(inp.kpe_suffix))
+    for b0, b1, c, r in br:
+        for b in range(b0, b1):
+            rows.ckv_suffix[b] = torch.cat([c, inp.ckv_suffix[b]])
+            rows.kpe_suffix[b] = torch.cat([r, inp.kpe_suffix[b]])
+    return rows, inp, br
+
+
+@pytest.mark.parametrize("case", ["root+branches", "branches only", "root only, no pages"])
+def test_tree_of_shared_prefixes(case, kernel_path):
+    """Several shared prefixes per step: a root shared by all requests plus one prefix per group of
+    requests, or flat groups, against the checker run on each request's whole context."""
+    from paper_2509_21081_b200 import binding as b
+    if kernel_path != "tcgen05":
+        pytest.skip("row ranges need the tcgen05 kernel")
+    B, H = 11, 32
+    lens = [0, 3, 64, 65, 130, 7, 200, 1, 90, 64, 30]
+    if case == "root+branches":
+        root_len, branches = 210, [(0, 150), (3, 0), (5, 333), (9, 70)]
+    elif case == "branches only":
+        root_len, branches = 0, [(0, 100), (4, 260), (8, 0), (10, 65)]
+    else:
+        root_len, branches, lens = 500, [], [0] * B
+    rows, inp, br = _tree_problem(B, H, root_len, branches, lens, seed=38)
+    ref, ref_lse = G.run_oracle(rows)
+    dev = "cuda"
+    w_uk, w_uv = inp.w_uk.to(dev), inp.w_uv.to(dev)
+    dims = b.make_dims(H)
+    handles = []
+
+    def prep(c, r):
+        h = b.typhoon_mla_prepare_shared(dims, c.to(dev), r.to(dev), w_uk, w_uv)
+        handles.append(h)
+        return h
+
+    levels = []
+    if root_len > 0:
+        levels.append(([prep(inp.ckv_shared, inp.kpe_shared)], [0, B]))
+    if br:
+        begins = [b0 for b0, _, _, _ in br] + [B]
+        prefixes = [prep(c, r) if c.shape[0] > 0 else None for _, _, c, r in br]
+        if begins[0] != 0:
+            begins, prefixes = [0] + begins, [None] + prefixes
+        levels.append((prefixes, begins))
+    use_pages = case != "root only, no pages"
+    pc = I.build_pages(inp)
+    max_pages = pc.block_table.shape[1] if use_pages else 0
+    ws = torch.empty(b.typhoon_mla_tree_workspace_bytes(levels, B, max_pages, 64), dtype=torch.uint8, device=dev)
+    assert ws.numel() > 0
+    out = torch.empty(B, H, 128, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(B, H, dtype=torch.float32, device=dev)
+    args = (pc.ckv_pages.to(dev), pc.kpe_pages.to(dev), 64, pc.block_table.to(dev), pc.seq_lens.to(dev)) if use_pages \
+        else (None, None, 64, None, None)
+    b.typhoon_mla_decode_tree(levels, inp.q_nope.to(dev), inp.q_pe.to(dev), *args, inp.scale, out, ws, lse_out=lse)
+    for h in handles:
+        assert b.typhoon_mla_device_status(h) == 0
+    G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse, what=f"tree: {case}")
+    for h in handles:
+        h.free()
+
+
 def test_invalid_arguments():
     from paper_2509_21081_b200 import binding as b
     cfg = _cfg("inval", B=2, H=16, Ls=64, lo=8, hi=8, seed=33)
