@@ -385,6 +385,86 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     return line
 
 
+def bench_extension(cfg, args, device_index):
+    """Measurement of the two extensions of the path (one GPU, device-resident inputs, two input sets
+    alternated, CUDA events): --sq S = S query tokens per request (rows = (request, token) pairs, causal
+    among the new tokens); --tree G:L = the config's prefix as the root of all requests plus G groups of
+    B/G requests with a further shared prefix of L tokens each.  One JSON line, queries = rows."""
+    import torch
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200 import inputs as I
+    dev = "cuda"
+    W, K = max(args.warmup, 3), max(args.steps, 1)
+    H, B, Ls = cfg.H, cfg.B, cfg.Ls
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp, poison=False)
+    dims = b.make_dims(H)
+    S_q = max(args.sq, 1)
+    rows = B * S_q
+    if args.tree:
+        G_, L_ = (int(x) for x in args.tree.split(":"))
+        assert B % G_ == 0 and S_q == 1
+    sets = []
+    for _ in range(2):
+        w_uk, w_uv = inp.w_uk.to(dev), inp.w_uv.to(dev)
+        root = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), w_uk, w_uv)
+        levels = [([root], [0, rows])]
+        if args.tree:
+            g = torch.Generator(device="cpu")
+            g.manual_seed(cfg.seed + 99)
+            br = [b.typhoon_mla_prepare_shared(dims, torch.randn(L_, 512, generator=g).to(torch.bfloat16).to(dev),
+                                               torch.randn(L_, 64, generator=g).to(torch.bfloat16).to(dev), w_uk, w_uv)
+                  for _ in range(G_)]
+            levels.append((br, [i * (B // G_) for i in range(G_ + 1)]))
+        bt, sl = pc.block_table.to(dev), pc.seq_lens.to(dev)
+        if S_q > 1:
+            bt, sl = b.typhoon_mla_expand_query_rows(bt, sl, S_q)
+        q_nope = inp.q_nope.to(dev).repeat_interleave(S_q, dim=0).contiguous()
+        q_pe = inp.q_pe.to(dev).repeat_interleave(S_q, dim=0).contiguous()
+        ws = torch.empty(b.typhoon_mla_tree_workspace_bytes(levels, rows, bt.shape[1], pc.page_size), dtype=torch.uint8,
+                         device=dev)
+        sets.append(dict(levels=levels, q_nope=q_nope, q_pe=q_pe, ckv=pc.ckv_pages.to(dev), kpe=pc.kpe_pages.to(dev),
+                         bt=bt, sl=sl, ws=ws, out=torch.empty(rows, H, 128, dtype=torch.bfloat16, device=dev)))
+
+    def step(i):
+        s = sets[i % 2]
+        b.typhoon_mla_decode_tree(s["levels"], s["q_nope"], s["q_pe"], s["ckv"], s["kpe"], pc.page_size, s["bt"], s["sl"],
+                                  inp.scale, s["out"], s["ws"])
+
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    launches = b.typhoon_mla_last_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(device_index) as clocks:
+        ev0.record()
+        for i in range(K):
+            step(i)
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / K
+    # algorithmic work: Table 1's hybrid terms with rows = B * S_q queries (the suffix is stored once per
+    # request), every shared prefix read once, plus the once-only reads of q and the weights and the write of out
+    sum_ln_rows = int(sets[0]["sl"].clamp(min=0).sum().item())
+    prefix_tokens_rows = rows * Ls + (rows * L_ if args.tree else 0)          # (query row, prefix token) pairs
+    prefix_tokens = Ls + (G_ * L_ if args.tree else 0)
+    flops = H * (640 * prefix_tokens_rows + 2176 * sum_ln_rows + 4 * 65536 * rows)
+    bytes_ = (512 * H + 128) * prefix_tokens + 4 * H * 65536 + 1152 * sum(inp.suffix_lens) + 640 * H * rows
+    pk = _peaks()
+    t_lb = max(flops / (pk["bf16_tflops"] * 1e12), bytes_ / (pk["hbm_gbs"] * 1e9))
+    what = (f"S_q={S_q} query tokens per request" if S_q > 1 else "") + \
+        (f"root prefix + {G_} groups with {L_} more shared tokens each" if args.tree else "")
+    return {"metric": METRIC, "value": rows / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: B={B} H={H} Ls={Ls} Ln=[{cfg.suffix_lo},{cfg.suffix_hi}], {what}",
+                       "rows": rows, "entry_point": "typhoon_mla_decode_tree",
+                       "l2": "2 full input sets used alternately"},
+            "clocks": clocks.summary(), "gpu_launches": launches * K,
+            "work": {"algorithmic_flops": flops, "algorithmic_bytes": bytes_, "t_lower_bound_ms": t_lb * 1e3,
+                     "step_frac_of_combined_roofline": t_lb / (ms * 1e-3), "peak_source": pk["source"]}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -396,6 +476,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (config 4 sweep)")
     ap.add_argument("--sweep", action="store_true", help="config 4 fan-out sweep over batch sizes and modes")
     ap.add_argument("--ref-heads", type=int, default=64, help="heads the CPU checker is timed on (scaled up)")
+    ap.add_argument("--sq", type=int, default=1, help="extension: query tokens per request (rows = B * S_q)")
+    ap.add_argument("--tree", default="", help="extension: G:L = G request groups with L more shared prefix tokens each")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -417,7 +499,14 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
     mode = {"auto": b.MODE_AUTO, "absorb": b.MODE_ABSORB, "hybrid": b.MODE_HYBRID, "naive": b.MODE_NAIVE}[args.mode]
 
-    if args.sweep:
+    if args.sq > 1 or args.tree:
+        if world > 1:
+            raise SystemExit("--sq / --tree are single-GPU measurements")
+        cfg = I.CONFIGS[args.config]
+        if args.batch:
+            cfg = cfg.with_batch(args.batch)
+        print(json.dumps(bench_extension(cfg, args, local)), flush=True)
+    elif args.sweep:
         base = I.CONFIGS["cfg4"]
         for B in I.CFG4_BATCHES:
             for m in (b.MODE_ABSORB, b.MODE_HYBRID, b.MODE_AUTO):
