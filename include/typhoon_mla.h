@@ -288,6 +288,13 @@ int typhoon_mla_set_kernel_path(int32_t path);
  * kernel on the caller's stream, one after the other (measurement aid).  Process-wide. */
 int typhoon_mla_set_overlap(int32_t enable);
 
+/* The kernels of a step are launched with the programmatic-stream-serialization attribute (default):
+ * a kernel may be scheduled while its predecessor in the stream is still running and waits, before its
+ * first access to global memory, until that predecessor has completed.  This hides most of the launch
+ * latency between the dependent kernels of a step.  0 gives ordinary stream-ordered launches
+ * (measurement aid; TYPHOON_MLA_PDL=0 in the environment sets the initial value).  Process-wide. */
+int typhoon_mla_set_programmatic_launch(int32_t enable);
+
 /* Work decomposition of the tcgen05 shared-prefix kernel (see typhoon_mla_naive_plan): 0 = the
  * library's choice (default), 1 = column split, 2 = stream-K.  Measurement and test aid; process-wide. */
 int typhoon_mla_set_naive_schedule(int32_t schedule);

@@ -93,6 +93,8 @@ def _load():
     lib.typhoon_mla_expand_query_rows.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.typhoon_mla_set_naive_schedule.restype = C.c_int
     lib.typhoon_mla_set_naive_schedule.argtypes = [i32]
+    lib.typhoon_mla_set_programmatic_launch.restype = C.c_int
+    lib.typhoon_mla_set_programmatic_launch.argtypes = [i32]
     lib.typhoon_mla_set_overlap.restype = C.c_int
     lib.typhoon_mla_set_overlap.argtypes = [i32]
     lib.typhoon_mla_device_status.restype = C.c_int
@@ -346,6 +348,10 @@ def typhoon_mla_expand_query_rows(block_table: torch.Tensor, seq_lens: torch.Ten
 
 def typhoon_mla_set_naive_schedule(schedule: int) -> None:
     _check(_lib.typhoon_mla_set_naive_schedule(schedule), "typhoon_mla_set_naive_schedule")
+
+
+def typhoon_mla_set_programmatic_launch(enable: bool) -> None:
+    _check(_lib.typhoon_mla_set_programmatic_launch(1 if enable else 0), "typhoon_mla_set_programmatic_launch")
 
 
 def typhoon_mla_set_overlap(enable: bool) -> None:

@@ -128,6 +128,8 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     volatile int* abort_flag = &sh->abort_flag;
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
+    pdl_trigger();
+    pdl_wait();   // the descriptors and Q_A read below are written by the preceding kernel
     if (threadIdx.x == 0) TRACE(0, 28);
     KT_BEGIN();
     TRACE_CTA(0);
@@ -641,8 +643,7 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     dim3 grid(n_chunks, (a.H + 63) / 64, a.B);
     const CUtensorMap* sh_c = a.n_shared_chunks > 0 ? tm_ckv_sh : &tm_ckv_pg;
     const CUtensorMap* sh_k = a.n_shared_chunks > 0 ? tm_kpe_sh : &tm_kpe_pg;
-    absorb_attn_sm100_kernel<<<grid, 384, smem, s>>>(tm_qa, tm_qp, *sh_c, *sh_k, tm_ckv_pg, tm_kpe_pg, p);
-    return cudaGetLastError();
+    return launch_pdl(absorb_attn_sm100_kernel, grid, dim3(384), smem, s, tm_qa, tm_qp, *sh_c, *sh_k, tm_ckv_pg, tm_kpe_pg, p);
 }
 
 }  // namespace tmla

@@ -13,6 +13,13 @@
 
 using namespace tmla;
 
+// Programmatic dependent launch of the step's kernels (tuning aid: TYPHOON_MLA_PDL=0 in the environment
+// gives ordinary stream-ordered launches).
+bool tmla::g_pdl = [] {
+    const char* v = std::getenv("TYPHOON_MLA_PDL");
+    return !(v && v[0] == '0');
+}();
+
 #include "handle.h"
 
 namespace {
@@ -422,6 +429,11 @@ int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* per
 
 int typhoon_mla_set_overlap(int32_t enable) {
     g_overlap = enable != 0;
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_set_programmatic_launch(int32_t enable) {
+    tmla::g_pdl = enable != 0;
     return TYPHOON_MLA_OK;
 }
 

@@ -5,6 +5,7 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "sm100.cuh"
 
 namespace tmla {
 namespace {
@@ -18,6 +19,8 @@ __global__ void __launch_bounds__(512) merge_latent_kernel(const float* __restri
                                                            const float* __restrict__ lse_part, int n_chunks,
                                                            int BH, __nv_bfloat16* __restrict__ o_lat,
                                                            float* __restrict__ lse) {
+    sm100::pdl_trigger();
+    sm100::pdl_wait();
     __shared__ float w_s[MERGE_MAX_CHUNKS];
     __shared__ float red[16];
     __shared__ float4 acc_s[3][128];
@@ -86,6 +89,8 @@ __global__ void __launch_bounds__(512) merge_latent_few_kernel(const float* __re
                                                                const float* __restrict__ lse_part, int n_chunks,
                                                                int BH, __nv_bfloat16* __restrict__ o_lat,
                                                                float* __restrict__ lse) {
+    sm100::pdl_trigger();
+    sm100::pdl_wait();
     const int bh = blockIdx.x * 4 + (threadIdx.x >> 7), col = threadIdx.x & 127;
     if (bh >= BH) return;
     float l[MERGE_FEW];
@@ -120,6 +125,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
                                                       const float* __restrict__ o_abs,
                                                       const float* __restrict__ lse_abs, int BH,
                                                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out) {
+    sm100::pdl_trigger();
+    sm100::pdl_wait();
     const int bh = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (bh >= BH) return;
@@ -244,11 +251,11 @@ cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int 
     if (B * H <= 0) return cudaSuccess;
     if (n_chunks > MERGE_MAX_CHUNKS) return cudaErrorInvalidValue;
     if (n_chunks <= MERGE_FEW) {
-        merge_latent_few_kernel<<<(B * H + 3) / 4, 512, 0, s>>>(o_part, lse_part, n_chunks, B * H,
-                                                                reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
+        return launch_pdl(merge_latent_few_kernel, dim3((B * H + 3) / 4), dim3(512), 0, s, o_part, lse_part, n_chunks, B * H,
+                          reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
     } else {
-        merge_latent_kernel<<<B * H, 512, 0, s>>>(o_part, lse_part, n_chunks, B * H,
-                                                  reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
+        return launch_pdl(merge_latent_kernel, dim3(B * H), dim3(512), 0, s, o_part, lse_part, n_chunks, B * H,
+                          reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
     }
     return cudaGetLastError();
 }
@@ -257,9 +264,8 @@ cudaError_t launch_combine(const float* o_naive, const float* lse_naive, int n_n
                            const float* lse_abs, int B, int H, void* out_bf16, float* lse_out, cudaStream_t s) {
     int BH = B * H;
     if (BH <= 0) return cudaSuccess;
-    combine_kernel<<<(BH + 7) / 8, 256, 0, s>>>(o_naive, lse_naive, n_naive, o_abs, lse_abs, BH,
-                                                reinterpret_cast<__nv_bfloat16*>(out_bf16), lse_out);
-    return cudaGetLastError();
+    return launch_pdl(combine_kernel, dim3((BH + 7) / 8), dim3(256), 0, s, o_naive, lse_naive, n_naive, o_abs, lse_abs, BH,
+                      reinterpret_cast<__nv_bfloat16*>(out_bf16), lse_out);
 }
 
 cudaError_t launch_transpose_bf16(const void* in, void* out, int R, int C, int batch, cudaStream_t s) {

@@ -58,6 +58,8 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
+    pdl_trigger();
+    pdl_wait();
     KT_BEGIN();
     const int KB = p.K / BK;
 
@@ -257,8 +259,7 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, c
                  ce ? 2 : (g.out_fp32 ? 1 : 0), ce ? *ce : CombineEpilogue{}};
     cudaFuncSetAttribute(gemm_tn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid(g.N / BN, (g.M + BM - 1) / BM, g.batch);
-    gemm_tn_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tmA, tmB, p);
-    return cudaGetLastError();
+    return launch_pdl(gemm_tn_sm100_kernel, grid, dim3(192), SMEM_BYTES, s, tmA, tmB, p);
 }
 
 }  // namespace tmla

@@ -6,6 +6,25 @@
 
 namespace tmla {
 
+// Launch with the programmatic-stream-serialization attribute when enabled (see sm100::pdl_wait): the
+// kernel must call pdl_wait() before its first access to global memory.
+extern bool g_pdl;
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+
 // C[z][m][n] = sum_k A[z][m][k] * B[z][n][k]   (both operands K-major, bf16, fp32 accumulate)
 struct GemmTN {
     const void* A; int64_t lda; int64_t a_batch;   // elements

@@ -141,6 +141,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     const int rng = blockIdx.x / p.m_groups, grp = blockIdx.x % p.m_groups;
+    pdl_trigger();   // the next kernel of the stream may be scheduled as soon as every CTA of this one has started
+    pdl_wait();      // nothing below touches global memory before the stream's earlier kernels are done
     KT_BEGIN();
     TRACE_CTA(0, 0);
 
@@ -696,10 +698,10 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     dim3 grid(p.n_ranges * p.m_groups, 1, 1);
     if (mode_y) {
         cudaFuncSetAttribute(naive_attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        naive_attn_sm100_kernel<64><<<grid, 384, smem, s>>>(tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        return launch_pdl(naive_attn_sm100_kernel<64>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     } else {
         cudaFuncSetAttribute(naive_attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        naive_attn_sm100_kernel<128><<<grid, 384, smem, s>>>(tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        return launch_pdl(naive_attn_sm100_kernel<128>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     }
     return cudaGetLastError();
 }

@@ -55,6 +55,8 @@ __global__ void __launch_bounds__(192, 1)
 q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_w, QAbsorbParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    pdl_trigger();
+    pdl_wait();
     KT_BEGIN();
     if ((int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
         if (blockIdx.x == 0) {
@@ -182,8 +184,7 @@ cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, v
                     (with_order && block_table != nullptr) ? reinterpret_cast<int4*>(desc) : nullptr};
     cudaFuncSetAttribute(q_absorb_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid((B + 127) / 128, H + (with_order ? 1 : 0), 1);
-    q_absorb_sm100_kernel<<<grid, 192, SMEM_BYTES, s>>>(tm_q, *tm_w, p);
-    return cudaGetLastError();
+    return launch_pdl(q_absorb_sm100_kernel, grid, dim3(192), SMEM_BYTES, s, tm_q, *tm_w, p);
 }
 
 }  // namespace tmla

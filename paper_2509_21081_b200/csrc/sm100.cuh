@@ -99,6 +99,12 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uin
 
 // ---------------------------------------------------------------- tensor memory
 // Allocation is done by one full warp; the base address lands in shared memory.
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the
+// stream is still running; pdl_wait() blocks until the predecessor has completed and its writes are
+// visible (a no-op for an ordinary launch), pdl_trigger() lets the successor's CTAs be scheduled early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 // Bulk copy shared -> global (both addresses 16-byte aligned, size a multiple of 16 bytes), tracked
 // by the issuing thread's bulk async-group.
 __device__ __forceinline__ void bulk_store(void* gdst, const void* ssrc, uint32_t bytes) {
