@@ -412,6 +412,48 @@ def test_tree_of_shared_prefixes(case, kernel_path):
         h.free()
 
 
+def test_random_switches_repeatable_and_consistent(kernel_path):
+    """Many small random problems with random work decomposition, stream overlap and launch mode: every
+    call is bitwise repeatable, no in-kernel wait expires, and the hybrid and absorb-only paths agree."""
+    import random
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    rnd = random.Random(77)
+    try:
+        for _ in range(40):
+            H = rnd.choice([16, 32, 64, 128])
+            B = rnd.choice([1, 2, 7, 33, 64, 65, 128, 129, 200, 300])
+            Ls = rnd.choice([0, 1, 63, 64, 65, 500, 1000, 2049])
+            hi = rnd.choice([0, 1, 64, 300])
+            ps = rnd.choice([64, 128])
+            b.typhoon_mla_set_naive_schedule(rnd.choice([0, 1, 2]))
+            b.typhoon_mla_set_overlap(rnd.choice([True, True, False]))
+            b.typhoon_mla_set_programmatic_launch(rnd.choice([True, True, False]))
+            cfg = _cfg("switches", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=rnd.randint(0, 10 ** 6), page_size=ps)
+            inp = I.make_inputs(cfg)
+            if Ls == 0 and max(inp.suffix_lens) == 0:
+                continue
+            pc = I.build_pages(inp, page_size=ps)
+            dec = TyphoonMLADecoder(H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(),
+                                    inp.scale, B, pc.block_table.shape[1], ps)
+            args = (inp.q_nope.cuda(), inp.q_pe.cuda(), pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), pc.block_table.cuda(),
+                    pc.seq_lens.cuda())
+            outs = {}
+            for mode in (HYBRID, ABSORB):
+                o = [dec.decode(*args, mode=mode).clone() for _ in range(3)]
+                assert b.typhoon_mla_device_status(dec.shared) == 0, f"{cfg} mode {mode}"
+                assert all(torch.equal(x, o[0]) for x in o[1:]), f"not repeatable: {cfg} mode {mode}"
+                assert torch.isfinite(o[0].float()).all(), f"non-finite: {cfg} mode {mode}"
+                outs[mode] = o[0].float()
+            d = (outs[HYBRID] - outs[ABSORB]).abs().max().item()
+            assert d <= 3e-2 * max(1.0, outs[ABSORB].abs().max().item()), f"hybrid vs absorb {d}: {cfg}"
+            dec.close()
+    finally:
+        b.typhoon_mla_set_naive_schedule(0)
+        b.typhoon_mla_set_overlap(True)
+        b.typhoon_mla_set_programmatic_launch(True)
+
+
 def test_invalid_arguments():
     from paper_2509_21081_b200 import binding as b
     cfg = _cfg("inval", B=2, H=16, Ls=64, lo=8, hi=8, seed=33)
