@@ -291,7 +291,9 @@ int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int3
     const typhoon_mla_dims_t& d = *dims;
     const double H = d.num_heads, L = (double)Ls;
     const double f_naive = 2.0 * B * H * L * (d.d_nope + d.d_rope + d.d_v);
-    const double f_absorb = 2.0 * B * H * L * (2.0 * d.kv_lora_rank + d.d_rope);
+    // (the absorb kernel works on groups of 64 heads: a partial group costs as much as a full one)
+    const double H_abs = std::ceil(H / 64.0) * 64.0;
+    const double f_absorb = 2.0 * B * H_abs * L * (2.0 * d.kv_lora_rank + d.d_rope);
     const double by_naive = 2.0 * L * (H * (d.d_nope + d.d_v) + d.d_rope);
     const double by_absorb = 2.0 * L * (d.kv_lora_rank + d.d_rope);
     // The absorb kernel re-reads the prefix per request and runs M = 64 tiles: measured on B200 it

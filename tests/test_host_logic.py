@@ -105,6 +105,10 @@ def test_crossover_rule(b):
     assert b.typhoon_mla_choose_mode_for(d, 16384, 8) == b.MODE_ABSORB
     assert b.typhoon_mla_choose_mode_for(d, 16384, 32) == b.MODE_HYBRID
     assert b.typhoon_mla_choose_mode_for(d, 16384, 512) == b.MODE_HYBRID
+    # 16 heads occupy a whole 64-head group of the absorb kernel: measured on B200 at L_s = 16384 the
+    # hybrid path wins from B = 16 (56 vs 72 us), which the rule has to reproduce
+    assert b.typhoon_mla_choose_mode_for(b.make_dims(16), 16384, 16) == b.MODE_HYBRID
+    assert b.typhoon_mla_choose_mode_for(b.make_dims(16), 16384, 2) == b.MODE_ABSORB
 
 
 def test_pure_entry_points_reject_bad_arguments(b):
