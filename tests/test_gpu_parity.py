@@ -552,3 +552,16 @@ def test_cfg2_long_prompt_sampled():
 @pytest.mark.parametrize("B", [1, 8, 128])
 def test_cfg4_fanout_sampled(B):
     _full_size_sampled(I.CONFIGS["cfg4"].with_batch(B), (AUTO, HYBRID), 8)
+
+
+def test_long_prefix_sampled():
+    """A prefix of 70 001 tokens (1094 tiles per head, not a tile multiple): tile indexing over long ranges,
+    many ring wrap-arounds per CTA, many absorb chunks in ABSORB mode."""
+    cfg = _cfg("long", B=3, H=16, Ls=70001, lo=1, hi=300, seed=51)
+    _full_size_sampled(cfg, (HYBRID, ABSORB), n_pairs=6)
+
+
+def test_more_requests_than_the_ordering_block_sorts():
+    """B = 4500 (> 4096): no longest-first order and no descriptors, 4500 CTAs per head group."""
+    cfg = _cfg("wide", B=4500, H=16, Ls=100, lo=0, hi=70, seed=52)
+    _full_size_sampled(cfg, (HYBRID, ABSORB), n_pairs=48, extremes=True)
