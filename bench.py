@@ -331,6 +331,27 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     alone = (k_bytes / a_s / 1e9) if roof["bound"] == "hbm" else (k_flops / a_s / 1e12)
     roof.update({"kernel_ms_alone": a_s * 1e3, "achieved_alone": alone, "frac_alone": alone / roof["peak"]})
 
+    # ---- per-stage times (the layout of the paper's Fig. 4 / Fig. 8: stage 1 = naive shared attention, stage 2
+    # = absorb attention, plus the projections and the merge), every kernel alone on the GPU: side stream
+    # off, ordinary launches, a CUDA-event pair around each launch
+    stages = None
+    if getattr(args, "stages", False):
+        b.typhoon_mla_set_overlap(False)
+        b.typhoon_mla_set_programmatic_launch(False)
+        stages = {}
+        n_st = max(5, min(K, 20))
+        for k_id, k_name in enumerate(b.KERNEL_NAMES):
+            for i in range(2):
+                step(i)
+            b.typhoon_mla_profile_begin(k_id, n_st)
+            for i in range(n_st):
+                step(i)
+            s_ms, s_n = b.typhoon_mla_profile_end()
+            if s_n:
+                stages[k_name + "_ms"] = s_ms / s_n
+        b.typhoon_mla_set_overlap(True)
+        b.typhoon_mla_set_programmatic_launch(True)
+
     # ---- end to end: per-step tensors from pinned host memory, result read back, every step
     e2e = None
     if with_e2e:
@@ -398,7 +419,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
             "config": {"workload": _workload_name(cfg), "mode": mode_name, "requested_mode": b.MODE_NAMES[mode],
                        "parallelism": f"replicas x{world} (shard by request, no exchange)",
                        "l2": f"{n_sets} full input sets used alternately, each larger than the 126 MB L2"},
-            "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches_per_step * K,
+            "clocks": clocks.summary(), "e2e": e2e, "stages": stages, "gpu_launches": launches_per_step * K,
             "roofline": roof, "cpu_baseline": cpu}
     return line
 
@@ -496,6 +517,7 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=64, help="heads the CPU checker is timed on (scaled up)")
     ap.add_argument("--sq", type=int, default=1, help="extension: query tokens per request (rows = B * S_q)")
     ap.add_argument("--tree", default="", help="extension: G:L = G request groups with L more shared prefix tokens each")
+    ap.add_argument("--stages", action="store_true", help="also time every kernel of the step alone (implied by --sweep)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -525,6 +547,7 @@ def main():
             cfg = cfg.with_batch(args.batch)
         print(json.dumps(bench_extension(cfg, args, local)), flush=True)
     elif args.sweep:
+        args.stages = True
         base = I.CONFIGS["cfg4"]
         for B in I.CFG4_BATCHES:
             for m in (b.MODE_ABSORB, b.MODE_HYBRID, b.MODE_AUTO):
