@@ -19,8 +19,9 @@
 //     S MMA halves the re-reads of Q from shared memory, the streams ping-pong between tensor
 //     core and softmax.
 //   * B <= 128 (mode Y, 64-token KV tiles): both streams use the same 128 query rows; stream i
-//     takes every second KV tile with its own softmax state.  HBM-bound regime: small tiles give
-//     deep K and V rings.
+//     takes every second KV tile with its own softmax state, and at the end of the segment
+//     stream 0 merges the two accumulators (same tensor-memory lanes) into one partial.
+//     HBM-bound regime: small tiles give deep K and V rings.
 //
 // Warp roles (384 threads): warp 0 = TMA producer for Q and the K ring, warp 2 = TMA producer
 // for the V ring, warp 1 = issuer of the S = Q K^T MMAs and TMEM owner, warp 3 = issuer of the
@@ -86,7 +87,7 @@ struct NaiveSm100Params {
     int n_tiles;           // KV tiles per head
     int n_ranges;          // R (grid = R * m_groups CTAs)
     int per, rem;          // T = R * per + rem: ranges [0, rem) hold per + 1 tiles, the others per
-    int n_seg_max;         // partial slots per head (x2 streams in mode Y)
+    int n_seg_max;         // partial slots per head (one per segment of the head)
     int k_stages, v_stages;
     float scale_log2;
     float* o_part;     // [n_slots][part_rows][H][128]
@@ -99,12 +100,16 @@ struct Barriers {
     uint64_t k_full[MAX_STAGES], k_empty[MAX_STAGES];
     uint64_t v_full[MAX_STAGES], v_empty[MAX_STAGES];
     uint64_t s_ready[2][2], p_ready[2][2], sbuf_free[2][2], o_free[2];
+    // 64-token tiles: stream 1 has published its softmax state (merge_m / merge_l) and its accumulator is
+    // complete; stream 0 then merges the two streams' results into one partial (128 arrivals per segment)
+    uint64_t merge_ready;
     // completion of PV product u of stream i goes to o_done[i][u & 1]: a waiter that knows product
     // u-2 has landed (every wait below does) then sees a barrier at most one completion from the
     // awaited one, which is what a parity wait can tell apart
     uint64_t o_done[2][2];
     uint32_t tmem_base;
     int abort_flag;
+    float merge_m[128], merge_l[128];   // stream 1's reference exponent and row sum, per query row
 };
 
 // One segment of a CTA's tile range.
@@ -243,7 +248,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             constexpr int n_bars = (int)(offsetof(Barriers, tmem_base) / sizeof(uint64_t));
             for (int i = lane; i < n_bars; i += 32) {
                 uint64_t* m = all + i;
-                const bool wg = (m >= &bar->p_ready[0][0] && m < &bar->sbuf_free[0][0]) || (m >= &bar->o_free[0] && m < &bar->o_done[0][0]);
+                const bool wg = (m >= &bar->p_ready[0][0] && m < &bar->sbuf_free[0][0]) || (m >= &bar->o_free[0] && m < &bar->o_done[0][0]);   // o_free, merge_ready
                 mbar_init(m, wg ? 128 : 1);
             }
             if (lane == 0) bar->abort_flag = 0;
@@ -412,6 +417,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         const int lg = (warp & 3) * 32;           // TMEM lane group of this warp
         const int r = lg + lane;                  // row within the 128-row tile
         int used = 0;                             // S-buffer uses (= PV products) of this stream so far
+        int segi = 0;                             // segments finished by this CTA
         bool ok = true;
         for (int g = g_begin; g < g_end && ok;) {
             const Segment s = segment_at(g);
@@ -519,49 +525,82 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             }
             if (!ok) break;
             TRACE_CTA(128, 3);
-            // ---- segment epilogue: normalised partial + LSE into this segment's slot
-            const int n_sub = MODE_Y ? 2 : 1;
-            const int slot = s.slot_seg * n_sub + (MODE_Y ? i : 0);
-            const bool owns_rows = MODE_Y || i == 0 || s.row0 + 128 < p.B;
+            // ---- segment epilogue: normalised partial + LSE into this segment's slot.  With 64-token tiles the two
+            // streams worked on the same query rows: stream 1 publishes its softmax state, stream 0 merges both
+            // accumulators (same tensor-memory lanes) and writes one partial.
+            const int slot = s.slot_seg;
+            const bool owns_rows = MODE_Y ? i == 0 : (i == 0 || s.row0 + 128 < p.B);
             if (nt > 0) {
                 const int u_last = used + nt - 1;
                 ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i][u_last & 1], (u_last >> 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                if (warp_has_rows) {
-                    const float inv = 1.f / l_sum;
-                    const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)i * 128u;
+            }
+            if (MODE_Y && i == 1) {
+                if (segi > 0) {   // stream 0 has read what the previous segment published (it frees O1 after that)
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_free[1], (segi - 1) & 1, abort_flag));
+                    if (!ok) break;
+                }
+                bar->merge_m[r] = nt > 0 ? m_ref : -INFINITY;
+                bar->merge_l[r] = nt > 0 ? l_sum : 0.f;
+                tc_fence_before();
+                mbar_arrive(&bar->merge_ready);
+            } else {
+                float a0 = 0.f, a1 = 0.f, lse2 = -INFINITY;   // weights of the two accumulators, LSE in base 2
+                if (MODE_Y) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&bar->merge_ready, segi & 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const float m1 = bar->merge_m[r], l1 = bar->merge_l[r];
+                    const float m = fmaxf(m_ref, m1);           // stream 0 always has a tile: m_ref is finite
+                    const float e0 = fast_exp2(m_ref - m), e1 = l1 > 0.f ? fast_exp2(m1 - m) : 0.f;
+                    const float l = l_sum * e0 + l1 * e1;
+                    a0 = e0 / l;
+                    a1 = e1 / l;
+                    lse2 = m + log2f(l);
+                } else if (nt > 0) {
+                    a0 = 1.f / l_sum;
+                    lse2 = m_ref + log2f(l_sum);
+                }
+                if (nt > 0 && warp_has_rows) {
+                    const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)(MODE_Y ? 0 : i) * 128u;
                     float* dst = p.o_part + (((int64_t)slot * p.part_rows + b) * p.H + s.h) * 128;
 #pragma unroll 1
                     for (int c = 0; c < 4; ++c) {
                         uint32_t orr[32];
                         tmem_ld32(o_addr + c * 32, orr);
                         tmem_ld_wait();
+                        float v[32];
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(orr[q]) * a0;
+                        if (MODE_Y && s.n_str1 > 0) {   // uniform over the CTA (the tensor-memory load is warp-collective)
+                            tmem_ld32(o_addr + 128u + c * 32, orr);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int q = 0; q < 32; ++q) v[q] = fmaf(__uint_as_float(orr[q]), a1, v[q]);
+                        }
                         if (b < p.B) {
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                float4 v = make_float4(__uint_as_float(orr[4 * q]) * inv, __uint_as_float(orr[4 * q + 1]) * inv,
-                                                       __uint_as_float(orr[4 * q + 2]) * inv, __uint_as_float(orr[4 * q + 3]) * inv);
-                                *reinterpret_cast<float4*>(dst + c * 32 + 4 * q) = v;
-                            }
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<float4*>(dst + c * 32 + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
                         }
                     }
-                    if (b < p.B) p.lse_part[((int64_t)slot * p.part_rows + b) * p.H + s.h] = (m_ref + log2f(l_sum)) * kLn2;
+                    if (b < p.B) p.lse_part[((int64_t)slot * p.part_rows + b) * p.H + s.h] = lse2 * kLn2;
+                } else if (nt == 0 && owns_rows && b < p.B) {
+                    p.lse_part[((int64_t)slot * p.part_rows + b) * p.H + s.h] = -INFINITY;   // this stream had no tile
                 }
-            } else if (owns_rows && b < p.B) {
-                p.lse_part[((int64_t)slot * p.part_rows + b) * p.H + s.h] = -INFINITY;   // this stream had no tile
-            }
-            // the segment that ends a column marks the column's unused slots as empty
-            if (s.last_of_col && owns_rows && b < p.B) {
-                for (int ss = s.slot_seg + 1; ss < p.n_seg_max; ++ss) {
-                    const int sl = ss * n_sub + (MODE_Y ? i : 0);
-                    p.lse_part[((int64_t)sl * p.part_rows + b) * p.H + s.h] = -INFINITY;
+                // the segment that ends a head marks the head's unused slots as empty
+                if (s.last_of_col && owns_rows && b < p.B) {
+                    for (int ss = s.slot_seg + 1; ss < p.n_seg_max; ++ss)
+                        p.lse_part[((int64_t)ss * p.part_rows + b) * p.H + s.h] = -INFINITY;
                 }
+                // the accumulator(s) just read may be overwritten by the next segment
+                TRACE_CTA(128, 4);
+                tc_fence_before();
+                mbar_arrive(&bar->o_free[i]);
+                if (MODE_Y) mbar_arrive(&bar->o_free[1]);
             }
-            // the accumulator of this stream may be overwritten by the next segment
-            TRACE_CTA(128, 4);
-            tc_fence_before();
-            mbar_arrive(&bar->o_free[i]);
+            ++segi;
             used += nt;
             g += s.cnt;
         }
@@ -598,7 +637,7 @@ int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 // may run in several waves); ns minimises waves x (tiles per CTA + a fixed cost of about six tile
 // times for the Q load and the pipeline fill).  "Stream-K" uses R = SMs / row groups resident
 // CTAs and gives every SM the same number of tiles at the price of a few more segments (each
-// pays the fixed cost and a pair of partial slots).  Stream-K is taken when its modelled cost is
+// pays the fixed cost and a partial slot).  Stream-K is taken when its modelled cost is
 // lower (by at least 5% in the HBM-bound regime of 64-token tiles).
 void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots) {
     const bool mode_y = B <= 128;
@@ -654,7 +693,7 @@ void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_r
         seg_max = std::max(seg_max, (int)(range_of(last) - range_of(first)) + 1);
     }
     *n_ranges = R;
-    *n_slots = seg_max * (mode_y ? 2 : 1);
+    *n_slots = seg_max;
 }
 
 cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
@@ -688,7 +727,7 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
         p.per = (int)(T / a.n_ranges);
         p.rem = (int)(T % a.n_ranges);
     }
-    p.n_seg_max = a.n_slots / (mode_y ? 2 : 1);
+    p.n_seg_max = a.n_slots;
     p.k_stages = mode_y ? 4 : 2;
     p.v_stages = mode_y ? 4 : 1;
     p.scale_log2 = a.scale * kLog2e;
