@@ -504,6 +504,92 @@ def bench_extension(cfg, args, device_index):
                      "step_frac_of_combined_roofline": t_lb / (ms * 1e-3), "peak_source": pk["source"]}}
 
 
+def bench_sharded(cfg, args, device_index, rank, world):
+    """--shard seq:G / head:G: one rank's share of a step whose context is sharded over G GPUs, by sequence
+    (slice of the prefix + the suffixes of the requests the rank owns -> fp32 partial, all-gather, combine of G
+    partials) or by head (H / G heads -> all-gather along heads).  Launched on G GPUs (torchrun, world == G) the
+    all-gather is NCCL's and inside the timed region; on one GPU the line is rank 0's compute (its partial step
+    plus the combine over G partials, the other ranks' partials being stand-in copies) and the exchange is
+    reported as bytes and as a modelled time at the pool's measured 770 GB/s per direction, not timed."""
+    import torch
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200 import inputs as I
+    from paper_2509_21081_b200 import sharded as S
+    kind, G_ = args.shard.split(":")
+    G_ = int(G_)
+    assert kind in ("seq", "head") and G_ >= 1 and world in (1, G_)
+    dev = "cuda"
+    W, K = max(args.warmup, 3), max(args.steps, 1)
+    H, B = cfg.H, cfg.B
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp, poison=False)
+    comm = S.TorchDistComm() if world > 1 else None
+    Dec = S.SequenceShardedDecoder if kind == "seq" else S.HeadShardedDecoder
+    sets = []
+    for _ in range(2):
+        dec = Dec(rank, G_, H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev), inp.w_uv.to(dev),
+                  inp.scale, B, pc.block_table.shape[1], comm=comm)
+        a = (inp.q_nope.to(dev), inp.q_pe.to(dev), pc.ckv_pages.to(dev), pc.kpe_pages.to(dev), pc.block_table.to(dev),
+             pc.seq_lens.to(dev))
+        if kind == "head":   # a rank is handed its own heads' queries
+            a = (a[0][:, dec.h0:dec.h1].contiguous(), a[1][:, dec.h0:dec.h1].contiguous()) + a[2:]
+        sets.append((dec, a))
+    mode = {"auto": b.MODE_AUTO, "absorb": b.MODE_ABSORB, "hybrid": b.MODE_HYBRID, "naive": b.MODE_NAIVE}[args.mode]
+    if kind == "seq":
+        o_parts = torch.zeros(G_, B, H, 128, dtype=torch.float32, device=dev)
+        lse_parts = torch.zeros(G_, B, H, dtype=torch.float32, device=dev)
+        out = torch.empty(B, H, 128, dtype=torch.bfloat16, device=dev)
+    else:
+        Hl = H // G_
+        out_l = torch.empty(B, Hl, 128, dtype=torch.bfloat16, device=dev)
+
+    def step(i):
+        dec, a = sets[i % 2]
+        if kind == "seq":
+            lens = lens_of[i % 2]
+            b.typhoon_mla_decode_partial(dec.shared, a[0], a[1], a[2], a[3], dec.page_size, a[4], lens, dec.scale,
+                                         o_parts[rank], lse_parts[rank], dec.workspace, mode=mode)
+            step.launches = b.typhoon_mla_last_launch_count() + 1
+            if comm is not None:
+                torch.distributed.all_gather_into_tensor(o_parts, o_parts[rank].clone())
+                torch.distributed.all_gather_into_tensor(lse_parts, lse_parts[rank].clone())
+            b.typhoon_mla_combine_partials(o_parts, lse_parts, out)
+        else:
+            b.typhoon_mla_decode(dec.shared, a[0], a[1], a[2], a[3], dec.page_size, a[4], a[5], dec.scale, out_l,
+                                 dec.workspace, mode=mode)
+            step.launches = b.typhoon_mla_last_launch_count()
+            if comm is not None:
+                comm.all_gather(out_l)
+    lens_of = [S.local_seq_lens(a[5], rank, G_) for _, a in sets]
+
+    for i in range(W):
+        step(i)
+    if kind == "seq" and comm is None:   # stand-ins for the other ranks' partials
+        for r in range(1, G_):
+            o_parts[r].copy_(o_parts[0]); lse_parts[r].copy_(lse_parts[0])
+    torch.cuda.synchronize()
+    if comm is not None:
+        torch.distributed.barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(device_index) as clocks:
+        ev0.record()
+        for i in range(K):
+            step(i)
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = max_over_ranks(ev0.elapsed_time(ev1) / K, world, "cuda") if world > 1 else ev0.elapsed_time(ev1) / K
+    xbytes = (G_ - 1) * B * H * 129 * 4 if kind == "seq" else (G_ - 1) * B * (H // G_) * 128 * 2   # received per rank
+    return {"metric": METRIC, "value": B / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{_workload_name(cfg)}, context sharded by {'sequence' if kind == 'seq' else 'head'} over {G_} GPUs",
+                       "shard": args.shard, "timed": "all ranks with the NCCL all-gather" if world > 1 else
+                       "rank 0's compute on one GPU (partial step + combine); exchange not timed",
+                       "l2": "2 full input sets used alternately"},
+            "clocks": clocks.summary(), "gpu_launches": step.launches * K,
+            "exchange": {"bytes_received_per_rank": xbytes, "modelled_us_at_770_GBps": xbytes / 770e9 * 1e6}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -517,6 +603,7 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=64, help="heads the CPU checker is timed on (scaled up)")
     ap.add_argument("--sq", type=int, default=1, help="extension: query tokens per request (rows = B * S_q)")
     ap.add_argument("--tree", default="", help="extension: G:L = G request groups with L more shared prefix tokens each")
+    ap.add_argument("--shard", default="", help="extension: seq:G or head:G = one rank's share of a context sharded over G GPUs")
     ap.add_argument("--stages", action="store_true", help="also time every kernel of the step alone (implied by --sweep)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -539,7 +626,14 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
     mode = {"auto": b.MODE_AUTO, "absorb": b.MODE_ABSORB, "hybrid": b.MODE_HYBRID, "naive": b.MODE_NAIVE}[args.mode]
 
-    if args.sq > 1 or args.tree:
+    if args.shard:
+        cfg = I.CONFIGS[args.config]
+        if args.batch:
+            cfg = cfg.with_batch(args.batch)
+        line = bench_sharded(cfg, args, local, rank, world)
+        if rank == 0:
+            print(json.dumps(line), flush=True)
+    elif args.sq > 1 or args.tree:
         if world > 1:
             raise SystemExit("--sq / --tree are single-GPU measurements")
         cfg = I.CONFIGS[args.config]

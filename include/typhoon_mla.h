@@ -158,6 +158,41 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* shared,
                        void* out, float* lse_out,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * A context sharded over several devices (Section 3.1: the shared part "can be
+ * parallelized across attention heads", the latent part across the sequence).
+ *
+ * Sequence sharding: every device holds a slice of the tokens (a slice of the
+ * shared prefix prepared as its own handle, and the suffix pages of the
+ * requests it owns; requests it does not own get seq_len 0) and calls
+ * typhoon_mla_decode_partial, which is typhoon_mla_decode except that the
+ * result over this device's tokens is returned un-rounded: out_partial fp32
+ * [B, H, 128] (normalised over this device's tokens) and lse_partial fp32
+ * [B, H] (natural log; -inf with a zero row where the device holds no token of
+ * a request; required).  The partials of all devices are gathered (one
+ * all-gather of B*H*129 floats per device) and merged by
+ * typhoon_mla_combine_partials: the log-sum-exp combine of Algorithm 1 line 8
+ * over n_parts partials, o_parts fp32 [n_parts, B, H, 128] and lse_parts fp32
+ * [n_parts, B, H] (device, 16-byte aligned) -> out bf16 [B, H, 128] and the
+ * optional lse_out fp32 [B, H].  Rows whose partials are all empty give zeros
+ * and -inf.  Head sharding needs no call of its own: a device prepares and
+ * decodes H / G heads (weights and queries sliced by head) and the bf16
+ * outputs are gathered along the head axis.
+ * Errors: as typhoon_mla_decode; INVALID_ARG for a null lse_partial or
+ * n_parts < 1.  Both calls only enqueue work on `stream`.
+ */
+int typhoon_mla_decode_partial(const typhoon_mla_shared_t* shared,
+                               const void* q_nope, const void* q_pe, int32_t B,
+                               const void* ckv_pages, const void* kpe_pages,
+                               int64_t ckv_token_stride, int64_t kpe_token_stride,
+                               int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                               const int32_t* seq_lens,
+                               float softmax_scale, int32_t mode,
+                               float* out_partial, float* lse_partial,
+                               void* workspace, size_t workspace_bytes, void* stream);
+int typhoon_mla_combine_partials(const float* o_parts, const float* lse_parts, int32_t n_parts,
+                                 int32_t B, int32_t H, void* out, float* lse_out, void* stream);
+
 /* Bytes of device staging typhoon_mla_decode_host needs (host, pure). */
 size_t typhoon_mla_host_staging_bytes(const typhoon_mla_shared_t* shared, int32_t B, int32_t max_pages);
 

@@ -57,6 +57,10 @@ def _load():
     lib.typhoon_mla_decode.argtypes = [vp, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, i32, vp, vp,
                                        vp, sz, vp]
     lib.typhoon_mla_tree_workspace_bytes.restype = sz
+    lib.typhoon_mla_decode_partial.restype = C.c_int
+    lib.typhoon_mla_decode_partial.argtypes = list(lib.typhoon_mla_decode.argtypes)
+    lib.typhoon_mla_combine_partials.restype = C.c_int
+    lib.typhoon_mla_combine_partials.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.typhoon_mla_tree_workspace_bytes.argtypes = [vp, i32, i32, i32, i32]
     lib.typhoon_mla_decode_tree.restype = C.c_int
     lib.typhoon_mla_decode_tree.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, vp, vp,
@@ -186,6 +190,32 @@ def typhoon_mla_decode(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages,
                                  _ptr(seq_lens), softmax_scale, mode, _ptr(out), _ptr(lse_out),
                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check(st, "typhoon_mla_decode")
+
+
+def typhoon_mla_decode_partial(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages, page_size, block_table,
+                               seq_lens, softmax_scale, out_partial, lse_partial, workspace, mode=MODE_AUTO,
+                               max_pages: Optional[int] = None, ckv_token_stride: Optional[int] = None,
+                               kpe_token_stride: Optional[int] = None) -> None:
+    """This device's share of a sharded context: fp32 out_partial [B, H, 128] and lse_partial [B, H]."""
+    B = q_nope.shape[0]
+    if max_pages is None:
+        max_pages = 0 if block_table is None else block_table.shape[1]
+    if ckv_token_stride is None:
+        ckv_token_stride = 512 if ckv_pages is None else ckv_pages.stride(-2)
+    if kpe_token_stride is None:
+        kpe_token_stride = 64 if kpe_pages is None else kpe_pages.stride(-2)
+    st = _lib.typhoon_mla_decode_partial(shared.handle, _ptr(q_nope), _ptr(q_pe), B, _ptr(ckv_pages), _ptr(kpe_pages),
+                                         ckv_token_stride, kpe_token_stride, page_size, _ptr(block_table), max_pages,
+                                         _ptr(seq_lens), softmax_scale, mode, _ptr(out_partial), _ptr(lse_partial),
+                                         _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
+    _check(st, "typhoon_mla_decode_partial")
+
+
+def typhoon_mla_combine_partials(o_parts, lse_parts, out, lse_out=None) -> None:
+    """o_parts fp32 [n, B, H, 128], lse_parts fp32 [n, B, H] -> out bf16 [B, H, 128] (+ lse_out fp32 [B, H])."""
+    n, B, H = lse_parts.shape
+    st = _lib.typhoon_mla_combine_partials(_ptr(o_parts), _ptr(lse_parts), n, B, H, _ptr(out), _ptr(lse_out), _stream())
+    _check(st, "typhoon_mla_combine_partials")
 
 
 class PrefixLevel(C.Structure):

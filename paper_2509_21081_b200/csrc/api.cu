@@ -507,7 +507,7 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
                 const Plan& pl, const void* q_nope, const void* q_pe, int32_t B, const void* ckv_pages,
                 const void* kpe_pages, int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size,
                 const int32_t* block_table, int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode,
-                void* out, float* lse_out, void* workspace, void* stream) {
+                void* out, float* lse_out, void* workspace, void* stream, bool out_fp32 = false) {
     const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     char* ws = reinterpret_cast<char*>(workspace);
@@ -625,6 +625,7 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
             CombineEpilogue ce;
             ce.o_naive = o_part_n; ce.lse_naive = lse_part_n; ce.n_naive = pl.n_slots_naive;
             ce.lse_abs = lse_a; ce.out = out; ce.lse_out = lse_out; ce.H = H;
+            ce.out_fp32 = out_fp32 ? 1 : 0;
             e = launch_gemm_tn_sm100(g2, sh->status, s, &ce);
             combined = true;
         } else {
@@ -640,7 +641,7 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
     if (!combined) {
         prof_before(TYPHOON_MLA_KERNEL_COMBINE, s);
         e = launch_combine(o_part_n, lse_part_n, pl.n_slots_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
-                           lse_out, s);
+                           lse_out, s, out_fp32);
         prof_after(TYPHOON_MLA_KERNEL_COMBINE, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
@@ -649,11 +650,11 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
     return TYPHOON_MLA_OK;
 }
 
-int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
+static int decode_impl(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
                        const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
                        int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
                        const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
-                       void* workspace, size_t workspace_bytes, void* stream) {
+                       void* workspace, size_t workspace_bytes, void* stream, bool out_fp32) {
     g_last_launches = 0;
     if (!sh || !q_nope || !q_pe || !out || B < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
@@ -676,7 +677,40 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const
     NaiveJob job{sh, 0, B, pl.n_split_naive, pl.n_slots_naive, 0};
     return decode_core(sh, &job, pl.n_split_naive > 0 ? 1 : 0, nullptr, 0, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
                        ckv_token_stride, kpe_token_stride, page_size, block_table, use_absorb ? max_pages : 0, seq_lens,
-                       softmax_scale, mode, out, lse_out, workspace, stream);
+                       softmax_scale, mode, out, lse_out, workspace, stream, out_fp32);
+}
+
+int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
+                       const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
+                       int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                       const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_impl(sh, q_nope, q_pe, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table,
+                       max_pages, seq_lens, softmax_scale, mode, out, lse_out, workspace, workspace_bytes, stream, false);
+}
+
+// ---- context sharded over several devices: per-device partial + merge -----------------------------
+int typhoon_mla_decode_partial(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
+                               const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
+                               int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table,
+                               int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode,
+                               float* out_partial, float* lse_partial, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+    if (!lse_partial) return TYPHOON_MLA_ERR_INVALID_ARG;
+    return decode_impl(sh, q_nope, q_pe, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table,
+                       max_pages, seq_lens, softmax_scale, mode, out_partial, lse_partial, workspace, workspace_bytes,
+                       stream, true);
+}
+
+int typhoon_mla_combine_partials(const float* o_parts, const float* lse_parts, int32_t n_parts, int32_t B, int32_t H,
+                                 void* out, float* lse_out, void* stream) {
+    if (!o_parts || !lse_parts || !out || n_parts < 1 || B < 1 || H < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!aligned16(o_parts) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const cudaError_t e = launch_combine(o_parts, lse_parts, n_parts, nullptr, nullptr, B, H, out, lse_out,
+                                         reinterpret_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_last_launches = 1;
+    return TYPHOON_MLA_OK;
 }
 // ---- several shared prefixes per step (tree-structured prompts) ------------------------------------
 namespace {

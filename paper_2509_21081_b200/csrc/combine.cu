@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
                                                       const float* __restrict__ lse_naive, int n_naive,
                                                       const float* __restrict__ o_abs,
                                                       const float* __restrict__ lse_abs, int BH,
-                                                      __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out) {
+                                                      void* __restrict__ out, float* __restrict__ lse_out, int out_fp32) {
     sm100::pdl_trigger();
     sm100::pdl_wait();
     const int bh = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -157,8 +157,12 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
         float inv = 1.f / z;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }
-    uint2 pk = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-    *reinterpret_cast<uint2*>(out + (int64_t)bh * 128 + lane * 4) = pk;
+    if (out_fp32) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + (int64_t)bh * 128 + lane * 4) = acc;
+    } else {
+        uint2 pk = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + (int64_t)bh * 128 + lane * 4) = pk;
+    }
     if (lse_out != nullptr && lane == 0) lse_out[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(z);
 }
 
@@ -261,11 +265,11 @@ cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int 
 }
 
 cudaError_t launch_combine(const float* o_naive, const float* lse_naive, int n_naive, const float* o_abs,
-                           const float* lse_abs, int B, int H, void* out_bf16, float* lse_out, cudaStream_t s) {
+                           const float* lse_abs, int B, int H, void* out, float* lse_out, cudaStream_t s, bool out_fp32) {
     int BH = B * H;
     if (BH <= 0) return cudaSuccess;
     return launch_pdl(combine_kernel, dim3((BH + 7) / 8), dim3(256), 0, s, o_naive, lse_naive, n_naive, o_abs, lse_abs, BH,
-                      reinterpret_cast<__nv_bfloat16*>(out_bf16), lse_out);
+                      out, lse_out, out_fp32 ? 1 : 0);
 }
 
 cudaError_t launch_transpose_bf16(const void* in, void* out, int R, int C, int batch, cudaStream_t s) {

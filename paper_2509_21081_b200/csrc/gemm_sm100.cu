@@ -160,6 +160,7 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
                     tmem_ld_wait();
                     if (!live) continue;
                     __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(ce.out) + bh * 128 + c * 32;
+                    float* dstf = reinterpret_cast<float*>(ce.out) + bh * 128 + c * 32;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         float o[8];
@@ -168,10 +169,15 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
                             const float oa = wa > 0.f ? wa * __uint_as_float(r[j * 8 + e]) : 0.f;
                             o[e] = (accn[c * 32 + j * 8 + e] + oa) * inv;
                         }
-                        uint4 v;
-                        v.x = pack_bf16(o[0], o[1]); v.y = pack_bf16(o[2], o[3]);
-                        v.z = pack_bf16(o[4], o[5]); v.w = pack_bf16(o[6], o[7]);
-                        *reinterpret_cast<uint4*>(dst + j * 8) = v;
+                        if (ce.out_fp32) {
+                            *reinterpret_cast<float4*>(dstf + j * 8) = make_float4(o[0], o[1], o[2], o[3]);
+                            *reinterpret_cast<float4*>(dstf + j * 8 + 4) = make_float4(o[4], o[5], o[6], o[7]);
+                        } else {
+                            uint4 v;
+                            v.x = pack_bf16(o[0], o[1]); v.y = pack_bf16(o[2], o[3]);
+                            v.z = pack_bf16(o[4], o[5]); v.w = pack_bf16(o[6], o[7]);
+                            *reinterpret_cast<uint4*>(dst + j * 8) = v;
+                        }
                     }
                 }
                 if (live && ce.lse_out) ce.lse_out[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(zsum);

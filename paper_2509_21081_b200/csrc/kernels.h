@@ -52,6 +52,7 @@ struct CombineEpilogue {
     void* out = nullptr;               // bf16 [B][H][128]
     float* lse_out = nullptr;          // optional [B][H]
     int H = 0;
+    int out_fp32 = 0;                  // `out` is fp32 [B][H][128] (a partial result for a later merge)
 };
 cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, const CombineEpilogue* ce = nullptr);
 
@@ -134,10 +135,11 @@ cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm
 cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,
                                 void* o_lat_bf16, float* lse, cudaStream_t s);
 
-// Final LSE combine (Algorithm 1 line 8) of n_naive naive partials and an optional absorb partial.
+// Final LSE combine (Algorithm 1 line 8) of n_naive naive partials and an optional absorb partial;
+// `out` is bf16 [B,H,128], or fp32 with out_fp32.
 cudaError_t launch_combine(const float* o_naive, const float* lse_naive, int n_naive,
                            const float* o_abs, const float* lse_abs,
-                           int B, int H, void* out_bf16, float* lse_out, cudaStream_t s);
+                           int B, int H, void* out, float* lse_out, cudaStream_t s, bool out_fp32 = false);
 
 // out[c][r] = in[r][c] for each of `batch` matrices [R][C] bf16.
 cudaError_t launch_transpose_bf16(const void* in, void* out, int R, int C, int batch, cudaStream_t s);

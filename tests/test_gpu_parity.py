@@ -565,3 +565,72 @@ def test_more_requests_than_the_ordering_block_sorts():
     """B = 4500 (> 4096): no longest-first order and no descriptors, 4500 CTAs per head group."""
     cfg = _cfg("wide", B=4500, H=16, Ls=100, lo=0, hi=70, seed=52)
     _full_size_sampled(cfg, (HYBRID, ABSORB), n_pairs=48, extremes=True)
+
+
+def _upload(inp, pc):
+    dev = "cuda"
+    return (inp.q_nope.to(dev), inp.q_pe.to(dev), pc.ckv_pages.to(dev), pc.kpe_pages.to(dev), pc.block_table.to(dev),
+            pc.seq_lens.to(dev))
+
+
+@pytest.mark.parametrize("world,Ls", [(2, 1000), (3, 700), (4, 130)])
+def test_sequence_sharded_ranks_one_after_the_other(world, Ls):
+    """The context sharded by sequence over `world` ranks, the ranks' partial steps run one after the other
+    on this GPU (no kernel waits for another): slices of the prefix (one of them empty when there are fewer
+    64-token blocks than ranks), suffixes owned round robin, fp32 partials merged by the combine entry point."""
+    from paper_2509_21081_b200 import binding as b, sharded as S
+    cfg = _cfg("seqshard", B=11, H=32, Ls=Ls, lo=0, hi=260, seed=60 + world)
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp, poison=True)
+    ref, ref_lse = G.run_oracle(inp)
+    args = _upload(inp, pc)
+    parts = []
+    for r in range(world):
+        dec = S.SequenceShardedDecoder(r, world, cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(),
+                                       inp.w_uv.cuda(), inp.scale, cfg.B, pc.block_table.shape[1])
+        parts.append(dec.partial(*args, mode=AUTO if r % 2 else HYBRID))
+        assert b.typhoon_mla_device_status(dec.shared) == 0
+        dec.close()
+    lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
+    out = S.merge_partials(torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]), lse)
+    G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse, what=f"sequence shards {world}")
+
+
+@pytest.mark.parametrize("world,H", [(2, 64), (4, 128)])
+def test_head_sharded_ranks_one_after_the_other(world, H):
+    from paper_2509_21081_b200 import binding as b, sharded as S
+    cfg = _cfg("headshard", B=6, H=H, Ls=300, lo=1, hi=150, seed=70 + world)
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp, poison=True)
+    ref, _ = G.run_oracle(inp)
+    args = _upload(inp, pc)
+    parts = []
+    for r in range(world):
+        dec = S.HeadShardedDecoder(r, world, cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(),
+                                   inp.w_uv.cuda(), inp.scale, cfg.B, pc.block_table.shape[1])
+        parts.append(dec.local(*args, mode=HYBRID))
+        assert b.typhoon_mla_device_status(dec.shared) == 0
+        dec.close()
+    out = S.join_heads(torch.stack(parts))
+    G.assert_parity(out.float().cpu().double().numpy(), ref, what=f"head shards {world}")
+
+
+def test_combine_partials_edge_cases():
+    """Partials that are all empty give a zero row and -inf; an empty partial next to a live one has no weight
+    even when its row holds NaN."""
+    from paper_2509_21081_b200 import sharded as S
+    g = torch.Generator().manual_seed(3)
+    o = torch.randn(3, 4, 16, 128, generator=g).cuda()
+    lse = torch.randn(3, 4, 16, generator=g).cuda()
+    lse[:, 0, :] = -math.inf                     # request 0: nothing anywhere
+    lse[1, 1, :] = -math.inf; o[1, 1] = math.nan   # request 1: rank 1 holds nothing, its row is garbage
+    lse_out = torch.empty(4, 16, device="cuda")
+    out = S.merge_partials(o, lse, lse_out).float().cpu()
+    assert torch.all(out[0] == 0) and torch.all(lse_out[0].cpu() == -math.inf)
+    o64, l64 = o.cpu().double(), lse.cpu().double()
+    w = torch.softmax(l64[:, 1:], dim=0)
+    w = torch.nan_to_num(w, nan=0.0)
+    o64 = torch.nan_to_num(o64, nan=0.0)
+    ref = (w.unsqueeze(-1) * o64[:, 1:]).sum(0)
+    assert torch.allclose(out[1:].double(), ref, atol=2e-2, rtol=1e-2)
+    assert torch.allclose(lse_out[1:].cpu().double(), torch.logsumexp(l64[:, 1:], dim=0), atol=1e-4)
