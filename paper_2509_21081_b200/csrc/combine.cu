@@ -55,13 +55,15 @@ __global__ void __launch_bounds__(512) merge_latent_kernel(const float* __restri
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (m != -INFINITY) {
         const float* src = o_part + (int64_t)bh * 512 + col * 4;
-#pragma unroll 4
+        // loads do not wait for the weights (eight in flight per thread); an empty chunk's slot was never
+        // written, so its value is dropped by a select
+#pragma unroll 8
         for (int c = grp; c < n_chunks; c += G) {
+            const float4 v = *reinterpret_cast<const float4*>(src + (int64_t)c * BH * 512);
             const float w = w_s[c];
-            if (w != 0.f) {
-                const float4 v = *reinterpret_cast<const float4*>(src + (int64_t)c * BH * 512);
-                acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-            }
+            const bool live = w != 0.f;
+            acc.x += live ? w * v.x : 0.f; acc.y += live ? w * v.y : 0.f;
+            acc.z += live ? w * v.z : 0.f; acc.w += live ? w * v.w : 0.f;
         }
     }
     if (grp > 0) acc_s[grp - 1][col] = acc;
@@ -83,8 +85,11 @@ __global__ void __launch_bounds__(512) merge_latent_kernel(const float* __restri
 
 // Few chunks per request (the common case at larger batch sizes): no shared memory, four (b, h) rows
 // per block of 512 threads, each thread owns 4 of a row's 512 latent columns and recomputes the (at most
-// MERGE_FEW) chunk weights itself.
+// NC) chunk weights itself.  The LSEs and the partial rows are all requested before any of them is used
+// (one memory round trip per thread); the slot of an empty chunk was never written, so its value is
+// dropped by a select, not multiplied by a zero weight.
 constexpr int MERGE_FEW = 16;
+template <int NC>
 __global__ void __launch_bounds__(512) merge_latent_few_kernel(const float* __restrict__ o_part,
                                                                const float* __restrict__ lse_part, int n_chunks,
                                                                int BH, __nv_bfloat16* __restrict__ o_lat,
@@ -93,22 +98,26 @@ __global__ void __launch_bounds__(512) merge_latent_few_kernel(const float* __re
     sm100::pdl_wait();
     const int bh = blockIdx.x * 4 + (threadIdx.x >> 7), col = threadIdx.x & 127;
     if (bh >= BH) return;
-    float l[MERGE_FEW];
+    float l[NC];
+    float4 v[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) l[c] = c < n_chunks ? lse_part[(int64_t)c * BH + bh] : -INFINITY;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+        v[c] = c < n_chunks ? *reinterpret_cast<const float4*>(o_part + ((int64_t)c * BH + bh) * 512 + col * 4)
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
     float m = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < MERGE_FEW; ++c) {
-        l[c] = c < n_chunks ? lse_part[(int64_t)c * BH + bh] : -INFINITY;
-        m = fmaxf(m, l[c]);
-    }
+    for (int c = 0; c < NC; ++c) m = fmaxf(m, l[c]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float z = 0.f;
     if (m != -INFINITY) {
 #pragma unroll
-        for (int c = 0; c < MERGE_FEW; ++c) {
-            if (l[c] == -INFINITY) continue;   // empty chunk (or none): its O slot was never written
-            const float w = __expf(l[c] - m);
-            const float4 v = *reinterpret_cast<const float4*>(o_part + ((int64_t)c * BH + bh) * 512 + col * 4);
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        for (int c = 0; c < NC; ++c) {
+            const bool live = l[c] != -INFINITY;
+            const float w = live ? __expf(l[c] - m) : 0.f;
+            acc.x += live ? w * v[c].x : 0.f; acc.y += live ? w * v[c].y : 0.f;
+            acc.z += live ? w * v[c].z : 0.f; acc.w += live ? w * v[c].w : 0.f;
             z += w;
         }
         const float inv = 1.f / z;
@@ -255,8 +264,12 @@ cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int 
     if (B * H <= 0) return cudaSuccess;
     if (n_chunks > MERGE_MAX_CHUNKS) return cudaErrorInvalidValue;
     if (n_chunks <= MERGE_FEW) {
-        return launch_pdl(merge_latent_few_kernel, dim3((B * H + 3) / 4), dim3(512), 0, s, o_part, lse_part, n_chunks, B * H,
-                          reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
+        const dim3 grid((B * H + 3) / 4);
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(o_lat_bf16);
+        if (n_chunks <= 2) return launch_pdl(merge_latent_few_kernel<2>, grid, dim3(512), 0, s, o_part, lse_part, n_chunks, B * H, o, lse);
+        if (n_chunks <= 4) return launch_pdl(merge_latent_few_kernel<4>, grid, dim3(512), 0, s, o_part, lse_part, n_chunks, B * H, o, lse);
+        if (n_chunks <= 8) return launch_pdl(merge_latent_few_kernel<8>, grid, dim3(512), 0, s, o_part, lse_part, n_chunks, B * H, o, lse);
+        return launch_pdl(merge_latent_few_kernel<MERGE_FEW>, grid, dim3(512), 0, s, o_part, lse_part, n_chunks, B * H, o, lse);
     } else {
         return launch_pdl(merge_latent_kernel, dim3(B * H), dim3(512), 0, s, o_part, lse_part, n_chunks, B * H,
                           reinterpret_cast<__nv_bfloat16*>(o_lat_bf16), lse);
