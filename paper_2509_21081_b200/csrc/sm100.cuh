@@ -229,6 +229,14 @@ __device__ __forceinline__ void tma_load_3d_if(uint32_t issue, void* dst, const 
             "r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(issue)
         : "memory");
 }
+// Request a box into L2 only (no shared memory, no completion): a later tma_load of the same box hits L2.
+__device__ __forceinline__ void tma_prefetch_3d_if(uint32_t issue, const CUtensorMap* m, int x, int y, int z) {
+    asm volatile(
+        "{\n.reg .pred q;\nsetp.ne.b32 q, %4, 0;\n"
+        "@q cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];\n}\n" ::
+            "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(z), "r"(issue)
+        : "memory");
+}
 __device__ __forceinline__ void tma_load_4d_if(uint32_t issue, void* dst, const CUtensorMap* m, uint64_t* bar, int x, int y, int z,
                                                int w) {
     asm volatile(
