@@ -503,6 +503,8 @@ struct EmptySlots {
 // Launch sequence of one step.  `sh` provides the weights, the absorb-side tensor maps, the side stream
 // and the status word; `mode` is resolved (ABSORB, HYBRID or NAIVE); `pl.n_slots_naive` is the total
 // number of naive partial slots.
+constexpr int kMergeProjectMaxB = 2;   // measured: from 3 requests on the GEMM form (weights read once) is faster
+
 static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n_jobs, const EmptySlots* empties, int n_empties,
                 const Plan& pl, const void* q_nope, const void* q_pe, int32_t B, const void* ckv_pages,
                 const void* kpe_pages, int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size,
@@ -604,6 +606,15 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
         prof_after(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         if (e != cudaSuccess) return cuda_fail(e);
         ++launches;
+        if (n_jobs == 0 && n_empties == 0 && n_chunks > 1 && B <= kMergeProjectMaxB) {
+            // absorb-only, a handful of requests: merge + projection + rounding in one launch
+            prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
+            e = launch_merge_project(o_part_a, lse_part_a, n_chunks, B, H, sh->w_uv, out, lse_out, out_fp32, s);
+            prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
+            if (e != cudaSuccess) return cuda_fail(e);
+            g_last_launches = launches + 1;
+            return TYPHOON_MLA_OK;
+        }
         if (!(tc && n_chunks == 1)) {   // a single-chunk tcgen05 launch has already written the merged result
             prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
             e = launch_merge_latent(o_part_a, lse_part_a, n_chunks, B, H, o_lat, lse_a, s);

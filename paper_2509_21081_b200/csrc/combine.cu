@@ -128,6 +128,109 @@ __global__ void __launch_bounds__(512) merge_latent_few_kernel(const float* __re
     if (col == 0) lse[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(z);
 }
 
+// Absorb-only step at small batch sizes: merge of the chunk partials, output projection O_A W_UV^T (Algorithm 1
+// line 7) and the final rounding in one launch.  One block per (request, head), 512 threads.  The 128 KB of the
+// head's W_UV (16 warps x 8 rows x 1 KB) are requested into L2 first and arrive while the chunk partials are merged
+// as in merge_latent_kernel; the merged latent row stays in fp32 in shared memory; every warp then forms 8 of the 128
+// outputs as dot products over 512 (16 elements per lane, butterfly sum).  Each block re-reads its head's weights,
+// so this form is for one or two requests (the GEMM form reads them once per 128 requests).
+__global__ void __launch_bounds__(512) merge_project_kernel(const float* __restrict__ o_part,
+                                                            const float* __restrict__ lse_part, int n_chunks, int B,
+                                                            int H, const __nv_bfloat16* __restrict__ w_uv,
+                                                            void* __restrict__ out, float* __restrict__ lse_out,
+                                                            int out_fp32) {
+    sm100::pdl_trigger();
+    sm100::pdl_wait();
+    __shared__ float w_s[MERGE_MAX_CHUNKS];
+    __shared__ float red[16];
+    __shared__ float4 acc_s[4][128];
+    const int h = blockIdx.x, b = blockIdx.y, BH = B * H, bh = b * H + h;
+    const int tid = threadIdx.x, grp = tid >> 7, col = tid & 127, warp = tid >> 5, lane = tid & 31;
+    // this warp's 8 weight rows (8 KB, contiguous): requested into L2 now, loaded after the merge
+    const __nv_bfloat16* wrow = w_uv + ((int64_t)h * 128 + warp * 8) * 512 + lane * 16;
+    {
+        const char* wl = reinterpret_cast<const char*>(w_uv + ((int64_t)h * 128 + warp * 8) * 512);
+        asm volatile("prefetch.global.L2 [%0];\n" ::"l"(wl + lane * 128));
+        asm volatile("prefetch.global.L2 [%0];\n" ::"l"(wl + 4096 + lane * 128));
+    }
+    float m = -INFINITY;
+    for (int c = tid; c < n_chunks; c += 512) {
+        const float l = lse_part[(int64_t)c * BH + bh];
+        w_s[c] = l;
+        m = fmaxf(m, l);
+    }
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    m = red[0];
+    for (int i = 1; i < 16; ++i) m = fmaxf(m, red[i]);
+    __syncthreads();
+    float z = 0.f;
+    for (int c = tid; c < n_chunks; c += 512) {
+        const float l = w_s[c];
+        const float w = (l == -INFINITY) ? 0.f : __expf(l - m);
+        w_s[c] = w;
+        z += w;
+    }
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    if (lane == 0) red[warp] = z;
+    __syncthreads();
+    z = 0.f;
+    for (int i = 0; i < 16; ++i) z += red[i];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (m != -INFINITY) {
+        const float* src = o_part + (int64_t)bh * 512 + col * 4;
+#pragma unroll 4
+        for (int c = grp; c < n_chunks; c += 4) {
+            const float4 v = *reinterpret_cast<const float4*>(src + (int64_t)c * BH * 512);
+            const float w = w_s[c];
+            const bool live = w != 0.f;   // an empty chunk's slot was never written
+            acc.x += live ? w * v.x : 0.f; acc.y += live ? w * v.y : 0.f;
+            acc.z += live ? w * v.z : 0.f; acc.w += live ? w * v.w : 0.f;
+        }
+    }
+    acc_s[grp][col] = acc;
+    __syncthreads();
+    // the merged, normalised latent row: this lane's 16 elements (float4 columns 4 lane .. 4 lane + 3)
+    const float inv = (m != -INFINITY) ? 1.f / z : 0.f;
+    float o[16];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float4 v = acc_s[0][lane * 4 + q];
+#pragma unroll
+        for (int g = 1; g < 4; ++g) {
+            const float4 u = acc_s[g][lane * 4 + q];
+            v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+        }
+        o[4 * q] = v.x * inv; o[4 * q + 1] = v.y * inv; o[4 * q + 2] = v.z * inv; o[4 * q + 3] = v.w * inv;
+    }
+    uint4 wv[8][2];   // 16 consecutive elements per lane and row (two 16-byte loads)
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        wv[r][0] = *reinterpret_cast<const uint4*>(wrow + r * 512);
+        wv[r][1] = *reinterpret_cast<const uint4*>(wrow + r * 512 + 8);
+    }
+    float res = 0.f;   // lane r < 8 keeps output row warp * 8 + r
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        const uint32_t wr[8] = {wv[r][0].x, wv[r][0].y, wv[r][0].z, wv[r][0].w, wv[r][1].x, wv[r][1].y, wv[r][1].z, wv[r][1].w};
+        float d = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const __nv_bfloat162 p2 = *reinterpret_cast<const __nv_bfloat162*>(&wr[e]);
+            d += __low2float(p2) * o[2 * e] + __high2float(p2) * o[2 * e + 1];
+        }
+        for (int s2 = 16; s2 > 0; s2 >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s2);
+        if (lane == r) res = d;
+    }
+    if (lane < 8) {
+        const int64_t idx = (int64_t)bh * 128 + warp * 8 + lane;
+        if (out_fp32) reinterpret_cast<float*>(out)[idx] = res;
+        else reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(res);
+    }
+    if (tid == 0 && lse_out != nullptr) lse_out[bh] = (m == -INFINITY) ? -INFINITY : m + __logf(z);
+}
+
 // One warp per (b, h); each lane owns 4 of the 128 output columns.
 __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ o_naive,
                                                       const float* __restrict__ lse_naive, int n_naive,
@@ -257,6 +360,14 @@ cudaError_t launch_expand_query_rows(const int32_t* block_table, const int32_t* 
     const unsigned blocks = (unsigned)std::min<int64_t>((n + 255) / 256, 1184);
     expand_query_rows_kernel<<<blocks, 256, 0, s>>>(block_table, seq_lens, B, max_pages, S_q, bt_rows, len_rows);
     return cudaGetLastError();
+}
+
+cudaError_t launch_merge_project(const float* o_part, const float* lse_part, int n_chunks, int B, int H, const void* w_uv,
+                                 void* out, float* lse_out, bool out_fp32, cudaStream_t s) {
+    if (B * H <= 0) return cudaSuccess;
+    if (n_chunks > MERGE_MAX_CHUNKS) return cudaErrorInvalidValue;
+    return launch_pdl(merge_project_kernel, dim3(H, B), dim3(512), 0, s, o_part, lse_part, n_chunks, B, H,
+                      reinterpret_cast<const __nv_bfloat16*>(w_uv), out, lse_out, out_fp32 ? 1 : 0);
 }
 
 cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,

@@ -135,6 +135,11 @@ cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm
 cudaError_t launch_merge_latent(const float* o_part, const float* lse_part, int n_chunks, int B, int H,
                                 void* o_lat_bf16, float* lse, cudaStream_t s);
 
+// Absorb-only step with one or two requests: merge of the chunk partials + W_UV projection (Algorithm 1 line 7)
+// + final rounding in one launch; w_uv is [H, 128, 512] bf16; out bf16 (or fp32) [B, H, 128], lse_out optional.
+cudaError_t launch_merge_project(const float* o_part, const float* lse_part, int n_chunks, int B, int H, const void* w_uv,
+                                 void* out, float* lse_out, bool out_fp32, cudaStream_t s);
+
 // Final LSE combine (Algorithm 1 line 8) of n_naive naive partials and an optional absorb partial;
 // `out` is bf16 [B,H,128], or fp32 with out_fp32.
 cudaError_t launch_combine(const float* o_naive, const float* lse_naive, int n_naive,

@@ -634,3 +634,27 @@ def test_combine_partials_edge_cases():
     ref = (w.unsqueeze(-1) * o64[:, 1:]).sum(0)
     assert torch.allclose(out[1:].double(), ref, atol=2e-2, rtol=1e-2)
     assert torch.allclose(lse_out[1:].cpu().double(), torch.logsumexp(l64[:, 1:], dim=0), atol=1e-4)
+
+
+@pytest.mark.parametrize("B", [1, 2, 3])
+def test_absorb_only_one_or_two_requests(B):
+    """Absorb-only steps of one or two requests take a single kernel for chunk merge, output projection and
+    rounding; three requests take the GEMM form.  Long context (many chunks), one empty suffix, bf16 and fp32
+    (partial) outputs."""
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    cfg = _cfg("fewreq", B=B, H=64, Ls=3000, lo=0, hi=0, seed=80 + B)
+    inp = I.make_inputs(cfg, suffix_lens=[0, 333, 70][:B])
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, launches = G.run_gpu(inp, ABSORB)
+    G.assert_parity(out, ref, lse, ref_lse, what=f"absorb-only B={B}")
+    pc = I.build_pages(inp, poison=True)
+    dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(), inp.scale,
+                            cfg.B, pc.block_table.shape[1])
+    o32 = torch.empty(B, cfg.H, 128, dtype=torch.float32, device="cuda")
+    l32 = torch.empty(B, cfg.H, dtype=torch.float32, device="cuda")
+    b.typhoon_mla_decode_partial(dec.shared, *_upload(inp, pc)[:4], cfg.page_size, *_upload(inp, pc)[4:], inp.scale, o32, l32,
+                                 dec.workspace, mode=ABSORB)
+    assert b.typhoon_mla_device_status(dec.shared) == 0
+    G.assert_parity(o32.cpu().double().numpy(), ref, l32.cpu().double().numpy(), ref_lse, what=f"absorb-only fp32 B={B}")
+    dec.close()
