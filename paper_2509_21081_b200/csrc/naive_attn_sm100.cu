@@ -22,6 +22,8 @@
 //     takes every second KV tile with its own softmax state, and at the end of the segment
 //     stream 0 merges the two accumulators (same tensor-memory lanes) into one partial.
 //     HBM-bound regime: small tiles give deep K and V rings.
+//     With B <= 64 the MMAs are issued with M = 64 (template flag M64): accumulator row r then
+//     sits in lane 32 (r / 16) + r % 16 and half of the softmax lanes hold no row.
 //
 // Warp roles (384 threads): warp 0 = TMA producer for Q and the K ring, warp 2 = TMA producer
 // for the V ring, warp 1 = issuer of the S = Q K^T MMAs and TMEM owner, warp 3 = issuer of the
@@ -122,7 +124,7 @@ struct Segment {
 };
 
 // TOK = tokens per KV tile: 64 (mode Y, B <= 128) or 128 (mode X, B > 128).
-template <int TOK>
+template <int TOK, bool M64>
 __global__ void __launch_bounds__(384, 1)
 naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_constant__ CUtensorMap tm_qp,
                         const __grid_constant__ CUtensorMap tm_kn, const __grid_constant__ CUtensorMap tm_kp,
@@ -317,7 +319,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         // ---------------- S = Q K^T issuer.  With two S buffers per stream it runs ahead of the softmax by
         // up to two steps; with one it follows the PV product of the previous step.
         const uint32_t ld = elect_one() ? 1u : 0u;
-        constexpr uint32_t idesc_s = idesc_bf16(128, TOK, false, false);
+        constexpr uint32_t idesc_s = idesc_bf16(M64 ? 64 : 128, TOK, false, false);
         int ring_base = 0, seg = 0;
         int used0 = 0, used1 = 0;                              // S-buffer uses so far, per stream
         bool ok = true;
@@ -365,7 +367,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     } else if (warp == 3) {
         // ---------------- O += P V issuer
         const uint32_t ld = elect_one() ? 1u : 0u;
-        constexpr uint32_t idesc_o = idesc_bf16(128, 128, false, false);
+        constexpr uint32_t idesc_o = idesc_bf16(M64 ? 64 : 128, 128, false, false);
         int ring_base = 0, seg = 0;
         int used0 = 0, used1 = 0;
         bool ok = true;
@@ -415,15 +417,20 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         // ---------------- softmax warpgroups
         const int i = (warp - 4) >> 2;            // stream
         const int lg = (warp & 3) * 32;           // TMEM lane group of this warp
-        const int r = lg + lane;                  // row within the 128-row tile
+        const int r = lg + lane;                  // this thread's tensor-memory lane
+        // query row of this thread within the tile: the lane itself, or, with M = 64 accumulators, 16 rows in
+        // the first 16 lanes of every 32-lane group (the other lanes hold no row; they only keep in step)
+        const bool lane_has_row = !M64 || lane < 16;
+        const int row = M64 ? (warp & 3) * 16 + lane : r;
         int used = 0;                             // S-buffer uses (= PV products) of this stream so far
         int segi = 0;                             // segments finished by this CTA
         bool ok = true;
         for (int g = g_begin; g < g_end && ok;) {
             const Segment s = segment_at(g);
-            const int b = s.row0 + (MODE_Y ? 0 : i * 128) + r;
+            const int tile_row0 = s.row0 + (MODE_Y ? 0 : i * 128);
+            const int b = lane_has_row ? tile_row0 + row : 0x3fffffff;
             const int nt = i == 0 ? s.n_str0 : s.n_str1;
-            const bool warp_has_rows = (b - lane) < p.B;   // warp-uniform: first row of this warp is a real request
+            const bool warp_has_rows = tile_row0 + (M64 ? (warp & 3) * 16 : lg) < p.B;   // warp-uniform: the warp's first row is a real request
             float m_ref = -INFINITY, l_sum = 0.f;
             for (int j = 0; j < nt && ok; ++j) {
                 const int u = used + j;
@@ -464,7 +471,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 const float mx = mx_raw * p.scale_log2;
                 if ((warp & 3) == 0) TRACE(j, 10 + 8 * i);
                 // lazy rescale: only when some row's maximum grew by more than 2^8
-                const bool grow = mx > m_ref + 8.f;
+                const bool grow = lane_has_row && mx > m_ref + 8.f;
                 if (j == 0) {
                     m_ref = mx;
                 } else if (__any_sync(0xffffffffu, grow)) {
@@ -736,11 +743,15 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     const int smem = (mode_y ? 1 : 2) * Q_TILE_BYTES + p.k_stages * k_tile + p.v_stages * v_tile + 1024 + (int)sizeof(Barriers) + 64;
     dim3 grid(p.n_ranges * p.m_groups, 1, 1);
     if (mode_y) {
-        cudaFuncSetAttribute(naive_attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        return launch_pdl(naive_attn_sm100_kernel<64>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        if (a.B <= 64) {   // half-height MMAs: the padding rows 64..127 of the query tile cost tensor-pipe time and power
+            cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            return launch_pdl(naive_attn_sm100_kernel<64, true>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        }
+        cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        return launch_pdl(naive_attn_sm100_kernel<64, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     } else {
-        cudaFuncSetAttribute(naive_attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        return launch_pdl(naive_attn_sm100_kernel<128>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        cudaFuncSetAttribute(naive_attn_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        return launch_pdl(naive_attn_sm100_kernel<128, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     }
     return cudaGetLastError();
 }
