@@ -32,7 +32,7 @@ UNIT = "queries/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (key: (config, kernel)); None where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("cfg1", "naive_attn"): 276_451_584,     # profiles/naive_attn_sm100_cfg1_and_cfg4_b512.md
+    ("cfg1", "naive_attn"): 275_993_856,     # profiles/naive_attn_sm100_cfg1_and_cfg4_b512.md
     ("cfg3", "absorb_attn"): 652_079_360,    # profiles/absorb_attn_sm100_cfg3.md
     ("cfg4_B512", "naive_attn"): 1_159_151_640,
 }
