@@ -238,9 +238,18 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     # previous step's data in the 126 MB L2 (each copy alone is larger than L2 for configs 1-4).
     n_sets = 2
     sets = []
-    for _ in range(n_sets):
-        dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev),
-                                inp.w_uv.to(dev), inp.scale, cfg.B, max_pages, pc.page_size)
+    prepare_ms = None
+    for k in range(n_sets):
+        dev_in = (inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev), inp.w_uv.to(dev))
+        # the one-off expansion of the prefix (not part of a step): timed on the second set, after the first
+        # has paid for context and module loading
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pe0.record()
+        dec = TyphoonMLADecoder(cfg.H, *dev_in, inp.scale, cfg.B, max_pages, pc.page_size)
+        pe1.record()
+        if k == 1:
+            torch.cuda.synchronize()
+            prepare_ms = pe0.elapsed_time(pe1)
         sets.append(dict(dec=dec, q_nope=inp.q_nope.to(dev), q_pe=inp.q_pe.to(dev), ckv=pc.ckv_pages.to(dev),
                          kpe=pc.kpe_pages.to(dev), bt=pc.block_table.to(dev), sl=pc.seq_lens.to(dev),
                          out=torch.empty(cfg.B, cfg.H, 128, dtype=torch.bfloat16, device=dev)))
@@ -420,6 +429,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
                        "parallelism": f"replicas x{world} (shard by request, no exchange)",
                        "l2": f"{n_sets} full input sets used alternately, each larger than the 126 MB L2"},
             "clocks": clocks.summary(), "e2e": e2e, "stages": stages, "gpu_launches": launches_per_step * K,
+            "prepare_shared_ms": prepare_ms,
             "roofline": roof, "cpu_baseline": cpu}
     return line
 
