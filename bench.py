@@ -514,6 +514,68 @@ def bench_extension(cfg, args, device_index):
                      "step_frac_of_combined_roofline": t_lb / (ms * 1e-3), "peak_source": pk["source"]}}
 
 
+def bench_naive_everywhere(cfg, args, device_index):
+    """--naive-suffix: the naive formulation on the shared AND the non-shared part (the paper's naive-only
+    curves in Fig. 8): every request's suffix is expanded once into per-head K/V (as a naive KV cache would hold
+    it; not part of the step) and attended with the shared-prefix kernel, one launch per request, next to the
+    shared prefix's launch; no absorb branch.  Built from typhoon_mla_decode_tree (level 0: the prefix for all
+    requests; level 1: one group per request whose "prefix" is that request's suffix).  B <= 255."""
+    import torch
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200 import inputs as I
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    dev = "cuda"
+    W, K = max(args.warmup, 3), max(args.steps, 1)
+    H, B = cfg.H, cfg.B
+    assert B <= 255, "one shared-prefix launch per request: at most 255 requests"
+    inp = I.make_inputs(cfg)
+    pc = I.build_pages(inp, poison=False)
+    dims = b.make_dims(H)
+    w_uk, w_uv = inp.w_uk.to(dev), inp.w_uv.to(dev)
+    q_nope, q_pe = inp.q_nope.to(dev), inp.q_pe.to(dev)
+    sets = []
+    for _ in range(2):
+        root = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), w_uk, w_uv)
+        own = [b.typhoon_mla_prepare_shared(dims, inp.ckv_suffix[r].to(dev), inp.kpe_suffix[r].to(dev), w_uk, w_uv)
+               if inp.ckv_suffix[r].shape[0] > 0 else None for r in range(B)]
+        levels = [([root], [0, B]), (own, list(range(B + 1)))]
+        ws = torch.empty(b.typhoon_mla_tree_workspace_bytes(levels, B, 0, pc.page_size), dtype=torch.uint8, device=dev)
+        sets.append(dict(levels=levels, ws=ws, out=torch.empty(B, H, 128, dtype=torch.bfloat16, device=dev)))
+
+    def step(i):
+        s = sets[i % 2]
+        b.typhoon_mla_decode_tree(s["levels"], q_nope, q_pe, None, None, pc.page_size, None, None, inp.scale, s["out"], s["ws"])
+
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    launches = b.typhoon_mla_last_launch_count()
+    # same result as the hybrid step (both are the same attention)
+    dec = TyphoonMLADecoder(H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), w_uk, w_uv, inp.scale, B, pc.block_table.shape[1])
+    ref = dec.decode(q_nope, q_pe, pc.ckv_pages.to(dev), pc.kpe_pages.to(dev), pc.block_table.to(dev), pc.seq_lens.to(dev),
+                     mode=b.MODE_HYBRID).float()
+    max_diff = float((sets[0]["out"].float() - ref).abs().max())
+    dec.close()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(device_index) as clocks:
+        ev0.record()
+        for i in range(K):
+            step(i)
+        ev1.record()
+        torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / K
+    sum_ln = sum(inp.suffix_lens)
+    bytes_naive = (512 * H + 128) * (cfg.Ls + sum_ln) + 640 * H * B     # every cached token's expanded K/V read once
+    return {"metric": METRIC, "value": B / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"{_workload_name(cfg)}, naive formulation on prefix and suffixes (one launch per request)",
+                       "entry_point": "typhoon_mla_decode_tree", "l2": "2 full input sets used alternately"},
+            "clocks": clocks.summary(), "gpu_launches": launches * K,
+            "check": {"max_abs_diff_vs_hybrid_step": max_diff},
+            "work": {"expanded_cache_bytes_read": bytes_naive}}
+
+
 def bench_sharded(cfg, args, device_index, rank, world):
     """--shard seq:G / head:G: one rank's share of a step whose context is sharded over G GPUs, by sequence
     (slice of the prefix + the suffixes of the requests the rank owns -> fp32 partial, all-gather, combine of G
@@ -613,6 +675,7 @@ def main():
     ap.add_argument("--ref-heads", type=int, default=64, help="heads the CPU checker is timed on (scaled up)")
     ap.add_argument("--sq", type=int, default=1, help="extension: query tokens per request (rows = B * S_q)")
     ap.add_argument("--tree", default="", help="extension: G:L = G request groups with L more shared prefix tokens each")
+    ap.add_argument("--naive-suffix", action="store_true", help="extension: naive formulation on the suffixes too (Fig. 8's naive-only curves)")
     ap.add_argument("--shard", default="", help="extension: seq:G or head:G = one rank's share of a context sharded over G GPUs")
     ap.add_argument("--stages", action="store_true", help="also time every kernel of the step alone (implied by --sweep)")
     ap.add_argument("--no-cpu", action="store_true")
@@ -636,7 +699,14 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
     mode = {"auto": b.MODE_AUTO, "absorb": b.MODE_ABSORB, "hybrid": b.MODE_HYBRID, "naive": b.MODE_NAIVE}[args.mode]
 
-    if args.shard:
+    if args.naive_suffix:
+        if world > 1:
+            raise SystemExit("--naive-suffix is a single-GPU measurement")
+        cfg = I.CONFIGS[args.config]
+        if args.batch:
+            cfg = cfg.with_batch(args.batch)
+        print(json.dumps(bench_naive_everywhere(cfg, args, local)), flush=True)
+    elif args.shard:
         cfg = I.CONFIGS[args.config]
         if args.batch:
             cfg = cfg.with_batch(args.batch)
