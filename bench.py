@@ -339,6 +339,10 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     a_s = (a_ms / max(a_n, 1)) * 1e-3
     alone = (k_bytes / a_s / 1e9) if roof["bound"] == "hbm" else (k_flops / a_s / 1e12)
     roof.update({"kernel_ms_alone": a_s * 1e3, "achieved_alone": alone, "frac_alone": alone / roof["peak"]})
+    # second column: the same fractions against the data-sheet peaks (8 TB/s HBM3e, 2.25 PFLOP/s dense bf16)
+    nominal = 8000.0 if roof["bound"] == "hbm" else 2250.0
+    roof.update({"nominal_peak": nominal, "frac_of_nominal": roof["achieved"] / nominal,
+                 "frac_alone_of_nominal": alone / nominal})
 
     # ---- per-stage times (the layout of the paper's Fig. 4 / Fig. 8: stage 1 = naive shared attention, stage 2
     # = absorb attention, plus the projections and the merge), every kernel alone on the GPU: side stream
