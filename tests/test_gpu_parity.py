@@ -658,3 +658,21 @@ def test_absorb_only_one_or_two_requests(B):
     assert b.typhoon_mla_device_status(dec.shared) == 0
     G.assert_parity(o32.cpu().double().numpy(), ref, l32.cpu().double().numpy(), ref_lse, what=f"absorb-only fp32 B={B}")
     dec.close()
+
+
+def test_partial_step_without_suffixes():
+    """The fp32 partial of a rank that holds prefix tokens only (no page table): the stand-alone combine writes it."""
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    cfg = _cfg("partial_naive", B=70, H=16, Ls=900, lo=0, hi=0, seed=91)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp, drop_suffix=True)
+    dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda(), inp.scale,
+                            cfg.B, 0)
+    o32 = torch.empty(cfg.B, cfg.H, 128, dtype=torch.float32, device="cuda")
+    l32 = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
+    b.typhoon_mla_decode_partial(dec.shared, inp.q_nope.cuda(), inp.q_pe.cuda(), None, None, cfg.page_size, None, None,
+                                 inp.scale, o32, l32, dec.workspace, mode=NAIVE)
+    assert b.typhoon_mla_device_status(dec.shared) == 0
+    G.assert_parity(o32.cpu().double().numpy(), ref, l32.cpu().double().numpy(), ref_lse, what="fp32 partial, prefix only")
+    dec.close()
