@@ -644,8 +644,9 @@ int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 // may run in several waves); ns minimises waves x (tiles per CTA + a fixed cost of about six tile
 // times for the Q load and the pipeline fill).  "Stream-K" uses R = SMs / row groups resident
 // CTAs and gives every SM the same number of tiles at the price of a few more segments (each
-// pays the fixed cost and a partial slot).  Stream-K is taken when its modelled cost is
-// lower (by at least 5% in the HBM-bound regime of 64-token tiles).
+// pays the fixed cost and a partial slot; with 64-token tiles a further slot per head is also charged
+// the extra read it causes in the combine).  Stream-K is taken when its modelled cost is lower (by at
+// least 5% in the HBM-bound regime of 64-token tiles).
 void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots) {
     const bool mode_y = B <= 128;
     const int tok = mode_y ? 64 : 128;
@@ -657,16 +658,30 @@ void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_r
         *n_slots = 0;
         return;
     }
+    // partial slots a head needs when the T tiles are cut into R ranges (ranges [0, rem) hold per + 1 tiles)
+    auto slots_for = [&](long long R) {
+        const long long per = T / R, rem = T % R, big = rem * (per + 1);
+        auto range_of = [&](long long t) { return t < big ? t / (per + 1) : rem + (t - big) / per; };
+        int seg_max = 1;
+        for (long long h = 0; h < H; ++h) {
+            const long long first = h * n_tiles, last = first + n_tiles - 1;
+            seg_max = std::max(seg_max, (int)(range_of(last) - range_of(first)) + 1);
+        }
+        return seg_max;
+    };
     // column split
     const long long base = (long long)H * m_groups;
     const double fixed = 6.0;
+    // every further partial slot is one more dependent read of B x H x 128 floats in the combine that follows
+    // (about 5 us, i.e. 8 tile times, measured with 64-token tiles; not significant next to 128-token tiles)
+    const double slot_cost = mode_y ? 8.0 : 0.0;
     int ns_best = 1;
     double cost_best = 1e30, eff_best = 0.0;
     for (int ns = 1; ns <= std::min(n_tiles, 32); ++ns) {
         const int per = (n_tiles + ns - 1) / ns;
         if (n_tiles % ns != 0) continue;   // equal parts only: every range stays inside one head
         const long long waves = (ns * base + n_sm - 1) / n_sm;
-        const double cost = (double)waves * (per + fixed);
+        const double cost = (double)waves * (per + fixed) + slot_cost * (ns - 1);
         if (cost < cost_best - 1e-9) {
             cost_best = cost;
             ns_best = ns;
@@ -678,7 +693,7 @@ void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_r
     const long long per_stream = (T + r_stream - 1) / r_stream;
     const long long waves_stream = ((long long)r_stream * m_groups + n_sm - 1) / n_sm;
     const double segs_stream = (per_stream >= n_tiles) ? (double)per_stream / n_tiles + 1.0 : 2.0;
-    const double cost_stream = (double)waves_stream * (per_stream + segs_stream * fixed);
+    const double cost_stream = (double)waves_stream * (per_stream + segs_stream * fixed) + slot_cost * (slots_for(r_stream) - 1);
     bool stream_k;
     if (schedule == 1) stream_k = false;
     else if (schedule == 2) stream_k = true;
@@ -691,16 +706,8 @@ void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_r
         stream_k = !hbm_bound_small && cost_stream < (mode_y ? 0.95 : 1.0) * cost_best;
     }
     const int R = stream_k ? r_stream : H * ns_best;
-    // ranges [0, rem) hold per + 1 tiles, the others per (the kernel uses the same partition)
-    const long long per = T / R, rem = T % R, big = rem * (per + 1);
-    auto range_of = [&](long long t) { return t < big ? t / (per + 1) : rem + (t - big) / per; };
-    int seg_max = 1;
-    for (long long h = 0; h < H; ++h) {
-        const long long first = h * n_tiles, last = first + n_tiles - 1;
-        seg_max = std::max(seg_max, (int)(range_of(last) - range_of(first)) + 1);
-    }
     *n_ranges = R;
-    *n_slots = seg_max;
+    *n_slots = slots_for(R);   // the kernel uses the same partition
 }
 
 cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
