@@ -149,6 +149,12 @@ def test_naive_plan_invariants(b):
     assert b.typhoon_mla_naive_plan(128, 64, 4096)[1:] == (128, 1, 1)
     assert b.typhoon_mla_naive_plan(128, 128, 26624)[1] == 148
     assert b.typhoon_mla_naive_plan(128, 512, 16384)[1:3] == (74, 2)
+    # every further partial slot is charged with 64-token tiles: shapes where equal ranges over all heads would
+    # need three or more slots per head keep one or two ranges per head (measured to be the faster choice)
+    assert b.typhoon_mla_naive_plan(128, 128, 16384)[1:] == (128, 1, 1)
+    assert b.typhoon_mla_naive_plan(64, 128, 8192)[1:] == (128, 1, 2)
+    assert b.typhoon_mla_naive_plan(16, 128, 8192)[1:] == (64, 1, 4)
+    assert b.typhoon_mla_naive_plan(64, 70, 20000)[1] == 148        # ... unless the column split wastes too much
     for bad in ((8, 1, 10, 0), (128, 0, 10, 0), (128, 1, 0, 0), (128, 1, 10, 3)):
         with pytest.raises(Exception):
             b.typhoon_mla_naive_plan(*bad)
