@@ -676,3 +676,106 @@ def test_partial_step_without_suffixes():
     assert b.typhoon_mla_device_status(dec.shared) == 0
     G.assert_parity(o32.cpu().double().numpy(), ref, l32.cpu().double().numpy(), ref_lse, what="fp32 partial, prefix only")
     dec.close()
+
+
+def test_random_trees_against_per_group_steps(kernel_path):
+    """Seeded random two-level trees (a root for all requests, branches for consecutive groups, some groups
+    without a branch, some trees without a root): every group's rows equal an ordinary step of that group over
+    the concatenation of root and branch (two runs of the library that share no launch plan)."""
+    if kernel_path == "warp_mma":
+        pytest.skip("row ranges need the tcgen05 kernel")
+    import random
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    rng = random.Random(11)
+    dev = "cuda"
+    for it in range(24):
+        H = rng.choice([16, 64, 128])
+        B = rng.choice([2, 5, 16, 40, 64, 100, 130, 260])
+        Ls = rng.choice([0, 64, 300, 1000, 3000])
+        hi = rng.choice([0, 50, 400])
+        n_groups = min(rng.choice([1, 2, 3, 5]), B)
+        cfg = _cfg("rtree", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=500 + it)
+        inp = I.make_inputs(cfg)
+        pc = I.build_pages(inp, poison=True)
+        gb = [0] + sorted(rng.sample(range(1, B), n_groups - 1)) + [B]
+        branch_len = [rng.choice([0, 1, 70, 500, 1500]) for _ in range(n_groups)]
+        gen = torch.Generator().manual_seed(it)
+        br_ckv = [torch.randn(n, 512, generator=gen).to(torch.bfloat16) for n in branch_len]
+        br_kpe = [torch.randn(n, 64, generator=gen).to(torch.bfloat16) for n in branch_len]
+        dims = b.make_dims(H)
+        w_uk, w_uv = inp.w_uk.to(dev), inp.w_uv.to(dev)
+        root = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), w_uk, w_uv) if Ls > 0 else None
+        brs = [b.typhoon_mla_prepare_shared(dims, c.to(dev), k.to(dev), w_uk, w_uv) if c.shape[0] > 0 else None
+               for c, k in zip(br_ckv, br_kpe)]
+        levels = ([([root], [0, B])] if root is not None else []) + ([(brs, gb)] if any(x is not None for x in brs) else [])
+        if not levels:
+            continue
+        args = _upload(inp, pc)
+        out = torch.empty(B, H, 128, dtype=torch.bfloat16, device=dev)
+        ws = torch.empty(b.typhoon_mla_tree_workspace_bytes(levels, B, pc.block_table.shape[1], 64), dtype=torch.uint8, device=dev)
+        b.typhoon_mla_decode_tree(levels, args[0], args[1], args[2], args[3], 64, args[4], args[5], inp.scale, out, ws)
+        handles = ([root] if root is not None else []) + [x for x in brs if x is not None]
+        assert b.typhoon_mla_device_status(handles[0]) == 0
+        for gi in range(n_groups):
+            r0, r1 = gb[gi], gb[gi + 1]
+            dec = TyphoonMLADecoder(H, torch.cat([inp.ckv_shared, br_ckv[gi]]).to(dev), torch.cat([inp.kpe_shared, br_kpe[gi]]).to(dev),
+                                    w_uk, w_uv, inp.scale, r1 - r0, pc.block_table.shape[1])
+            ref = dec.decode(args[0][r0:r1].contiguous(), args[1][r0:r1].contiguous(), args[2], args[3],
+                             args[4][r0:r1].contiguous(), args[5][r0:r1].contiguous(), mode=AUTO).float()
+            dec.close()
+            o = out[r0:r1].float()
+            assert torch.isfinite(o).all()
+            err = float((o - ref).abs().max()) / max(1.0, float(ref.abs().max()))
+            assert err < 2e-2, (it, gi, dict(H=H, B=B, Ls=Ls, hi=hi, groups=gb, branch=branch_len), err)
+        for x in handles:
+            x.free()
+
+
+def test_random_shards_against_the_whole_step():
+    """Seeded random sequence shardings (2 to 5 ranks, prefixes shorter than one block per rank included, ranks in
+    different modes) and two-way head shardings: merged partials equal the single-device step."""
+    import random
+    from paper_2509_21081_b200 import binding as b, sharded as S
+    from paper_2509_21081_b200.decoder import TyphoonMLADecoder
+    rng = random.Random(12)
+    dev = "cuda"
+    for it in range(30):
+        B = rng.choice([1, 2, 3, 7, 16, 33, 64, 65, 130, 200])
+        H = rng.choice([16, 32, 64, 128])
+        Ls = rng.choice([0, 1, 63, 64, 65, 200, 513, 1500, 4000])
+        hi = rng.choice([0, 1, 70, 300, 900])
+        world = rng.choice([2, 3, 4, 5])
+        if Ls == 0 and hi == 0:
+            continue
+        cfg = _cfg("rshard", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=1000 + it)
+        inp = I.make_inputs(cfg)
+        pc = I.build_pages(inp, poison=True)
+        args = _upload(inp, pc)
+        dev_in = (inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev), inp.w_uv.to(dev))
+        dec = TyphoonMLADecoder(H, *dev_in, inp.scale, B, pc.block_table.shape[1])
+        lse_ref = torch.empty(B, H, device=dev)
+        ref = dec.decode(*args, mode=AUTO, lse_out=lse_ref).float()
+        dec.close()
+        parts = []
+        for r in range(world):
+            d = S.SequenceShardedDecoder(r, world, H, *dev_in, inp.scale, B, pc.block_table.shape[1])
+            parts.append(d.partial(*args, mode=rng.choice([AUTO, HYBRID, ABSORB])))
+            assert b.typhoon_mla_device_status(d.shared) == 0
+            d.close()
+        lse = torch.empty(B, H, device=dev)
+        out = S.merge_partials(torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]), lse).float()
+        scale = max(1.0, float(ref.abs().max()))
+        fin = torch.isfinite(lse_ref)
+        assert torch.isfinite(out).all() and torch.equal(torch.isfinite(lse), fin)
+        assert float((out - ref).abs().max()) / scale < 2e-2, (it, dict(B=B, H=H, Ls=Ls, hi=hi, world=world))
+        if fin.any():
+            assert float((lse[fin] - lse_ref[fin]).abs().max()) < 2e-2
+        if H % 32 == 0:
+            halves = []
+            for r in range(2):
+                d = S.HeadShardedDecoder(r, 2, H, *dev_in, inp.scale, B, pc.block_table.shape[1])
+                halves.append(d.local(*args, mode=AUTO))
+                d.close()
+            o2 = S.join_heads(torch.stack(halves)).float()
+            assert float((o2 - ref).abs().max()) / scale < 2e-2, (it, "heads")
