@@ -368,11 +368,11 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     # ---- end to end: per-step tensors from pinned host memory, result read back, every step
     e2e = None
     if with_e2e:
-        # Four steps are kept in flight ("lanes"), each on its own stream with its own decoder (prepared
+        # Eight steps are kept in flight ("lanes"), each on its own stream with its own decoder (prepared
         # prefix, workspace, staging) and pinned buffers, so that the copies of one step overlap the kernels
         # of the others, as a serving loop with several micro-batches would do.  Every step still copies
         # its inputs in and its result out.  Lane k reads the device-resident caches of input set k % 2.
-        n_lanes = int(os.environ.get("TYPHOON_MLA_BENCH_LANES", "4"))
+        n_lanes = int(os.environ.get("TYPHOON_MLA_BENCH_LANES", "8"))
         lanes = []
         for k in range(n_lanes):
             s = sets[k % n_sets]
@@ -403,19 +403,25 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         for i in range(W):
             step_host(i)
         join()
-        barrier()
-        ev0.record()
-        fork()
-        for i in range(K):
-            step_host(i)
-        join()
-        ev1.record()
-        barrier()
-        e_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / K
+        # the region is short (K steps of ~0.1 ms) and sensitive to a hiccup of the launching thread: it is
+        # timed three times and the median is reported
+        e_runs = []
+        for _ in range(3):
+            barrier()
+            ev0.record()
+            fork()
+            for i in range(K):
+                step_host(i)
+            join()
+            ev1.record()
+            barrier()
+            e_runs.append(max_over_ranks(ev0.elapsed_time(ev1), world, dev) / K)
+        e_ms = sorted(e_runs)[1]
         h2d = inp.q_nope.numel() * 2 + inp.q_pe.numel() * 2 + pc.block_table.numel() * 4 + pc.seq_lens.numel() * 4
         d2h = cfg.B * cfg.H * 128 * 2
         e2e = {"value": whole_job_value(cfg.B, world, e_ms), "unit": UNIT, "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "runs_ms_per_step": e_runs,
                "pipelining": f"{n_lanes} steps in flight on {n_lanes} streams (own decoder, workspace, staging and pinned buffers each)"}
 
     cpu = None
