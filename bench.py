@@ -29,13 +29,15 @@ if ROOT not in sys.path:
 METRIC = "mla_decode_attention_queries_per_s"
 UNIT = "queries/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (key: (config, kernel)); None where no capture exists.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture
+# of that kernel at that configuration (key: (config, kernel)); None where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("cfg1", "naive_attn"): 275_993_856,     # profiles/naive_attn_sm100_cfg1_and_cfg4_b512.md
-    ("cfg3", "absorb_attn"): 652_079_360,    # profiles/absorb_attn_sm100_cfg3.md
+    ("cfg1", "naive_attn"): 275_993_856,
+    ("cfg3", "absorb_attn"): 652_079_360,
     ("cfg4_B512", "naive_attn"): 1_159_151_640,
 }
+MIN_REGION_MS = 50.0      # every timed region is repeated until this much GPU time has been measured
+MAX_REPEATS = 400
 
 
 def _peaks():
@@ -159,6 +161,7 @@ class ClockSampler:
     def summary(self):
         idle = {"GpuIdle", "None", "ApplicationsClocksSetting"}
         return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
+                "sm_min_mhz": (min(self.samples) if self.samples else None),
                 "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
                 "reasons": sorted(r for r in self.reasons if r not in idle)}
 
@@ -222,7 +225,11 @@ def _workload_name(cfg):
             f"page={cfg.page_size} d=(128,64,128,512) bf16")
 
 
-def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with_e2e=True):
+def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with_e2e=True, max_steps=None):
+    """One configuration: K steps per timed region, the region repeated until MIN_REGION_MS of GPU time
+    has been measured (median of the repeats reported; the clock sampler runs over all of them), then
+    the dominant kernel's duration inside the step and alone, optionally per-stage times, the end-to-end
+    figures and the CPU checker."""
     import torch
     from paper_2509_21081_b200 import binding as b
     from paper_2509_21081_b200 import inputs as I
@@ -266,42 +273,55 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         torch.cuda.synchronize()
 
     W, K = max(args.warmup, 3), max(args.steps, 1)
+    if max_steps:
+        K = min(K, max_steps)
     for i in range(W):
         step(i)
     torch.cuda.synchronize()
     launches_per_step = b.typhoon_mla_last_launch_count()
+    assert b.typhoon_mla_check_status(sets[0]["dec"].shared) == 0 and b.typhoon_mla_check_status(sets[1]["dec"].shared) == 0
     kid, kname, k_bytes, k_flops = dominant_kernel(cfg, inp.suffix_lens, mode_name)
 
-    # ---- device-resident timing: K steps, nothing else on the stream
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    with ClockSampler(device_index) as clocks:
+
+    def region(fn, n):
+        """n calls of fn bracketed by a barrier + synchronize on both sides; device time in ms (max over ranks)."""
+        barrier()
         ev0.record()
-        for i in range(K):
-            step(i)
+        for i in range(n):
+            fn(i)
         ev1.record()
         barrier()
-    total_ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
-    ms_per_step = total_ms / K
+        return max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+
+    def repeated(fn, n):
+        """Repeats the n-call region until MIN_REGION_MS of device time has been measured (at least 3
+        times); returns the per-call times of the repeats."""
+        runs, total = [], 0.0
+        while (total < MIN_REGION_MS or len(runs) < 3) and len(runs) < MAX_REPEATS:
+            ms = region(fn, n)
+            runs.append(ms / n)
+            total += ms
+        return runs
+
+    # ---- device-resident timing: regions of exactly K steps, nothing else on the stream
+    with ClockSampler(device_index) as clocks:
+        step_runs = repeated(step, K)
+    ms_per_step = statistics.median(step_runs)
     value = whole_job_value(cfg.B, world, ms_per_step)
 
-    # ---- the same K steps again with a pair of CUDA events around every launch of the dominant kernel
+    # ---- the same steps again with a pair of CUDA events around every launch of the dominant kernel
     # (on the stream it is launched on).  Event records cost several microseconds per step and, with
     # programmatic launches, change the order in which the two streams' kernels get their SMs (an event in
     # front of a kernel delays it behind the side stream's kernels), so this second timed region runs with
     # ordinary stream-ordered launches and is only used for the kernel's duration inside a step; its own
     # step time is reported next to it.
+    n_prof = int(min(2000, max(K, MIN_REGION_MS / max(ms_per_step, 1e-3))))
     b.typhoon_mla_set_programmatic_launch(False)
     for i in range(3):
         step(i)
-    b.typhoon_mla_profile_begin(kid, K)
-    barrier()
-    ev0.record()
-    for i in range(K):
-        step(i)
-    ev1.record()
-    barrier()
-    instrumented_ms_per_step = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / K
+    b.typhoon_mla_profile_begin(kid, n_prof)
+    instrumented_ms_per_step = region(step, n_prof) / n_prof
     k_ms, k_n = b.typhoon_mla_profile_end()
     b.typhoon_mla_set_programmatic_launch(True)
 
@@ -315,9 +335,12 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         roof = {"bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / pk["hbm_gbs"]}
     else:
+        # timed inside a long loop under the power cap: the sustained figure is the denominator; the
+        # fraction of the burst figure is printed next to it
         achieved = k_flops / k_avg_s / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                "frac": achieved / pk["bf16_tflops_sustained"]}
+                "frac": achieved / pk["bf16_tflops_sustained"], "frac_of_burst_peak": achieved / pk["bf16_tflops"],
+                "burst_peak": pk["bf16_tflops"]}
     roof.update({"traffic": NCU_TRAFFIC_BYTES.get((cfg.name, kname)), "kernel": kname,
                  "kernel_ms": k_avg_s * 1e3, "launches_timed": k_n,
                  "ms_per_step_with_kernel_events": instrumented_ms_per_step, "peak_source": pk["source"],
@@ -328,7 +351,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     # The same kernel with the side stream switched off (every kernel alone on the GPU), outside the
     # timed region: what the kernel reaches when it does not share the machine.
     b.typhoon_mla_set_overlap(False)
-    n_alone = max(5, min(K, 50))
+    n_alone = int(min(2000, max(5, min(K, 50), 0.5 * MIN_REGION_MS / max(ms_per_step, 1e-3))))
     for i in range(3):
         step(i)
     b.typhoon_mla_profile_begin(kid, n_alone)
@@ -339,6 +362,8 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     a_s = (a_ms / max(a_n, 1)) * 1e-3
     alone = (k_bytes / a_s / 1e9) if roof["bound"] == "hbm" else (k_flops / a_s / 1e12)
     roof.update({"kernel_ms_alone": a_s * 1e3, "achieved_alone": alone, "frac_alone": alone / roof["peak"]})
+    if roof["bound"] == "tensor":
+        roof["frac_alone_of_burst_peak"] = alone / pk["bf16_tflops"]
     # second column: the same fractions against the data-sheet peaks (8 TB/s HBM3e, 2.25 PFLOP/s dense bf16)
     nominal = 8000.0 if roof["bound"] == "hbm" else 2250.0
     roof.update({"nominal_peak": nominal, "frac_of_nominal": roof["achieved"] / nominal,
@@ -403,10 +428,10 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         for i in range(W):
             step_host(i)
         join()
-        # the region is short (K steps of ~0.1 ms) and sensitive to a hiccup of the launching thread: it is
-        # timed three times and the median is reported
-        e_runs = []
-        for _ in range(3):
+        # regions of K steps (fork, K host-fed steps round robin over the lanes, join), repeated like the
+        # device-resident regions; the median is reported
+        e_runs, total = [], 0.0
+        while (total < MIN_REGION_MS or len(e_runs) < 3) and len(e_runs) < MAX_REPEATS:
             barrier()
             ev0.record()
             fork()
@@ -415,14 +440,35 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
             join()
             ev1.record()
             barrier()
-            e_runs.append(max_over_ranks(ev0.elapsed_time(ev1), world, dev) / K)
-        e_ms = sorted(e_runs)[1]
+            ms = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
+            e_runs.append(ms / K)
+            total += ms
+        e_ms = statistics.median(e_runs)
+        # One step in flight, as a decode loop sees it: copy in, step, copy out, wait for the result, then the
+        # next step (lane 0 and lane 1 alternately so that L2 does not hold the previous step's cache lines).
+        # Host clock around the loop: the launch path and the wake-up after the synchronise are part of it.
+        n_lat = int(min(2000, max(K, MIN_REGION_MS / max(e_ms, 1e-3))))
+        for i in range(3):
+            step_host(i % 2)
+            lanes[i % 2]["stream"].synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(n_lat):
+            step_host(i % 2)
+            lanes[i % 2]["stream"].synchronize()
+        lat_ms = (time.perf_counter() - t0) * 1e3 / n_lat
+        lat_ms = max_over_ranks(lat_ms, world, dev)
         h2d = inp.q_nope.numel() * 2 + inp.q_pe.numel() * 2 + pc.block_table.numel() * 4 + pc.seq_lens.numel() * 4
         d2h = cfg.B * cfg.H * 128 * 2
         e2e = {"value": whole_job_value(cfg.B, world, e_ms), "unit": UNIT, "ms_per_step": e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "runs_ms_per_step": e_runs,
-               "pipelining": f"{n_lanes} steps in flight on {n_lanes} streams (own decoder, workspace, staging and pinned buffers each)"}
+               "repeats": len(e_runs), "min_ms_per_step": min(e_runs), "max_ms_per_step": max(e_runs),
+               "pipelining": f"{n_lanes} steps in flight on {n_lanes} streams (own decoder, workspace, staging and pinned buffers each)",
+               "e2e_latency_ms": lat_ms, "e2e_latency_steps": n_lat,
+               "e2e_latency_value": whole_job_value(cfg.B, world, lat_ms),
+               "e2e_latency_note": "one step in flight: pinned host inputs copied in, step, result copied out, stream synchronised, host clock"}
+        for ln in lanes[n_sets:]:
+            ln["dec"].close()
 
     cpu = None
     if with_cpu and rank == 0 and world == 1:
@@ -437,11 +483,46 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": _workload_name(cfg), "mode": mode_name, "requested_mode": b.MODE_NAMES[mode],
                        "parallelism": f"replicas x{world} (shard by request, no exchange)",
-                       "l2": f"{n_sets} full input sets used alternately, each larger than the 126 MB L2"},
+                       "l2": f"{n_sets} full input sets used alternately, each larger than the 126 MB L2",
+                       "timing": f"regions of {K} steps repeated until {MIN_REGION_MS:g} ms of device time; median of the repeats"},
+            "timed_regions": {"repeats": len(step_runs), "min_ms_per_step": min(step_runs), "max_ms_per_step": max(step_runs)},
             "clocks": clocks.summary(), "e2e": e2e, "stages": stages, "gpu_launches": launches_per_step * K,
             "prepare_shared_ms": prepare_ms,
             "roofline": roof, "cpu_baseline": cpu}
     return line
+
+
+# Configurations reported next to the headline one in the default run: the other benchmark configurations,
+# the fan-out sweep at the batch sizes on either side of the crossover and in the compute-bound regime.
+EXTRA_CONFIGS = (("cfg2", 0), ("cfg3", 0), ("cfg4", 8), ("cfg4", 128), ("cfg4", 512), ("cfg4", 1024))
+
+
+def bench_extra_configs(args, rank, world, device_index):
+    """Short lines for the other benchmark configurations (mode AUTO, same timing method, at most 20 steps per
+    region): step time, resolved mode, the dominant kernel and its roofline fractions inside the step and
+    alone, the sampled clocks."""
+    import gc
+    import torch
+    from paper_2509_21081_b200 import binding as b
+    from paper_2509_21081_b200 import inputs as I
+    out = []
+    for name, batch in EXTRA_CONFIGS:
+        cfg = I.CONFIGS[name]
+        if batch:
+            cfg = cfg.with_batch(batch)
+        ln = bench_config(cfg, args, b.MODE_AUTO, rank, world, device_index, with_cpu=False, with_e2e=False, max_steps=20)
+        r = ln["roofline"]
+        out.append({"workload": ln["config"]["workload"], "mode": ln["config"]["mode"], "value": ln["value"],
+                    "ms_per_step": ln["ms_per_step"], "steps": ln["steps"], "timed_regions": ln["timed_regions"],
+                    "gpu_launches": ln["gpu_launches"], "dominant_kernel": r["kernel"], "bound": r["bound"],
+                    "peak": r["peak"], "unit": r["unit"], "achieved": r["achieved"], "frac": r["frac"],
+                    "achieved_alone": r["achieved_alone"], "frac_alone": r["frac_alone"],
+                    "frac_of_burst_peak": r.get("frac_of_burst_peak"), "frac_alone_of_burst_peak": r.get("frac_alone_of_burst_peak"),
+                    "frac_of_nominal": r["frac_of_nominal"], "kernel_ms": r["kernel_ms"], "kernel_ms_alone": r["kernel_ms_alone"],
+                    "step_frac_of_combined_roofline": r["step_frac_of_combined_roofline"], "clocks": ln["clocks"]})
+        gc.collect()
+        torch.cuda.empty_cache()
+    return out
 
 
 def bench_extension(cfg, args, device_index):
@@ -690,6 +771,7 @@ def main():
     ap.add_argument("--stages", action="store_true", help="also time every kernel of the step alone (implied by --sweep)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="headline configuration only (skip the other configurations' short lines)")
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -744,6 +826,8 @@ def main():
             cfg = cfg.with_batch(args.batch)
         line = bench_config(cfg, args, mode, rank, world, local, with_cpu=not args.no_cpu,
                             with_e2e=not args.no_e2e)
+        if args.config == "cfg1" and not args.batch and args.mode == "auto" and not args.no_extra:
+            line["extra_configs"] = bench_extra_configs(args, rank, world, local)
         if rank == 0:
             print(json.dumps(line), flush=True)
     if world > 1:

@@ -109,10 +109,13 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims /* host */,
  * NULL is accepted. */
 int typhoon_mla_free(typhoon_mla_shared_t* shared);
 
-/* Bytes of scratch typhoon_mla_decode needs for this problem size in the worst
- * case over modes (host, pure).  Returns 0 on invalid arguments. */
+/* Bytes of scratch typhoon_mla_decode needs for this problem size in `mode`
+ * (TYPHOON_MLA_MODE_AUTO: the worst case over the modes AUTO may resolve to, so the
+ * same workspace serves every step whatever the crossover rule picks).  Host, pure:
+ * it reads the handle and touches no process-wide state, so it may be called from
+ * any thread at any time.  Returns 0 on invalid arguments. */
 size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* shared, int32_t B,
-                                   int32_t max_pages, int32_t page_size);
+                                   int32_t max_pages, int32_t page_size, int32_t mode);
 
 /*
  * One decode-attention step for B requests (Algorithm 1).
@@ -124,6 +127,14 @@ size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* shared, int32_t B
  *   kpe_pages    bf16 rope keys, same addressing with kpe_token_stride, 64 wide
  *                (strides in elements, multiples of 8; a fused 576-wide page
  *                layout can be passed by pointing both into it)
+ *   num_pages    number of physical pages in ckv_pages / kpe_pages (>= 1 when
+ *                max_pages > 0).  It bounds every read of the paged cache: a
+ *                block-table entry inside a request's length that is negative
+ *                or >= num_pages is never dereferenced -- its tokens read as
+ *                zeros -- and sets bit TYPHOON_MLA_STATUS_BAD_PAGE of the
+ *                handle's status word (typhoon_mla_check_status); the output
+ *                rows of that request are then meaningless, the call does not
+ *                fault.
  *   block_table  int32 [B, max_pages]: physical page of each logical page;
  *                entries at or beyond ceil(seq_lens[b] / page_size) are ignored
  *   seq_lens     int32 [B]: suffix length of each request, may be 0; values
@@ -152,7 +163,8 @@ int typhoon_mla_decode(const typhoon_mla_shared_t* shared,
                        const void* q_nope, const void* q_pe, int32_t B,
                        const void* ckv_pages, const void* kpe_pages,
                        int64_t ckv_token_stride, int64_t kpe_token_stride,
-                       int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                       int32_t page_size, int32_t num_pages,
+                       const int32_t* block_table, int32_t max_pages,
                        const int32_t* seq_lens,
                        float softmax_scale, int32_t mode,
                        void* out, float* lse_out,
@@ -185,7 +197,8 @@ int typhoon_mla_decode_partial(const typhoon_mla_shared_t* shared,
                                const void* q_nope, const void* q_pe, int32_t B,
                                const void* ckv_pages, const void* kpe_pages,
                                int64_t ckv_token_stride, int64_t kpe_token_stride,
-                               int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                               int32_t page_size, int32_t num_pages,
+                               const int32_t* block_table, int32_t max_pages,
                                const int32_t* seq_lens,
                                float softmax_scale, int32_t mode,
                                float* out_partial, float* lse_partial,
@@ -208,7 +221,8 @@ int typhoon_mla_decode_host(const typhoon_mla_shared_t* shared,
                             const void* q_nope_host, const void* q_pe_host, int32_t B,
                             const void* ckv_pages, const void* kpe_pages,
                             int64_t ckv_token_stride, int64_t kpe_token_stride,
-                            int32_t page_size, const int32_t* block_table_host, int32_t max_pages,
+                            int32_t page_size, int32_t num_pages,
+                            const int32_t* block_table_host, int32_t max_pages,
                             const int32_t* seq_lens_host,
                             float softmax_scale, int32_t mode,
                             void* out_host,
@@ -277,7 +291,8 @@ int typhoon_mla_decode_tree(const typhoon_mla_prefix_level_t* levels /* host */,
                             const void* q_nope, const void* q_pe, int32_t B,
                             const void* ckv_pages, const void* kpe_pages,
                             int64_t ckv_token_stride, int64_t kpe_token_stride,
-                            int32_t page_size, const int32_t* block_table, int32_t max_pages,
+                            int32_t page_size, int32_t num_pages,
+                            const int32_t* block_table, int32_t max_pages,
                             const int32_t* seq_lens, float softmax_scale,
                             void* out, float* lse_out,
                             void* workspace, size_t workspace_bytes, void* stream);
@@ -295,53 +310,21 @@ int typhoon_mla_expand_query_rows(const int32_t* block_table, const int32_t* seq
                                   int32_t max_pages, int32_t S_q, int32_t* block_table_rows,
                                   int32_t* seq_lens_rows, void* stream);
 
-/* Work decomposition the tcgen05 shared-prefix kernel (Algorithm 1 line 4) would use for a problem
- * size: tokens per KV tile (64 for B <= 128, else 128), number of contiguous tile ranges the H * n_tiles
- * tiles are cut into, query-row groups per range (CTAs = ranges * row_groups) and partial slots written
- * per (request, head).  schedule: 0 = the library's choice, 1 = every range inside one head ("column
- * split"), 2 = ranges of equal size over all heads ("stream-K").  Host, pure (a function of the sizes
- * only, so the decomposition and with it the summation order are reproducible).  INVALID_ARG for
- * B < 1, L_s < 1, unsupported H or schedule outside 0..2; no output is written then. */
-int typhoon_mla_naive_plan(int32_t num_heads, int32_t B, int64_t L_s, int32_t schedule,
-                           int32_t* tile_tokens /* host */, int32_t* n_ranges /* host */,
-                           int32_t* row_groups /* host */, int32_t* n_slots /* host */);
-
-/* Read-only views of what the handle owns (for tests and accounting):
- * k_nope bf16 [H, Ls_padded/64, 2, 64, 64]; v_t bf16 [H, Ls_padded/64, 128, 64]. */
-int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
-                            const void** k_nope, const void** v_t,
-                            int64_t* Ls /* host */, int64_t* Ls_padded /* host */,
-                            int64_t* owned_bytes /* host */);
-
-/* Which implementation of the tensor-core kernels runs: the tcgen05/TMEM/TMA kernels (default) or
- * the warp-MMA kernels.  Process-wide; affects later prepare_shared and decode calls. */
-enum { TYPHOON_MLA_PATH_TCGEN05 = 0, TYPHOON_MLA_PATH_WARP_MMA = 1 };
-int typhoon_mla_set_kernel_path(int32_t path);
-
-/* In a hybrid step the absorb branch (Algorithm 1 lines 5-6) runs on a stream owned by the handle,
- * beside the naive kernel (line 4), and is joined before the projection (default).  0 keeps every
- * kernel on the caller's stream, one after the other (measurement aid).  Process-wide. */
-int typhoon_mla_set_overlap(int32_t enable);
-
-/* The kernels of a step are launched with the programmatic-stream-serialization attribute (default):
- * a kernel may be scheduled while its predecessor in the stream is still running and waits, before its
- * first access to global memory, until that predecessor has completed.  This hides most of the launch
- * latency between the dependent kernels of a step.  0 gives ordinary stream-ordered launches
- * (measurement aid; TYPHOON_MLA_PDL=0 in the environment sets the initial value).  Process-wide. */
-int typhoon_mla_set_programmatic_launch(int32_t enable);
-
-/* Work decomposition of the tcgen05 shared-prefix kernel (see typhoon_mla_naive_plan): 0 = the
- * library's choice (default), 1 = column split, 2 = stream-K.  Measurement and test aid; process-wide. */
-int typhoon_mla_set_naive_schedule(int32_t schedule);
-
-/* Synchronises `stream` and reads the handle's device status word.  Every in-kernel wait of the
- * tcgen05 kernels has a deadline; if one expired, the kernel abandoned its work, the word is
- * non-zero and this returns TYPHOON_MLA_ERR_DEVICE_CHECK (results of that launch are invalid). */
-int typhoon_mla_device_status(const typhoon_mla_shared_t* shared, void* stream, int32_t* status /* host */);
-
-/* Copy the expanded caches into caller buffers of H * Ls_padded * 128 bf16
- * elements each (device memory), on `stream`. */
-int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_dst, void* v_t_dst, void* stream);
+/*
+ * Device-side checks.  The handle owns one status word in device memory, zero after
+ * typhoon_mla_prepare_shared.  Kernels never trap or assert; instead they OR a bit into the word:
+ *   TYPHOON_MLA_STATUS_WAIT_EXPIRED  a bounded in-kernel wait ran out (every wait on a copy or a tensor-core
+ *                                    completion has a deadline of about one second); the kernel abandoned its
+ *                                    work and the results of that launch are invalid
+ *   TYPHOON_MLA_STATUS_BAD_PAGE      a block-table entry inside a request's length was negative or >= num_pages;
+ *                                    it was not dereferenced (its tokens read as zeros)
+ * typhoon_mla_check_status synchronises `stream`, copies the word to *word (host, may be NULL), clears it on the
+ * device when `clear` is non-zero, and returns TYPHOON_MLA_ERR_DEVICE_CHECK if it was non-zero, else OK.  This is
+ * the library's stand-in for a memory checker on systems where none can be run; it is off the hot path (a decode
+ * call never reads the word back).  Bits 0-7 of the word name the kernel whose wait expired (diagnostic only).
+ */
+enum { TYPHOON_MLA_STATUS_WAIT_EXPIRED = 0xff, TYPHOON_MLA_STATUS_BAD_PAGE = 0x100 };
+int typhoon_mla_check_status(const typhoon_mla_shared_t* shared, void* stream, int32_t* word /* host */, int32_t clear);
 
 /*
  * Shared-prefix attention without any allocation (the paper has no counterpart:
@@ -373,35 +356,6 @@ int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_d
 int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* shared,
                                      const void* q_nope, const void* q_pe, int32_t B,
                                      float softmax_scale, void* out, float* lse_out, void* stream);
-
-/* Longest-first order used for ragged suffixes: perm[0..B) (device, int32) = request indices sorted
- * by descending seq_lens (device, int32), ties by ascending index.  B <= 4096.  Exposed for tests. */
-int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* perm, void* stream);
-
-/* Kernel kinds of the decode step, in launch order (Algorithm 1 lines 4-8). */
-enum {
-    TYPHOON_MLA_KERNEL_NAIVE_ATTN = 0,  /* line 4 */
-    TYPHOON_MLA_KERNEL_Q_ABSORB = 1,    /* line 5 */
-    TYPHOON_MLA_KERNEL_ABSORB_ATTN = 2, /* line 6 */
-    TYPHOON_MLA_KERNEL_MERGE = 3,       /* merge of line 6's KV splits */
-    TYPHOON_MLA_KERNEL_W_UV = 4,        /* line 7 */
-    TYPHOON_MLA_KERNEL_COMBINE = 5,     /* line 8 */
-    TYPHOON_MLA_NUM_KERNELS = 6
-};
-
-/*
- * Measurement aid: between profile_begin and profile_end every decode call of
- * the process records a pair of CUDA events around the launch of the chosen
- * kernel kind, on the stream the kernel is launched on (up to max_launches
- * launches).  profile_end waits for the recorded events and returns the summed
- * device time in milliseconds and the number of launches timed.  Host, not
- * thread-safe; begin allocates events, decode itself still allocates nothing.
- */
-int typhoon_mla_profile_begin(int32_t kernel_id, int32_t max_launches);
-int typhoon_mla_profile_end(double* total_ms /* host */, int32_t* launches /* host */);
-
-/* Number of kernels the last typhoon_mla_decode call of this thread launched. */
-int typhoon_mla_last_launch_count(void);
 
 /* The cudaError_t (as int) behind the last TYPHOON_MLA_ERR_CUDA of this thread. */
 int typhoon_mla_last_cuda_error(void);

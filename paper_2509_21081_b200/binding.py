@@ -52,9 +52,9 @@ def _load():
     lib.typhoon_mla_free.restype = C.c_int
     lib.typhoon_mla_free.argtypes = [vp]
     lib.typhoon_mla_workspace_bytes.restype = sz
-    lib.typhoon_mla_workspace_bytes.argtypes = [vp, i32, i32, i32]
+    lib.typhoon_mla_workspace_bytes.argtypes = [vp, i32, i32, i32, i32]
     lib.typhoon_mla_decode.restype = C.c_int
-    lib.typhoon_mla_decode.argtypes = [vp, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, i32, vp, vp,
+    lib.typhoon_mla_decode.argtypes = [vp, vp, vp, i32, vp, vp, i64, i64, i32, i32, vp, i32, vp, f32, i32, vp, vp,
                                        vp, sz, vp]
     lib.typhoon_mla_tree_workspace_bytes.restype = sz
     lib.typhoon_mla_decode_partial.restype = C.c_int
@@ -63,12 +63,12 @@ def _load():
     lib.typhoon_mla_combine_partials.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     lib.typhoon_mla_tree_workspace_bytes.argtypes = [vp, i32, i32, i32, i32]
     lib.typhoon_mla_decode_tree.restype = C.c_int
-    lib.typhoon_mla_decode_tree.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, vp, vp,
+    lib.typhoon_mla_decode_tree.argtypes = [vp, i32, vp, vp, i32, vp, vp, i64, i64, i32, i32, vp, i32, vp, f32, vp, vp,
                                             vp, sz, vp]
     lib.typhoon_mla_host_staging_bytes.restype = sz
     lib.typhoon_mla_host_staging_bytes.argtypes = [vp, i32, i32]
     lib.typhoon_mla_decode_host.restype = C.c_int
-    lib.typhoon_mla_decode_host.argtypes = [vp, vp, vp, i32, vp, vp, i64, i64, i32, vp, i32, vp, f32, i32, vp,
+    lib.typhoon_mla_decode_host.argtypes = [vp, vp, vp, i32, vp, vp, i64, i64, i32, i32, vp, i32, vp, f32, i32, vp,
                                             vp, sz, vp, sz, vp]
     lib.typhoon_mla_choose_mode.restype = C.c_int
     lib.typhoon_mla_choose_mode.argtypes = [vp, i32, i64]
@@ -83,7 +83,7 @@ def _load():
     lib.typhoon_mla_cost_model.restype = C.c_int
     lib.typhoon_mla_cost_model.argtypes = [C.POINTER(Dims), i32, i64, i64, i64, i64, C.POINTER(i64), C.POINTER(i64)]
     lib.typhoon_mla_naive_plan.restype = C.c_int
-    lib.typhoon_mla_naive_plan.argtypes = [i32, i32, i64, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    lib.typhoon_mla_naive_plan.argtypes = [i32, i32, i64, i32, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
     lib.typhoon_mla_shared_view.restype = C.c_int
     lib.typhoon_mla_shared_view.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), C.POINTER(i64),
                                             C.POINTER(i64)]
@@ -101,8 +101,12 @@ def _load():
     lib.typhoon_mla_set_programmatic_launch.argtypes = [i32]
     lib.typhoon_mla_set_overlap.restype = C.c_int
     lib.typhoon_mla_set_overlap.argtypes = [i32]
-    lib.typhoon_mla_device_status.restype = C.c_int
-    lib.typhoon_mla_device_status.argtypes = [vp, vp, C.POINTER(i32)]
+    lib.typhoon_mla_check_status.restype = C.c_int
+    lib.typhoon_mla_check_status.argtypes = [vp, vp, C.POINTER(i32), i32]
+    lib.typhoon_mla_test_wait_expiry.restype = C.c_int
+    lib.typhoon_mla_test_wait_expiry.argtypes = [vp, i64, i32, vp]
+    lib.typhoon_mla_set_stacked_absorb.restype = C.c_int
+    lib.typhoon_mla_set_stacked_absorb.argtypes = [i32]
     lib.typhoon_mla_naive_shared_noalloc.restype = C.c_int
     lib.typhoon_mla_naive_shared_noalloc.argtypes = [vp, vp, vp, i32, f32, vp, vp, vp]
     lib.typhoon_mla_profile_begin.restype = C.c_int
@@ -170,14 +174,22 @@ def typhoon_mla_free(handle) -> None:
     _check(_lib.typhoon_mla_free(handle), "typhoon_mla_free")
 
 
-def typhoon_mla_workspace_bytes(shared: SharedPrefix, B: int, max_pages: int, page_size: int) -> int:
-    return int(_lib.typhoon_mla_workspace_bytes(shared.handle, B, max_pages, page_size))
+def typhoon_mla_workspace_bytes(shared: SharedPrefix, B: int, max_pages: int, page_size: int,
+                                mode: int = MODE_AUTO) -> int:
+    return int(_lib.typhoon_mla_workspace_bytes(shared.handle, B, max_pages, page_size, mode))
+
+
+def _num_pages(num_pages: Optional[int], ckv_pages) -> int:
+    """Physical pages of the cache: the leading extent of the page array unless given."""
+    if num_pages is not None:
+        return int(num_pages)
+    return 0 if ckv_pages is None else int(ckv_pages.shape[0])
 
 
 def typhoon_mla_decode(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages, page_size, block_table,
                        seq_lens, softmax_scale, out, workspace, mode=MODE_AUTO, lse_out=None,
                        max_pages: Optional[int] = None, ckv_token_stride: Optional[int] = None,
-                       kpe_token_stride: Optional[int] = None) -> None:
+                       kpe_token_stride: Optional[int] = None, num_pages: Optional[int] = None) -> None:
     B = q_nope.shape[0]
     if max_pages is None:
         max_pages = 0 if block_table is None else block_table.shape[1]
@@ -186,7 +198,8 @@ def typhoon_mla_decode(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages,
     if kpe_token_stride is None:
         kpe_token_stride = 64 if kpe_pages is None else kpe_pages.stride(-2)
     st = _lib.typhoon_mla_decode(shared.handle, _ptr(q_nope), _ptr(q_pe), B, _ptr(ckv_pages), _ptr(kpe_pages),
-                                 ckv_token_stride, kpe_token_stride, page_size, _ptr(block_table), max_pages,
+                                 ckv_token_stride, kpe_token_stride, page_size, _num_pages(num_pages, ckv_pages),
+                                 _ptr(block_table), max_pages,
                                  _ptr(seq_lens), softmax_scale, mode, _ptr(out), _ptr(lse_out),
                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check(st, "typhoon_mla_decode")
@@ -195,7 +208,7 @@ def typhoon_mla_decode(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages,
 def typhoon_mla_decode_partial(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kpe_pages, page_size, block_table,
                                seq_lens, softmax_scale, out_partial, lse_partial, workspace, mode=MODE_AUTO,
                                max_pages: Optional[int] = None, ckv_token_stride: Optional[int] = None,
-                               kpe_token_stride: Optional[int] = None) -> None:
+                               kpe_token_stride: Optional[int] = None, num_pages: Optional[int] = None) -> None:
     """This device's share of a sharded context: fp32 out_partial [B, H, 128] and lse_partial [B, H]."""
     B = q_nope.shape[0]
     if max_pages is None:
@@ -205,7 +218,8 @@ def typhoon_mla_decode_partial(shared: SharedPrefix, q_nope, q_pe, ckv_pages, kp
     if kpe_token_stride is None:
         kpe_token_stride = 64 if kpe_pages is None else kpe_pages.stride(-2)
     st = _lib.typhoon_mla_decode_partial(shared.handle, _ptr(q_nope), _ptr(q_pe), B, _ptr(ckv_pages), _ptr(kpe_pages),
-                                         ckv_token_stride, kpe_token_stride, page_size, _ptr(block_table), max_pages,
+                                         ckv_token_stride, kpe_token_stride, page_size, _num_pages(num_pages, ckv_pages),
+                                         _ptr(block_table), max_pages,
                                          _ptr(seq_lens), softmax_scale, mode, _ptr(out_partial), _ptr(lse_partial),
                                          _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check(st, "typhoon_mla_decode_partial")
@@ -244,14 +258,15 @@ def typhoon_mla_tree_workspace_bytes(levels, B: int, max_pages: int, page_size: 
 
 
 def typhoon_mla_decode_tree(levels, q_nope, q_pe, ckv_pages, kpe_pages, page_size, block_table, seq_lens,
-                            softmax_scale, out, workspace, lse_out=None) -> None:
+                            softmax_scale, out, workspace, lse_out=None, num_pages: Optional[int] = None) -> None:
     arr, keep = _marshal_levels(levels)
     B = q_nope.shape[0]
     max_pages = 0 if block_table is None else block_table.shape[1]
     st = _lib.typhoon_mla_decode_tree(
         C.cast(arr, C.c_void_p), len(levels), _ptr(q_nope), _ptr(q_pe), B, _ptr(ckv_pages), _ptr(kpe_pages),
         512 if ckv_pages is None else ckv_pages.stride(-2), 64 if kpe_pages is None else kpe_pages.stride(-2),
-        page_size, _ptr(block_table), max_pages, _ptr(seq_lens), softmax_scale, _ptr(out), _ptr(lse_out),
+        page_size, _num_pages(num_pages, ckv_pages), _ptr(block_table), max_pages, _ptr(seq_lens), softmax_scale,
+        _ptr(out), _ptr(lse_out),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check(st, "typhoon_mla_decode_tree")
 
@@ -262,13 +277,14 @@ def typhoon_mla_host_staging_bytes(shared: SharedPrefix, B: int, max_pages: int)
 
 def typhoon_mla_decode_host(shared: SharedPrefix, q_nope_host, q_pe_host, ckv_pages, kpe_pages, page_size,
                             block_table_host, seq_lens_host, softmax_scale, out_host, staging, workspace,
-                            mode=MODE_AUTO) -> None:
+                            mode=MODE_AUTO, num_pages: Optional[int] = None) -> None:
     B = q_nope_host.shape[0]
     max_pages = 0 if block_table_host is None else block_table_host.shape[1]
     st = _lib.typhoon_mla_decode_host(
         shared.handle, _ptr(q_nope_host), _ptr(q_pe_host), B, _ptr(ckv_pages), _ptr(kpe_pages),
         512 if ckv_pages is None else ckv_pages.stride(-2), 64 if kpe_pages is None else kpe_pages.stride(-2),
-        page_size, _ptr(block_table_host), max_pages, _ptr(seq_lens_host), softmax_scale, mode, _ptr(out_host),
+        page_size, _num_pages(num_pages, ckv_pages), _ptr(block_table_host), max_pages, _ptr(seq_lens_host),
+        softmax_scale, mode, _ptr(out_host),
         _ptr(staging), staging.numel() * staging.element_size(),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     _check(st, "typhoon_mla_decode_host")
@@ -297,10 +313,10 @@ def typhoon_mla_cost_model(dims: Dims, kind: int, B: int, S_q: int, L_s: int, L_
     return m.value, w.value
 
 
-def typhoon_mla_naive_plan(num_heads: int, B: int, L_s: int, schedule: int = 0):
+def typhoon_mla_naive_plan(num_heads: int, B: int, L_s: int, schedule: int = 0, num_sms: int = 0):
     """(tile_tokens, n_ranges, row_groups, n_slots) of the shared-prefix kernel's work decomposition."""
     t, r, g, sl = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
-    _check(_lib.typhoon_mla_naive_plan(num_heads, B, L_s, schedule, C.byref(t), C.byref(r), C.byref(g), C.byref(sl)),
+    _check(_lib.typhoon_mla_naive_plan(num_heads, B, L_s, schedule, num_sms, C.byref(t), C.byref(r), C.byref(g), C.byref(sl)),
            "typhoon_mla_naive_plan")
     return t.value, r.value, g.value, sl.value
 
@@ -359,11 +375,26 @@ def typhoon_mla_set_kernel_path(path: int) -> None:
     _check(_lib.typhoon_mla_set_kernel_path(path), "typhoon_mla_set_kernel_path")
 
 
-def typhoon_mla_device_status(shared: SharedPrefix) -> int:
-    """Synchronises the current stream; raises if an in-kernel wait expired."""
+STATUS_WAIT_EXPIRED, STATUS_BAD_PAGE = 0xFF, 0x100
+
+
+def typhoon_mla_check_status(shared: SharedPrefix, clear: bool = False, raise_on_error: bool = True) -> int:
+    """Synchronises the current stream and returns the handle's device status word; raises if it is
+    non-zero (a bounded in-kernel wait ran out, or a page id was out of range) unless told not to."""
     v = C.c_int32()
-    _check(_lib.typhoon_mla_device_status(shared.handle, _stream(), C.byref(v)), "typhoon_mla_device_status")
+    st = _lib.typhoon_mla_check_status(shared.handle, _stream(), C.byref(v), 1 if clear else 0)
+    if raise_on_error or st not in (0, 6):
+        _check(st, "typhoon_mla_check_status")
     return v.value
+
+
+def typhoon_mla_test_wait_expiry(shared: SharedPrefix, deadline_cycles: int, code: int = 0x40) -> None:
+    _check(_lib.typhoon_mla_test_wait_expiry(shared.handle, deadline_cycles, code, _stream()),
+           "typhoon_mla_test_wait_expiry")
+
+
+def typhoon_mla_set_stacked_absorb(enable: bool) -> None:
+    _check(_lib.typhoon_mla_set_stacked_absorb(1 if enable else 0), "typhoon_mla_set_stacked_absorb")
 
 
 def typhoon_mla_expand_query_rows(block_table: torch.Tensor, seq_lens: torch.Tensor, S_q: int):

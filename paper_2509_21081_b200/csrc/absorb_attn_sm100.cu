@@ -23,27 +23,13 @@
 //
 // Tensor memory (512 columns allocated): S^T[buf] at 64 buf (2 buffers), O^T block
 // m (128 latent rows x 64 heads) at 128 + 64 m.
+#include <algorithm>
 #include <cstddef>
 
 #include "kernels.h"
 #include "sm100.cuh"
 
 
-#ifdef TMLA_TRACE
-static __device__ unsigned long long g_kt_absorb[2] = {~0ull, 0ull};
-__device__ __forceinline__ unsigned long long kt_now_absorb() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_absorb[0], kt_now_absorb()); } while (0)
-#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_absorb[1], kt_now_absorb()); } while (0)
-extern "C" int typhoon_mla_debug_kt_absorb(unsigned long long* out) {
-    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_absorb, 16);
-    unsigned long long init[2] = {~0ull, 0ull};
-    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_absorb, init, 16);
-    return (int)e;
-}
-#else
-#define KT_BEGIN() do {} while (0)
-#define KT_END() do {} while (0)
-#endif
 
 namespace tmla {
 namespace {
@@ -56,22 +42,13 @@ constexpr int TILE_BYTES = 9 * SLAB_BYTES;       // 8 latent slabs + 1 rope slab
 constexpr int STAGES = 2;
 constexpr float kRescaleThreshold = 8.f;         // log2 units
 
-#ifdef TMLA_TRACE
-__device__ long long g_trace_ab[64 * 32];
-__device__ long long g_trace_cta[4096 * 2];
-__device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TRACE_CTA(which) do { if (threadIdx.x == 0) { int lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); if (lin < 4096) g_trace_cta[lin * 2 + (which)] = gtimer(); } } while (0)
-#define TRACE(step, slot) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (step) >= 0 && (step) < 64 && (threadIdx.x & 31) == 0) g_trace_ab[(step) * 32 + (slot)] = clock64(); } while (0)
-#else
-#define TRACE(step, slot) do {} while (0)
-#define TRACE_CTA(which) do {} while (0)
-#endif
 
 struct AbsorbSm100Params {
     int B, H;
     int chunk, n_shared_chunks, n_suffix_chunks;
     int Ls_absorb;
     int page_size, max_pages;
+    int num_pages;         // physical pages of the paged cache: ids outside [0, num_pages) are not dereferenced
     const int32_t* block_table;
     const int32_t* seq_lens;
     const int32_t* order;
@@ -104,6 +81,8 @@ struct Shared {
     alignas(16) float inv[2][32];   // [warpgroup][column]: inverse row sums for the epilogue
 };
 
+constexpr int kAbsorbSmem = (STAGES + 1) * TILE_BYTES + 1024 + (int)sizeof(Shared) + 64;
+
 __device__ __forceinline__ bool wg_vote_or(int bar_id, bool pred) {
     uint32_t r;
     asm volatile(
@@ -130,9 +109,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     pdl_trigger();
     pdl_wait();   // the descriptors and Q_A read below are written by the preceding kernel
-    if (threadIdx.x == 0) TRACE(0, 28);
-    KT_BEGIN();
-    TRACE_CTA(0);
     const int chunk = blockIdx.x, h0 = blockIdx.y * 64;
     // one 16-byte load gives the request, its suffix length and its first two pages (else three
     // dependent loads stand between the kernel's start and its first copy)
@@ -165,6 +141,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     const uint32_t ld0 = (warp == 0 && elect_one()) ? 1u : 0u;
     // physical page and slot of tile j (the block-table read is issued ahead of the wait for a free
     // ring slot so that its latency is off the critical path)
+    bool bad_page = false;   // producer warp only: a page id of the caller's table was out of range
     auto page_of = [&](int j, int& page, int& slot) {
         const int t0 = tok_begin + j * TOK;
         if (shared_seg) {
@@ -174,12 +151,17 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             const int idx = t0 / p.page_size;
             page = (p.desc != nullptr && idx < 2) ? (idx == 0 ? pg0 : pg1) : __shfl_sync(0xffffffffu, bt[idx], 0);
             slot = t0 % p.page_size;
+            // The tensor map ends at num_pages: a coordinate at or past it reads as zeros instead of touching
+            // memory the caller does not own.  The violation is reported through the status word.
+            if ((unsigned)page >= (unsigned)p.num_pages) {
+                bad_page = true;
+                page = p.num_pages;
+            }
         }
     };
     auto issue_group = [&](int j, int g, int page, int slot) {
         const int s = j & 1;
         uint8_t* dst = sKV + s * TILE_BYTES;
-        if (g == 0) TRACE(j, 0);
         mbar_arrive_expect_tx_if(ld0, &sh->kv_full[s][g], (g == 3 ? 3 : 2) * SLAB_BYTES);
         tma_load_3d_if(ld0, dst + (2 * g) * SLAB_BYTES, tc, &sh->kv_full[s][g], (2 * g) * 64, slot, page);
         tma_load_3d_if(ld0, dst + (2 * g + 1) * SLAB_BYTES, tc, &sh->kv_full[s][g], (2 * g + 1) * 64, slot, page);
@@ -284,9 +266,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     }
                 }
                 if (!ok) break;
-                TRACE(j, 1);
                 umma_commit_if(ld, &sh->s_ready[s]);
-                TRACE(j, 2);
             }
         } else if (warp == 3) {
             // ---------------- O^T += C^T * P^T issuer (4 blocks of M = 128 latent rows, N = 64 heads, K = 64 tokens)
@@ -297,7 +277,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 const int s = j & 1;
                 ok = mbar_wait_warp(&sh->p_ready[s], (j >> 1) & 1, abort_flag);
                 if (!ok) break;
-                TRACE(j, 3);
                 tc_fence_after();
                 const uint32_t ca = smem_u32(sKV + s * TILE_BYTES);
                 const uint32_t pa = ca + 8 * SLAB_BYTES;     // P^T lives in the rope slab
@@ -314,7 +293,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     umma_commit_if(ld, &sh->kv_empty[s][m]);
                 }
                 umma_commit_if(ld, &sh->o_done[s]);
-                TRACE(j, 4);
             }
         } else if (warp >= 4) {
             // ---------------- softmax warpgroups
@@ -339,7 +317,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             for (int j = 0; j < n_tiles; ++j) {
                 const int s = j & 1;
                 bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->s_ready[s], (j >> 1) & 1, abort_flag));
-                if (warp == 4) TRACE(j, 8);
                 const int t0 = tok_begin + j * TOK;
                 const int n_valid = min(TOK, tok_end - t0);
                 const bool valid = has_token && r < n_valid;
@@ -364,9 +341,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                         pk[c] = pack_bf16(fast_exp2(d0), fast_exp2(d1));
                     }
                 }
-                if (warp == 4) TRACE(j, 9);
                 const bool rescale = wg_vote_or(bar_id, exceed);
-                if (warp == 4) TRACE(j, 10);
                 if (*abort_flag) break;                      // uniform across the warpgroup after the barrier
                 if (rescale) {
                     // exact column maxima of this tile across the 64 token lanes: warp-wide integer max of
@@ -415,7 +390,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                         pk[c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(sr[2 * c]), p.scale_log2, neg_mr[2 * c])),
                                           fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), p.scale_log2, neg_mr[2 * c + 1])));
                 }
-                if (warp == 4) TRACE(j, 11);
                 // per-thread partial row sums (of the bf16-rounded values), P^T row into the rope slab
                 uint8_t* tile = sKV + s * TILE_BYTES;
                 if (has_token) {
@@ -445,7 +419,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 fence_proxy_async();
                 tc_fence_before();
                 mbar_arrive(&sh->p_ready[s]);
-                if (warp == 4) TRACE(j, 12);
             }
 
             // ---------------- epilogue: row sums across lanes, normalised partial, LSE
@@ -504,16 +477,13 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     const float4 v = *reinterpret_cast<const float4*>(&sh->inv[cg][c]);
                     inv[c] = v.x; inv[c + 1] = v.y; inv[c + 2] = v.z; inv[c + 3] = v.w;
                 }
-                if (warp == 4) TRACE(0, 13);
                 const bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->o_done[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, abort_flag));
                 tc_fence_after();
-                if (warp == 4) TRACE(0, 14);
                 if (ok && !*abort_flag) {
                     // The normalised O (head-major rows of 512 latent values) is staged in the KV ring, which
                     // no product reads any more, as the contiguous block of up to 64 head rows it forms in
                     // global memory, and leaves with one bulk copy.
                     const bool direct = p.o_lat_direct != nullptr;
-                    if (warp == 4) TRACE(0, 15);
 #pragma unroll 1
                     for (int m = 0; m < 4; ++m) {
                         uint32_t orr[32];
@@ -536,9 +506,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             }
             // Both warpgroups have staged their heads, or at least one has set the abort flag (every
             // thread of the two warpgroups gets here: named barrier 3, 256 threads).
-            if (warp == 4) TRACE(0, 16);
             asm volatile("bar.sync 3, 256;\n" ::: "memory");
-            if (warp == 4) TRACE(0, 17);
             if (threadIdx.x == 128 && staged && !*abort_flag) {
                 const int n_heads = min(64, p.H - h0);
                 if (p.o_lat_direct) {
@@ -549,7 +517,6 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 }
                 bulk_commit();
                 bulk_wait_read();   // the staging buffer must outlive the copy; the kernel end publishes the writes
-                TRACE(0, 18);
             }
         }
     } else if (warp >= 4) {
@@ -569,14 +536,12 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
 
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0) TRACE(0, 29);
-    TRACE_CTA(1);
+    if (threadIdx.x == 0 && bad_page && p.status) atomicOr(p.status, 0x100);
     if (*abort_flag) {
-        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 3);
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, 3);
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
         __syncthreads();
     }
-    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
@@ -601,14 +566,10 @@ cudaError_t make_kv_tmaps(const void* ckv, const void* kpe, int64_t ckv_stride, 
 
 }  // namespace
 
-#ifdef TMLA_TRACE
-extern "C" int typhoon_mla_debug_read_trace_absorb_cta(long long* dst) {
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_cta, sizeof(long long) * 4096 * 2);
+
+cudaError_t set_attrs_absorb_sm100() {
+    return cudaFuncSetAttribute(absorb_attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAbsorbSmem);
 }
-extern "C" int typhoon_mla_debug_read_trace_absorb(long long* dst) {
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_ab, sizeof(long long) * 64 * 32);
-}
-#endif
 
 cudaError_t make_absorb_shared_tmaps(const void* ckv, const void* kpe, int64_t Ls_pad, CUtensorMap* tm_ckv,
                                      CUtensorMap* tm_kpe) {
@@ -636,9 +597,9 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
         if (e != cudaSuccess) return e;
     }
     if (a.n_suffix_chunks > 0) {
-        // the number of physical pages is not part of the interface: the caller's block table is trusted
+        // the maps end at the caller's last physical page: anything past it reads as zeros
         cudaError_t e = make_kv_tmaps(a.ckv_pages, a.kpe_pages, a.ckv_stride, a.kpe_stride, a.page_size,
-                                      (uint64_t)1 << 24, &tm_ckv_pg, &tm_kpe_pg);
+                                      (uint64_t)std::max(a.num_pages, 1), &tm_ckv_pg, &tm_kpe_pg);
         if (e != cudaSuccess) return e;
     } else {
         tm_ckv_pg = *tm_ckv_sh;
@@ -648,15 +609,14 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     p.B = a.B; p.H = a.H;
     p.chunk = a.chunk; p.n_shared_chunks = a.n_shared_chunks; p.n_suffix_chunks = a.n_suffix_chunks;
     p.Ls_absorb = a.Ls_absorb;
-    p.page_size = a.page_size; p.max_pages = a.max_pages;
+    p.page_size = a.page_size; p.max_pages = a.max_pages; p.num_pages = a.num_pages;
     p.block_table = a.block_table; p.seq_lens = a.seq_lens; p.order = a.order;
     p.desc = reinterpret_cast<const int4*>(a.desc);
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = status;
     p.o_lat_direct = n_chunks == 1 ? reinterpret_cast<__nv_bfloat16*>(o_lat_direct) : nullptr;
     p.lse_direct = lse_direct;
-    const int smem = (STAGES + 1) * TILE_BYTES + 1024 + (int)sizeof(Shared) + 64;
-    cudaFuncSetAttribute(absorb_attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    const int smem = kAbsorbSmem;
     dim3 grid(n_chunks, (a.H + 63) / 64, a.B);
     const CUtensorMap* sh_c = a.n_shared_chunks > 0 ? tm_ckv_sh : &tm_ckv_pg;
     const CUtensorMap* sh_k = a.n_shared_chunks > 0 ? tm_kpe_sh : &tm_kpe_pg;

@@ -2,6 +2,7 @@
 // workspace plan, the crossover rule (Eq. 1 / Table 1) and the launch sequence
 // of one decode step (Algorithm 1).
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstdlib>
@@ -9,18 +10,14 @@
 #include <new>
 
 #include "../../include/typhoon_mla.h"
+#include "../../include/typhoon_mla_internal.h"
 #include "kernels.h"
 
 using namespace tmla;
 
-// Programmatic dependent launch of the step's kernels (tuning aid: TYPHOON_MLA_PDL=0 in the environment
-// gives ordinary stream-ordered launches).
-bool tmla::g_pdl = [] {
-    const char* v = std::getenv("TYPHOON_MLA_PDL");
-    return !(v && v[0] == '0');
-}();
-
 #include "handle.h"
+
+thread_local bool tmla::tl_pdl = true;
 
 namespace {
 
@@ -45,20 +42,27 @@ inline void prof_after(int id, cudaStream_t s) {
     }
 }
 
-int g_kernel_path = TYPHOON_MLA_PATH_TCGEN05;
-// Run the absorb branch of a hybrid step on a side stream next to the naive kernel (tuning aid:
-// TYPHOON_MLA_OVERLAP=0 in the environment keeps everything on the caller's stream).
-bool g_overlap = [] {
-    const char* v = std::getenv("TYPHOON_MLA_OVERLAP");
-    return !(v && v[0] == '0');
-}();
+// Process-wide switches (test and measurement hooks) and the hardware model of the crossover rule.  They
+// are atomics; an API call takes one snapshot at its start and plans and launches from that snapshot only.
+std::atomic<int> g_kernel_path{TYPHOON_MLA_PATH_TCGEN05};
+std::atomic<bool> g_overlap{true};          // absorb branch of a hybrid step on the handle's side stream
+std::atomic<bool> g_pdl{true};              // programmatic dependent launch of the step's kernels
+std::atomic<int> g_naive_schedule{0};
+std::atomic<bool> g_stacked_absorb{true};   // absorb-only steps: batch-stacked kernel over the shared prefix
+constexpr double kDefTensor = 1.0e15, kDefHbm = 6.0e12, kDefFixed = 6.0e-6, kDefAbsorbEff = 0.5;
+std::atomic<double> g_tensor_flops{kDefTensor};        // sustained rate the attention kernels reach, FLOP/s
+std::atomic<double> g_hbm_bytes{kDefHbm};              // bytes/s
+std::atomic<double> g_hybrid_fixed_s{kDefFixed};       // extra launches + combine of the hybrid path
+std::atomic<double> g_absorb_efficiency{kDefAbsorbEff};   // absorb kernel's share of g_tensor_flops (calibrated on B200)
 
-// Hardware model of the crossover rule (defaults: measured on B200).
-double g_tensor_flops = 1.0e15;      // sustained rate the attention kernels reach, FLOP/s
-double g_hbm_bytes = 6.0e12;         // bytes/s
-double g_hybrid_fixed_s = 6.0e-6;    // extra launches + combine of the hybrid path
-constexpr double kDefTensor = 1.0e15, kDefHbm = 6.0e12, kDefFixed = 6.0e-6;
-double g_absorb_efficiency = 0.5;           // absorb kernel's share of g_tensor_flops (calibrated on B200)
+struct Settings {
+    int kernel_path, naive_schedule;
+    bool overlap, pdl, stacked_absorb;
+    bool tc() const { return kernel_path == TYPHOON_MLA_PATH_TCGEN05; }
+};
+Settings snapshot() {
+    return Settings{g_kernel_path.load(), g_naive_schedule.load(), g_overlap.load(), g_pdl.load(), g_stacked_absorb.load()};
+}
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -72,6 +76,10 @@ int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
     return TYPHOON_MLA_ERR_CUDA;
 }
+}  // namespace
+int tmla::api_cuda_fail(cudaError_t e) { return cuda_fail(e); }
+void tmla::api_set_last_launches(int n) { g_last_launches = n; }
+namespace {
 
 // ---- workspace plan --------------------------------------------------------
 struct Plan {
@@ -85,40 +93,22 @@ struct Plan {
     size_t off_order, off_desc, off_qabs, off_opart_a, off_lsepart_a, off_olat, off_lse_a, off_oabs, off_opart_n, off_lsepart_n, total;
 };
 
-constexpr int kNumSM = 148;
+constexpr int kDefaultNumSM = 148;        // a B200; used where no device is at hand (pure planning queries)
 constexpr int kMaxAbsorbChunks = 1024;   // chunks per request the merge kernel accepts
 
-// Tuning aids for the tcgen05 naive kernel: TYPHOON_MLA_NAIVE_CTAS overrides the SM count the plan
-// fills, TYPHOON_MLA_NAIVE_SCHEDULE ("split" or "streamk") the initial value of typhoon_mla_set_naive_schedule.
-int naive_sm_budget() {
-    if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_CTAS")) {
-        const int v = std::atoi(ov);
-        if (v >= 1 && v <= kNumSM) return v;
-    }
-    return kNumSM;
-}
-int g_naive_schedule = [] {   // process-wide; TYPHOON_MLA_NAIVE_SCHEDULE sets the initial value
-    if (const char* ov = std::getenv("TYPHOON_MLA_NAIVE_SCHEDULE")) {
-        if (std::strcmp(ov, "split") == 0) return 1;
-        if (std::strcmp(ov, "streamk") == 0) return 2;
-    }
-    return 0;
-}();
-int naive_schedule() { return g_naive_schedule; }
-
-int naive_splits(int B, int H, int64_t Ls) {
+int naive_splits(int B, int H, int64_t Ls, int n_sm) {
     if (Ls <= 0) return 0;
     int n_tiles = (int)((Ls + 63) / 64);
     int base = ((B + 63) / 64) * H;
-    int want = (4 * kNumSM + base - 1) / base;
+    int want = (4 * n_sm + base - 1) / base;
     return std::max(1, std::min({want, n_tiles, 64}));
 }
 
-void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chunk, int* n_sh, int* n_sf) {
+void absorb_chunks(bool tc, int n_sm, int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chunk, int* n_sh, int* n_sf) {
     const int units = B * ((H + 63) / 64);
     const int64_t longest = std::max<int64_t>(std::max(Ls_absorb, cap_suffix), 1);
     int64_t c;
-    if (g_kernel_path == TYPHOON_MLA_PATH_TCGEN05) {
+    if (tc) {
         // One CTA per SM: minimise waves x (tiles per chunk + fixed cost in tile units) over the number of
         // chunks the longest segment is cut into.
         const double fixed = 3.0;
@@ -128,7 +118,7 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
             const int64_t ch = round_up((longest + parts - 1) / parts, 64);
             const int64_t ctas = (int64_t)units * ((Ls_absorb + ch - 1) / ch + (cap_suffix + ch - 1) / ch);
             if (ctas / units > kMaxAbsorbChunks) continue;   // limit of the merge kernel
-            const int64_t waves = (ctas + kNumSM - 1) / kNumSM;
+            const int64_t waves = (ctas + n_sm - 1) / n_sm;
             // a split segment writes and re-reads fp32 partials (64 heads x 2 KB, both ways): about 3.5 tiles
             // worth of traffic per chunk
             const double split_cost = (ctas > units) ? 3.5 : 0.0;
@@ -140,7 +130,7 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
             if (ch <= 64) break;
         }
     } else {
-        const int target = std::max(1, (2 * kNumSM + units - 1) / units);
+        const int target = std::max(1, (2 * n_sm + units - 1) / units);
         c = std::max<int64_t>(round_up((longest + target - 1) / target, 64), 256);
         while ((Ls_absorb + c - 1) / c + (cap_suffix + c - 1) / c > kMaxAbsorbChunks) c *= 2;
     }
@@ -149,25 +139,27 @@ void absorb_chunks(int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chu
     *n_sf = (int)((cap_suffix + c - 1) / c);
 }
 
-Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size, int mode, int naive_slots_override = -1) {
+// `mode` is resolved (ABSORB, HYBRID or NAIVE); `tc` and `schedule` come from the caller's settings snapshot.
+Plan make_plan(const typhoon_mla_shared* sh, bool tc, int schedule, int B, int max_pages, int page_size, int mode,
+               int naive_slots_override = -1) {
     Plan p{};
     const int H = sh->dims.num_heads;
+    const int n_sm = sh->num_sms > 0 ? sh->num_sms : kDefaultNumSM;
     p.mode = mode;
     const int64_t cap = (int64_t)max_pages * page_size;
     const bool use_naive = (mode != TYPHOON_MLA_MODE_ABSORB) && sh->Ls > 0;
     const bool use_absorb = (mode != TYPHOON_MLA_MODE_NAIVE);
-    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
     if (naive_slots_override >= 0) {   // several shared-prefix launches planned by the caller
         p.n_split_naive = naive_slots_override > 0 ? 1 : 0;
         p.n_slots_naive = naive_slots_override;
     } else if (use_naive && tc) {
-        naive_sm100_plan(B, H, sh->Ls, naive_sm_budget(), naive_schedule(), &p.n_split_naive, &p.n_slots_naive);   // n_split_naive = tile ranges
+        naive_sm100_plan(B, H, sh->Ls, n_sm, schedule, &p.n_split_naive, &p.n_slots_naive);   // n_split_naive = tile ranges
     } else {
-        p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls) : 0;
+        p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls, n_sm) : 0;
         p.n_slots_naive = p.n_split_naive;
     }
     if (use_absorb) {
-        absorb_chunks(B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
+        absorb_chunks(tc, n_sm, B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
                       &p.n_suffix_chunks);
     }
     const int n_chunks = p.n_shared_chunks + p.n_suffix_chunks;
@@ -190,6 +182,12 @@ Plan make_plan(const typhoon_mla_shared* sh, int B, int max_pages, int page_size
     p.off_lsepart_n = take((size_t)p.n_slots_naive * BH * 4);
     p.total = off;
     return p;
+}
+
+// The handle's buffers, stream and events live on the device it was prepared on.
+bool on_handle_device(const typhoon_mla_shared* sh) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == sh->device;
 }
 
 int resolve_mode(const typhoon_mla_shared* sh, int B, int max_pages, int mode) {
@@ -228,13 +226,13 @@ double typhoon_mla_batch_threshold(const typhoon_mla_dims_t* d, int32_t S_q, dou
     return (d_qk + d->d_v) / ((double)S_q * (2.0 * d->kv_lora_rank + d->d_rope)) * (T / M);
 }
 
-int typhoon_mla_naive_plan(int32_t num_heads, int32_t B, int64_t L_s, int32_t schedule, int32_t* tile_tokens,
-                           int32_t* n_ranges, int32_t* row_groups, int32_t* n_slots) {
-    if (B < 1 || L_s < 1 || L_s > (int64_t)1 << 30 || schedule < 0 || schedule > 2) return TYPHOON_MLA_ERR_INVALID_ARG;
+int typhoon_mla_naive_plan(int32_t num_heads, int32_t B, int64_t L_s, int32_t schedule, int32_t num_sms,
+                           int32_t* tile_tokens, int32_t* n_ranges, int32_t* row_groups, int32_t* n_slots) {
+    if (B < 1 || L_s < 1 || L_s > (int64_t)1 << 30 || schedule < 0 || schedule > 2 || num_sms < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (num_heads < 16 || num_heads > 128 || num_heads % 16) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!tile_tokens || !n_ranges || !row_groups || !n_slots) return TYPHOON_MLA_ERR_INVALID_ARG;
     int r = 0, sl = 0;
-    naive_sm100_plan(B, num_heads, L_s, kNumSM, schedule, &r, &sl);
+    naive_sm100_plan(B, num_heads, L_s, num_sms > 0 ? num_sms : kDefaultNumSM, schedule, &r, &sl);
     *tile_tokens = naive_sm100_tile_tokens(B);
     *n_ranges = r;
     *row_groups = B <= 128 ? 1 : (B + 255) / 256;
@@ -271,14 +269,14 @@ int typhoon_mla_cost_model(const typhoon_mla_dims_t* d, int32_t kind, int64_t B,
 }
 
 int typhoon_mla_set_hw_model(double tensor_flops, double hbm_bytes_per_s, double hybrid_fixed_s) {
-    g_tensor_flops = tensor_flops > 0 ? tensor_flops : kDefTensor;
-    g_hbm_bytes = hbm_bytes_per_s > 0 ? hbm_bytes_per_s : kDefHbm;
-    g_hybrid_fixed_s = hybrid_fixed_s >= 0 ? hybrid_fixed_s : kDefFixed;
+    g_tensor_flops.store(tensor_flops > 0 ? tensor_flops : kDefTensor);
+    g_hbm_bytes.store(hbm_bytes_per_s > 0 ? hbm_bytes_per_s : kDefHbm);
+    g_hybrid_fixed_s.store(hybrid_fixed_s >= 0 ? hybrid_fixed_s : kDefFixed);
     return TYPHOON_MLA_OK;
 }
 
 int typhoon_mla_set_absorb_efficiency(double fraction) {
-    g_absorb_efficiency = (fraction > 0.0 && fraction <= 1.0) ? fraction : 0.5;
+    g_absorb_efficiency.store((fraction > 0.0 && fraction <= 1.0) ? fraction : kDefAbsorbEff);
     return TYPHOON_MLA_OK;
 }
 
@@ -298,8 +296,9 @@ int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int3
     const double by_absorb = 2.0 * L * (d.kv_lora_rank + d.d_rope);
     // The absorb kernel re-reads the prefix per request and runs M = 64 tiles: measured on B200 it
     // reaches about half of the tensor throughput the naive kernel does, hence the factor.
-    const double t_hybrid = std::max(f_naive / g_tensor_flops, by_naive / g_hbm_bytes) + g_hybrid_fixed_s;
-    const double t_absorb = std::max(f_absorb / (g_absorb_efficiency * g_tensor_flops), by_absorb / g_hbm_bytes);
+    const double T = g_tensor_flops.load(), M = g_hbm_bytes.load();
+    const double t_hybrid = std::max(f_naive / T, by_naive / M) + g_hybrid_fixed_s.load();
+    const double t_absorb = std::max(f_absorb / (g_absorb_efficiency.load() * T), by_absorb / M);
     return t_hybrid < t_absorb ? TYPHOON_MLA_MODE_HYBRID : TYPHOON_MLA_MODE_ABSORB;
 }
 
@@ -334,9 +333,26 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
                    !aligned16(ckv_shared) || !aligned16(kpe_shared)))
         return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!aligned16(w_uk) || !aligned16(w_uv) || Ls > (int64_t)1 << 24) return TYPHOON_MLA_ERR_INVALID_ARG;
-    int dev = 0;
+    int dev = 0, n_sm = 0;
     cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    // opt-in shared-memory sizes of every kernel, once per device and off the decode path
+    if (e == cudaSuccess) e = set_attrs_naive_sm100();
+    if (e == cudaSuccess) e = set_attrs_absorb_sm100();
+    if (e == cudaSuccess) e = set_attrs_gemm_sm100();
+    if (e == cudaSuccess) e = set_attrs_q_absorb_sm100();
+    if (e == cudaSuccess) e = set_attrs_attn_mma();
+    if (e == cudaSuccess) e = set_attrs_gemm_tn();
     if (e != cudaSuccess) return cuda_fail(e);
+    // The allocation-free entry point keeps its scratch in a device array of the library image.  The module
+    // that holds it is loaded lazily, and loading it takes device memory: do it here, where allocating is
+    // allowed, so that the entry point itself never has to.
+    {
+        const int st = noalloc_resolve_scratch_for_current_device();
+        if (st != TYPHOON_MLA_OK) return st;
+    }
+    const Settings cfg = snapshot();
+    tmla::tl_pdl = cfg.pdl;
 
     typhoon_mla_shared* sh = new (std::nothrow) typhoon_mla_shared();
     if (!sh) return TYPHOON_MLA_ERR_ALLOC;
@@ -346,6 +362,7 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
     sh->Ls_pad = round_up(Ls, 128);
     sh->w_uv = w_uv;
     sh->device = dev;
+    sh->num_sms = n_sm;
     const int H = dims->num_heads;
     const size_t Lp = (size_t)sh->Ls_pad;
     const size_t b_k = (size_t)H * Lp * 128 * 2, b_ckv = Lp * 512 * 2, b_kpe = Lp * 64 * 2,
@@ -362,7 +379,7 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
         return TYPHOON_MLA_ERR_ALLOC;
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    const bool tc = cfg.tc();
     {
         int lo = 0, hi = 0;
         cudaDeviceGetStreamPriorityRange(&lo, &hi);   // hi is the numerically lowest = highest priority
@@ -430,36 +447,49 @@ int typhoon_mla_order_by_length(const int32_t* seq_lens, int32_t B, int32_t* per
 }
 
 int typhoon_mla_set_overlap(int32_t enable) {
-    g_overlap = enable != 0;
+    g_overlap.store(enable != 0);
     return TYPHOON_MLA_OK;
 }
 
 int typhoon_mla_set_programmatic_launch(int32_t enable) {
-    tmla::g_pdl = enable != 0;
+    g_pdl.store(enable != 0);
     return TYPHOON_MLA_OK;
 }
 
 int typhoon_mla_set_naive_schedule(int32_t schedule) {
     if (schedule < 0 || schedule > 2) return TYPHOON_MLA_ERR_INVALID_ARG;
-    g_naive_schedule = schedule;
+    g_naive_schedule.store(schedule);
     return TYPHOON_MLA_OK;
 }
 
 int typhoon_mla_set_kernel_path(int32_t path) {
     if (path != TYPHOON_MLA_PATH_TCGEN05 && path != TYPHOON_MLA_PATH_WARP_MMA) return TYPHOON_MLA_ERR_INVALID_ARG;
-    g_kernel_path = path;
+    g_kernel_path.store(path);
     return TYPHOON_MLA_OK;
 }
 
-int typhoon_mla_device_status(const typhoon_mla_shared_t* sh, void* stream, int32_t* status) {
-    if (!sh || !status) return TYPHOON_MLA_ERR_INVALID_ARG;
+int typhoon_mla_set_stacked_absorb(int32_t enable) {
+    g_stacked_absorb.store(enable != 0);
+    return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_check_status(const typhoon_mla_shared_t* sh, void* stream, int32_t* word, int32_t clear) {
+    if (!sh) return TYPHOON_MLA_ERR_INVALID_ARG;
     int v = 0;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(&v, sh->status, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && clear) e = cudaMemsetAsync(sh->status, 0, sizeof(int), s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
-    *status = v;
+    if (word) *word = v;
     return v == 0 ? TYPHOON_MLA_OK : TYPHOON_MLA_ERR_DEVICE_CHECK;
+}
+
+int typhoon_mla_test_wait_expiry(const typhoon_mla_shared_t* sh, int64_t deadline_cycles, int32_t code, void* stream) {
+    if (!sh || code < 1 || code > 255) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const long long d = std::min<long long>(std::max<long long>(deadline_cycles, 1000), 100000000LL);
+    const cudaError_t e = launch_wait_expiry_selftest(sh->status, d, code, reinterpret_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
 }
 
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* sh, void* k_nope_dst, void* v_t_dst, void* stream) {
@@ -472,17 +502,21 @@ int typhoon_mla_shared_export(const typhoon_mla_shared_t* sh, void* k_nope_dst, 
     return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
 }
 
-size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* sh, int32_t B, int32_t max_pages, int32_t page_size) {
+size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* sh, int32_t B, int32_t max_pages, int32_t page_size,
+                                   int32_t mode) {
     if (!sh || B < 1 || max_pages < 0 || (page_size != 64 && page_size != 128)) return 0;
-    // worst case over modes and kernel paths
-    const int saved = g_kernel_path;
+    if (mode < TYPHOON_MLA_MODE_AUTO || mode > TYPHOON_MLA_MODE_NAIVE) return 0;
+    // Worst case over the modes `mode` can resolve to, over both kernel implementations and over the work
+    // decompositions a test hook may select: a workspace sized here serves whatever the switches are set to when
+    // the step runs.  Only local values are used; no process-wide state is read or written.
     size_t worst = 0;
-    for (int path : {TYPHOON_MLA_PATH_TCGEN05, TYPHOON_MLA_PATH_WARP_MMA}) {
-        g_kernel_path = path;
-        worst = std::max(worst, make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_ABSORB).total);
-        worst = std::max(worst, make_plan(sh, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID).total);
+    for (int m : {TYPHOON_MLA_MODE_ABSORB, TYPHOON_MLA_MODE_HYBRID, TYPHOON_MLA_MODE_NAIVE}) {
+        if (mode != TYPHOON_MLA_MODE_AUTO && mode != m && !(mode == TYPHOON_MLA_MODE_HYBRID && sh->Ls == 0)) continue;
+        const int pages = m == TYPHOON_MLA_MODE_NAIVE ? 0 : max_pages;
+        for (bool tc : {true, false})
+            for (int schedule : {0, 1, 2})
+                worst = std::max(worst, make_plan(sh, tc, schedule, B, pages, page_size, m).total);
     }
-    g_kernel_path = saved;
     return worst + 256;
 }
 
@@ -505,12 +539,14 @@ struct EmptySlots {
 // number of naive partial slots.
 constexpr int kMergeProjectMaxB = 2;   // measured: from 3 requests on the GEMM form (weights read once) is faster
 
-static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n_jobs, const EmptySlots* empties, int n_empties,
+static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const NaiveJob* jobs, int n_jobs,
+                const EmptySlots* empties, int n_empties,
                 const Plan& pl, const void* q_nope, const void* q_pe, int32_t B, const void* ckv_pages,
-                const void* kpe_pages, int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size,
+                const void* kpe_pages, int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size, int32_t num_pages,
                 const int32_t* block_table, int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode,
                 void* out, float* lse_out, void* workspace, void* stream, bool out_fp32 = false) {
     const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
+    tmla::tl_pdl = cfg.pdl;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     char* ws = reinterpret_cast<char*>(workspace);
     const int H = sh->dims.num_heads;
@@ -524,12 +560,12 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
 
     const int n_chunks = pl.n_shared_chunks + pl.n_suffix_chunks;
     const bool have_absorb = use_absorb && n_chunks > 0;
-    const bool tc = g_kernel_path == TYPHOON_MLA_PATH_TCGEN05;
+    const bool tc = cfg.tc();
     // In a hybrid step the absorb branch (lines 5-6) does not depend on the naive kernel (line 4): it runs
     // on the handle's (high-priority) side stream, forked behind the caller's stream here and joined
     // before the projection.
     cudaStream_t s_main = s;
-    const bool forked = g_overlap && have_absorb && n_jobs > 0 && sh->side_stream != nullptr;
+    const bool forked = cfg.overlap && have_absorb && n_jobs > 0 && sh->side_stream != nullptr;
     if (forked) {
         e = cudaEventRecord(sh->ev_fork, s_main);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(sh->side_stream, sh->ev_fork, 0);
@@ -544,7 +580,7 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
         float* op = o_part_n + ((size_t)jb.slot0 * B + jb.row0) * H * 128;
         float* lp = lse_part_n + ((size_t)jb.slot0 * B + jb.row0) * H;
         prof_before(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
-        if (g_kernel_path == TYPHOON_MLA_PATH_TCGEN05) {
+        if (tc) {
             NaiveAttnSm100 na{qn, qp, &jb.sh->tm_kn, &jb.sh->tm_kp, &jb.sh->tm_vt, jb.rows, H, (int)jb.sh->Ls,
                               jb.n_ranges, jb.n_slots_level, softmax_scale, op, lp, sh->status, B};
             e = launch_naive_attn_sm100(na, s);
@@ -597,9 +633,9 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
         float* lse_part_a = reinterpret_cast<float*>(ws + pl.off_lsepart_a);
         void* o_lat = ws + pl.off_olat;
         AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
-                      ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages,
+                      ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, num_pages, block_table, max_pages,
                       seq_lens, order, desc, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
-                      o_part_a, lse_part_a};
+                      o_part_a, lse_part_a, sh->status};
         prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         e = tc ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, o_lat, lse_a, sh->status, s)
                : launch_absorb_attn_mma(ab, s);
@@ -663,11 +699,13 @@ static int decode_core(const typhoon_mla_shared* sh, const NaiveJob* jobs, int n
 
 static int decode_impl(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
                        const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
-                       int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
-                       const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
-                       void* workspace, size_t workspace_bytes, void* stream, bool out_fp32) {
+                       int64_t kpe_token_stride, int32_t page_size, int32_t num_pages, const int32_t* block_table,
+                       int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out,
+                       float* lse_out, void* workspace, size_t workspace_bytes, void* stream, bool out_fp32) {
     g_last_launches = 0;
     if (!sh || !q_nope || !q_pe || !out || B < 1 || max_pages < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!on_handle_device(sh)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const Settings cfg = snapshot();
     if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (mode < TYPHOON_MLA_MODE_AUTO || mode > TYPHOON_MLA_MODE_NAIVE) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
@@ -675,48 +713,50 @@ static int decode_impl(const typhoon_mla_shared_t* sh, const void* q_nope, const
     mode = resolve_mode(sh, B, max_pages, mode);
     const bool use_absorb = mode != TYPHOON_MLA_MODE_NAIVE;
     if (use_absorb && max_pages > 0) {
-        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens) return TYPHOON_MLA_ERR_INVALID_ARG;
+        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens || num_pages < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
         if (!aligned16(ckv_pages) || !aligned16(kpe_pages) || ckv_token_stride < 512 || kpe_token_stride < 64 ||
             ckv_token_stride % 8 || kpe_token_stride % 8)
             return TYPHOON_MLA_ERR_INVALID_ARG;
     }
     if (mode == TYPHOON_MLA_MODE_NAIVE && sh->Ls == 0) max_pages = 0;
-    const Plan pl = make_plan(sh, B, use_absorb ? max_pages : 0, page_size, mode);
+    const Plan pl = make_plan(sh, cfg.tc(), cfg.naive_schedule, B, use_absorb ? max_pages : 0, page_size, mode);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
 
     NaiveJob job{sh, 0, B, pl.n_split_naive, pl.n_slots_naive, 0};
-    return decode_core(sh, &job, pl.n_split_naive > 0 ? 1 : 0, nullptr, 0, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
-                       ckv_token_stride, kpe_token_stride, page_size, block_table, use_absorb ? max_pages : 0, seq_lens,
-                       softmax_scale, mode, out, lse_out, workspace, stream, out_fp32);
+    return decode_core(cfg, sh, &job, pl.n_split_naive > 0 ? 1 : 0, nullptr, 0, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
+                       ckv_token_stride, kpe_token_stride, page_size, num_pages, block_table, use_absorb ? max_pages : 0,
+                       seq_lens, softmax_scale, mode, out, lse_out, workspace, stream, out_fp32);
 }
 
 int typhoon_mla_decode(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
                        const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
-                       int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table, int32_t max_pages,
-                       const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out, float* lse_out,
-                       void* workspace, size_t workspace_bytes, void* stream) {
-    return decode_impl(sh, q_nope, q_pe, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table,
-                       max_pages, seq_lens, softmax_scale, mode, out, lse_out, workspace, workspace_bytes, stream, false);
+                       int64_t kpe_token_stride, int32_t page_size, int32_t num_pages, const int32_t* block_table,
+                       int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode, void* out,
+                       float* lse_out, void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_impl(sh, q_nope, q_pe, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, num_pages,
+                       block_table, max_pages, seq_lens, softmax_scale, mode, out, lse_out, workspace, workspace_bytes, stream,
+                       false);
 }
 
 // ---- context sharded over several devices: per-device partial + merge -----------------------------
 int typhoon_mla_decode_partial(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe, int32_t B,
                                const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
-                               int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table,
-                               int32_t max_pages, const int32_t* seq_lens, float softmax_scale, int32_t mode,
-                               float* out_partial, float* lse_partial, void* workspace, size_t workspace_bytes,
-                               void* stream) {
+                               int64_t kpe_token_stride, int32_t page_size, int32_t num_pages,
+                               const int32_t* block_table, int32_t max_pages, const int32_t* seq_lens,
+                               float softmax_scale, int32_t mode, float* out_partial, float* lse_partial,
+                               void* workspace, size_t workspace_bytes, void* stream) {
     if (!lse_partial) return TYPHOON_MLA_ERR_INVALID_ARG;
-    return decode_impl(sh, q_nope, q_pe, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, block_table,
-                       max_pages, seq_lens, softmax_scale, mode, out_partial, lse_partial, workspace, workspace_bytes,
-                       stream, true);
+    return decode_impl(sh, q_nope, q_pe, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, num_pages,
+                       block_table, max_pages, seq_lens, softmax_scale, mode, out_partial, lse_partial, workspace,
+                       workspace_bytes, stream, true);
 }
 
 int typhoon_mla_combine_partials(const float* o_parts, const float* lse_parts, int32_t n_parts, int32_t B, int32_t H,
                                  void* out, float* lse_out, void* stream) {
     if (!o_parts || !lse_parts || !out || n_parts < 1 || B < 1 || H < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!aligned16(o_parts) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
+    tmla::tl_pdl = g_pdl.load();
     const cudaError_t e = launch_combine(o_parts, lse_parts, n_parts, nullptr, nullptr, B, H, out, lse_out,
                                          reinterpret_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);
@@ -732,7 +772,7 @@ struct TreePlan {
     EmptySlots empties[kMaxTreeJobs];
     int n_jobs = 0, n_empties = 0, total_slots = 0;
 };
-int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, TreePlan* tp) {
+int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, int schedule, TreePlan* tp) {
     if (!levels || n_levels < 1 || n_levels > kMaxLevels || B < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
     for (int l = 0; l < n_levels && !tp->sh0; ++l) {
         if (!levels[l].prefixes || !levels[l].group_begin || levels[l].n_groups < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
@@ -755,7 +795,7 @@ int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, Tre
             if (!sh || sh->Ls == 0 || r1 == r0) continue;
             if (tp->n_jobs == kMaxTreeJobs) return TYPHOON_MLA_ERR_INVALID_ARG;
             int ranges = 0, slots = 0;
-            naive_sm100_plan(r1 - r0, H, sh->Ls, naive_sm_budget(), naive_schedule(), &ranges, &slots);
+            naive_sm100_plan(r1 - r0, H, sh->Ls, sh->num_sms > 0 ? sh->num_sms : kDefaultNumSM, schedule, &ranges, &slots);
             tp->jobs[tp->n_jobs++] = NaiveJob{sh, r0, r1 - r0, ranges, 0, slot0};
             level_slots = std::max(level_slots, slots);
         }
@@ -777,15 +817,20 @@ int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, Tre
 
 size_t typhoon_mla_tree_workspace_bytes(const typhoon_mla_prefix_level_t* levels, int32_t n_levels, int32_t B,
                                         int32_t max_pages, int32_t page_size) {
-    if (max_pages < 0 || (page_size != 64 && page_size != 128) || g_kernel_path != TYPHOON_MLA_PATH_TCGEN05) return 0;
-    TreePlan tp;
-    if (plan_tree(levels, n_levels, B, &tp) != TYPHOON_MLA_OK) return 0;
-    return make_plan(tp.sh0, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID, tp.total_slots).total + 256;
+    if (max_pages < 0 || (page_size != 64 && page_size != 128)) return 0;
+    // worst case over the work decompositions a test hook may select (the tree step needs the tcgen05 kernels)
+    size_t worst = 0;
+    for (int schedule : {0, 1, 2}) {
+        TreePlan tp;
+        if (plan_tree(levels, n_levels, B, schedule, &tp) != TYPHOON_MLA_OK) return 0;
+        worst = std::max(worst, make_plan(tp.sh0, true, schedule, B, max_pages, page_size, TYPHOON_MLA_MODE_HYBRID, tp.total_slots).total);
+    }
+    return worst + 256;
 }
 
 int typhoon_mla_decode_tree(const typhoon_mla_prefix_level_t* levels, int32_t n_levels, const void* q_nope,
                             const void* q_pe, int32_t B, const void* ckv_pages, const void* kpe_pages,
-                            int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size,
+                            int64_t ckv_token_stride, int64_t kpe_token_stride, int32_t page_size, int32_t num_pages,
                             const int32_t* block_table, int32_t max_pages, const int32_t* seq_lens, float softmax_scale,
                             void* out, float* lse_out, void* workspace, size_t workspace_bytes, void* stream) {
     g_last_launches = 0;
@@ -793,24 +838,26 @@ int typhoon_mla_decode_tree(const typhoon_mla_prefix_level_t* levels, int32_t n_
     if (page_size != 64 && page_size != 128) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!aligned16(q_nope) || !aligned16(q_pe) || !aligned16(out)) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return TYPHOON_MLA_ERR_INVALID_ARG;
-    if (g_kernel_path != TYPHOON_MLA_PATH_TCGEN05) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;
+    const Settings cfg = snapshot();
+    if (!cfg.tc()) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;
     if (max_pages > 0) {
-        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens) return TYPHOON_MLA_ERR_INVALID_ARG;
+        if (!ckv_pages || !kpe_pages || !block_table || !seq_lens || num_pages < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
         if (!aligned16(ckv_pages) || !aligned16(kpe_pages) || ckv_token_stride < 512 || kpe_token_stride < 64 ||
             ckv_token_stride % 8 || kpe_token_stride % 8)
             return TYPHOON_MLA_ERR_INVALID_ARG;
     }
     TreePlan tp;
-    const int rc = plan_tree(levels, n_levels, B, &tp);
+    const int rc = plan_tree(levels, n_levels, B, cfg.naive_schedule, &tp);
     if (rc != TYPHOON_MLA_OK) return rc;
+    if (!on_handle_device(tp.sh0)) return TYPHOON_MLA_ERR_INVALID_ARG;
     // NAIVE when there is no page table (nothing for the absorb branch), else Algorithm 1 with several line-4 launches
     const int mode = max_pages == 0 ? TYPHOON_MLA_MODE_NAIVE : TYPHOON_MLA_MODE_HYBRID;
-    const Plan pl = make_plan(tp.sh0, B, max_pages, page_size, mode, tp.total_slots);
+    const Plan pl = make_plan(tp.sh0, true, cfg.naive_schedule, B, max_pages, page_size, mode, tp.total_slots);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
-    return decode_core(tp.sh0, tp.jobs, tp.n_jobs, tp.empties, tp.n_empties, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
-                       ckv_token_stride, kpe_token_stride, page_size, block_table, max_pages, seq_lens, softmax_scale,
-                       mode, out, lse_out, workspace, stream);
+    return decode_core(cfg, tp.sh0, tp.jobs, tp.n_jobs, tp.empties, tp.n_empties, pl, q_nope, q_pe, B, ckv_pages, kpe_pages,
+                       ckv_token_stride, kpe_token_stride, page_size, num_pages, block_table, max_pages, seq_lens,
+                       softmax_scale, mode, out, lse_out, workspace, stream);
 }
 
 int typhoon_mla_profile_begin(int32_t kernel_id, int32_t max_launches) {
@@ -861,8 +908,9 @@ size_t typhoon_mla_host_staging_bytes(const typhoon_mla_shared_t* sh, int32_t B,
 
 int typhoon_mla_decode_host(const typhoon_mla_shared_t* sh, const void* q_nope_host, const void* q_pe_host, int32_t B,
                             const void* ckv_pages, const void* kpe_pages, int64_t ckv_token_stride,
-                            int64_t kpe_token_stride, int32_t page_size, const int32_t* block_table_host,
-                            int32_t max_pages, const int32_t* seq_lens_host, float softmax_scale, int32_t mode,
+                            int64_t kpe_token_stride, int32_t page_size, int32_t num_pages,
+                            const int32_t* block_table_host, int32_t max_pages, const int32_t* seq_lens_host,
+                            float softmax_scale, int32_t mode,
                             void* out_host, void* staging, size_t staging_bytes, void* workspace,
                             size_t workspace_bytes, void* stream) {
     if (!sh || !q_nope_host || !q_pe_host || !out_host || !staging || B < 1 || max_pages < 0)
@@ -886,7 +934,7 @@ int typhoon_mla_decode_host(const typhoon_mla_shared_t* sh, const void* q_nope_h
     }
     if (e != cudaSuccess) return cuda_fail(e);
     int st_code = typhoon_mla_decode(sh, d_qn, d_qp, B, ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride,
-                                     page_size, reinterpret_cast<const int32_t*>(d_bt), max_pages,
+                                     page_size, num_pages, reinterpret_cast<const int32_t*>(d_bt), max_pages,
                                      reinterpret_cast<const int32_t*>(d_sl), softmax_scale, mode, d_out, nullptr,
                                      workspace, workspace_bytes, stream);
     if (st_code != TYPHOON_MLA_OK) return st_code;

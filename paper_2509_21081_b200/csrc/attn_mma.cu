@@ -276,7 +276,13 @@ __global__ void __launch_bounds__(256) absorb_attn_mma_kernel(AbsorbAttn p) {
                 src = ch < 64 ? ckv_s + (int64_t)t * 512 + ch * 8 : kpe_s + (int64_t)t * 64 + (ch - 64) * 8;
             } else {
                 int t = ok ? tok : tok_begin;
-                int64_t slot = (int64_t)bt[t / p.page_size] * p.page_size + (t % p.page_size);
+                int pg = bt[t / p.page_size];
+                if ((unsigned)pg >= (unsigned)p.num_pages) {   // not dereferenced: the token reads as zeros
+                    if (ok && p.status) atomicOr(p.status, 0x100);
+                    ok = false;
+                    pg = 0;
+                }
+                int64_t slot = (int64_t)pg * p.page_size + (t % p.page_size);
                 src = ch < 64 ? ckv_p + slot * p.ckv_stride + ch * 8 : kpe_p + slot * p.kpe_stride + (ch - 64) * 8;
             }
             cp_async16(smem_u32(sKV + swz<72>(row, ch)), src, ok);
@@ -397,9 +403,14 @@ __global__ void __launch_bounds__(256) absorb_attn_mma_kernel(AbsorbAttn p) {
 
 }  // namespace
 
+cudaError_t set_attrs_attn_mma() {
+    cudaError_t e = cudaFuncSetAttribute(naive_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NA_SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(absorb_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AB_SMEM_BYTES);
+    return e;
+}
+
 cudaError_t launch_naive_attn_mma(const NaiveAttn& p, cudaStream_t s) {
     if (p.B <= 0 || p.Ls <= 0 || p.n_split <= 0) return cudaSuccess;
-    cudaFuncSetAttribute(naive_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NA_SMEM_BYTES);
     dim3 grid(p.n_split, (p.B + NA_ROWS - 1) / NA_ROWS, p.H);
     naive_attn_mma_kernel<<<grid, 128, NA_SMEM_BYTES, s>>>(p);
     return cudaGetLastError();
@@ -408,7 +419,6 @@ cudaError_t launch_naive_attn_mma(const NaiveAttn& p, cudaStream_t s) {
 cudaError_t launch_absorb_attn_mma(const AbsorbAttn& p, cudaStream_t s) {
     int n_chunks = p.n_shared_chunks + p.n_suffix_chunks;
     if (p.B <= 0 || n_chunks <= 0) return cudaSuccess;
-    cudaFuncSetAttribute(absorb_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AB_SMEM_BYTES);
     dim3 grid(n_chunks, (p.H + AB_ROWS - 1) / AB_ROWS, p.B);
     absorb_attn_mma_kernel<<<grid, 256, AB_SMEM_BYTES, s>>>(p);
     return cudaGetLastError();

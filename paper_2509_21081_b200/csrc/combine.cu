@@ -340,6 +340,26 @@ __global__ void __launch_bounds__(256) expand_query_rows_kernel(const int32_t* _
 
 }  // namespace
 
+// Test kernel for the bounded wait of the tcgen05 kernels: a barrier on which nothing arrives, the same
+// mbar_wait with a short deadline, the same report through the status word, a normal return.
+static __global__ void wait_expiry_selftest_kernel(int* status, long long deadline_cycles, int code) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(&bar, 1);
+        abort_flag = 0;
+        sm100::fence_mbar_init();
+    }
+    __syncthreads();
+    const bool ok = sm100::mbar_wait(&bar, 0, &abort_flag, deadline_cycles);   // nobody arrives: runs out
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_flag) && status) atomicOr(status, code);
+}
+cudaError_t launch_wait_expiry_selftest(int* status, long long deadline_cycles, int code, cudaStream_t s) {
+    wait_expiry_selftest_kernel<<<1, 32, 0, s>>>(status, deadline_cycles, code);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_order_by_length(const int32_t* seq_lens, int B, int32_t* perm, cudaStream_t s) {
     if (B <= 0 || B > 4096) return cudaErrorInvalidValue;
     order_by_length_kernel<<<1, 1024, 0, s>>>(seq_lens, B, perm);

@@ -12,21 +12,6 @@
 #include "sm100.cuh"
 
 
-#ifdef TMLA_TRACE
-static __device__ unsigned long long g_kt_gemm[2] = {~0ull, 0ull};
-__device__ __forceinline__ unsigned long long kt_now_gemm() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_gemm[0], kt_now_gemm()); } while (0)
-#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_gemm[1], kt_now_gemm()); } while (0)
-extern "C" int typhoon_mla_debug_kt_gemm(unsigned long long* out) {
-    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_gemm, 16);
-    unsigned long long init[2] = {~0ull, 0ull};
-    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_gemm, init, 16);
-    return (int)e;
-}
-#else
-#define KT_BEGIN() do {} while (0)
-#define KT_END() do {} while (0)
-#endif
 
 namespace tmla {
 namespace {
@@ -60,7 +45,6 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, z = blockIdx.z;
     pdl_trigger();
     pdl_wait();
-    KT_BEGIN();
     const int KB = p.K / BK;
 
     if (threadIdx.x == 0) {
@@ -221,15 +205,18 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
     if (*abort_flag) {
         // A wait gave up: leave time for copies already in flight to land before the CTA's
         // shared memory is released, and report.
-        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 1);
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, 1);
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
-    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 128);
 }
 
 }  // namespace
+
+cudaError_t set_attrs_gemm_sm100() {
+    return cudaFuncSetAttribute(gemm_tn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+}
 
 cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, const CombineEpilogue* ce) {
     if (g.M <= 0 || g.batch <= 0) return cudaSuccess;
@@ -263,7 +250,6 @@ cudaError_t launch_gemm_tn_sm100(const GemmTN& g, int* status, cudaStream_t s, c
     }
     GemmParams p{g.C, g.ldc, g.c_batch, g.M, g.N, g.K, g.c_block_n, g.c_tile64 ? 1 : 0, g.a_batch != 0, g.b_batch != 0, a_swap ? 1 : 0, status,
                  ce ? 2 : (g.out_fp32 ? 1 : 0), ce ? *ce : CombineEpilogue{}};
-    cudaFuncSetAttribute(gemm_tn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid(g.N / BN, (g.M + BM - 1) / BM, g.batch);
     return launch_pdl(gemm_tn_sm100_kernel, grid, dim3(192), SMEM_BYTES, s, tmA, tmB, p);
 }

@@ -131,14 +131,16 @@ cudaError_t launch_gemm_tn(const GemmTN& g, cudaStream_t s) {
     if (g.N % BN != 0 || g.K % BK != 0) return cudaErrorInvalidValue;
     dim3 grid(g.N / BN, (g.M + BM - 1) / BM, g.batch);
     size_t smem = (size_t)STAGES * STAGE_ELEMS * sizeof(__nv_bfloat16);
-    if (g.out_fp32) {
-        cudaFuncSetAttribute(gemm_tn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        gemm_tn_kernel<true><<<grid, 256, smem, s>>>(g);
-    } else {
-        cudaFuncSetAttribute(gemm_tn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        gemm_tn_kernel<false><<<grid, 256, smem, s>>>(g);
-    }
+    if (g.out_fp32) gemm_tn_kernel<true><<<grid, 256, smem, s>>>(g);
+    else gemm_tn_kernel<false><<<grid, 256, smem, s>>>(g);
     return cudaGetLastError();
+}
+
+cudaError_t set_attrs_gemm_tn() {
+    const int smem = (int)((size_t)STAGES * STAGE_ELEMS * sizeof(__nv_bfloat16));
+    cudaError_t e = cudaFuncSetAttribute(gemm_tn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    return e;
 }
 
 }  // namespace tmla

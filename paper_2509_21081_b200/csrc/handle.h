@@ -23,5 +23,6 @@ struct typhoon_mla_shared {
     cudaEvent_t ev_fork, ev_join;
     int* status;    // device word: non-zero after a bounded in-kernel wait expired
     size_t owned_bytes;
-    int device;
+    int device;     // device the handle was prepared on; every call checks that it is the current one
+    int num_sms;    // multiprocessors of that device (the work decompositions fill them)
 };

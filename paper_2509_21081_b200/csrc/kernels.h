@@ -7,8 +7,19 @@
 namespace tmla {
 
 // Launch with the programmatic-stream-serialization attribute when enabled (see sm100::pdl_wait): the
-// kernel must call pdl_wait() before its first access to global memory.
-extern bool g_pdl;
+// kernel must call pdl_wait() before its first access to global memory.  The switch is per thread: an API
+// call copies its snapshot of the process-wide setting here before it launches anything.
+extern thread_local bool tl_pdl;
+
+// Opt-in shared-memory sizes of the kernels, set once per device (by typhoon_mla_prepare_shared, with that
+// device current) instead of before every launch.
+cudaError_t set_attrs_naive_sm100();
+cudaError_t set_attrs_absorb_sm100();
+cudaError_t set_attrs_stacked_sm100();
+cudaError_t set_attrs_gemm_sm100();
+cudaError_t set_attrs_q_absorb_sm100();
+cudaError_t set_attrs_attn_mma();
+cudaError_t set_attrs_gemm_tn();
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
     cudaLaunchConfig_t cfg{};
@@ -20,7 +31,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_pdl ? 1 : 0;
+    cfg.numAttrs = tl_pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -103,6 +114,7 @@ struct AbsorbAttn {
     const void* ckv_shared; const void* kpe_shared; int Ls_absorb;  // shared prefix handled here (ABSORB mode) or 0
     const void* ckv_pages; const void* kpe_pages;
     int64_t ckv_stride, kpe_stride; int page_size;
+    int num_pages;                                 // physical pages in ckv_pages / kpe_pages; ids outside are not read
     const int32_t* block_table; int max_pages; const int32_t* seq_lens;
     const int32_t* order;                          // optional [B]: request handled by block z (longest first)
     const int32_t* desc;                           // optional [B][4]: per launch position, see launch_q_absorb_sm100
@@ -111,6 +123,7 @@ struct AbsorbAttn {
     float scale;
     float* o_part;   // [n_chunks][B][H][512], each normalised
     float* lse_part; // [n_chunks][B][H]
+    int* status = nullptr;   // device word: bit 0x100 is set when a page id was out of range
 };
 cudaError_t launch_absorb_attn_mma(const AbsorbAttn& p, cudaStream_t s);
 
@@ -145,6 +158,18 @@ cudaError_t launch_merge_project(const float* o_part, const float* lse_part, int
 cudaError_t launch_combine(const float* o_naive, const float* lse_naive, int n_naive,
                            const float* o_abs, const float* lse_abs,
                            int B, int H, void* out, float* lse_out, cudaStream_t s, bool out_fp32 = false);
+
+// One block that waits, with the given deadline in SM clocks, on a barrier nothing arrives on, then ORs `code`
+// into *status (test of the bounded-wait mechanism; no copies, no tensor memory).
+cudaError_t launch_wait_expiry_selftest(int* status, long long deadline_cycles, int code, cudaStream_t s);
+
+// typhoon_mla_naive_shared_noalloc: looks up (once per device) the device address of the built-in scratch array
+// for the current device.  Returns a TYPHOON_MLA_* status.
+int noalloc_resolve_scratch_for_current_device();
+// Bookkeeping shared by the entry points that live outside api.cu: records the CUDA error behind a
+// TYPHOON_MLA_ERR_CUDA (returns that status) and the number of kernels the call launched, both per thread.
+int api_cuda_fail(cudaError_t e);
+void api_set_last_launches(int n);
 
 // out[c][r] = in[r][c] for each of `batch` matrices [R][C] bf16.
 cudaError_t launch_transpose_bf16(const void* in, void* out, int R, int C, int batch, cudaStream_t s);

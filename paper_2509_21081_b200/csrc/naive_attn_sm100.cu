@@ -47,21 +47,6 @@
 #include "sm100.cuh"
 
 
-#ifdef TMLA_TRACE
-static __device__ unsigned long long g_kt_naive[2] = {~0ull, 0ull};
-__device__ __forceinline__ unsigned long long kt_now_naive() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_naive[0], kt_now_naive()); } while (0)
-#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_naive[1], kt_now_naive()); } while (0)
-extern "C" int typhoon_mla_debug_kt_naive(unsigned long long* out) {
-    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_naive, 16);
-    unsigned long long init[2] = {~0ull, 0ull};
-    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_naive, init, 16);
-    return (int)e;
-}
-#else
-#define KT_BEGIN() do {} while (0)
-#define KT_END() do {} while (0)
-#endif
 
 namespace tmla {
 namespace {
@@ -70,17 +55,8 @@ using namespace sm100;
 
 constexpr int Q_TILE_BYTES = 128 * 192 * 2;   // 3 slabs [128][64] bf16
 
-#ifdef TMLA_TRACE
-__device__ long long g_trace_ncta[4096 * 8];
-__device__ __forceinline__ long long gtimer() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TRACE_CTA(tid, which) do { if ((int)threadIdx.x == (tid) && blockIdx.x < 4096) g_trace_ncta[blockIdx.x * 8 + (which)] = gtimer(); } while (0)
-__device__ long long g_trace_nstep[64 * 32];
-#define TRACE(step, slot) do { if (blockIdx.x == 3 && (step) >= 0 && (step) < 64 && (threadIdx.x & 31) == 0) g_trace_nstep[(step) * 32 + (slot)] = clock64(); } while (0)
-#else
-#define TRACE_CTA(tid, which) do {} while (0)
-#define TRACE(step, slot) do {} while (0)
-#endif
 constexpr int MAX_STAGES = 4;
+constexpr int kNaiveSmemMax = 227 * 1024;   // opt-in limit set once per device; every launch stays below it
 
 struct NaiveSm100Params {
     int B, H, Ls, Ls_pad;
@@ -150,8 +126,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     const int rng = blockIdx.x / p.m_groups, grp = blockIdx.x % p.m_groups;
     pdl_trigger();   // the next kernel of the stream may be scheduled as soon as every CTA of this one has started
     pdl_wait();      // nothing below touches global memory before the stream's earlier kernels are done
-    KT_BEGIN();
-    TRACE_CTA(0, 0);
 
     // this CTA's contiguous range of the global tile sequence (T < 2^31: 32-bit arithmetic)
     const int g_begin = rng * p.per + min(rng, p.rem);
@@ -257,7 +231,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             fence_mbar_init();
             __syncwarp();
             asm volatile("bar.sync 1, 64;\n" ::: "memory");
-            TRACE_CTA(0, 6);
             issue_q(s0);
             issue_k(s0, 0, 0);
             asm volatile("bar.sync 2, 64;\n" ::: "memory");
@@ -266,15 +239,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     } else if (threadIdx.x == 0) {
         bar->abort_flag = 0;
     }
-    TRACE_CTA(0, 7);
     if (warp == 1) tmem_alloc(&bar->tmem_base, 512);
-    TRACE_CTA(32, 3);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     // broadcast through a shuffle so that the compiler knows the value is warp-uniform
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
-    TRACE_CTA(0, 1);
 
     if (warp == 0) {
         // ---------------- Q + K producer
@@ -341,7 +311,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         if (!ok) break;
                     }
                     tc_fence_after();
-                    TRACE(j, 0 + i);
                     const uint32_t qa = smem_u32(sQ + (MODE_Y ? 0 : i) * Q_TILE_BYTES);
                     const uint32_t ka = smem_u32(sK + st * K_TILE_BYTES);
                     const uint32_t d = tmem_base + s_col(i, u);
@@ -354,7 +323,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (slab | k) != 0);
                     }
                     umma_commit_if(ld, &bar->s_ready[i][u % NB]);
-                    TRACE(j, 2 + i);
                     if (last_user) umma_commit_if(ld, &bar->k_empty[st]);   // last user releases the ring slot
                 }
             }
@@ -390,7 +358,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         if (!ok) break;
                     }
                     tc_fence_after();
-                    TRACE(j, 4 + i);
                     const uint32_t va = smem_u32(sV + st * V_TILE_BYTES);
                     const uint32_t pa = tmem_base + s_col(i, u);
                     const uint32_t d = tmem_base + 256u + (uint32_t)i * 128u;
@@ -403,7 +370,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                             umma_ts_if(ld, d, pa + 8 * (bi * 4 + k), db + 2 * k, idesc_o, (j | bi | k) != 0);
                     }
                     umma_commit_if(ld, &bar->o_done[i][u & 1]);
-                    TRACE(j, 6 + i);
                     umma_commit_if(ld, &bar->sbuf_free[i][u % NB]);
                     if (last_user) umma_commit_if(ld, &bar->v_empty[st]);
                 }
@@ -435,12 +401,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             for (int j = 0; j < nt && ok; ++j) {
                 const int u = used + j;
                 const int buf = u % NB;
-                if ((warp & 3) == 0) TRACE(j, 8 + 8 * i);
                 ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_ready[i][buf], (u / NB) & 1, abort_flag));
-                if ((warp & 3) == 0) TRACE(j, 9 + 8 * i);
                 if (!ok) break;
                 tc_fence_after();
-                if (used + j == 0) TRACE_CTA(128, 2);
                 if (!warp_has_rows) {
                     // all 32 rows of this warp are padding past B: their P rows may hold anything (rows of
                     // the MMA are independent and these output rows are never stored); just keep in step
@@ -469,7 +432,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     for (int c = 0; c < 64; ++c) mx_raw = fmaxf(mx_raw, __uint_as_float(sr[c >> 5][c & 31]));
                 }
                 const float mx = mx_raw * p.scale_log2;
-                if ((warp & 3) == 0) TRACE(j, 10 + 8 * i);
                 // lazy rescale: only when some row's maximum grew by more than 2^8
                 const bool grow = lane_has_row && mx > m_ref + 8.f;
                 if (j == 0) {
@@ -525,13 +487,10 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     tmem_st32(s_addr + half * 32, pk);
                 }
                 tmem_st_wait();
-                if ((warp & 3) == 0) TRACE(j, 11 + 8 * i);
                 tc_fence_before();
                 mbar_arrive(&bar->p_ready[i][buf]);
-                if ((warp & 3) == 0) TRACE(j, 12 + 8 * i);
             }
             if (!ok) break;
-            TRACE_CTA(128, 3);
             // ---- segment epilogue: normalised partial + LSE into this segment's slot.  With 64-token tiles the two
             // streams worked on the same query rows: stream 1 publishes its softmax state, stream 0 merges both
             // accumulators (same tensor-memory lanes) and writes one partial.
@@ -602,7 +561,6 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         p.lse_part[((int64_t)ss * p.part_rows + b) * p.H + s.h] = -INFINITY;
                 }
                 // the accumulator(s) just read may be overwritten by the next segment
-                TRACE_CTA(128, 4);
                 tc_fence_before();
                 mbar_arrive(&bar->o_free[i]);
                 if (MODE_Y) mbar_arrive(&bar->o_free[1]);
@@ -615,26 +573,16 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 
     tc_fence_before();
     __syncthreads();
-    TRACE_CTA(0, 5);
     if (*abort_flag) {
-        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 2);
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
         for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
         __syncthreads();
     }
-    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
 }  // namespace
 
-#ifdef TMLA_TRACE
-extern "C" int typhoon_mla_debug_read_trace_naive_step(long long* dst) {
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_nstep, sizeof(long long) * 64 * 32);
-}
-extern "C" int typhoon_mla_debug_read_trace_naive_cta(long long* dst) {
-    return (int)cudaMemcpyFromSymbol(dst, g_trace_ncta, sizeof(long long) * 4096 * 8);
-}
-#endif
 
 int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 
@@ -749,18 +697,20 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     const int k_tile = tok * 384, v_tile = mode_y ? 16384 : 32768;
     const int smem = (mode_y ? 1 : 2) * Q_TILE_BYTES + p.k_stages * k_tile + p.v_stages * v_tile + 1024 + (int)sizeof(Barriers) + 64;
     dim3 grid(p.n_ranges * p.m_groups, 1, 1);
+    if (smem > kNaiveSmemMax) return cudaErrorInvalidValue;
     if (mode_y) {
-        if (a.B <= 64) {   // half-height MMAs: the padding rows 64..127 of the query tile cost tensor-pipe time and power
-            cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (a.B <= 64)   // half-height MMAs: the padding rows 64..127 of the query tile cost tensor-pipe time and power
             return launch_pdl(naive_attn_sm100_kernel<64, true>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
-        }
-        cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         return launch_pdl(naive_attn_sm100_kernel<64, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
-    } else {
-        cudaFuncSetAttribute(naive_attn_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        return launch_pdl(naive_attn_sm100_kernel<128, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     }
-    return cudaGetLastError();
+    return launch_pdl(naive_attn_sm100_kernel<128, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+}
+
+cudaError_t set_attrs_naive_sm100() {
+    cudaError_t e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    return e;
 }
 
 cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const void* v_t, int H, int64_t Ls_pad,

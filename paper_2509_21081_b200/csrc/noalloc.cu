@@ -8,8 +8,12 @@
 // latency-critical loop in which cudaMalloc/cudaFree are banned because they
 // synchronise the device and take the driver's allocator lock.  For them this
 // file keeps the scratch in a fixed device array that is part of the library
-// image: it exists on every GPU that loads the library, from load to exit,
-// whether or not the entry point is ever called.
+// image.  CUDA loads the module that holds the array lazily, at the first
+// lookup of its address on a device, and loading it is what takes the 32 MiB
+// of device memory.  typhoon_mla_prepare_shared therefore does that lookup for
+// its device (preparing a prefix allocates anyway and happens before serving
+// starts); from then on the array stays until the process exits, and this
+// entry point only reads a cached pointer.
 #include <mutex>
 
 #include "handle.h"
@@ -29,47 +33,62 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 void* g_scratch_ptr[kMaxDevices] = {};
 
-int scratch_for_current_device(void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TYPHOON_MLA_ERR_CUDA;
+// Cached address for device `dev`, or null if it has not been resolved yet.
+void* cached_scratch(int dev) {
+    if (dev < 0 || dev >= kMaxDevices) return nullptr;
     std::lock_guard<std::mutex> lock(g_mu);
-    if (!g_scratch_ptr[dev]) {
-        void* p = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-        if (e != cudaSuccess || p == nullptr) {
-            cudaGetLastError();
-            return TYPHOON_MLA_ERR_CUDA;
-        }
-        g_scratch_ptr[dev] = p;
-    }
-    *out = g_scratch_ptr[dev];
-    return TYPHOON_MLA_OK;
+    return g_scratch_ptr[dev];
 }
 
 }  // namespace
 
+int tmla::noalloc_resolve_scratch_for_current_device() {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return api_cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return TYPHOON_MLA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_scratch_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return api_cuda_fail(e != cudaSuccess ? e : cudaErrorInvalidSymbol);
+        }
+        g_scratch_ptr[dev] = p;
+    }
+    return TYPHOON_MLA_OK;
+}
+
 extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, const void* q_nope, const void* q_pe,
                                                  int32_t B, float softmax_scale, void* out, float* lse_out,
                                                  void* stream) {
+    api_set_last_launches(0);
     if (!sh || !q_nope || !q_pe || !out || B < 1) return TYPHOON_MLA_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(q_nope) | reinterpret_cast<uintptr_t>(q_pe) | reinterpret_cast<uintptr_t>(out)) & 15u)
         return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || softmax_scale > 3.0e38f) return TYPHOON_MLA_ERR_INVALID_ARG;   // positive, finite
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return api_cuda_fail(e);
+    if (dev != sh->device) return TYPHOON_MLA_ERR_INVALID_ARG;   // the handle's caches live on another device
     const int H = sh->dims.num_heads;
     const size_t rows = (size_t)B * H;
     const size_t per_split = rows * 128 * sizeof(float) + ((rows * sizeof(float) + 255) / 256) * 256;
     if (per_split > kScratchBytes) return TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED;
 
-    void* scratch = nullptr;
-    int st = scratch_for_current_device(&scratch);
-    if (st != TYPHOON_MLA_OK) return st;
+    // resolved when the handle was prepared on this device
+    void* scratch = cached_scratch(sh->device);
+    if (!scratch) return TYPHOON_MLA_ERR_INVALID_ARG;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
     // As many KV splits as fit, up to what fills the GPU about four times over.
     int n_split = 0;
     if (sh->Ls > 0) {
+        const int n_sm = sh->num_sms > 0 ? sh->num_sms : 148;
         const int n_tiles = (int)((sh->Ls + 63) / 64);
         const int base = ((B + 63) / 64) * H;
-        int want = (4 * 148 + base - 1) / base;
+        int want = (4 * n_sm + base - 1) / base;
         int fit = (int)(kScratchBytes / per_split);
         n_split = want < fit ? want : fit;
         if (n_split > n_tiles) n_split = n_tiles;
@@ -82,12 +101,17 @@ extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, 
     // Every (split, request, head) slot that the combine reads is written by the attention
     // kernel of the same call (empty splits write lse = -inf), so nothing has to start at zero
     // and the previous call's contents never leak into this one.
+    tl_pdl = false;   // ordinary stream-ordered launches
+    int launches = 0;
     if (n_split > 0) {
         NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad, n_split,
                      softmax_scale, o_part, lse_part};
-        if (launch_naive_attn_mma(na, s) != cudaSuccess) return TYPHOON_MLA_ERR_CUDA;
+        e = launch_naive_attn_mma(na, s);
+        if (e != cudaSuccess) return api_cuda_fail(e);
+        ++launches;
     }
-    if (launch_combine(o_part, lse_part, n_split, nullptr, nullptr, B, H, out, lse_out, s) != cudaSuccess)
-        return TYPHOON_MLA_ERR_CUDA;
+    e = launch_combine(o_part, lse_part, n_split, nullptr, nullptr, B, H, out, lse_out, s);
+    if (e != cudaSuccess) return api_cuda_fail(e);
+    api_set_last_launches(launches + 1);
     return TYPHOON_MLA_OK;
 }

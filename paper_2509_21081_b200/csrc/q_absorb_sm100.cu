@@ -12,21 +12,6 @@
 #include "sm100.cuh"
 
 
-#ifdef TMLA_TRACE
-static __device__ unsigned long long g_kt_qabs[2] = {~0ull, 0ull};
-__device__ __forceinline__ unsigned long long kt_now_qabs() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define KT_BEGIN() do { if (threadIdx.x == 0) atomicMin(&g_kt_qabs[0], kt_now_qabs()); } while (0)
-#define KT_END() do { if (threadIdx.x == 0) atomicMax(&g_kt_qabs[1], kt_now_qabs()); } while (0)
-extern "C" int typhoon_mla_debug_kt_qabs(unsigned long long* out) {
-    cudaError_t e = cudaMemcpyFromSymbol(out, g_kt_qabs, 16);
-    unsigned long long init[2] = {~0ull, 0ull};
-    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_kt_qabs, init, 16);
-    return (int)e;
-}
-#else
-#define KT_BEGIN() do {} while (0)
-#define KT_END() do {} while (0)
-#endif
 
 namespace tmla {
 namespace {
@@ -57,7 +42,6 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     pdl_trigger();
     pdl_wait();
-    KT_BEGIN();
     if ((int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
         if (blockIdx.x == 0) {
             block_order_by_length(p.seq_lens, p.B, p.order, reinterpret_cast<unsigned long long*>(smem));
@@ -152,15 +136,18 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
-        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 4);
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, 4);
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
-    KT_END();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
 }  // namespace
+
+cudaError_t set_attrs_q_absorb_sm100() {
+    return cudaFuncSetAttribute(q_absorb_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+}
 
 cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w) {
     uint64_t dims[3] = {128, 512, (uint64_t)H};
@@ -182,7 +169,6 @@ cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, v
     const bool with_order = seq_lens != nullptr && order != nullptr && B <= 4096;
     QAbsorbParams p{q_abs, B, H, status, seq_lens, order, block_table, max_pages, page_size,
                     (with_order && block_table != nullptr) ? reinterpret_cast<int4*>(desc) : nullptr};
-    cudaFuncSetAttribute(q_absorb_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     dim3 grid((B + 127) / 128, H + (with_order ? 1 : 0), 1);
     return launch_pdl(q_absorb_sm100_kernel, grid, dim3(192), SMEM_BYTES, s, tm_q, *tm_w, p);
 }

@@ -39,7 +39,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // then skips its remaining work and falls through to the common teardown.
 // `abort_flag` lives in shared memory.
 constexpr long long kWaitDeadlineCycles = 2000000000LL;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long deadline_cycles = kWaitDeadlineCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -47,7 +48,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitDeadlineCycles) {
+            if (clock64() - t0 > deadline_cycles) {
                 *abort_flag = 1;
                 return false;
             }

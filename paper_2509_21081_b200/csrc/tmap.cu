@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "sm100.cuh"
@@ -28,6 +29,30 @@ cudaError_t make_tmap_bf16(CUtensorMap* out, const void* base, int rank, const u
     });
     if (!g_encode) return cudaErrorNotSupported;
     if (rank < 2 || rank > 5) return cudaErrorInvalidValue;
+    // A decode step re-creates the same handful of descriptors (queries, workspace buffers, page arrays)
+    // every call.  The encoding is a pure function of its arguments, so each host thread remembers the
+    // last few results and a repeated request costs one comparison instead of a driver call.
+    struct Key {
+        const void* base; int rank; uint64_t dims[5]; uint64_t strides[4]; uint32_t box[5];
+    };
+    struct Entry { Key key; CUtensorMap map; bool valid; };
+    constexpr int kCacheEntries = 32;
+    thread_local Entry cache[kCacheEntries] = {};
+    thread_local int next_slot = 0;
+    Key key;
+    std::memset(&key, 0, sizeof(key));
+    key.base = base; key.rank = rank;
+    for (int i = 0; i < rank; ++i) {
+        key.dims[i] = dims[i];
+        key.box[i] = box[i];
+        if (i > 0) key.strides[i - 1] = strides_bytes[i - 1];
+    }
+    for (int i = 0; i < kCacheEntries; ++i) {
+        if (cache[i].valid && std::memcmp(&cache[i].key, &key, sizeof(Key)) == 0) {
+            *out = cache[i].map;
+            return cudaSuccess;
+        }
+    }
     cuuint64_t gdim[5];
     cuuint64_t gstr[5];
     cuuint32_t bx[5], es[5];
@@ -40,7 +65,13 @@ cudaError_t make_tmap_bf16(CUtensorMap* out, const void* base, int rank, const u
     CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
                           bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    Entry& e = cache[next_slot];
+    next_slot = (next_slot + 1) % kCacheEntries;
+    e.key = key;
+    e.map = *out;
+    e.valid = true;
+    return cudaSuccess;
 }
 
 }  // namespace tmla

@@ -30,7 +30,7 @@ def run_gpu(inp, mode, page_size=None, pages=None, want_lse=True, poison=True, m
         out = dec.decode(inp.q_nope.to(dev), inp.q_pe.to(dev), pc.ckv_pages.to(dev), pc.kpe_pages.to(dev),
                          pc.block_table.to(dev), pc.seq_lens.to(dev), mode=mode, lse_out=lse)
     launches = b.typhoon_mla_last_launch_count()
-    assert b.typhoon_mla_device_status(dec.shared) == 0   # synchronises; raises if an in-kernel wait expired
+    assert b.typhoon_mla_check_status(dec.shared) == 0   # synchronises; raises if an in-kernel wait expired
     res = out.float().cpu().double().numpy(), (lse.cpu().double().numpy() if want_lse else None), launches
     dec.close()
     return res

@@ -226,7 +226,7 @@ def test_expansion_matches_plain_matmul():
     dims = b.make_dims(cfg.H)
     w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
     sh = b.typhoon_mla_prepare_shared(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
-    assert b.typhoon_mla_device_status(sh) == 0
+    assert b.typhoon_mla_check_status(sh) == 0
     k, vt = b.typhoon_mla_shared_export(sh)
     Ls, Lp, owned = b.typhoon_mla_shared_view(sh)
     torch.cuda.synchronize()
@@ -294,7 +294,7 @@ def test_decode_captured_in_a_cuda_graph(kernel_path):
     dec.decode(*args, mode=HYBRID, out=out)
     torch.cuda.synchronize()
     assert torch.equal(out, replayed) and not torch.equal(out, direct)
-    assert b.typhoon_mla_device_status(dec.shared) == 0
+    assert b.typhoon_mla_check_status(dec.shared) == 0
     dec.close()
 
 
@@ -328,7 +328,7 @@ def test_several_query_tokens_per_request(S_q):
         lse = torch.empty(B * S_q, H, dtype=torch.float32, device="cuda")
         out = dec.decode(rows.q_nope.cuda(), rows.q_pe.cuda(), pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), bt_rows,
                          sl_rows, mode=mode, lse_out=lse)
-        assert b.typhoon_mla_device_status(dec.shared) == 0
+        assert b.typhoon_mla_check_status(dec.shared) == 0
         G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse,
                         what=f"S_q={S_q} mode {mode}")
     dec.close()
@@ -406,7 +406,7 @@ def test_tree_of_shared_prefixes(case, kernel_path):
         else (None, None, 64, None, None)
     b.typhoon_mla_decode_tree(levels, inp.q_nope.to(dev), inp.q_pe.to(dev), *args, inp.scale, out, ws, lse_out=lse)
     for h in handles:
-        assert b.typhoon_mla_device_status(h) == 0
+        assert b.typhoon_mla_check_status(h) == 0
     G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse, what=f"tree: {case}")
     for h in handles:
         h.free()
@@ -441,7 +441,7 @@ def test_random_switches_repeatable_and_consistent(kernel_path):
             outs = {}
             for mode in (HYBRID, ABSORB):
                 o = [dec.decode(*args, mode=mode).clone() for _ in range(3)]
-                assert b.typhoon_mla_device_status(dec.shared) == 0, f"{cfg} mode {mode}"
+                assert b.typhoon_mla_check_status(dec.shared) == 0, f"{cfg} mode {mode}"
                 assert all(torch.equal(x, o[0]) for x in o[1:]), f"not repeatable: {cfg} mode {mode}"
                 assert torch.isfinite(o[0].float()).all(), f"non-finite: {cfg} mode {mode}"
                 outs[mode] = o[0].float()
@@ -495,7 +495,7 @@ def test_fused_page_layout_and_strides():
         lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
         out = dec.decode(inp.q_nope.cuda(), inp.q_pe.cuda(), ckv_view, kpe_view, pc.block_table.cuda(),
                          pc.seq_lens.cuda(), mode=mode, lse_out=lse)
-        assert b.typhoon_mla_device_status(dec.shared) == 0
+        assert b.typhoon_mla_check_status(dec.shared) == 0
         G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse,
                         what=f"fused layout mode {mode}")
     dec.close()
@@ -535,23 +535,79 @@ def _full_size_sampled(cfg, modes, n_pairs, extremes=False):
     return res
 
 
-def test_cfg1_full_size_sampled():
-    """DeepSeek-v3 dims, B=64, Ls=4096, Ln=512 -- the benchmark's launch configuration, checked on
-    sampled (request, head) rows computed one by one by the CPU checker."""
-    _full_size_sampled(I.CONFIGS["cfg1"], (HYBRID, ABSORB, AUTO), 48)
+def _checked_requests(cfg, inp, n_min=16):
+    """Requests whose rows the checker computes for ALL heads: the first and the last request of every
+    query-row group of the shared-prefix kernel, the rows on either side of a row-tile boundary, the
+    shortest and the longest suffix, and seeded random ones up to n_min."""
+    B = cfg.B
+    if B <= n_min:
+        return list(range(B))
+    chosen = {0, B - 1, int(np.argmin(inp.suffix_lens)), int(np.argmax(inp.suffix_lens))}
+    for g0 in range(0, B, 256):                      # a CTA of the 128-token-tile kernel owns 256 query rows ...
+        chosen |= {g0, min(g0 + 255, B - 1)}
+    chosen |= {min(127, B - 1), min(128, B - 1)}     # ... as two row tiles of 128
+    r = np.random.default_rng(cfg.seed + 17)
+    while len(chosen) < n_min:
+        chosen.add(int(r.integers(B)))
+    return sorted(chosen)
 
 
-def test_cfg3_kimi_like_sampled():
-    _full_size_sampled(I.CONFIGS["cfg3"], (HYBRID,), 24, extremes=True)
+def _full_size_all_heads(cfg, modes, kernel_path, all_rows=False):
+    """A benchmark configuration at full size, in the launch configuration the benchmark times: the float64
+    checker computes every head of the checked requests (every request with all_rows), so that every head,
+    every tile range and partial slot of the shared-prefix kernel and every query-row group is compared;
+    next to it the whole output tensor of the tcgen05 kernels is compared with that of the warp-MMA kernels
+    (both are checked against the float64 rows): a second net over the rows the checker does not reach."""
+    from paper_2509_21081_b200 import binding as b
+    if kernel_path != "tcgen05":
+        pytest.skip("both kernel paths run inside the tcgen05 parametrisation of this test")
+    inp = I.make_inputs(cfg)
+    reqs = list(range(cfg.B)) if all_rows else _checked_requests(cfg, inp)
+    pairs = [(r, h) for r in reqs for h in range(cfg.H)]
+    ref, ref_lse = G.run_oracle(inp, pairs=pairs)
+    mask = ~np.isnan(ref_lse)
+    assert mask.sum() == len(reqs) * cfg.H
+    for mode in modes:
+        outs = {}
+        for path in (b.PATH_TCGEN05, b.PATH_WARP_MMA):
+            b.typhoon_mla_set_kernel_path(path)
+            out, lse, _ = G.run_gpu(inp, mode)
+            assert np.isfinite(out).all()
+            G.assert_parity(out, ref, lse, ref_lse, mask=mask, what=f"{cfg.name} mode {mode} path {path}")
+            outs[path] = (out, lse)
+        b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05)
+        (o_t, l_t), (o_w, l_w) = outs[b.PATH_TCGEN05], outs[b.PATH_WARP_MMA]
+        # two implementations with different summation orders and both within the bars of the float64 rows:
+        # their difference over the whole tensor stays within twice those bars, row by row as well
+        d = np.abs(o_t - o_w)
+        assert d.max() <= 2 * G.MAX_ABS_TOL
+        rn = np.linalg.norm(o_w.reshape(-1, 128), axis=1)
+        re = np.linalg.norm((o_t - o_w).reshape(-1, 128), axis=1)
+        assert np.linalg.norm(o_t - o_w) / np.linalg.norm(o_w) <= 2 * G.REL_FRO_TOL
+        assert np.max(re / np.maximum(rn, 1e-30)) <= 8 * G.REL_FRO_TOL, f"{cfg.name} mode {mode}: worst row tcgen05 vs warp-MMA"
+        assert np.max(np.abs(l_t - l_w)) <= 2 * G.LSE_TOL
 
 
-def test_cfg2_long_prompt_sampled():
-    _full_size_sampled(I.CONFIGS["cfg2"], (HYBRID,), 16, extremes=True)
+def test_cfg1_full_size_all_rows(kernel_path):
+    """DeepSeek-v3 dims, B=64, Ls=4096, Ln=512 -- the benchmark's headline configuration: every
+    (request, head) row against the float64 checker, in the hybrid mode AUTO resolves to and absorb-only."""
+    _full_size_all_heads(I.CONFIGS["cfg1"], (AUTO, ABSORB), kernel_path, all_rows=True)
 
 
-@pytest.mark.parametrize("B", [1, 8, 128])
-def test_cfg4_fanout_sampled(B):
-    _full_size_sampled(I.CONFIGS["cfg4"].with_batch(B), (AUTO, HYBRID), 8)
+def test_cfg3_kimi_like_all_heads(kernel_path):
+    _full_size_all_heads(I.CONFIGS["cfg3"], (HYBRID,), kernel_path)
+
+
+def test_cfg2_long_prompt_all_heads(kernel_path):
+    _full_size_all_heads(I.CONFIGS["cfg2"], (HYBRID,), kernel_path)
+
+
+@pytest.mark.parametrize("B", [1, 8, 32, 128, 512, 1024])
+def test_cfg4_fanout_all_heads(B, kernel_path):
+    """The fan-out sweep at every batch size of the benchmark, in the mode AUTO picks (absorb-only at 1 and 8,
+    hybrid above) and, up to 128 requests, in the other one as well."""
+    modes = (AUTO,) if B > 128 else (AUTO, HYBRID if B <= 8 else ABSORB)
+    _full_size_all_heads(I.CONFIGS["cfg4"].with_batch(B), modes, kernel_path)
 
 
 def test_long_prefix_sampled():
@@ -589,7 +645,7 @@ def test_sequence_sharded_ranks_one_after_the_other(world, Ls):
         dec = S.SequenceShardedDecoder(r, world, cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(),
                                        inp.w_uv.cuda(), inp.scale, cfg.B, pc.block_table.shape[1])
         parts.append(dec.partial(*args, mode=AUTO if r % 2 else HYBRID))
-        assert b.typhoon_mla_device_status(dec.shared) == 0
+        assert b.typhoon_mla_check_status(dec.shared) == 0
         dec.close()
     lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
     out = S.merge_partials(torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]), lse)
@@ -609,7 +665,7 @@ def test_head_sharded_ranks_one_after_the_other(world, H):
         dec = S.HeadShardedDecoder(r, world, cfg.H, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(),
                                    inp.w_uv.cuda(), inp.scale, cfg.B, pc.block_table.shape[1])
         parts.append(dec.local(*args, mode=HYBRID))
-        assert b.typhoon_mla_device_status(dec.shared) == 0
+        assert b.typhoon_mla_check_status(dec.shared) == 0
         dec.close()
     out = S.join_heads(torch.stack(parts))
     G.assert_parity(out.float().cpu().double().numpy(), ref, what=f"head shards {world}")
@@ -655,7 +711,7 @@ def test_absorb_only_one_or_two_requests(B):
     l32 = torch.empty(B, cfg.H, dtype=torch.float32, device="cuda")
     b.typhoon_mla_decode_partial(dec.shared, *_upload(inp, pc)[:4], cfg.page_size, *_upload(inp, pc)[4:], inp.scale, o32, l32,
                                  dec.workspace, mode=ABSORB)
-    assert b.typhoon_mla_device_status(dec.shared) == 0
+    assert b.typhoon_mla_check_status(dec.shared) == 0
     G.assert_parity(o32.cpu().double().numpy(), ref, l32.cpu().double().numpy(), ref_lse, what=f"absorb-only fp32 B={B}")
     dec.close()
 
@@ -673,7 +729,7 @@ def test_partial_step_without_suffixes():
     l32 = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device="cuda")
     b.typhoon_mla_decode_partial(dec.shared, inp.q_nope.cuda(), inp.q_pe.cuda(), None, None, cfg.page_size, None, None,
                                  inp.scale, o32, l32, dec.workspace, mode=NAIVE)
-    assert b.typhoon_mla_device_status(dec.shared) == 0
+    assert b.typhoon_mla_check_status(dec.shared) == 0
     G.assert_parity(o32.cpu().double().numpy(), ref, l32.cpu().double().numpy(), ref_lse, what="fp32 partial, prefix only")
     dec.close()
 
@@ -716,7 +772,7 @@ def test_random_trees_against_per_group_steps(kernel_path):
         ws = torch.empty(b.typhoon_mla_tree_workspace_bytes(levels, B, pc.block_table.shape[1], 64), dtype=torch.uint8, device=dev)
         b.typhoon_mla_decode_tree(levels, args[0], args[1], args[2], args[3], 64, args[4], args[5], inp.scale, out, ws)
         handles = ([root] if root is not None else []) + [x for x in brs if x is not None]
-        assert b.typhoon_mla_device_status(handles[0]) == 0
+        assert b.typhoon_mla_check_status(handles[0]) == 0
         for gi in range(n_groups):
             r0, r1 = gb[gi], gb[gi + 1]
             dec = TyphoonMLADecoder(H, torch.cat([inp.ckv_shared, br_ckv[gi]]).to(dev), torch.cat([inp.kpe_shared, br_kpe[gi]]).to(dev),
@@ -761,7 +817,7 @@ def test_random_shards_against_the_whole_step():
         for r in range(world):
             d = S.SequenceShardedDecoder(r, world, H, *dev_in, inp.scale, B, pc.block_table.shape[1])
             parts.append(d.partial(*args, mode=rng.choice([AUTO, HYBRID, ABSORB])))
-            assert b.typhoon_mla_device_status(d.shared) == 0
+            assert b.typhoon_mla_check_status(d.shared) == 0
             d.close()
         lse = torch.empty(B, H, device=dev)
         out = S.merge_partials(torch.stack([p[0] for p in parts]), torch.stack([p[1] for p in parts]), lse).float()

@@ -20,14 +20,28 @@ def b():
     return binding
 
 
-def test_exports_every_declared_symbol(b):
-    hdr = open(os.path.join(ROOT, "include", "typhoon_mla.h")).read()
+def _declared(header):
+    hdr = open(os.path.join(ROOT, "include", header)).read()
     hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    names = set(re.findall(r"\b(typhoon_mla_[a-z_0-9]+)\s*\(", hdr))
-    assert {"typhoon_mla_prepare_shared", "typhoon_mla_decode", "typhoon_mla_free"} <= names
+    return set(re.findall(r"\b(typhoon_mla_[a-z_0-9]+)\s*\(", hdr))
+
+
+def test_exports_every_declared_symbol(b):
+    public, internal = _declared("typhoon_mla.h"), _declared("typhoon_mla_internal.h")
+    assert {"typhoon_mla_prepare_shared", "typhoon_mla_decode", "typhoon_mla_free", "typhoon_mla_workspace_bytes",
+            "typhoon_mla_choose_mode", "typhoon_mla_check_status", "typhoon_mla_status_string"} <= public
+    # process-wide switches and measurement hooks are not part of the public header
+    assert not {n for n in public if n.startswith("typhoon_mla_set_") and n not in
+                ("typhoon_mla_set_hw_model", "typhoon_mla_set_absorb_efficiency")}
+    assert not {n for n in public if "profile" in n or "debug" in n}
     lib = ctypes.CDLL(b.LIB_PATH)
-    for n in sorted(names):
-        assert hasattr(lib, n), f"{n} declared in the header but not exported"
+    for n in sorted(public | internal):
+        assert hasattr(lib, n), f"{n} declared in a header but not exported"
+    # and nothing is exported that no header declares
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", b.LIB_PATH], capture_output=True, text=True).stdout
+    exported = {ln.split()[-1] for ln in out.splitlines() if " T typhoon_mla_" in ln}
+    assert exported <= (public | internal), exported - (public | internal)
 
 
 def test_status_strings(b):
@@ -112,7 +126,7 @@ def test_crossover_rule(b):
 
 
 def test_pure_entry_points_reject_bad_arguments(b):
-    assert b._lib.typhoon_mla_workspace_bytes(None, 4, 4, 64) == 0
+    assert b._lib.typhoon_mla_workspace_bytes(None, 4, 4, 64, 0) == 0
     assert b._lib.typhoon_mla_free(None) == 0
     assert b.typhoon_mla_batch_threshold(b.make_dims(128), 0, 1.0, 1.0) < 0
     with pytest.raises(b.TyphoonMLAError):
