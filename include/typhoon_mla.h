@@ -336,17 +336,25 @@ int typhoon_mla_check_status(const typhoon_mla_shared_t* shared, void* stream, i
  * loop where cudaMalloc/cudaFree are forbidden because they synchronise the
  * device -- and therefore cannot pass a workspace.  The KV-split partials live
  * in a fixed array of TYPHOON_MLA_NOALLOC_SCRATCH_BYTES inside the library
- * image (each GPU that loads the library holds it until the process exits).
+ * image.  CUDA loads the part of the image that holds the array when its
+ * address is first looked up on a device, and it is that load which takes the
+ * 32 MiB of device memory: typhoon_mla_prepare_shared does the lookup (with
+ * its device current, checking the result), so the memory is taken while the
+ * caller is still setting up and allocation is still possible, and this entry
+ * point only reads a cached device pointer.  From then on every GPU on which
+ * a prefix was prepared holds the array until the process exits.
  *
  *   q_nope bf16 [B, H, 128], q_pe bf16 [B, H, 64], out bf16 [B, H, 128],
  *   lse_out optional fp32 [B, H]; all device pointers, 16-byte aligned.
  *
  * Limit: B * H * 516 bytes (rounded up to 256) must fit in the array, i.e.
  * B * H <= 65024 (B <= 508 at H = 128); larger problems are rejected with
- * TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED and nothing is launched.
- * The call uses no cudaMalloc/cudaFree and no allocating library routine.
- * The first call on each device looks up the array's device address
- * (cudaGetSymbolAddress, with that device current); make that first call
+ * TYPHOON_MLA_ERR_STATIC_SCRATCH_EXCEEDED, a bad scale or a handle of another
+ * device with INVALID_ARG; a rejected call launches nothing and writes nothing.
+ * The call uses no cudaMalloc/cudaFree and no allocating library routine, and
+ * runs the same shared-prefix kernel as typhoon_mla_decode (with fewer partial
+ * slots when the library's own choice would not fit the array).  Because the
+ * address lookup happens in typhoon_mla_prepare_shared, prepare the prefix
  * before any stream capture begins.  All calls on a device share the one
  * array, which keeps the previous call's contents; every slot a call reads it
  * has written itself, so no clearing is needed, but two calls whose kernels

@@ -1,6 +1,9 @@
 // Absorb attention over latent tokens (Algorithm 1 line 6) on tcgen05 / TMEM / TMA.
 //
-// Work item (CTA) = (request b, group of 64 heads, KV chunk).  The problem is run
+// Work item (CTA) = (64 query rows, KV chunk).  Over a request's own suffix the rows are 64 heads of that
+// request.  Over the shared prefix (absorb-only steps) every request attends to the same tokens, so the rows are
+// 64 consecutive rows of the stacked [B * H] query matrix: with fewer than 64 heads per request (a head-sharded
+// model) several requests fill one tile instead of each padding its own.  The problem is run
 // transposed so that the 64 x 512 latent accumulator fits tensor memory:
 //     S^T [64 tokens, 64 heads] = KV_tile [64, 576] * Q_g^T [576, 64]
 //     O^T [512 latent, 64 heads] += C_tile^T [512, 64 tokens] * P^T [64 tokens, 64 heads]
@@ -46,6 +49,8 @@ constexpr float kRescaleThreshold = 8.f;         // log2 units
 struct AbsorbSm100Params {
     int B, H;
     int chunk, n_shared_chunks, n_suffix_chunks;
+    int shared_groups;     // row groups per shared-prefix chunk
+    int stacked;           // shared-prefix row groups cut from the stacked [B * H] query matrix (else per request)
     int Ls_absorb;
     int page_size, max_pages;
     int num_pages;         // physical pages of the paged cache: ids outside [0, num_pages) are not dereferenced
@@ -109,19 +114,40 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
     pdl_trigger();
     pdl_wait();   // the descriptors and Q_A read below are written by the preceding kernel
-    const int chunk = blockIdx.x, h0 = blockIdx.y * 64;
-    // one 16-byte load gives the request, its suffix length and its first two pages (else three
-    // dependent loads stand between the kernel's start and its first copy)
-    int b, len_b = -1, pg0 = -1, pg1 = -1;
-    if (p.desc != nullptr) {
-        const int4 d = p.desc[blockIdx.z];
-        b = d.x; len_b = d.y; pg0 = d.z; pg1 = d.w;
+    // Work items in launch order: the shared-prefix items (chunk fastest, then row group), then the suffix items
+    // (chunk fastest, then head group, then request position in longest-first order).
+    const int n_shared_items = p.n_shared_chunks * p.shared_groups;
+    const bool shared_seg = (int)blockIdx.x < n_shared_items;
+    int chunk, row0, n_rows, b = 0, len_b = -1, pg0 = -1, pg1 = -1;
+    if (shared_seg) {
+        chunk = blockIdx.x % p.n_shared_chunks;
+        const int g = blockIdx.x / p.n_shared_chunks;
+        if (p.stacked) {                       // 64 consecutive rows of the stacked query matrix
+            row0 = g * 64;
+            n_rows = min(64, p.B * p.H - row0);
+        } else {                               // 64 heads of one request
+            const int hg = (p.H + 63) / 64;
+            b = g / hg;
+            row0 = b * p.H + (g % hg) * 64;
+            n_rows = min(64, p.H - (g % hg) * 64);
+        }
     } else {
-        b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
+        const int i = blockIdx.x - n_shared_items, hg = (p.H + 63) / 64;
+        chunk = p.n_shared_chunks + i % p.n_suffix_chunks;
+        const int y = (i / p.n_suffix_chunks) % hg, z = i / (p.n_suffix_chunks * hg);
+        // one 16-byte load gives the request, its suffix length and its first two pages (else three
+        // dependent loads stand between the kernel's start and its first copy)
+        if (p.desc != nullptr) {
+            const int4 d = p.desc[z];
+            b = d.x; len_b = d.y; pg0 = d.z; pg1 = d.w;
+        } else {
+            b = p.order ? p.order[z] : z;
+        }
+        row0 = b * p.H + y * 64;
+        n_rows = min(64, p.H - y * 64);
     }
 
     // token range of this chunk
-    const bool shared_seg = chunk < p.n_shared_chunks;
     int seg_len, tok_begin;
     if (shared_seg) {
         seg_len = p.Ls_absorb;
@@ -203,8 +229,8 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
         if (n_tiles > 0) {
             mbar_arrive_expect_tx_if(ld0, &sh->q_full, TILE_BYTES);
 #pragma unroll 1
-            for (int s = 0; s < 8; ++s) tma_load_3d_if(ld0, sQ + s * SLAB_BYTES, &tm_qa, &sh->q_full, s * 64, h0, b);
-            tma_load_3d_if(ld0, sQ + 8 * SLAB_BYTES, &tm_qp, &sh->q_full, 0, h0, b);
+            for (int s = 0; s < 8; ++s) tma_load_2d_if(ld0, sQ + s * SLAB_BYTES, &tm_qa, &sh->q_full, s * 64, row0);
+            tma_load_2d_if(ld0, sQ + 8 * SLAB_BYTES, &tm_qp, &sh->q_full, 0, row0);
             for (int j = 0; j < min(n_tiles, STAGES); ++j) {
                 int page, slot;
                 page_of(j, page, slot);
@@ -220,10 +246,12 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, sh->tmem_base, 0);
 
+    int tiles_issued = min(n_tiles, STAGES);   // producer warp: tiles whose copies were issued (upper bound), for the abort path
     if (n_tiles > 0) {
         if (warp == 0) {
             // ---------------- producer: the rest of the KV ring (Q and the first tiles are already in flight)
             for (int j = STAGES; j < n_tiles; ++j) {
+                tiles_issued = j + 1;
                 int page, slot;
                 page_of(j, page, slot);
                 bool ok = true;
@@ -296,7 +324,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             }
         } else if (warp >= 4) {
             // ---------------- softmax warpgroups
-            const int cg = (warp - 4) >> 2;                 // column group: heads h0 + 32 cg .. + 31
+            const int cg = (warp - 4) >> 2;                 // column group: query rows row0 + 32 cg .. + 31
             const int q = warp & 3;                         // TMEM lane quadrant of this warp
             const int bar_id = 1 + cg;
             const bool has_token = lane < 16;               // M = 64 layout: 16 token rows per quadrant
@@ -463,11 +491,11 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                 if (q == 0) {   // lane = head column: its inverse row sum and LSE
                     const float l = sh->red[cg][0][lane] + sh->red[cg][1][lane] + sh->red[cg][2][lane] + sh->red[cg][3][lane];
                     sh->inv[cg][lane] = 1.f / l;
-                    const int h = h0 + cg * 32 + lane;
-                    if (h < p.H) {
+                    const int r = cg * 32 + lane;
+                    if (r < n_rows) {
                         const float lse = (mref[lane] + log2f(l)) * kLn2;
-                        if (p.o_lat_direct) p.lse_direct[(int64_t)b * p.H + h] = lse;
-                        else p.lse_part[((int64_t)chunk * p.B + b) * p.H + h] = lse;
+                        if (p.o_lat_direct) p.lse_direct[row0 + r] = lse;
+                        else p.lse_part[(int64_t)chunk * p.B * p.H + row0 + r] = lse;
                     }
                 }
                 wg_sync(bar_id);
@@ -508,12 +536,10 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             // thread of the two warpgroups gets here: named barrier 3, 256 threads).
             asm volatile("bar.sync 3, 256;\n" ::: "memory");
             if (threadIdx.x == 128 && staged && !*abort_flag) {
-                const int n_heads = min(64, p.H - h0);
                 if (p.o_lat_direct) {
-                    bulk_store(p.o_lat_direct + ((int64_t)b * p.H + h0) * 512, sKV, (uint32_t)n_heads * 1024u);
+                    bulk_store(p.o_lat_direct + (int64_t)row0 * 512, sKV, (uint32_t)n_rows * 1024u);
                 } else {
-                    const int64_t row_base = ((int64_t)chunk * p.B + b) * p.H;
-                    bulk_store(p.o_part + (row_base + h0) * 512, sKV, (uint32_t)n_heads * 2048u);
+                    bulk_store(p.o_part + ((int64_t)chunk * p.B * p.H + row0) * 512, sKV, (uint32_t)n_rows * 2048u);
                 }
                 bulk_commit();
                 bulk_wait_read();   // the staging buffer must outlive the copy; the kernel end publishes the writes
@@ -522,14 +548,14 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     } else if (warp >= 4) {
         // empty chunk: weight zero in the merge
         const int i = threadIdx.x - 128;
-        if (i < 64 && h0 + i < p.H) {
+        if (i < n_rows) {
             if (p.o_lat_direct) {
                 // a request without any latent token: zero latent output, weight zero in the combine
-                p.lse_direct[(int64_t)b * p.H + h0 + i] = -INFINITY;
+                p.lse_direct[row0 + i] = -INFINITY;
                 for (int l = 0; l < 512; l += 8)
-                    *reinterpret_cast<uint4*>(p.o_lat_direct + ((int64_t)b * p.H + h0 + i) * 512 + l) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(p.o_lat_direct + (int64_t)(row0 + i) * 512 + l) = make_uint4(0, 0, 0, 0);
             } else {
-                p.lse_part[((int64_t)chunk * p.B + b) * p.H + h0 + i] = -INFINITY;
+                p.lse_part[(int64_t)chunk * p.B * p.H + row0 + i] = -INFINITY;
             }
         }
     }
@@ -538,8 +564,14 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
     __syncthreads();
     if (threadIdx.x == 0 && bad_page && p.status) atomicOr(p.status, 0x100);
     if (*abort_flag) {
+        // A wait gave up.  Before the CTA's shared memory is released the producer warp waits (with a limit) on the
+        // barriers of the tiles it issued last and of the query tile: only those copies can still be in flight.
+        if (warp == 0 && n_tiles > 0) {
+            for (int j = max(0, tiles_issued - STAGES); j < tiles_issued; ++j)
+                for (int g = 0; g < 4; ++g) mbar_drain(&sh->kv_full[j & 1][g], (j >> 1) & 1);
+            mbar_drain(&sh->q_full, 0);
+        }
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, 3);
-        for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
         __syncthreads();
     }
     if (warp == 1) tmem_dealloc(tmem_base, 512);
@@ -582,18 +614,19 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     if (a.B <= 0 || n_chunks <= 0) return cudaSuccess;
     if (a.chunk % TOK != 0) return cudaErrorInvalidValue;
     CUtensorMap tm_qa, tm_qp, tm_ckv_pg, tm_kpe_pg;
-    {
-        uint64_t dims[3] = {512, (uint64_t)a.H, (uint64_t)a.B};
-        uint64_t str[2] = {512 * 2, (uint64_t)a.H * 512 * 2};
-        uint32_t box[3] = {64, 64, 1};
-        cudaError_t e = make_tmap_bf16(&tm_qa, a.q_abs, 3, dims, str, box);
+    {   // the queries as one [B * H, 512] matrix: a box is 64 consecutive rows (of one request or across requests);
+        // rows past the end read as zeros
+        uint64_t dims[2] = {512, (uint64_t)a.H * (uint64_t)a.B};
+        uint64_t str[1] = {512 * 2};
+        uint32_t box[2] = {64, 64};
+        cudaError_t e = make_tmap_bf16(&tm_qa, a.q_abs, 2, dims, str, box);
         if (e != cudaSuccess) return e;
     }
     {
-        uint64_t dims[3] = {64, (uint64_t)a.H, (uint64_t)a.B};
-        uint64_t str[2] = {64 * 2, (uint64_t)a.H * 64 * 2};
-        uint32_t box[3] = {64, 64, 1};
-        cudaError_t e = make_tmap_bf16(&tm_qp, a.q_pe, 3, dims, str, box);
+        uint64_t dims[2] = {64, (uint64_t)a.H * (uint64_t)a.B};
+        uint64_t str[1] = {64 * 2};
+        uint32_t box[2] = {64, 64};
+        cudaError_t e = make_tmap_bf16(&tm_qp, a.q_pe, 2, dims, str, box);
         if (e != cudaSuccess) return e;
     }
     if (a.n_suffix_chunks > 0) {
@@ -608,6 +641,9 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     AbsorbSm100Params p{};
     p.B = a.B; p.H = a.H;
     p.chunk = a.chunk; p.n_shared_chunks = a.n_shared_chunks; p.n_suffix_chunks = a.n_suffix_chunks;
+    const int head_groups = (a.H + 63) / 64;
+    p.stacked = a.stacked ? 1 : 0;
+    p.shared_groups = a.stacked ? (int)(((int64_t)a.B * a.H + 63) / 64) : a.B * head_groups;
     p.Ls_absorb = a.Ls_absorb;
     p.page_size = a.page_size; p.max_pages = a.max_pages; p.num_pages = a.num_pages;
     p.block_table = a.block_table; p.seq_lens = a.seq_lens; p.order = a.order;
@@ -617,7 +653,7 @@ cudaError_t launch_absorb_attn_sm100(const AbsorbAttn& a, const CUtensorMap* tm_
     p.o_lat_direct = n_chunks == 1 ? reinterpret_cast<__nv_bfloat16*>(o_lat_direct) : nullptr;
     p.lse_direct = lse_direct;
     const int smem = kAbsorbSmem;
-    dim3 grid(n_chunks, (a.H + 63) / 64, a.B);
+    dim3 grid(a.n_shared_chunks * p.shared_groups + a.n_suffix_chunks * head_groups * a.B, 1, 1);
     const CUtensorMap* sh_c = a.n_shared_chunks > 0 ? tm_ckv_sh : &tm_ckv_pg;
     const CUtensorMap* sh_k = a.n_shared_chunks > 0 ? tm_kpe_sh : &tm_kpe_pg;
     return launch_pdl(absorb_attn_sm100_kernel, grid, dim3(384), smem, s, tm_qa, tm_qp, *sh_c, *sh_k, tm_ckv_pg, tm_kpe_pg, p);

@@ -104,8 +104,11 @@ int naive_splits(int B, int H, int64_t Ls, int n_sm) {
     return std::max(1, std::min({want, n_tiles, 64}));
 }
 
-void absorb_chunks(bool tc, int n_sm, int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chunk, int* n_sh, int* n_sf) {
+void absorb_chunks(bool tc, bool stacked, int n_sm, int B, int H, int64_t Ls_absorb, int64_t cap_suffix, int* chunk, int* n_sh,
+                   int* n_sf) {
     const int units = B * ((H + 63) / 64);
+    // CTAs per shared-prefix chunk: 64-row groups of the stacked [B * H] query matrix, or of each request
+    const int units_sh = (tc && stacked) ? (int)(((int64_t)B * H + 63) / 64) : units;
     const int64_t longest = std::max<int64_t>(std::max(Ls_absorb, cap_suffix), 1);
     int64_t c;
     if (tc) {
@@ -116,12 +119,13 @@ void absorb_chunks(bool tc, int n_sm, int B, int H, int64_t Ls_absorb, int64_t c
         c = round_up(longest, 64);
         for (int parts = 1; parts <= 512; ++parts) {
             const int64_t ch = round_up((longest + parts - 1) / parts, 64);
-            const int64_t ctas = (int64_t)units * ((Ls_absorb + ch - 1) / ch + (cap_suffix + ch - 1) / ch);
-            if (ctas / units > kMaxAbsorbChunks) continue;   // limit of the merge kernel
+            const int64_t per_req = (Ls_absorb + ch - 1) / ch + (cap_suffix + ch - 1) / ch;
+            const int64_t ctas = (int64_t)units_sh * ((Ls_absorb + ch - 1) / ch) + (int64_t)units * ((cap_suffix + ch - 1) / ch);
+            if (per_req > kMaxAbsorbChunks) continue;   // limit of the merge kernel
             const int64_t waves = (ctas + n_sm - 1) / n_sm;
             // a split segment writes and re-reads fp32 partials (64 heads x 2 KB, both ways): about 3.5 tiles
             // worth of traffic per chunk
-            const double split_cost = (ctas > units) ? 3.5 : 0.0;
+            const double split_cost = (per_req > 1) ? 3.5 : 0.0;
             const double cost = (double)waves * ((double)ch / 64.0 + fixed + split_cost);
             if (cost < best_cost - 1e-9) {
                 best_cost = cost;
@@ -141,7 +145,7 @@ void absorb_chunks(bool tc, int n_sm, int B, int H, int64_t Ls_absorb, int64_t c
 
 // `mode` is resolved (ABSORB, HYBRID or NAIVE); `tc` and `schedule` come from the caller's settings snapshot.
 Plan make_plan(const typhoon_mla_shared* sh, bool tc, int schedule, int B, int max_pages, int page_size, int mode,
-               int naive_slots_override = -1) {
+               int naive_slots_override = -1, bool stacked = true) {
     Plan p{};
     const int H = sh->dims.num_heads;
     const int n_sm = sh->num_sms > 0 ? sh->num_sms : kDefaultNumSM;
@@ -159,7 +163,7 @@ Plan make_plan(const typhoon_mla_shared* sh, bool tc, int schedule, int B, int m
         p.n_slots_naive = p.n_split_naive;
     }
     if (use_absorb) {
-        absorb_chunks(tc, n_sm, B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
+        absorb_chunks(tc, stacked, n_sm, B, H, mode == TYPHOON_MLA_MODE_ABSORB ? sh->Ls : 0, cap, &p.chunk, &p.n_shared_chunks,
                       &p.n_suffix_chunks);
     }
     const int n_chunks = p.n_shared_chunks + p.n_suffix_chunks;
@@ -289,9 +293,10 @@ int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int3
     const typhoon_mla_dims_t& d = *dims;
     const double H = d.num_heads, L = (double)Ls;
     const double f_naive = 2.0 * B * H * L * (d.d_nope + d.d_rope + d.d_v);
-    // (the absorb kernel works on groups of 64 heads: a partial group costs as much as a full one)
-    const double H_abs = std::ceil(H / 64.0) * 64.0;
-    const double f_absorb = 2.0 * B * H_abs * L * (2.0 * d.kv_lora_rank + d.d_rope);
+    // (the absorb kernel works on groups of 64 rows of the stacked [B * H] query matrix: a partial group costs as
+    // much as a full one)
+    const double rows_abs = std::ceil(B * H / 64.0) * 64.0;
+    const double f_absorb = 2.0 * rows_abs * L * (2.0 * d.kv_lora_rank + d.d_rope);
     const double by_naive = 2.0 * L * (H * (d.d_nope + d.d_v) + d.d_rope);
     const double by_absorb = 2.0 * L * (d.kv_lora_rank + d.d_rope);
     // The absorb kernel re-reads the prefix per request and runs M = 64 tiles: measured on B200 it
@@ -515,7 +520,8 @@ size_t typhoon_mla_workspace_bytes(const typhoon_mla_shared_t* sh, int32_t B, in
         const int pages = m == TYPHOON_MLA_MODE_NAIVE ? 0 : max_pages;
         for (bool tc : {true, false})
             for (int schedule : {0, 1, 2})
-                worst = std::max(worst, make_plan(sh, tc, schedule, B, pages, page_size, m).total);
+                for (bool stacked : {true, false})
+                    worst = std::max(worst, make_plan(sh, tc, schedule, B, pages, page_size, m, -1, stacked).total);
     }
     return worst + 256;
 }
@@ -635,7 +641,7 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         AbsorbAttn ab{q_abs, q_pe, sh->ckv, sh->kpe, mode == TYPHOON_MLA_MODE_ABSORB ? (int)sh->Ls : 0,
                       ckv_pages, kpe_pages, ckv_token_stride, kpe_token_stride, page_size, num_pages, block_table, max_pages,
                       seq_lens, order, desc, B, H, pl.chunk, pl.n_shared_chunks, pl.n_suffix_chunks, softmax_scale,
-                      o_part_a, lse_part_a, sh->status};
+                      o_part_a, lse_part_a, sh->status, cfg.stacked_absorb};
         prof_before(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
         e = tc ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, o_lat, lse_a, sh->status, s)
                : launch_absorb_attn_mma(ab, s);
@@ -719,7 +725,7 @@ static int decode_impl(const typhoon_mla_shared_t* sh, const void* q_nope, const
             return TYPHOON_MLA_ERR_INVALID_ARG;
     }
     if (mode == TYPHOON_MLA_MODE_NAIVE && sh->Ls == 0) max_pages = 0;
-    const Plan pl = make_plan(sh, cfg.tc(), cfg.naive_schedule, B, use_absorb ? max_pages : 0, page_size, mode);
+    const Plan pl = make_plan(sh, cfg.tc(), cfg.naive_schedule, B, use_absorb ? max_pages : 0, page_size, mode, -1, cfg.stacked_absorb);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return TYPHOON_MLA_ERR_INVALID_ARG;
     if (workspace_bytes < pl.total) return TYPHOON_MLA_ERR_WORKSPACE_TOO_SMALL;
 

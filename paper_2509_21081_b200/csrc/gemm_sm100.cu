@@ -64,12 +64,14 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_holder, 0);
 
+    int kb_issued = 0;   // producer warp: operand tiles issued (upper bound), for the abort path
     if (warp == 0) {
         // producer: the whole warp runs the loop, the elected lane issues
         const uint32_t ld = elect_one() ? 1u : 0u;
         for (int kb = 0; kb < KB; ++kb) {
             const int s = kb % STAGES;
             if (!mbar_wait_warp(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag)) break;
+            kb_issued = kb + 1;
             mbar_arrive_expect_tx_if(ld, &full[s], STAGE_BYTES);
             uint8_t* sa = smem + s * STAGE_BYTES;
             if (p.a_swap) tma_load_3d_if(ld, sa, &tmA, &full[s], kb * BK, z, m0);
@@ -203,10 +205,11 @@ __global__ void __launch_bounds__(192) gemm_tn_sm100_kernel(const __grid_constan
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
-        // A wait gave up: leave time for copies already in flight to land before the CTA's
-        // shared memory is released, and report.
+        // A wait gave up: before the CTA's shared memory is released the producer warp waits (with a limit) for the
+        // operand tiles it issued last, the only copies that can still be in flight; then report.
+        if (warp == 0)
+            for (int kb = max(0, kb_issued - STAGES); kb < kb_issued; ++kb) mbar_drain(&full[kb % STAGES], (kb / STAGES) & 1);
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, 1);
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
     if (warp == 1) tmem_dealloc(tmem_base, 128);

@@ -124,6 +124,7 @@ struct AbsorbAttn {
     float* o_part;   // [n_chunks][B][H][512], each normalised
     float* lse_part; // [n_chunks][B][H]
     int* status = nullptr;   // device word: bit 0x100 is set when a page id was out of range
+    bool stacked = false;    // tcgen05 kernel: shared-prefix chunks take 64-row groups of the stacked [B*H] queries
 };
 cudaError_t launch_absorb_attn_mma(const AbsorbAttn& p, cudaStream_t s);
 

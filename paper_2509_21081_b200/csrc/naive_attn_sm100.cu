@@ -77,7 +77,9 @@ struct Barriers {
     uint64_t q_full, q_free;
     uint64_t k_full[MAX_STAGES], k_empty[MAX_STAGES];
     uint64_t v_full[MAX_STAGES], v_empty[MAX_STAGES];
-    uint64_t s_ready[2][2], p_ready[2][2], sbuf_free[2][2], o_free[2];
+    // p_half (128-token tiles): the first 64 tokens' probabilities of a tile are in place, so the PV product can start
+    // on them while the softmax warpgroup is still working on the second 64
+    uint64_t s_ready[2][2], p_ready[2][2], p_half[2], sbuf_free[2][2], o_free[2];
     // 64-token tiles: stream 1 has published its softmax state (merge_m / merge_l) and its accumulator is
     // complete; stream 0 then merges the two streams' results into one partial (128 arrivals per segment)
     uint64_t merge_ready;
@@ -246,6 +248,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     // broadcast through a shuffle so that the compiler knows the value is warp-uniform
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
 
+    int k_issued = 0, v_issued = 0, q_issued = 0;   // producer warps: copies issued (upper bounds), for the abort path
     if (warp == 0) {
         // ---------------- Q + K producer
         int ring = 0, seg = 0;
@@ -271,6 +274,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             }
             g += s.cnt;
         }
+        k_issued = ring;
+        q_issued = max(seg, 1);
     } else if (warp == 2) {
         // ---------------- V producer
         const uint32_t ld = ld2;
@@ -285,6 +290,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             }
             g += s.cnt;
         }
+        v_issued = ring;
     } else if (warp == 1) {
         // ---------------- S = Q K^T issuer.  With two S buffers per stream it runs ahead of the softmax by
         // up to two steps; with one it follows the PV product of the previous step.
@@ -351,7 +357,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         if (!ok) break;
                     }
                     const int u = (i == 0 ? used0 : used1) + j;
-                    ok = mbar_wait_warp(&bar->p_ready[i][u % NB], (u / NB) & 1, abort_flag);
+                    ok = MODE_Y ? mbar_wait_warp(&bar->p_ready[i][u % NB], (u / NB) & 1, abort_flag)
+                                : mbar_wait_warp(&bar->p_half[i], u & 1, abort_flag);
                     if (!ok) break;
                     if (j == 0 && seg > 0) {   // the previous segment's epilogue has read this accumulator
                         ok = mbar_wait_warp(&bar->o_free[i], (seg - 1) & 1, abort_flag);
@@ -364,11 +371,17 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     const bool last_user = MODE_Y || i == 1 || s.n_str1 == 0;
 #pragma unroll
                     for (int bi = 0; bi < BLK; ++bi) {
+                        if (bi == 1) {   // second 64 tokens of a 128-token tile: the rest of the probabilities
+                            ok = mbar_wait_warp(&bar->p_ready[i][u % NB], (u / NB) & 1, abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
                         const uint64_t db = smem_desc_k_sw128(va + bi * 16384);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
                             umma_ts_if(ld, d, pa + 8 * (bi * 4 + k), db + 2 * k, idesc_o, (j | bi | k) != 0);
                     }
+                    if (!ok) break;
                     umma_commit_if(ld, &bar->o_done[i][u & 1]);
                     umma_commit_if(ld, &bar->sbuf_free[i][u % NB]);
                     if (last_user) umma_commit_if(ld, &bar->v_empty[st]);
@@ -397,7 +410,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const int b = lane_has_row ? tile_row0 + row : 0x3fffffff;
             const int nt = i == 0 ? s.n_str0 : s.n_str1;
             const bool warp_has_rows = tile_row0 + (M64 ? (warp & 3) * 16 : lg) < p.B;   // warp-uniform: the warp's first row is a real request
-            float m_ref = -INFINITY, l_sum = 0.f;
+            float m_ref = -INFINITY;
+            uint64_t l_sum2 = pack_f32x2(0.f, 0.f), l_sum2b = pack_f32x2(0.f, 0.f);   // row sum of the probabilities, as four partial sums
+            const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
             for (int j = 0; j < nt && ok; ++j) {
                 const int u = used + j;
                 const int buf = u % NB;
@@ -408,6 +423,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     // all 32 rows of this warp are padding past B: their P rows may hold anything (rows of
                     // the MMA are independent and these output rows are never stored); just keep in step
                     tc_fence_before();
+                    if (!MODE_Y) mbar_arrive(&bar->p_half[i]);
                     mbar_arrive(&bar->p_ready[i][buf]);
                     continue;
                 }
@@ -416,7 +432,10 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 const int valid = min(TOK, p.Ls - tile * TOK);
                 // pass 1: row maximum of the raw logits (the scale is positive, so it commutes with the
                 // maximum); the ragged tail is masked with -inf in place
-                float mx_raw = -INFINITY;
+                // (four independent running maxima and, below, two pairs of running sums: the tile's softmax is one
+                // link of the chain S product -> softmax -> PV product -> next S product of its stream, so the length
+                // of its dependent instruction chains counts, not only the number of instructions)
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 uint32_t sr[2][32];
 #pragma unroll
                 for (int half = 0; half < BLK; ++half) {
@@ -429,9 +448,11 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                             if (half * 64 + c >= valid) sr[c >> 5][c & 31] = 0xff800000u;   // -inf
                     }
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) mx_raw = fmaxf(mx_raw, __uint_as_float(sr[c >> 5][c & 31]));
+                    for (int c = 0; c < 64; c += 2)
+                        mx4[(c >> 1) & 3] = max3(mx4[(c >> 1) & 3], __uint_as_float(sr[c >> 5][c & 31]),
+                                                 __uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]));
                 }
-                const float mx = mx_raw * p.scale_log2;
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
                 // lazy rescale: only when some row's maximum grew by more than 2^8
                 const bool grow = lane_has_row && mx > m_ref + 8.f;
                 if (j == 0) {
@@ -444,7 +465,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     const float m_new = grow ? mx : m_ref;
                     const float f = fast_exp2(m_ref - m_new);
                     m_ref = m_new;
-                    l_sum *= f;
+                    l_sum2 = mul_f32x2(add_f32x2(l_sum2, l_sum2b), pack_f32x2(f, f));
+                    l_sum2b = pack_f32x2(0.f, 0.f);
                     const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)i * 128u;
 #pragma unroll 1
                     for (int c = 0; c < 4; ++c) {
@@ -460,37 +482,62 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 // pass 2: p = 2^(s * scale - m_ref) (one FMA and one ex2 per element), packed to bf16 over
                 // the S columns (P column c holds tokens 2c, 2c+1); with 128-token tiles the logits are read
                 // again, 64 at a time, to stay within the register budget
-                const float neg_m = -m_ref;
+                const uint64_t neg_m2 = pack_f32x2(-m_ref, -m_ref);
+                // probabilities of 32 logits held in `src`: 16 packed bf16 pairs, sums into the four partial sums
+                auto probs32 = [&](const uint32_t (&src)[32], uint32_t (&dst)[16]) {
 #pragma unroll
-                for (int half = 0; half < BLK; ++half) {
-                    if (BLK == 2) {
-                        tmem_ld32(s_addr + half * 64, sr[0]);
-                        tmem_ld32(s_addr + half * 64 + 32, sr[1]);
+                    for (int c = 0; c < 16; ++c) {
+                        // two logits per instruction: distance to the reference exponent, probabilities, running sums
+                        float x0, x1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(src[2 * c]), __uint_as_float(src[2 * c + 1])), scale2, neg_m2), x0, x1);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        dst[c] = pack_bf16(p0, p1);
+                        if (c & 1) l_sum2b = add_f32x2(l_sum2b, pack_f32x2(p0, p1));
+                        else l_sum2 = add_f32x2(l_sum2, pack_f32x2(p0, p1));
+                    }
+                };
+                if (BLK == 1) {
+                    // the 64 logits of pass 1 are still in registers
+                    uint32_t pk[2][16];
+                    probs32(sr[0], pk[0]);
+                    tmem_st16(s_addr, pk[0]);
+                    probs32(sr[1], pk[1]);
+                    tmem_st16(s_addr + 16, pk[1]);
+                } else {
+                    // 128-token tiles: the logits are read again, 32 at a time with the next 32 already requested, to stay
+                    // within the register budget.  Quarter q covers S columns [32 q, 32 q + 32) and writes P columns
+                    // [16 q, 16 q + 16): those overlap only S columns that are already in registers or consumed.
+                    tmem_ld32(s_addr, sr[0]);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
                         tmem_ld_wait();
+                        if (q < 3) tmem_ld32(s_addr + (q + 1) * 32, sr[(q + 1) & 1]);
                         if (valid < TOK) {
 #pragma unroll
-                            for (int c = 0; c < 64; ++c)
-                                if (half * 64 + c >= valid) sr[c >> 5][c & 31] = 0xff800000u;
+                            for (int c = 0; c < 32; ++c)
+                                if (q * 32 + c >= valid) sr[q & 1][c] = 0xff800000u;
+                        }
+                        uint32_t pk[16];
+                        probs32(sr[q & 1], pk);
+                        tmem_st16(s_addr + q * 16, pk);
+                        if (q == 1) {   // first half of the tile's probabilities in place
+                            tmem_st_wait();
+                            tc_fence_before();
+                            mbar_arrive(&bar->p_half[i]);
                         }
                     }
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[(2 * c) >> 5][(2 * c) & 31]), p.scale_log2, neg_m));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[(2 * c + 1) >> 5][(2 * c + 1) & 31]), p.scale_log2, neg_m));
-                        const uint32_t w = pack_bf16(p0, p1);
-                        pk[c] = w;
-                        l_sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
-                    }
-                    // in the 128-token case the second half's logits (S columns 64-127) are loaded before
-                    // P columns 32-63 are written, and P columns 0-31 only cover S columns already consumed
-                    tmem_st32(s_addr + half * 32, pk);
                 }
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(&bar->p_ready[i][buf]);
             }
             if (!ok) break;
+            float l_sum;
+            {
+                float a, c;
+                unpack_f32x2(add_f32x2(l_sum2, l_sum2b), a, c);
+                l_sum = a + c;
+            }
             // ---- segment epilogue: normalised partial + LSE into this segment's slot.  With 64-token tiles the two
             // streams worked on the same query rows: stream 1 publishes its softmax state, stream 0 merges both
             // accumulators (same tensor-memory lanes) and writes one partial.
@@ -574,8 +621,19 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
+        // A wait gave up.  Before the CTA's shared memory is released, each producer warp waits (with a limit) on the
+        // barriers of the ring positions it issued last: the copies against them are the only ones that can still be
+        // in flight.
+        if (warp == 0 && g_begin < g_end) {
+            for (int pos = max(0, k_issued - p.k_stages); pos < k_issued; ++pos)
+                mbar_drain(&bar->k_full[pos % p.k_stages], (pos / p.k_stages) & 1);
+            mbar_drain(&bar->q_full, (q_issued - 1) & 1);
+        }
+        if (warp == 2 && g_begin < g_end) {
+            for (int pos = max(0, v_issued - p.v_stages); pos < v_issued; ++pos)
+                mbar_drain(&bar->v_full[pos % p.v_stages], (pos / p.v_stages) & 1);
+        }
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
-        for (int k = 0; k < 64; ++k) __nanosleep(2000);   // let copies already in flight land
         __syncthreads();
     }
     if (warp == 1) tmem_dealloc(tmem_base, 512);

@@ -82,35 +82,33 @@ extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, 
     if (!scratch) return TYPHOON_MLA_ERR_INVALID_ARG;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
-    // As many KV splits as fit, up to what fills the GPU about four times over.
-    int n_split = 0;
+    // Work decomposition of the shared-prefix kernel (the same tcgen05 kernel the regular entry point runs): the
+    // library's choice if its partial slots fit the array, else one tile range per head, which needs one slot.
+    const int n_sm = sh->num_sms > 0 ? sh->num_sms : 148;
+    int n_ranges = 0, n_slots = 0;
     if (sh->Ls > 0) {
-        const int n_sm = sh->num_sms > 0 ? sh->num_sms : 148;
-        const int n_tiles = (int)((sh->Ls + 63) / 64);
-        const int base = ((B + 63) / 64) * H;
-        int want = (4 * n_sm + base - 1) / base;
-        int fit = (int)(kScratchBytes / per_split);
-        n_split = want < fit ? want : fit;
-        if (n_split > n_tiles) n_split = n_tiles;
-        if (n_split > 64) n_split = 64;
-        if (n_split < 1) n_split = 1;
+        naive_sm100_plan(B, H, sh->Ls, n_sm, 0, &n_ranges, &n_slots);
+        if ((size_t)n_slots * per_split > kScratchBytes) {
+            n_ranges = H;
+            n_slots = 1;
+        }
     }
     float* o_part = reinterpret_cast<float*>(scratch);
     float* lse_part = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(scratch) +
-                                               (size_t)(n_split > 0 ? n_split : 1) * rows * 128 * sizeof(float));
-    // Every (split, request, head) slot that the combine reads is written by the attention
-    // kernel of the same call (empty splits write lse = -inf), so nothing has to start at zero
-    // and the previous call's contents never leak into this one.
+                                               (size_t)(n_slots > 0 ? n_slots : 1) * rows * 128 * sizeof(float));
+    // Every (slot, request, head) entry that the combine reads is written by the attention kernel of the same
+    // call (slots a head does not use get lse = -inf), so nothing has to start at zero and the previous call's
+    // contents never leak into this one.
     tl_pdl = false;   // ordinary stream-ordered launches
     int launches = 0;
-    if (n_split > 0) {
-        NaiveAttn na{q_nope, q_pe, sh->k_nope, sh->v_t, sh->kpe, B, H, (int)sh->Ls, (int)sh->Ls_pad, n_split,
-                     softmax_scale, o_part, lse_part};
-        e = launch_naive_attn_mma(na, s);
+    if (n_slots > 0) {
+        NaiveAttnSm100 na{q_nope, q_pe, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt, B, H, (int)sh->Ls, n_ranges, n_slots,
+                          softmax_scale, o_part, lse_part, sh->status, B};
+        e = launch_naive_attn_sm100(na, s);
         if (e != cudaSuccess) return api_cuda_fail(e);
         ++launches;
     }
-    e = launch_combine(o_part, lse_part, n_split, nullptr, nullptr, B, H, out, lse_out, s);
+    e = launch_combine(o_part, lse_part, n_slots, nullptr, nullptr, B, H, out, lse_out, s);
     if (e != cudaSuccess) return api_cuda_fail(e);
     api_set_last_launches(launches + 1);
     return TYPHOON_MLA_OK;

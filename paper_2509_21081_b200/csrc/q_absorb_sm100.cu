@@ -136,8 +136,11 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
+        // A wait gave up: all copies of this CTA were issued up front against full[0..3]; wait for them (with a limit)
+        // before the shared memory is released, then report.
+        if (warp == 0)
+            for (int n = 0; n < 4; ++n) mbar_drain(&full[n], 0);
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, 4);
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
     if (warp == 1) tmem_dealloc(tmem_base, 512);

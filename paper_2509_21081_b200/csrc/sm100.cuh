@@ -56,6 +56,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
+// After a wait has given up: copies that were issued earlier may still be landing in this CTA's shared memory.
+// The producer waits, again with a limit (about a millisecond), for the phase `parity` of a barrier it issued
+// a copy against; it ignores the abort flag.  Used only on the way out of a CTA that abandons its work.
+__device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > 2000000LL) break;
+    }
+}
+
 // Warp-collective form: all 32 lanes poll, the result is made warp-uniform.  Role warps run
 // their loops with all lanes (uniform control flow lets the compiler keep descriptors, addresses
 // and coordinates in uniform registers) and elect one lane only for the issuing instruction.
@@ -245,6 +255,38 @@ __device__ __forceinline__ void tma_load_4d_if(uint32_t issue, void* dst, const 
         "@q cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n}\n" ::
             "r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(issue)
         : "memory");
+}
+
+// ---------------------------------------------------------------- packed fp32 arithmetic
+// Two fp32 lanes per instruction (sm_100): the softmax loops do their scale-and-subtract and their row sums
+// on pairs, which halves the issue slots those take next to the exponentials.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 // ---------------------------------------------------------------- TMEM <-> registers

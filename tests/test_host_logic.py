@@ -119,10 +119,14 @@ def test_crossover_rule(b):
     assert b.typhoon_mla_choose_mode_for(d, 16384, 8) == b.MODE_ABSORB
     assert b.typhoon_mla_choose_mode_for(d, 16384, 32) == b.MODE_HYBRID
     assert b.typhoon_mla_choose_mode_for(d, 16384, 512) == b.MODE_HYBRID
-    # 16 heads occupy a whole 64-head group of the absorb kernel: measured on B200 at L_s = 16384 the
-    # hybrid path wins from B = 16 (56 vs 72 us), which the rule has to reproduce
-    assert b.typhoon_mla_choose_mode_for(b.make_dims(16), 16384, 16) == b.MODE_HYBRID
-    assert b.typhoon_mla_choose_mode_for(b.make_dims(16), 16384, 2) == b.MODE_ABSORB
+    # The absorb kernel takes 64-row groups of the stacked [B * H] query matrix over the shared prefix, so with 16
+    # heads per device four requests share a group.  Measured on B200 at L_s = 16384, H = 16: absorb-only 42 / 50 /
+    # 56 / 77 us at B = 16 / 24 / 32 / 48 against 56 / 58 / 58 / 59 us hybrid; H = 32: 54 / 68 us at B = 16 / 24
+    # against 60 / 63; H = 48: 66 / 112 us at B = 16 / 32 against 93 / 96.  The rule has to reproduce the sides.
+    for H, B, want in ((16, 2, b.MODE_ABSORB), (16, 16, b.MODE_ABSORB), (16, 24, b.MODE_ABSORB), (16, 48, b.MODE_HYBRID),
+                       (32, 16, b.MODE_ABSORB), (32, 24, b.MODE_HYBRID), (48, 16, b.MODE_ABSORB), (48, 32, b.MODE_HYBRID),
+                       (128, 20, b.MODE_ABSORB), (128, 24, b.MODE_HYBRID)):
+        assert b.typhoon_mla_choose_mode_for(b.make_dims(H), 16384, B) == want, (H, B)
 
 
 def test_pure_entry_points_reject_bad_arguments(b):
