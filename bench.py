@@ -32,9 +32,9 @@ UNIT = "queries/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture
 # of that kernel at that configuration (key: (config, kernel)); None where no capture exists.
 NCU_TRAFFIC_BYTES = {
-    ("cfg1", "naive_attn"): 275_993_856,
-    ("cfg3", "absorb_attn"): 652_079_360,
-    ("cfg4_B512", "naive_attn"): 1_159_151_640,
+    ("cfg1", "naive_attn"): 275_997_696,
+    ("cfg3", "absorb_attn"): 652_403_968,
+    ("cfg4_B512", "naive_attn"): 1_163_312_528,
 }
 MIN_REGION_MS = 50.0      # every timed region is repeated until this much GPU time has been measured
 MAX_REPEATS = 400
@@ -298,7 +298,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         """Repeats the n-call region until MIN_REGION_MS of device time has been measured (at least 3
         times); returns the per-call times of the repeats."""
         runs, total = [], 0.0
-        while (total < MIN_REGION_MS or len(runs) < 3) and len(runs) < MAX_REPEATS:
+        while (total < MIN_REGION_MS or len(runs) < (3 if MIN_REGION_MS > 0 else 1)) and len(runs) < MAX_REPEATS:
             ms = region(fn, n)
             runs.append(ms / n)
             total += ms
@@ -431,7 +431,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         # regions of K steps (fork, K host-fed steps round robin over the lanes, join), repeated like the
         # device-resident regions; the median is reported
         e_runs, total = [], 0.0
-        while (total < MIN_REGION_MS or len(e_runs) < 3) and len(e_runs) < MAX_REPEATS:
+        while (total < MIN_REGION_MS or len(e_runs) < (3 if MIN_REGION_MS > 0 else 1)) and len(e_runs) < MAX_REPEATS:
             barrier()
             ev0.record()
             fork()
@@ -771,8 +771,11 @@ def main():
     ap.add_argument("--stages", action="store_true", help="also time every kernel of the step alone (implied by --sweep)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
+                    help="device time every timed region is repeated up to (0: each region once, e.g. under a profiler)")
     ap.add_argument("--no-extra", action="store_true", help="headline configuration only (skip the other configurations' short lines)")
     args = ap.parse_args()
+    globals()["MIN_REGION_MS"] = max(args.min_region_ms, 0.0)
 
     if args.impl == "reference":
         run_reference(args)

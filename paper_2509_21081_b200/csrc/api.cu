@@ -620,7 +620,7 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         prof_before(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (tc) {
             if (order) desc = reinterpret_cast<int32_t*>(ws + pl.off_desc);
-            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->status, order ? seq_lens : nullptr, order,
+            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->num_sms, sh->status, order ? seq_lens : nullptr, order,
                                       block_table, max_pages, page_size, desc, s);
         } else {
             GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,

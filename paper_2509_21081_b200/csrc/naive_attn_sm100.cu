@@ -410,7 +410,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const int b = lane_has_row ? tile_row0 + row : 0x3fffffff;
             const int nt = i == 0 ? s.n_str0 : s.n_str1;
             const bool warp_has_rows = tile_row0 + (M64 ? (warp & 3) * 16 : lg) < p.B;   // warp-uniform: the warp's first row is a real request
-            float m_ref = -INFINITY;
+            float m_ref = -INFINITY, m_ref_b = -INFINITY;   // (M = 64: reference exponents of this thread's rows A and B)
             uint64_t l_sum2 = pack_f32x2(0.f, 0.f), l_sum2b = pack_f32x2(0.f, 0.f);   // row sum of the probabilities, as four partial sums
             const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
             for (int j = 0; j < nt && ok; ++j) {
@@ -430,6 +430,85 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 const uint32_t s_addr = tmem_base + ((uint32_t)lg << 16) + s_col(i, u);
                 const int tile = tile_of(s, entry_of(j, i));
                 const int valid = min(TOK, p.Ls - tile * TOK);
+                if (M64) {
+                    // M = 64 accumulators: the warp's 16 rows sit in the first 16 lanes of its lane group.  They are
+                    // read as fragments, so that all 32 threads work: thread t holds 16 of the 64 logits of row
+                    // t/4 ("A") and of row t/4 + 8 ("B"), in column pairs 8g + 2(t%4) + {0, 1}, which are exactly the
+                    // token pairs that share a packed P column (4g + t%4).  Row maxima need two shuffles within the
+                    // four threads of a row; row sums stay per thread until the end of the segment.
+                    uint32_t sr[32];
+                    tmem_ld_16x256b_x8(s_addr, sr);
+                    tmem_ld_wait();
+                    const int q4 = lane & 3;
+                    if (valid < TOK) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (8 * (c >> 2) + 2 * q4 + (c & 1) >= valid) sr[c] = 0xff800000u;   // -inf
+                    }
+                    float mxa = -INFINITY, mxb = -INFINITY, mxa2 = -INFINITY, mxb2 = -INFINITY;
+#pragma unroll
+                    for (int gq = 0; gq < 8; gq += 2) {
+                        mxa = max3(mxa, __uint_as_float(sr[4 * gq]), __uint_as_float(sr[4 * gq + 1]));
+                        mxb = max3(mxb, __uint_as_float(sr[4 * gq + 2]), __uint_as_float(sr[4 * gq + 3]));
+                        mxa2 = max3(mxa2, __uint_as_float(sr[4 * gq + 4]), __uint_as_float(sr[4 * gq + 5]));
+                        mxb2 = max3(mxb2, __uint_as_float(sr[4 * gq + 6]), __uint_as_float(sr[4 * gq + 7]));
+                    }
+                    mxa = fmaxf(mxa, mxa2);
+                    mxb = fmaxf(mxb, mxb2);
+                    mxa = fmaxf(mxa, __shfl_xor_sync(0xffffffffu, mxa, 1));
+                    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, 1));
+                    mxa = fmaxf(mxa, __shfl_xor_sync(0xffffffffu, mxa, 2)) * p.scale_log2;
+                    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, 2)) * p.scale_log2;
+                    // lazy rescale: only when some row's maximum grew by more than 2^8
+                    const bool grow_a = mxa > m_ref + 8.f, grow_b = mxb > m_ref_b + 8.f;
+                    if (j == 0) {
+                        m_ref = mxa;
+                        m_ref_b = mxb;
+                    } else if (__any_sync(0xffffffffu, grow_a || grow_b)) {
+                        // the previous PV of this stream must have landed before O is touched
+                        ok = __all_sync(0xffffffffu, mbar_wait(&bar->o_done[i][(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const float fa = grow_a ? fast_exp2(m_ref - mxa) : 1.f, fb = grow_b ? fast_exp2(m_ref_b - mxb) : 1.f;
+                        if (grow_a) m_ref = mxa;
+                        if (grow_b) m_ref_b = mxb;
+                        l_sum2 = mul_f32x2(l_sum2, pack_f32x2(fa, fa));
+                        l_sum2b = mul_f32x2(l_sum2b, pack_f32x2(fb, fb));
+                        // the accumulator is rescaled row by row through the one-lane-per-thread shape: lane l < 16 of
+                        // the group holds row l, whose factor lives in the threads 4 (l % 8) .. + 3 (A for l < 8, else B)
+                        const float va = __shfl_sync(0xffffffffu, fa, 4 * (lane & 7)), vb = __shfl_sync(0xffffffffu, fb, 4 * (lane & 7));
+                        const float f = (lane & 8) ? vb : va;
+                        const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)i * 128u;
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t orr[32];
+                            tmem_ld32(o_addr + c * 32, orr);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int qq = 0; qq < 32; ++qq) orr[qq] = __float_as_uint(__uint_as_float(orr[qq]) * f);
+                            tmem_st32(o_addr + c * 32, orr);
+                        }
+                        tmem_st_wait();
+                    }
+                    const uint64_t nma = pack_f32x2(-m_ref, -m_ref), nmb = pack_f32x2(-m_ref_b, -m_ref_b);
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int gq = 0; gq < 8; ++gq) {
+                        float x0, x1, y0, y1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[4 * gq]), __uint_as_float(sr[4 * gq + 1])), scale2, nma), x0, x1);
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[4 * gq + 2]), __uint_as_float(sr[4 * gq + 3])), scale2, nmb), y0, y1);
+                        const float pa0 = fast_exp2(x0), pa1 = fast_exp2(x1), pb0 = fast_exp2(y0), pb1 = fast_exp2(y1);
+                        pk[2 * gq] = pack_bf16(pa0, pa1);          // row A, P column 4 gq + t%4
+                        pk[2 * gq + 1] = pack_bf16(pb0, pb1);      // row B, same column
+                        l_sum2 = add_f32x2(l_sum2, pack_f32x2(pa0, pa1));
+                        l_sum2b = add_f32x2(l_sum2b, pack_f32x2(pb0, pb1));
+                    }
+                    tmem_st_16x128b_x8(s_addr, pk);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    mbar_arrive(&bar->p_ready[i][buf]);
+                    continue;
+                }
                 // pass 1: row maximum of the raw logits (the scale is positive, so it commutes with the
                 // maximum); the ragged tail is masked with -inf in place
                 // (four independent running maxima and, below, two pairs of running sums: the tile's softmax is one
@@ -533,7 +612,23 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             }
             if (!ok) break;
             float l_sum;
-            {
+            if (M64) {
+                // this thread's partial sums of rows A and B -> whole-row sums (four threads per row), then the values
+                // of the row that the one-lane-per-thread epilogue below handles in this lane: lane l < 16 holds row l
+                float a0, a1, b0, b1;
+                unpack_f32x2(l_sum2, a0, a1);
+                unpack_f32x2(l_sum2b, b0, b1);
+                float la = a0 + a1, lb = b0 + b1;
+                la += __shfl_xor_sync(0xffffffffu, la, 1);
+                lb += __shfl_xor_sync(0xffffffffu, lb, 1);
+                la += __shfl_xor_sync(0xffffffffu, la, 2);
+                lb += __shfl_xor_sync(0xffffffffu, lb, 2);
+                const int src = 4 * (lane & 7);
+                const float la_r = __shfl_sync(0xffffffffu, la, src), lb_r = __shfl_sync(0xffffffffu, lb, src);
+                const float ma_r = __shfl_sync(0xffffffffu, m_ref, src), mb_r = __shfl_sync(0xffffffffu, m_ref_b, src);
+                l_sum = (lane & 8) ? lb_r : la_r;
+                m_ref = (lane & 8) ? mb_r : ma_r;
+            } else {
                 float a, c;
                 unpack_f32x2(add_f32x2(l_sum2, l_sum2b), a, c);
                 l_sum = a + c;

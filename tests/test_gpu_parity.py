@@ -835,3 +835,23 @@ def test_random_shards_against_the_whole_step():
                 d.close()
             o2 = S.join_heads(torch.stack(halves)).float()
             assert float((o2 - ref).abs().max()) / scale < 2e-2, (it, "heads")
+
+
+@pytest.mark.parametrize("H,B", [(16, 7), (16, 37), (48, 5), (32, 64), (64, 3)])
+def test_absorb_row_groups_stacked_and_per_request(H, B, kernel_path):
+    """Absorb-only steps over the shared prefix take 64-row groups of the stacked [B * H] query matrix (requests
+    share a tile when a device has fewer than 64 heads) or, with the switch off, of every request: both against
+    the checker, with ragged suffixes so that the per-request suffix items run next to the stacked prefix items."""
+    from paper_2509_21081_b200 import binding as b
+    if kernel_path != "tcgen05":
+        pytest.skip("row groups are a property of the tcgen05 kernel")
+    cfg = _cfg("stack", B=B, H=H, Ls=1100, lo=0, hi=150, seed=300 + H + B)
+    inp = I.make_inputs(cfg)
+    ref, ref_lse = G.run_oracle(inp)
+    try:
+        for stacked in (True, False):
+            b.typhoon_mla_set_stacked_absorb(stacked)
+            out, lse, _ = G.run_gpu(inp, ABSORB)
+            G.assert_parity(out, ref, lse, ref_lse, what=f"H={H} B={B} stacked={stacked}")
+    finally:
+        b.typhoon_mla_set_stacked_absorb(True)
