@@ -30,15 +30,15 @@ cudaError_t make_tmap_bf16(CUtensorMap* out, const void* base, int rank, const u
     if (!g_encode) return cudaErrorNotSupported;
     if (rank < 2 || rank > 5) return cudaErrorInvalidValue;
     // A decode step re-creates the same handful of descriptors (queries, workspace buffers, page arrays)
-    // every call.  The encoding is a pure function of its arguments, so each host thread remembers the
-    // last few results and a repeated request costs one comparison instead of a driver call.
+    // every call.  The encoding is a pure function of its arguments, so each host thread remembers results in a
+    // direct-mapped table (a serving loop with several steps in flight has a few dozen live descriptors) and a
+    // repeated request costs one hash and one comparison instead of a driver call.
     struct Key {
         const void* base; int rank; uint64_t dims[5]; uint64_t strides[4]; uint32_t box[5];
     };
     struct Entry { Key key; CUtensorMap map; bool valid; };
-    constexpr int kCacheEntries = 32;
+    constexpr int kCacheEntries = 256;
     thread_local Entry cache[kCacheEntries] = {};
-    thread_local int next_slot = 0;
     Key key;
     std::memset(&key, 0, sizeof(key));
     key.base = base; key.rank = rank;
@@ -47,11 +47,15 @@ cudaError_t make_tmap_bf16(CUtensorMap* out, const void* base, int rank, const u
         key.box[i] = box[i];
         if (i > 0) key.strides[i - 1] = strides_bytes[i - 1];
     }
-    for (int i = 0; i < kCacheEntries; ++i) {
-        if (cache[i].valid && std::memcmp(&cache[i].key, &key, sizeof(Key)) == 0) {
-            *out = cache[i].map;
-            return cudaSuccess;
-        }
+    uint64_t hsh = 1469598103934665603ull;   // FNV-1a over the key's bytes
+    {
+        const unsigned char* kb = reinterpret_cast<const unsigned char*>(&key);
+        for (size_t i = 0; i < sizeof(Key); ++i) hsh = (hsh ^ kb[i]) * 1099511628211ull;
+    }
+    Entry& slot = cache[(hsh ^ (hsh >> 17)) % kCacheEntries];
+    if (slot.valid && std::memcmp(&slot.key, &key, sizeof(Key)) == 0) {
+        *out = slot.map;
+        return cudaSuccess;
     }
     cuuint64_t gdim[5];
     cuuint64_t gstr[5];
@@ -66,11 +70,9 @@ cudaError_t make_tmap_bf16(CUtensorMap* out, const void* base, int rank, const u
                           bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    Entry& e = cache[next_slot];
-    next_slot = (next_slot + 1) % kCacheEntries;
-    e.key = key;
-    e.map = *out;
-    e.valid = true;
+    slot.key = key;
+    slot.map = *out;
+    slot.valid = true;
     return cudaSuccess;
 }
 
