@@ -327,59 +327,71 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             const int cg = (warp - 4) >> 2;                 // column group: query rows row0 + 32 cg .. + 31
             const int q = warp & 3;                         // TMEM lane quadrant of this warp
             const int bar_id = 1 + cg;
-            const bool has_token = lane < 16;               // M = 64 layout: 16 token rows per quadrant
-            const int r = 16 * q + lane;                    // token row within the tile (valid when has_token)
+            // S^T has M = 64: the 16 token rows of this warp's quadrant sit in its first 16 tensor-memory lanes.  They
+            // are read as fragments so that all 32 threads work: thread t holds, for the tokens ra = 16 q + t/4 and
+            // rb = ra + 8, the logits of the columns 8g + 2(t%4) + {0, 1} (g = 0..3) of this warpgroup's 32 columns.
+            const int qq = lane & 3;
+            const int ra = 16 * q + (lane >> 2), rb = ra + 8;
             const uint32_t lane_base = (uint32_t)(32 * q) << 16;
-            // Per-thread state: partial row sums of this thread's token slot.  The reference exponents
-            // are the same for every thread of the warpgroup and live in shared memory.
-            float l_part[32];
+            // Per-thread state: partial sums of this thread's eight columns over its two token rows.  The reference
+            // exponents are the same for every thread of the warpgroup and live in shared memory.
+            float l_part[8];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) l_part[c] = 0.f;
+            for (int c = 0; c < 8; ++c) l_part[c] = 0.f;
             volatile float* mref = sh->mref[cg];
             if (q == 0) mref[lane] = -INFINITY;
             wg_sync(bar_id);
-            float neg_mr[32];      // register copy of -m_ref, refreshed after every rescale event
+            float neg_mr[8];       // register copy of -m_ref of this thread's columns, refreshed after every rescale event
 #pragma unroll
-            for (int c = 0; c < 32; ++c) neg_mr[c] = INFINITY;
+            for (int c = 0; c < 8; ++c) neg_mr[c] = INFINITY;
 
             for (int j = 0; j < n_tiles; ++j) {
                 const int s = j & 1;
                 bool ok = __all_sync(0xffffffffu, mbar_wait(&sh->s_ready[s], (j >> 1) & 1, abort_flag));
                 const int t0 = tok_begin + j * TOK;
                 const int n_valid = min(TOK, tok_end - t0);
-                const bool valid = has_token && r < n_valid;
-                uint32_t sr[32], pk[16];
+                uint32_t sr[16], pka[4], pkb[4];   // logits; packed probabilities of row a / row b (columns 8g+2qq, +1)
                 bool exceed = false;
                 if (ok) {
                     tc_fence_after();
-                    tmem_ld32(tmem_base + lane_base + (uint32_t)(s * 64 + cg * 32), sr);
+                    tmem_ld_16x256b_x4(tmem_base + lane_base + (uint32_t)(s * 64 + cg * 32), sr);
                     tmem_ld_wait();
                     // one pass: distance of the scaled logit to the reference (one FMA), probability
-                    // (speculative: final unless the warpgroup votes for a rescale).  Lanes without a valid
-                    // token carry -inf.
-                    if (!valid) {
+                    // (speculative: final unless the warpgroup votes for a rescale).  Token rows past the end
+                    // carry -inf.
+                    if (ra >= n_valid) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) sr[c] = 0xff800000u;
+                        for (int g = 0; g < 4; ++g) sr[4 * g] = sr[4 * g + 1] = 0xff800000u;
+                    }
+                    if (rb >= n_valid) {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) sr[4 * g + 2] = sr[4 * g + 3] = 0xff800000u;
                     }
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float d0 = fmaf(__uint_as_float(sr[2 * c]), p.scale_log2, neg_mr[2 * c]);
-                        const float d1 = fmaf(__uint_as_float(sr[2 * c + 1]), p.scale_log2, neg_mr[2 * c + 1]);
-                        exceed |= (d0 > kRescaleThreshold) | (d1 > kRescaleThreshold);
-                        pk[c] = pack_bf16(fast_exp2(d0), fast_exp2(d1));
+                    for (int g = 0; g < 4; ++g) {
+                        const float a0 = fmaf(__uint_as_float(sr[4 * g]), p.scale_log2, neg_mr[2 * g]);
+                        const float a1 = fmaf(__uint_as_float(sr[4 * g + 1]), p.scale_log2, neg_mr[2 * g + 1]);
+                        const float b0 = fmaf(__uint_as_float(sr[4 * g + 2]), p.scale_log2, neg_mr[2 * g]);
+                        const float b1 = fmaf(__uint_as_float(sr[4 * g + 3]), p.scale_log2, neg_mr[2 * g + 1]);
+                        exceed |= (a0 > kRescaleThreshold) | (a1 > kRescaleThreshold) | (b0 > kRescaleThreshold) | (b1 > kRescaleThreshold);
+                        pka[g] = pack_bf16(fast_exp2(a0), fast_exp2(a1));
+                        pkb[g] = pack_bf16(fast_exp2(b0), fast_exp2(b1));
                     }
                 }
                 const bool rescale = wg_vote_or(bar_id, exceed);
                 if (*abort_flag) break;                      // uniform across the warpgroup after the barrier
                 if (rescale) {
-                    // exact column maxima of this tile across the 64 token lanes: warp-wide integer max of
-                    // order-preserving keys, then across the four warps through shared memory
+                    // exact column maxima of this tile across the 64 token rows: over this thread's two rows, then
+                    // over the eight threads of the warp that hold the same columns (lanes t%4 equal), then across the
+                    // four warps through shared memory
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const int bits = __float_as_int(__uint_as_float(sr[c]) * p.scale_log2);
-                        const int key = bits >= 0 ? bits : bits ^ 0x7fffffff;
-                        const int mk = __reduce_max_sync(0xffffffffu, key);
-                        if (lane == c) sh->red[cg][q][c] = __int_as_float(mk >= 0 ? mk : mk ^ 0x7fffffff);
+                    for (int c = 0; c < 8; ++c) {
+                        const int g = c >> 1, e = c & 1;
+                        float v = fmaxf(__uint_as_float(sr[4 * g + e]), __uint_as_float(sr[4 * g + 2 + e])) * p.scale_log2;
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 4));
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 8));
+                        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 16));
+                        if (lane < 4) sh->red[cg][q][8 * g + 2 * qq + e] = v;
                     }
                     wg_sync(bar_id);
                     const float cm = fmaxf(fmaxf(sh->red[cg][0][lane], sh->red[cg][1][lane]), fmaxf(sh->red[cg][2][lane], sh->red[cg][3][lane]));
@@ -390,7 +402,7 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     if (q == 0) mref[lane] = m_new;
                     wg_sync(bar_id);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) l_part[c] *= __shfl_sync(0xffffffffu, f_lane, c);
+                    for (int c = 0; c < 8; ++c) l_part[c] *= __shfl_sync(0xffffffffu, f_lane, 8 * (c >> 1) + 2 * qq + (c & 1));
                     if (j > 0) {
                         // rescale this column group's 32 columns of all four O^T blocks (all 128 lanes), once
                         // the previous tile's accumulation has landed
@@ -412,27 +424,26 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
                     }
                     // probabilities again, against the new references
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) neg_mr[c] = -mref[c];
+                    for (int c = 0; c < 8; ++c) neg_mr[c] = -mref[8 * (c >> 1) + 2 * qq + (c & 1)];
 #pragma unroll
-                    for (int c = 0; c < 16; ++c)
-                        pk[c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(sr[2 * c]), p.scale_log2, neg_mr[2 * c])),
-                                          fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1]), p.scale_log2, neg_mr[2 * c + 1])));
+                    for (int g = 0; g < 4; ++g) {
+                        pka[g] = pack_bf16(fast_exp2(fmaf(__uint_as_float(sr[4 * g]), p.scale_log2, neg_mr[2 * g])),
+                                           fast_exp2(fmaf(__uint_as_float(sr[4 * g + 1]), p.scale_log2, neg_mr[2 * g + 1])));
+                        pkb[g] = pack_bf16(fast_exp2(fmaf(__uint_as_float(sr[4 * g + 2]), p.scale_log2, neg_mr[2 * g])),
+                                           fast_exp2(fmaf(__uint_as_float(sr[4 * g + 3]), p.scale_log2, neg_mr[2 * g + 1])));
+                    }
                 }
-                // per-thread partial row sums (of the bf16-rounded values), P^T row into the rope slab
+                // per-thread partial column sums (of the bf16-rounded values), P^T into the rope slab
                 uint8_t* tile = sKV + s * TILE_BYTES;
-                if (has_token) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        l_part[2 * c] += __uint_as_float(pk[c] << 16);
-                        l_part[2 * c + 1] += __uint_as_float(pk[c] & 0xffff0000u);
-                    }
-                    // MN-major P^T: row r (token) = 64 heads = 128 bytes, 16-byte chunks swizzled by r & 7
-                    uint8_t* prow = tile + 8 * SLAB_BYTES + r * 128;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int ch = (cg * 4 + i) ^ (r & 7);
-                        *reinterpret_cast<uint4*>(prow + ch * 16) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-                    }
+                for (int g = 0; g < 4; ++g) {
+                    l_part[2 * g] += __uint_as_float(pka[g] << 16) + __uint_as_float(pkb[g] << 16);
+                    l_part[2 * g + 1] += __uint_as_float(pka[g] & 0xffff0000u) + __uint_as_float(pkb[g] & 0xffff0000u);
+                    // MN-major P^T: row (token) = 64 heads = 128 bytes, 16-byte chunks swizzled by row & 7; this
+                    // thread's column pair is word qq of chunk cg * 4 + g (the four threads of a row fill the chunk)
+                    const int ch = cg * 4 + g;
+                    *reinterpret_cast<uint32_t*>(tile + 8 * SLAB_BYTES + ra * 128 + ((ch ^ (ra & 7)) * 16) + qq * 4) = pka[g];
+                    *reinterpret_cast<uint32_t*>(tile + 8 * SLAB_BYTES + rb * 128 + ((ch ^ (rb & 7)) * 16) + qq * 4) = pkb[g];
                 }
                 if (n_valid < TOK) {
                     // ragged tail: latent rows of tokens past the end may hold anything (even NaN);
@@ -454,38 +465,16 @@ absorb_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid
             // warpgroup reaches the same named barriers)
             bool staged = false;
             if (!wg_vote_or(bar_id, *abort_flag != 0)) {
-                // Row sums first (they do not depend on the accumulator, whose last product is still
-                // running): a transposing butterfly over the 32 lanes leaves lane c with column c's sum
-                // over this warp's token rows (31 shuffles), then the four warps add up through shared memory.
-                float a16[16], a8[8], a4[4], a2[2];
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const bool up = (lane & 16) != 0;
-                    const float keep = up ? l_part[c + 16] : l_part[c], send = up ? l_part[c] : l_part[c + 16];
-                    a16[c] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-                }
+                // Column sums first (they do not depend on the accumulator, whose last product is still running):
+                // over the eight threads of the warp that hold the same columns, then the four warps add up through
+                // shared memory.
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    const bool up = (lane & 8) != 0;
-                    const float keep = up ? a16[c + 8] : a16[c], send = up ? a16[c] : a16[c + 8];
-                    a8[c] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const bool up = (lane & 4) != 0;
-                    const float keep = up ? a8[c + 4] : a8[c], send = up ? a8[c] : a8[c + 4];
-                    a4[c] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-                }
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    const bool up = (lane & 2) != 0;
-                    const float keep = up ? a4[c + 2] : a4[c], send = up ? a4[c] : a4[c + 2];
-                    a2[c] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-                }
-                {
-                    const bool up = (lane & 1) != 0;
-                    const float keep = up ? a2[1] : a2[0], send = up ? a2[0] : a2[1];
-                    sh->red[cg][q][lane] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+                    float v = l_part[c];
+                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                    if (lane < 4) sh->red[cg][q][8 * (c >> 1) + 2 * qq + (c & 1)] = v;
                 }
                 wg_sync(bar_id);
                 if (q == 0) {   // lane = head column: its inverse row sum and LSE
