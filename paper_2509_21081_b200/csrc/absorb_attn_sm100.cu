@@ -22,7 +22,9 @@
 // Warp roles (384 threads): warp 0 = TMA producer (Q once, KV ring), warp 1 =
 // S^T issuer and TMEM owner, warp 3 = O^T issuer, warps 4-7 / 8-11 = softmax
 // warpgroup for head columns 0-31 / 32-63.  S^T uses M = 64: token row r lives in
-// TMEM lane 32 (r / 16) + r % 16, so lanes 0-15 of every softmax warp own a token.
+// TMEM lane 32 (r / 16) + r % 16, i.e. in the first 16 lanes of a warp's lane
+// group.  The softmax warps read it with the 16-lane fragment shape, so that all 32
+// threads hold logits: two token rows and eight columns each.
 //
 // Tensor memory (512 columns allocated): S^T[buf] at 64 buf (2 buffers), O^T block
 // m (128 latent rows x 64 heads) at 128 + 64 m.
