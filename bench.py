@@ -393,11 +393,14 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     # ---- end to end: per-step tensors from pinned host memory, result read back, every step
     e2e = None
     if with_e2e:
-        # Eight steps are kept in flight ("lanes"), each on its own stream with its own decoder (prepared
+        # Twelve steps are kept in flight ("lanes"), each on its own stream with its own decoder (prepared
         # prefix, workspace, staging) and pinned buffers, so that the copies of one step overlap the kernels
         # of the others, as a serving loop with several micro-batches would do.  Every step still copies
         # its inputs in and its result out.  Lane k reads the device-resident caches of input set k % 2.
-        n_lanes = int(os.environ.get("TYPHOON_MLA_BENCH_LANES", "8"))
+        # (A lane's copy out waits for its kernels, and the copy queues run in submission order, so with only
+        # a few lanes the next lanes' copies in sit behind it: measured 237-250 / 180 / 105-147 / 95 / 95 us per
+        # step with 2 / 4 / 6 / 8 / 12 lanes on one GPU.)
+        n_lanes = int(os.environ.get("TYPHOON_MLA_BENCH_LANES", "12"))
         lanes = []
         for k in range(n_lanes):
             s = sets[k % n_sets]
