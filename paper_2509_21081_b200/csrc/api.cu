@@ -314,6 +314,9 @@ int typhoon_mla_choose_mode(const typhoon_mla_shared_t* sh, int32_t B, int64_t t
 
 int typhoon_mla_free(typhoon_mla_shared_t* sh) {
     if (!sh) return TYPHOON_MLA_OK;
+    // the handle's buffers, stream and events belong to the device it was prepared on, whatever device is current now
+    int cur = -1;
+    const bool switched = cudaGetDevice(&cur) == cudaSuccess && cur != sh->device && cudaSetDevice(sh->device) == cudaSuccess;
     cudaDeviceSynchronize();
     cudaFree(sh->k_nope);
     cudaFree(sh->v_t);
@@ -324,6 +327,8 @@ int typhoon_mla_free(typhoon_mla_shared_t* sh) {
     if (sh->side_stream) cudaStreamDestroy(sh->side_stream);
     if (sh->ev_fork) cudaEventDestroy(sh->ev_fork);
     if (sh->ev_join) cudaEventDestroy(sh->ev_join);
+    if (switched) cudaSetDevice(cur);
+    cudaGetLastError();   // a failure while releasing must not surface in the caller's next launch
     delete sh;
     return TYPHOON_MLA_OK;
 }
@@ -577,6 +582,13 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         if (e == cudaSuccess) e = cudaStreamWaitEvent(sh->side_stream, sh->ev_fork, 0);
         if (e != cudaSuccess) return cuda_fail(e);
     }
+    // A failure after the fork still joins the side stream back into the caller's stream, so that the caller's stream
+    // stays the only one with work of this call pending (and a stream capture is not left with an open branch).
+    bool open_fork = forked;
+    auto fail = [&](cudaError_t err) {
+        if (open_fork && cudaEventRecord(sh->ev_join, sh->side_stream) == cudaSuccess) cudaStreamWaitEvent(s_main, sh->ev_join, 0);
+        return cuda_fail(err);
+    };
 
     // --- naive shared-prefix attention (Algorithm 1 line 4), one launch per (prefix, row range)
     for (int j = 0; j < n_jobs; ++j) {
@@ -597,14 +609,14 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
             e = launch_naive_attn_mma(na, s);
         }
         prof_after(TYPHOON_MLA_KERNEL_NAIVE_ATTN, s);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
         ++launches;
     }
     for (int j = 0; j < n_empties; ++j) {
         const EmptySlots& es = empties[j];
         e = launch_fill_neg_inf(lse_part_n + ((size_t)es.slot0 * B + es.row0) * H, es.n_slots, (int64_t)B * H,
                                 (int64_t)es.rows * H, s);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
         ++launches;
     }
     bool combined = false;
@@ -632,7 +644,7 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
             }
         }
         prof_after(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
         ++launches;
         // --- absorb attention over latent tokens (Algorithm 1 line 6)
         float* o_part_a = reinterpret_cast<float*>(ws + pl.off_opart_a);
@@ -646,14 +658,14 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         e = tc ? launch_absorb_attn_sm100(ab, &sh->tm_ckv, &sh->tm_kpe_tok, o_lat, lse_a, sh->status, s)
                : launch_absorb_attn_mma(ab, s);
         prof_after(TYPHOON_MLA_KERNEL_ABSORB_ATTN, s);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
         ++launches;
         if (n_jobs == 0 && n_empties == 0 && n_chunks > 1 && B <= kMergeProjectMaxB) {
             // absorb-only, a handful of requests: merge + projection + rounding in one launch
             prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
             e = launch_merge_project(o_part_a, lse_part_a, n_chunks, B, H, sh->w_uv, out, lse_out, out_fp32, s);
             prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
-            if (e != cudaSuccess) return cuda_fail(e);
+            if (e != cudaSuccess) return fail(e);
             g_last_launches = launches + 1;
             return TYPHOON_MLA_OK;
         }
@@ -661,12 +673,13 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
             prof_before(TYPHOON_MLA_KERNEL_MERGE, s);
             e = launch_merge_latent(o_part_a, lse_part_a, n_chunks, B, H, o_lat, lse_a, s);
             prof_after(TYPHOON_MLA_KERNEL_MERGE, s);
-            if (e != cudaSuccess) return cuda_fail(e);
+            if (e != cudaSuccess) return fail(e);
             ++launches;
         }
         if (forked) {
             e = cudaEventRecord(sh->ev_join, sh->side_stream);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(s_main, sh->ev_join, 0);
+            open_fork = false;
             if (e != cudaSuccess) return cuda_fail(e);
             s = s_main;
         }
@@ -687,7 +700,7 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
             e = launch_gemm_tn(g2, s);
         }
         prof_after(TYPHOON_MLA_KERNEL_W_UV, s);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
         ++launches;
     }
     // --- LSE combine (Algorithm 1 line 8)
@@ -696,7 +709,7 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         e = launch_combine(o_part_n, lse_part_n, pl.n_slots_naive, have_absorb ? o_abs : nullptr, lse_a, B, H, out,
                            lse_out, s, out_fp32);
         prof_after(TYPHOON_MLA_KERNEL_COMBINE, s);
-        if (e != cudaSuccess) return cuda_fail(e);
+        if (e != cudaSuccess) return fail(e);
         ++launches;
     }
     g_last_launches = launches;
@@ -797,7 +810,7 @@ int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, int
             const int r0 = lv.group_begin[g], r1 = lv.group_begin[g + 1];
             if (r1 < r0) return TYPHOON_MLA_ERR_INVALID_ARG;
             const typhoon_mla_shared* sh = lv.prefixes[g];
-            if (sh && sh->dims.num_heads != H) return TYPHOON_MLA_ERR_INVALID_ARG;
+            if (sh && (sh->dims.num_heads != H || sh->device != tp->sh0->device)) return TYPHOON_MLA_ERR_INVALID_ARG;
             if (!sh || sh->Ls == 0 || r1 == r0) continue;
             if (tp->n_jobs == kMaxTreeJobs) return TYPHOON_MLA_ERR_INVALID_ARG;
             int ranges = 0, slots = 0;
