@@ -105,6 +105,29 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims /* host */,
                                const void* w_uk, const void* w_uv,
                                void* stream, typhoon_mla_shared_t** out_handle /* host */);
 
+/*
+ * The same with the expanded K_nope and V stored in 8 bits (half the footprint and half the
+ * bytes a step streams; the paper assumes 8-bit caches only in its memory-footprint
+ * analysis, Section 4 "HBM Footprint", and does not fix an encoding; this is the library's):
+ * OCP E4M3 codes (1-4-3 bits, bias 7, no infinities, largest value 448), round to
+ * nearest even, saturating, of the 16-bit expanded cache divided by one power of two per
+ * head and tensor (the smallest 2^e with amax / 2^e <= 448).  Rope keys, the copy of the
+ * latent cache, the per-request caches and the queries stay 16-bit; the attention kernel
+ * widens the codes exactly and computes as in the 16-bit path (half-precision operands,
+ * fp32 accumulation), so the only error added is that of the encoding.  Queries must be
+ * within half precision's range (|q| < 65504).  The handle is used like any other
+ * (decode, decode_tree, decode_partial, the no-alloc call; AUTO / ABSORB / HYBRID /
+ * NAIVE); the shared-prefix kernel then works on row groups of 64 requests, so for
+ * B > 128 it is slower than with the 16-bit cache.  A 16-bit scratch of the size of one
+ * expanded tensor is taken from and returned to the stream's memory pool inside the call.
+ * Arguments and errors as typhoon_mla_prepare_shared.
+ */
+int typhoon_mla_prepare_shared_fp8(const typhoon_mla_dims_t* dims /* host */,
+                                   const void* ckv_shared, const void* kpe_shared,
+                                   int64_t Ls, int64_t ld_ckv, int64_t ld_kpe,
+                                   const void* w_uk, const void* w_uv,
+                                   void* stream, typhoon_mla_shared_t** out_handle /* host */);
+
 /* Release the handle and the device memory it owns (synchronises the device).
  * NULL is accepted. */
 int typhoon_mla_free(typhoon_mla_shared_t* shared);

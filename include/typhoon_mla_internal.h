@@ -40,6 +40,13 @@ int typhoon_mla_shared_view(const typhoon_mla_shared_t* shared,
  * elements each (device memory), on `stream`. */
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* shared, void* k_nope_dst, void* v_t_dst, void* stream);
 
+/* A handle from typhoon_mla_prepare_shared_fp8: the E4M3 codes in logical order, K_nope as
+ * uint8 [H, Ls_padded, 128] (token rows), V as uint8 [H, Ls_padded/64, 128, 64] (V^T in 64-token
+ * blocks), and the scales as float [2][H] (K_nope, then V); device buffers, on `stream`.
+ * INVALID_ARG for a 16-bit handle (and typhoon_mla_shared_export for an 8-bit one). */
+int typhoon_mla_shared_export_fp8(const typhoon_mla_shared_t* shared, void* k_codes_dst, void* v_codes_dst,
+                                  float* scales_dst, void* stream);
+
 /* Which implementation of the tensor-core kernels runs: the tcgen05/TMEM/TMA kernels (default) or
  * the warp-MMA kernels kept as an on-GPU cross-check.  Affects later prepare_shared and decode calls. */
 enum { TYPHOON_MLA_PATH_TCGEN05 = 0, TYPHOON_MLA_PATH_WARP_MMA = 1 };

@@ -49,6 +49,8 @@ def _load():
     lib.typhoon_mla_status_string.argtypes = [C.c_int]
     lib.typhoon_mla_prepare_shared.restype = C.c_int
     lib.typhoon_mla_prepare_shared.argtypes = [C.POINTER(Dims), vp, vp, i64, i64, i64, vp, vp, vp, C.POINTER(vp)]
+    lib.typhoon_mla_prepare_shared_fp8.restype = C.c_int
+    lib.typhoon_mla_prepare_shared_fp8.argtypes = [C.POINTER(Dims), vp, vp, i64, i64, i64, vp, vp, vp, C.POINTER(vp)]
     lib.typhoon_mla_free.restype = C.c_int
     lib.typhoon_mla_free.argtypes = [vp]
     lib.typhoon_mla_workspace_bytes.restype = sz
@@ -89,6 +91,8 @@ def _load():
                                             C.POINTER(i64)]
     lib.typhoon_mla_shared_export.restype = C.c_int
     lib.typhoon_mla_shared_export.argtypes = [vp, vp, vp, vp]
+    lib.typhoon_mla_shared_export_fp8.restype = C.c_int
+    lib.typhoon_mla_shared_export_fp8.argtypes = [vp, vp, vp, vp, vp]
     lib.typhoon_mla_set_kernel_path.restype = C.c_int
     lib.typhoon_mla_set_kernel_path.argtypes = [i32]
     lib.typhoon_mla_order_by_length.restype = C.c_int
@@ -167,6 +171,19 @@ def typhoon_mla_prepare_shared(dims: Dims, ckv_shared: torch.Tensor, kpe_shared:
     st = _lib.typhoon_mla_prepare_shared(C.byref(dims), _ptr(ckv_shared), _ptr(kpe_shared), Ls, ld_ckv, ld_kpe,
                                          _ptr(w_uk), _ptr(w_uv), _stream(), C.byref(h))
     _check(st, "typhoon_mla_prepare_shared")
+    return SharedPrefix(h, dims, (w_uk, w_uv))
+
+
+def typhoon_mla_prepare_shared_fp8(dims: Dims, ckv_shared: torch.Tensor, kpe_shared: torch.Tensor,
+                                   w_uk: torch.Tensor, w_uv: torch.Tensor) -> SharedPrefix:
+    """The same with the expanded K_nope / V stored as E4M3 codes (one power-of-two scale per head and tensor)."""
+    Ls = ckv_shared.shape[0]
+    h = C.c_void_p()
+    ld_ckv = ckv_shared.stride(0) if Ls > 0 else 512
+    ld_kpe = kpe_shared.stride(0) if Ls > 0 else 64
+    st = _lib.typhoon_mla_prepare_shared_fp8(C.byref(dims), _ptr(ckv_shared), _ptr(kpe_shared), Ls, ld_ckv, ld_kpe,
+                                             _ptr(w_uk), _ptr(w_uv), _stream(), C.byref(h))
+    _check(st, "typhoon_mla_prepare_shared_fp8")
     return SharedPrefix(h, dims, (w_uk, w_uv))
 
 
@@ -338,6 +355,19 @@ def typhoon_mla_shared_export(shared: SharedPrefix):
     vt = torch.empty(H, Lp // 64, 128, 64, dtype=torch.bfloat16, device="cuda")
     _check(_lib.typhoon_mla_shared_export(shared.handle, _ptr(kt), _ptr(vt), _stream()), "typhoon_mla_shared_export")
     return kt, vt
+
+
+def typhoon_mla_shared_export_fp8(shared: SharedPrefix):
+    """Codes and scales of an 8-bit handle: K codes uint8 [H, Ls_pad, 128], V codes uint8 [H, Ls_pad/64, 128, 64]
+    (V^T in 64-token blocks), scales float32 [2, H] (K_nope, V)."""
+    _, Lp, _ = typhoon_mla_shared_view(shared)
+    H = shared.dims.num_heads
+    kc = torch.empty(H, Lp, 128, dtype=torch.uint8, device="cuda")
+    vc = torch.empty(H, Lp // 64, 128, 64, dtype=torch.uint8, device="cuda")
+    sc = torch.empty(2, H, dtype=torch.float32, device="cuda")
+    _check(_lib.typhoon_mla_shared_export_fp8(shared.handle, _ptr(kc), _ptr(vc), _ptr(sc), _stream()),
+           "typhoon_mla_shared_export_fp8")
+    return kc, vc, sc
 
 
 def typhoon_mla_last_launch_count() -> int:

@@ -157,7 +157,7 @@ Plan make_plan(const typhoon_mla_shared* sh, bool tc, int schedule, int B, int m
         p.n_split_naive = naive_slots_override > 0 ? 1 : 0;
         p.n_slots_naive = naive_slots_override;
     } else if (use_naive && tc) {
-        naive_sm100_plan(B, H, sh->Ls, n_sm, schedule, &p.n_split_naive, &p.n_slots_naive);   // n_split_naive = tile ranges
+        naive_sm100_plan(B, H, sh->Ls, n_sm, schedule, &p.n_split_naive, &p.n_slots_naive, sh->fp8 != 0);   // n_split_naive = tile ranges
     } else {
         p.n_split_naive = use_naive ? naive_splits(B, H, sh->Ls, n_sm) : 0;
         p.n_slots_naive = p.n_split_naive;
@@ -324,6 +324,9 @@ int typhoon_mla_free(typhoon_mla_shared_t* sh) {
     cudaFree(sh->kpe);
     cudaFree(sh->w_uk_t);
     cudaFree(sh->status);
+    cudaFree(sh->k8);
+    cudaFree(sh->v8);
+    cudaFree(sh->fp8_f);
     if (sh->side_stream) cudaStreamDestroy(sh->side_stream);
     if (sh->ev_fork) cudaEventDestroy(sh->ev_fork);
     if (sh->ev_join) cudaEventDestroy(sh->ev_join);
@@ -333,9 +336,9 @@ int typhoon_mla_free(typhoon_mla_shared_t* sh) {
     return TYPHOON_MLA_OK;
 }
 
-int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_shared, const void* kpe_shared,
-                               int64_t Ls, int64_t ld_ckv, int64_t ld_kpe, const void* w_uk, const void* w_uv,
-                               void* stream, typhoon_mla_shared_t** out_handle) {
+static int prepare_impl(const typhoon_mla_dims_t* dims, const void* ckv_shared, const void* kpe_shared,
+                        int64_t Ls, int64_t ld_ckv, int64_t ld_kpe, const void* w_uk, const void* w_uv,
+                        void* stream, typhoon_mla_shared_t** out_handle, bool fp8) {
     if (!dims || !out_handle || !w_uk || !w_uv || Ls < 0) return TYPHOON_MLA_ERR_INVALID_ARG;
     *out_handle = nullptr;
     if (!dims_supported(*dims)) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;
@@ -383,12 +386,28 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
         sh->owned_bytes += bytes;
         return true;
     };
-    if (!alloc(&sh->k_nope, b_k) || !alloc(&sh->v_t, b_k) || !alloc(&sh->ckv, b_ckv) || !alloc(&sh->kpe, b_kpe) ||
-        !alloc(&sh->w_uk_t, b_w) || !alloc(reinterpret_cast<void**>(&sh->status), 256)) {
+    sh->fp8 = (fp8 && Ls > 0) ? 1 : 0;
+    bool ok_alloc = alloc(&sh->ckv, b_ckv) && alloc(&sh->kpe, b_kpe) && alloc(&sh->w_uk_t, b_w) &&
+                    alloc(reinterpret_cast<void**>(&sh->status), 256);
+    if (ok_alloc && !sh->fp8) ok_alloc = alloc(&sh->k_nope, b_k) && alloc(&sh->v_t, b_k);
+    if (ok_alloc && sh->fp8)
+        ok_alloc = alloc(&sh->k8, b_k / 2) && alloc(&sh->v8, b_k / 2) &&
+                   alloc(reinterpret_cast<void**>(&sh->fp8_f), (size_t)H * 5 * sizeof(float));
+    if (!ok_alloc) {
         typhoon_mla_free(sh);
         return TYPHOON_MLA_ERR_ALLOC;
     }
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // 8-bit cache: each tensor is expanded into a 16-bit scratch of the stream's memory pool, encoded from there,
+    // and the scratch is handed back in stream order (no synchronisation)
+    void* scratch16 = nullptr;
+    if (sh->fp8 && cudaMallocAsync(&scratch16, b_k, s) != cudaSuccess) {
+        cudaGetLastError();
+        typhoon_mla_free(sh);
+        return TYPHOON_MLA_ERR_ALLOC;
+    }
+    void* const k_dst = sh->fp8 ? scratch16 : sh->k_nope;
+    void* const v_dst = sh->fp8 ? scratch16 : sh->v_t;
     const bool tc = cfg.tc();
     {
         int lo = 0, hi = 0;
@@ -398,6 +417,7 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sh->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sh->ev_join, cudaEventDisableTiming);
     if (e != cudaSuccess) {
+        if (scratch16) cudaFreeAsync(scratch16, s);
         typhoon_mla_free(sh);
         return cuda_fail(e);
     }
@@ -407,18 +427,29 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
         e = launch_copy_pad_rows(ckv_shared, ld_ckv, sh->ckv, (int)Ls, (int)Lp, 512, s);
         if (e == cudaSuccess) e = launch_copy_pad_rows(kpe_shared, ld_kpe, sh->kpe, (int)Ls, (int)Lp, 64, s);
         if (e == cudaSuccess) {  // K_nope[h] = ckv * W_UK[h]^T
-            GemmTN g{sh->ckv, 512, 0, w_uk, 512, 128 * 512, sh->k_nope, 128, (int64_t)Lp * 128,
+            GemmTN g{sh->ckv, 512, 0, w_uk, 512, 128 * 512, k_dst, 128, (int64_t)Lp * 128,
                      (int)Lp, 128, 512, H, false, 0, true};
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
+            if (e == cudaSuccess && sh->fp8)
+                e = launch_quantize_e4m3(k_dst, false, H, (int64_t)Lp, sh->k8, reinterpret_cast<uint32_t*>(sh->fp8_f + 4 * H),
+                                         sh->fp8_f, sh->fp8_f + 2 * H, s);
         }
         if (e == cudaSuccess) {  // V^T[h] = W_UV[h] * ckv^T
-            GemmTN g{w_uv, 512, 128 * 512, sh->ckv, 512, 0, sh->v_t, (int64_t)Lp, (int64_t)(128 * Lp),
+            GemmTN g{w_uv, 512, 128 * 512, sh->ckv, 512, 0, v_dst, (int64_t)Lp, (int64_t)(128 * Lp),
                      128, (int)Lp, 512, H, false, 64};
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
+            if (e == cudaSuccess && sh->fp8)
+                e = launch_quantize_e4m3(v_dst, true, H, (int64_t)Lp, sh->v8, reinterpret_cast<uint32_t*>(sh->fp8_f + 4 * H),
+                                         sh->fp8_f + H, sh->fp8_f + 3 * H, s);
         }
     }
+    if (scratch16) {
+        const cudaError_t ef = cudaFreeAsync(scratch16, s);
+        if (e == cudaSuccess) e = ef;
+    }
     if (e == cudaSuccess && Ls > 0)
-        e = make_naive_sm100_tmaps(sh->k_nope, sh->kpe, sh->v_t, H, sh->Ls_pad, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt);
+        e = sh->fp8 ? make_naive_fp8_tmaps(sh->k8, sh->kpe, sh->v8, H, sh->Ls_pad, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt)
+                    : make_naive_sm100_tmaps(sh->k_nope, sh->kpe, sh->v_t, H, sh->Ls_pad, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt);
     if (e == cudaSuccess) e = make_q_absorb_tmap(sh->w_uk_t, H, &sh->tm_wuk_t);
     if (e == cudaSuccess && Ls > 0) e = make_absorb_shared_tmaps(sh->ckv, sh->kpe, sh->Ls_pad, &sh->tm_ckv, &sh->tm_kpe_tok);
     if (e != cudaSuccess) {
@@ -427,6 +458,18 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_s
     }
     *out_handle = sh;
     return TYPHOON_MLA_OK;
+}
+
+int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims, const void* ckv_shared, const void* kpe_shared,
+                               int64_t Ls, int64_t ld_ckv, int64_t ld_kpe, const void* w_uk, const void* w_uv,
+                               void* stream, typhoon_mla_shared_t** out_handle) {
+    return prepare_impl(dims, ckv_shared, kpe_shared, Ls, ld_ckv, ld_kpe, w_uk, w_uv, stream, out_handle, false);
+}
+
+int typhoon_mla_prepare_shared_fp8(const typhoon_mla_dims_t* dims, const void* ckv_shared, const void* kpe_shared,
+                                   int64_t Ls, int64_t ld_ckv, int64_t ld_kpe, const void* w_uk, const void* w_uv,
+                                   void* stream, typhoon_mla_shared_t** out_handle) {
+    return prepare_impl(dims, ckv_shared, kpe_shared, Ls, ld_ckv, ld_kpe, w_uk, w_uv, stream, out_handle, true);
 }
 
 int typhoon_mla_shared_view(const typhoon_mla_shared_t* sh, const void** k_nope, const void** v_t, int64_t* Ls,
@@ -503,12 +546,24 @@ int typhoon_mla_test_wait_expiry(const typhoon_mla_shared_t* sh, int64_t deadlin
 }
 
 int typhoon_mla_shared_export(const typhoon_mla_shared_t* sh, void* k_nope_dst, void* v_t_dst, void* stream) {
-    if (!sh || !k_nope_dst || !v_t_dst) return TYPHOON_MLA_ERR_INVALID_ARG;
+    if (!sh || !k_nope_dst || !v_t_dst || sh->fp8) return TYPHOON_MLA_ERR_INVALID_ARG;
     const size_t bytes = (size_t)sh->dims.num_heads * (size_t)sh->Ls_pad * 128 * 2;
     if (bytes == 0) return TYPHOON_MLA_OK;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(k_nope_dst, sh->k_nope, bytes, cudaMemcpyDeviceToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(v_t_dst, sh->v_t, bytes, cudaMemcpyDeviceToDevice, s);
+    return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
+}
+
+int typhoon_mla_shared_export_fp8(const typhoon_mla_shared_t* sh, void* k_codes_dst, void* v_codes_dst, float* scales_dst,
+                                  void* stream) {
+    if (!sh || !k_codes_dst || !v_codes_dst || !scales_dst || !sh->fp8) return TYPHOON_MLA_ERR_INVALID_ARG;
+    const int H = sh->dims.num_heads;
+    const size_t n = (size_t)H * (size_t)sh->Ls_pad * 128;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_unpermute_codes(sh->k8, k_codes_dst, n, s);
+    if (e == cudaSuccess) e = launch_unpermute_codes(sh->v8, v_codes_dst, n, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(scales_dst, sh->fp8_f, (size_t)2 * H * sizeof(float), cudaMemcpyDeviceToDevice, s);
     return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
 }
 
@@ -575,6 +630,9 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
     // In a hybrid step the absorb branch (lines 5-6) does not depend on the naive kernel (line 4): it runs
     // on the handle's (high-priority) side stream, forked behind the caller's stream here and joined
     // before the projection.
+    if (!tc)   // row ranges and the 8-bit cache need the tcgen05 kernel
+        for (int j = 0; j < n_jobs; ++j)
+            if (jobs[j].rows != B || jobs[j].sh->fp8) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;
     cudaStream_t s_main = s;
     const bool forked = cfg.overlap && have_absorb && n_jobs > 0 && sh->side_stream != nullptr;
     if (forked) {
@@ -601,9 +659,9 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         if (tc) {
             NaiveAttnSm100 na{qn, qp, &jb.sh->tm_kn, &jb.sh->tm_kp, &jb.sh->tm_vt, jb.rows, H, (int)jb.sh->Ls,
                               jb.n_ranges, jb.n_slots_level, softmax_scale, op, lp, sh->status, B};
+            if (jb.sh->fp8) na.fp8_mult = jb.sh->fp8_f + 2 * H;
             e = launch_naive_attn_sm100(na, s);
         } else {
-            if (jb.rows != B) return TYPHOON_MLA_ERR_UNSUPPORTED_DIMS;   // row ranges need the tcgen05 kernel
             NaiveAttn na{qn, qp, jb.sh->k_nope, jb.sh->v_t, jb.sh->kpe, B, H, (int)jb.sh->Ls, (int)jb.sh->Ls_pad,
                          jb.n_ranges, softmax_scale, op, lp};
             e = launch_naive_attn_mma(na, s);
@@ -814,7 +872,8 @@ int plan_tree(const typhoon_mla_prefix_level_t* levels, int n_levels, int B, int
             if (!sh || sh->Ls == 0 || r1 == r0) continue;
             if (tp->n_jobs == kMaxTreeJobs) return TYPHOON_MLA_ERR_INVALID_ARG;
             int ranges = 0, slots = 0;
-            naive_sm100_plan(r1 - r0, H, sh->Ls, sh->num_sms > 0 ? sh->num_sms : kDefaultNumSM, schedule, &ranges, &slots);
+            naive_sm100_plan(r1 - r0, H, sh->Ls, sh->num_sms > 0 ? sh->num_sms : kDefaultNumSM, schedule, &ranges, &slots,
+                             sh->fp8 != 0);
             tp->jobs[tp->n_jobs++] = NaiveJob{sh, r0, r1 - r0, ranges, 0, slot0};
             level_slots = std::max(level_slots, slots);
         }

@@ -25,4 +25,11 @@ struct typhoon_mla_shared {
     size_t owned_bytes;
     int device;     // device the handle was prepared on; every call checks that it is the current one
     int num_sms;    // multiprocessors of that device (the work decompositions fill them)
+    // 8-bit expanded cache (typhoon_mla_prepare_shared_fp8): k_nope and v_t are null, the codes live here and
+    // tm_kn / tm_vt describe the code arrays
+    int fp8;
+    void* k8;       // E4M3 codes [H, Ls_pad, 128]: token rows of 128 dims
+    void* v8;       // E4M3 codes [H, Ls_pad/64, 128, 64]: V^T in 64-token blocks
+    float* fp8_f;   // device [4][H] floats: scale of K_nope, scale of V, 2^8 * scale of K_nope, 2^8 * scale of V;
+                    // then [H] words of scratch for the amax reduction
 };

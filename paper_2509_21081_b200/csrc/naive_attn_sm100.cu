@@ -56,6 +56,7 @@ using namespace sm100;
 constexpr int Q_TILE_BYTES = 128 * 192 * 2;   // 3 slabs [128][64] bf16
 
 constexpr int MAX_STAGES = 4;
+constexpr int MAX_Q_STAGES = 8;
 constexpr int kNaiveSmemMax = 227 * 1024;   // opt-in limit set once per device; every launch stays below it
 
 struct NaiveSm100Params {
@@ -67,6 +68,8 @@ struct NaiveSm100Params {
     int per, rem;          // T = R * per + rem: ranges [0, rem) hold per + 1 tiles, the others per
     int n_seg_max;         // partial slots per head (one per segment of the head)
     int k_stages, v_stages;
+    int kq_stages, vq_stages;   // 8-bit cache: depth of the staging rings the copies land in
+    const float* mult;          // 8-bit cache: [2][H] factors 2^8 * scale of K_nope and of V, per head
     float scale_log2;
     float* o_part;     // [n_slots][part_rows][H][128]
     float* lse_part;   // [n_slots][part_rows][H]
@@ -87,6 +90,9 @@ struct Barriers {
     // u-2 has landed (every wait below does) then sees a barrier at most one completion from the
     // awaited one, which is what a parity wait can tell apart
     uint64_t o_done[2][2];
+    // 8-bit cache: staging rings filled by bulk copies (K codes + rope keys; V codes) and emptied by the conversion
+    // warpgroup, which fills the 16-bit rings k_full / v_full guard; q_conv: the query tile is in half precision
+    uint64_t kq_full[MAX_Q_STAGES], kq_empty[MAX_Q_STAGES], vq_full[MAX_Q_STAGES], vq_empty[MAX_Q_STAGES], q_conv;
     uint32_t tmem_base;
     int abort_flag;
     float merge_m[128], merge_l[128];   // stream 1's reference exponent and row sum, per query row
@@ -102,8 +108,9 @@ struct Segment {
 };
 
 // TOK = tokens per KV tile: 64 (mode Y, B <= 128) or 128 (mode X, B > 128).
-template <int TOK, bool M64>
-__global__ void __launch_bounds__(384, 1)
+// FP8: the expanded cache is stored as E4M3 codes (see the conversion warpgroup below); 64 query rows per CTA.
+template <int TOK, bool M64, bool FP8>
+__global__ void __launch_bounds__(FP8 ? 512 : 384, 1)
 naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_constant__ CUtensorMap tm_qp,
                         const __grid_constant__ CUtensorMap tm_kn, const __grid_constant__ CUtensorMap tm_kp,
                         const __grid_constant__ CUtensorMap tm_vt, NaiveSm100Params p) {
@@ -111,17 +118,24 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     constexpr int NB = MODE_Y ? 2 : 1;                  // S buffers per stream
     constexpr int BLK = TOK / 64;                       // 64-token blocks per tile
     constexpr int K_SLAB = TOK * 128;                   // bytes of one [TOK][64] K slab
-    constexpr int K_TILE_BYTES = 3 * K_SLAB;
+    constexpr int K_TILE_BYTES = (FP8 ? 2 : 3) * K_SLAB;   // (8-bit cache: the rope slab stays in the staging ring)
     constexpr int V_TILE_BYTES = BLK * 16384;           // BLK slabs [128 dims][64 tokens]
-    constexpr int ROWS = MODE_Y ? 128 : 256;            // query rows per column
+    constexpr int ROWS = FP8 ? 64 : (MODE_Y ? 128 : 256);   // query rows per column
+    static_assert(!FP8 || (M64 && TOK == 64), "the 8-bit cache path is built for 64-row, 64-token tiles");
+    constexpr int Q_SLAB = (FP8 ? 64 : 128) * 128;      // bytes of one [rows][64] slab of the query tile
+    constexpr int Q_BYTES = 3 * Q_SLAB;
+    constexpr int KQ_BYTES = 16384, VQ_BYTES = 8192;    // staging slots: K codes 8 KB + rope keys 8 KB; V codes 8 KB
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     constexpr int n_q_tiles = MODE_Y ? 1 : 2;
     uint8_t* sQ = smem;
-    uint8_t* sK = sQ + n_q_tiles * Q_TILE_BYTES;
+    uint8_t* sK = sQ + n_q_tiles * Q_BYTES;
     uint8_t* sV = sK + p.k_stages * K_TILE_BYTES;
-    Barriers* bar = reinterpret_cast<Barriers*>(sV + p.v_stages * V_TILE_BYTES);
+    uint8_t* sKq = sV + p.v_stages * V_TILE_BYTES;      // staging rings (8-bit cache only)
+    uint8_t* sVq = sKq + (FP8 ? p.kq_stages : 0) * KQ_BYTES;
+    Barriers* bar = reinterpret_cast<Barriers*>(sVq + (FP8 ? p.vq_stages : 0) * VQ_BYTES);
+    const int k_depth = FP8 ? p.kq_stages : p.k_stages, v_depth = FP8 ? p.vq_stages : p.v_stages;   // rings the copies land in
     volatile int* abort_flag = &bar->abort_flag;
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
@@ -170,15 +184,24 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     const uint32_t ld0 = (warp == 0 && elect_one()) ? 1u : 0u;
     auto issue_q = [&](const Segment& s) {
         const int nq = (s.n_str1 > 0 && !MODE_Y) ? 2 : 1;
-        mbar_arrive_expect_tx_if(ld0, &bar->q_full, nq * Q_TILE_BYTES);
+        mbar_arrive_expect_tx_if(ld0, &bar->q_full, nq * Q_BYTES);
         for (int t = 0; t < nq; ++t) {
-            uint8_t* dst = sQ + t * Q_TILE_BYTES;
+            uint8_t* dst = sQ + t * Q_BYTES;
             tma_load_3d_if(ld0, dst, &tm_qn, &bar->q_full, 0, s.h, s.row0 + t * 128);
-            tma_load_3d_if(ld0, dst + 16384, &tm_qn, &bar->q_full, 64, s.h, s.row0 + t * 128);
-            tma_load_3d_if(ld0, dst + 32768, &tm_qp, &bar->q_full, 0, s.h, s.row0 + t * 128);
+            tma_load_3d_if(ld0, dst + Q_SLAB, &tm_qn, &bar->q_full, 64, s.h, s.row0 + t * 128);
+            tma_load_3d_if(ld0, dst + 2 * Q_SLAB, &tm_qp, &bar->q_full, 0, s.h, s.row0 + t * 128);
         }
     };
     auto issue_k = [&](const Segment& s, int e, int ring_pos) {
+        if (FP8) {   // one 64-token block of codes (as 64 rows of 128 bytes) and its rope keys into a staging slot
+            const int sq = ring_pos % p.kq_stages;
+            uint8_t* dst = sKq + sq * KQ_BYTES;
+            const int blk = tile_of(s, e);
+            mbar_arrive_expect_tx_if(ld0, &bar->kq_full[sq], KQ_BYTES);
+            tma_load_3d_if(ld0, dst, &tm_kn, &bar->kq_full[sq], 0, blk * 64, s.h);
+            tma_load_2d_if(ld0, dst + 8192, &tm_kp, &bar->kq_full[sq], 0, blk * 64);
+            return;
+        }
         const int st = ring_pos % p.k_stages;
         uint8_t* dst = sK + st * K_TILE_BYTES;
         const int blk0 = tile_of(s, e) * BLK;
@@ -192,6 +215,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         }
     };
     auto issue_v = [&](const Segment& s, int e, int ring_pos, uint32_t ld) {
+        if (FP8) {
+            const int sq = ring_pos % p.vq_stages;
+            mbar_arrive_expect_tx_if(ld, &bar->vq_full[sq], VQ_BYTES);
+            tma_load_3d_if(ld, sVq + sq * VQ_BYTES, &tm_vt, &bar->vq_full[sq], 0, tile_of(s, e) * 64, s.h);
+            return;
+        }
         const int st = ring_pos % p.v_stages;
         const int blk0 = tile_of(s, e) * BLK;
         mbar_arrive_expect_tx_if(ld, &bar->v_full[st], V_TILE_BYTES);
@@ -207,8 +236,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     int n_pre_k = 0, n_pre_v = 0;
     if (g_begin < g_end) {
         const Segment s0 = segment_at(g_begin);
-        n_pre_k = min(p.k_stages, s0.cnt);
-        n_pre_v = min(p.v_stages, s0.cnt);
+        n_pre_k = min(k_depth, s0.cnt);
+        n_pre_v = min(v_depth, s0.cnt);
         if (warp == 2) {
             if (lane == 0) prefetch_tmap(&tm_qn);
             if (lane == 1) prefetch_tmap(&tm_qp);
@@ -227,7 +256,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             for (int i = lane; i < n_bars; i += 32) {
                 uint64_t* m = all + i;
                 const bool wg = (m >= &bar->p_ready[0][0] && m < &bar->sbuf_free[0][0]) || (m >= &bar->o_free[0] && m < &bar->o_done[0][0]);   // o_free, merge_ready
-                mbar_init(m, wg ? 128 : 1);
+                // (a K staging slot is released by two parties: the conversion warpgroup and the S products that read its rope keys)
+                const bool two = FP8 && m >= &bar->kq_empty[0] && m < &bar->vq_full[0];
+                mbar_init(m, wg ? 128 : (two ? 2 : 1));
             }
             if (lane == 0) bar->abort_flag = 0;
             fence_mbar_init();
@@ -257,11 +288,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const Segment s = segment_at(g);
             // K tiles first (they only need free ring slots), so that they are in flight while the
             // previous segment's last S products still hold the Q tile
-            const int head_k = min(s.cnt, p.k_stages);
+            const int head_k = min(s.cnt, k_depth);
+            uint64_t* const k_slot_free = FP8 ? bar->kq_empty : bar->k_empty;   // ring the K copies land in
             int e = 0;
             for (; e < head_k && ok; ++e, ++ring) {
                 if (ring < n_pre_k) continue;                 // issued before the setup barrier
-                ok = mbar_wait_warp(&bar->k_empty[ring % p.k_stages], ((ring / p.k_stages) & 1) ^ 1, abort_flag);
+                ok = mbar_wait_warp(&k_slot_free[ring % k_depth], ((ring / k_depth) & 1) ^ 1, abort_flag);
                 if (ok) issue_k(s, e, ring);
             }
             if (seg > 0 && ok) {
@@ -269,7 +301,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 if (ok) issue_q(s);
             }
             for (; e < s.cnt && ok; ++e, ++ring) {
-                ok = mbar_wait_warp(&bar->k_empty[ring % p.k_stages], ((ring / p.k_stages) & 1) ^ 1, abort_flag);
+                ok = mbar_wait_warp(&k_slot_free[ring % k_depth], ((ring / k_depth) & 1) ^ 1, abort_flag);
                 if (ok) issue_k(s, e, ring);
             }
             g += s.cnt;
@@ -285,7 +317,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const Segment s = segment_at(g);
             for (int e = 0; e < s.cnt && ok; ++e, ++ring) {
                 if (ring < n_pre_v) continue;                 // issued before the setup barrier
-                ok = mbar_wait_warp(&bar->v_empty[ring % p.v_stages], ((ring / p.v_stages) & 1) ^ 1, abort_flag);
+                uint64_t* const v_slot_free = FP8 ? bar->vq_empty : bar->v_empty;
+                ok = mbar_wait_warp(&v_slot_free[ring % v_depth], ((ring / v_depth) & 1) ^ 1, abort_flag);
                 if (ok) issue_v(s, e, ring, ld);
             }
             g += s.cnt;
@@ -296,12 +329,14 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         // up to two steps; with one it follows the PV product of the previous step.
         const uint32_t ld = elect_one() ? 1u : 0u;
         constexpr uint32_t idesc_s = idesc_bf16(M64 ? 64 : 128, TOK, false, false);
+        constexpr uint32_t idesc_s_nope = FP8 ? idesc_f16(M64 ? 64 : 128, TOK, false, false) : idesc_s;
         int ring_base = 0, seg = 0;
         int used0 = 0, used1 = 0;                              // S-buffer uses so far, per stream
         bool ok = true;
         for (int g = g_begin; g < g_end && ok; ++seg) {
             const Segment s = segment_at(g);
             ok = mbar_wait_warp(&bar->q_full, seg & 1, abort_flag);
+            if (FP8 && ok) ok = mbar_wait_warp(&bar->q_conv, seg & 1, abort_flag);   // nope part converted to half precision
             for (int j = 0; j < s.n_str0 && ok; ++j) {
                 for (int i = 0; i < 2 && ok; ++i) {
                     if (j >= (i == 0 ? s.n_str0 : s.n_str1)) continue;
@@ -310,6 +345,10 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     if (MODE_Y || i == 0) {                       // mode X: stream 1 reuses stream 0's tile
                         ok = mbar_wait_warp(&bar->k_full[st], (ring / p.k_stages) & 1, abort_flag);
                         if (!ok) break;
+                        if (FP8) {   // the rope keys of the tile are read from the staging slot itself
+                            ok = mbar_wait_warp(&bar->kq_full[ring % p.kq_stages], (ring / p.kq_stages) & 1, abort_flag);
+                            if (!ok) break;
+                        }
                     }
                     const int u = (i == 0 ? used0 : used1) + j;
                     if (u >= NB) {   // the PV product that read P from this S buffer NB uses ago must be done
@@ -317,19 +356,22 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         if (!ok) break;
                     }
                     tc_fence_after();
-                    const uint32_t qa = smem_u32(sQ + (MODE_Y ? 0 : i) * Q_TILE_BYTES);
+                    const uint32_t qa = smem_u32(sQ + (MODE_Y ? 0 : i) * Q_BYTES);
                     const uint32_t ka = smem_u32(sK + st * K_TILE_BYTES);
+                    const uint32_t rope = FP8 ? smem_u32(sKq + (ring % p.kq_stages) * KQ_BYTES + 8192) : ka + 2 * K_SLAB;
                     const uint32_t d = tmem_base + s_col(i, u);
                     const bool last_user = MODE_Y || i == 1 || s.n_str1 == 0;
 #pragma unroll
                     for (int slab = 0; slab < 3; ++slab) {
-                        const uint64_t da = smem_desc_k_sw128(qa + slab * 16384);
-                        const uint64_t db = smem_desc_k_sw128(ka + slab * K_SLAB);
+                        const uint64_t da = smem_desc_k_sw128(qa + slab * Q_SLAB);
+                        const uint64_t db = smem_desc_k_sw128(slab == 2 ? rope : ka + slab * K_SLAB);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_ss_if(ld, d, da + 2 * k, db + 2 * k, idesc_s, (slab | k) != 0);
+                        for (int k = 0; k < 4; ++k)
+                            umma_ss_if(ld, d, da + 2 * k, db + 2 * k, slab == 2 ? idesc_s : idesc_s_nope, (slab | k) != 0);
                     }
                     umma_commit_if(ld, &bar->s_ready[i][u % NB]);
                     if (last_user) umma_commit_if(ld, &bar->k_empty[st]);   // last user releases the ring slot
+                    if (FP8) umma_commit_if(ld, &bar->kq_empty[ring % p.kq_stages]);   // ... and its share of the staging slot
                 }
             }
             umma_commit_if(ld, &bar->q_free);                     // the Q tile may be replaced
@@ -341,7 +383,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     } else if (warp == 3) {
         // ---------------- O += P V issuer
         const uint32_t ld = elect_one() ? 1u : 0u;
-        constexpr uint32_t idesc_o = idesc_bf16(M64 ? 64 : 128, 128, false, false);
+        constexpr uint32_t idesc_o = FP8 ? idesc_f16(M64 ? 64 : 128, 128, false, false) : idesc_bf16(M64 ? 64 : 128, 128, false, false);
         int ring_base = 0, seg = 0;
         int used0 = 0, used1 = 0;
         bool ok = true;
@@ -392,7 +434,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             ring_base += s.cnt;
             g += s.cnt;
         }
-    } else if (warp >= 4) {
+    } else if (warp >= 4 && warp < 12) {
         // ---------------- softmax warpgroups
         const int i = (warp - 4) >> 2;            // stream
         const int lg = (warp & 3) * 32;           // TMEM lane group of this warp
@@ -412,7 +454,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const bool warp_has_rows = tile_row0 + (M64 ? (warp & 3) * 16 : lg) < p.B;   // warp-uniform: the warp's first row is a real request
             float m_ref = -INFINITY, m_ref_b = -INFINITY;   // (M = 64: reference exponents of this thread's rows A and B)
             uint64_t l_sum2 = pack_f32x2(0.f, 0.f), l_sum2b = pack_f32x2(0.f, 0.f);   // row sum of the probabilities, as four partial sums
-            const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+            // (8-bit cache: the accumulated logits are the true ones divided by 2^8 * scale of this head's K, see below)
+            const float scale_l2 = FP8 ? p.scale_log2 * p.mult[s.h] : p.scale_log2;
+            const uint64_t scale2 = pack_f32x2(scale_l2, scale_l2);
             for (int j = 0; j < nt && ok; ++j) {
                 const int u = used + j;
                 const int buf = u % NB;
@@ -457,8 +501,8 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     mxb = fmaxf(mxb, mxb2);
                     mxa = fmaxf(mxa, __shfl_xor_sync(0xffffffffu, mxa, 1));
                     mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, 1));
-                    mxa = fmaxf(mxa, __shfl_xor_sync(0xffffffffu, mxa, 2)) * p.scale_log2;
-                    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, 2)) * p.scale_log2;
+                    mxa = fmaxf(mxa, __shfl_xor_sync(0xffffffffu, mxa, 2)) * scale_l2;
+                    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, 2)) * scale_l2;
                     // lazy rescale: only when some row's maximum grew by more than 2^8
                     const bool grow_a = mxa > m_ref + 8.f, grow_b = mxb > m_ref_b + 8.f;
                     if (j == 0) {
@@ -498,8 +542,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[4 * gq]), __uint_as_float(sr[4 * gq + 1])), scale2, nma), x0, x1);
                         unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[4 * gq + 2]), __uint_as_float(sr[4 * gq + 3])), scale2, nmb), y0, y1);
                         const float pa0 = fast_exp2(x0), pa1 = fast_exp2(x1), pb0 = fast_exp2(y0), pb1 = fast_exp2(y1);
-                        pk[2 * gq] = pack_bf16(pa0, pa1);          // row A, P column 4 gq + t%4
-                        pk[2 * gq + 1] = pack_bf16(pb0, pb1);      // row B, same column
+                        // (8-bit cache: V is converted to half precision, so the probabilities are too)
+                        pk[2 * gq] = FP8 ? pack_f16(pa0, pa1) : pack_bf16(pa0, pa1);          // row A, P column 4 gq + t%4
+                        pk[2 * gq + 1] = FP8 ? pack_f16(pb0, pb1) : pack_bf16(pb0, pb1);      // row B, same column
                         l_sum2 = add_f32x2(l_sum2, pack_f32x2(pa0, pa1));
                         l_sum2b = add_f32x2(l_sum2b, pack_f32x2(pb0, pb1));
                     }
@@ -531,7 +576,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         mx4[(c >> 1) & 3] = max3(mx4[(c >> 1) & 3], __uint_as_float(sr[c >> 5][c & 31]),
                                                  __uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]));
                 }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_l2;
                 // lazy rescale: only when some row's maximum grew by more than 2^8
                 const bool grow = lane_has_row && mx > m_ref + 8.f;
                 if (j == 0) {
@@ -670,6 +715,11 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     a0 = 1.f / l_sum;
                     lse2 = m_ref + log2f(l_sum);
                 }
+                if (FP8) {   // the accumulators hold P times the V codes' half-precision images: 2^-8 / scale of the true values
+                    const float vm = p.mult[p.H + s.h];
+                    a0 *= vm;
+                    a1 *= vm;
+                }
                 if (nt > 0 && warp_has_rows) {
                     const uint32_t o_addr = tmem_base + ((uint32_t)lg << 16) + 256u + (uint32_t)(MODE_Y ? 0 : i) * 128u;
                     float* dst = p.o_part + (((int64_t)slot * p.part_rows + b) * p.H + s.h) * 128;
@@ -711,6 +761,107 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             used += nt;
             g += s.cnt;
         }
+    } else if (FP8) {
+        // ---------------- conversion warpgroup (warps 12-15; 8-bit cache only).
+        // The expanded K_nope and V of the prefix are stored as E4M3 codes with one power-of-two scale per head.
+        // Bulk copies bring 8 KB blocks of codes into staging slots; this warpgroup rewrites each block as the
+        // half-precision operand tile the MMAs read (same 128-byte-swizzled layouts as the 16-bit path).  A code
+        // (s eeee mmm) becomes the half-precision bit pattern s 0eeee mmm0000000: the same number times 2^-8,
+        // subnormal codes included, by two masks, a shift and an OR per pair.  The factors 2^8 * scale go where they
+        // cost nothing.  K: the query's nope part is only converted to half precision (once per segment, here), its
+        // rope part is divided by the factor (a power of two: exact), so the accumulated logits are the true ones
+        // divided by it, and the softmax scale is multiplied by it.  V: into the final normalisation.  The bytes of every 4-code group are stored in the order (0, 2, 1, 3), so
+        // that the pairs (0, 1) and (2, 3) come out of one 32-bit word without a byte shuffle.
+        const int ct = threadIdx.x - 384;
+        auto wg_sync = [] { asm volatile("bar.sync 3, 128;\n" ::: "memory"); };
+        auto widen = [](uint32_t w, uint32_t& lo, uint32_t& hi) {
+            const uint32_t v = w << 8;
+            lo = (v & 0x80008000u) | ((v & 0x7f007f00u) >> 1);   // codes 0, 1 of the group
+            hi = (w & 0x80008000u) | ((w & 0x7f007f00u) >> 1);   // codes 2, 3
+        };
+        // one 8 KB staging block (64 rows of 128 bytes, 16-byte chunks swizzled by the row) -> 16 KB operand tile.
+        // K: row = token, chunk = 16 dims, tile = two [64 tokens][64 dims] slabs.  V: row = two dims (64 tokens
+        // each), chunk = 16 tokens of one dim, tile = [128 dims][64 tokens].
+        auto convert = [&](const uint8_t* src, uint8_t* dst, bool is_v) {
+#pragma unroll
+            for (int it = 0; it < 4; ++it) {
+                const int u = it * 128 + ct, r = u >> 3, c = u & 7;
+                const uint4 w = *reinterpret_cast<const uint4*>(src + r * 128 + ((c ^ (r & 7)) << 4));
+                uint4 o0, o1;
+                widen(w.x, o0.x, o0.y);
+                widen(w.y, o0.z, o0.w);
+                widen(w.z, o1.x, o1.y);
+                widen(w.w, o1.z, o1.w);
+                const int row = is_v ? 2 * r + (c >> 2) : r;          // row of the operand tile
+                const int slab = is_v ? 0 : (c >> 2);
+                const int c0 = 2 * (c & 3);
+                uint8_t* d = dst + slab * 8192 + row * 128;
+                *reinterpret_cast<uint4*>(d + ((c0 ^ (row & 7)) << 4)) = o0;
+                *reinterpret_cast<uint4*>(d + (((c0 + 1) ^ (row & 7)) << 4)) = o1;
+            }
+        };
+        auto convert_k = [&](int ring) {
+            const int sq = ring % p.kq_stages, st = ring % p.k_stages;
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&bar->kq_full[sq], (ring / p.kq_stages) & 1, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(&bar->k_empty[st], ((ring / p.k_stages) & 1) ^ 1, abort_flag));
+            if (!ok) return false;
+            convert(sKq + sq * KQ_BYTES, sK + st * K_TILE_BYTES, false);
+            fence_proxy_async();   // the MMAs read the tile through the async proxy
+            wg_sync();
+            if (ct == 0) {
+                mbar_arrive(&bar->k_full[st]);
+                mbar_arrive(&bar->kq_empty[sq]);
+            }
+            return true;
+        };
+        auto convert_v = [&](int ring) {
+            const int sq = ring % p.vq_stages, st = ring % p.v_stages;
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&bar->vq_full[sq], (ring / p.vq_stages) & 1, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(&bar->v_empty[st], ((ring / p.v_stages) & 1) ^ 1, abort_flag));
+            if (!ok) return false;
+            convert(sVq + sq * VQ_BYTES, sV + st * V_TILE_BYTES, true);
+            fence_proxy_async();
+            wg_sync();
+            if (ct == 0) {
+                mbar_arrive(&bar->v_full[st]);
+                mbar_arrive(&bar->vq_empty[sq]);
+            }
+            return true;
+        };
+        int ring_base = 0, seg = 0;
+        bool ok = true;
+        for (int g = g_begin; g < g_end && ok; ++seg) {
+            const Segment s = segment_at(g);
+            // query tile (three slabs of 64 rows): nope part to half precision, rope part divided by 2^8 * scale
+            ok = __all_sync(0xffffffffu, mbar_wait(&bar->q_full, seg & 1, abort_flag));
+            if (!ok) break;
+            {
+                const float inv_km = __fdiv_rn(1.f, p.mult[s.h]);   // a power of two: exact
+#pragma unroll
+                for (int it = 0; it < 12; ++it) {
+                    uint4* qv = reinterpret_cast<uint4*>(sQ) + it * 128 + ct;
+                    uint4 w = *qv;
+                    uint32_t* e = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&e[k]));
+                        e[k] = it < 8 ? pack_f16(f.x, f.y) : pack_bf16(f.x * inv_km, f.y * inv_km);
+                    }
+                    *qv = w;
+                }
+                fence_proxy_async();
+                wg_sync();
+                if (ct == 0) mbar_arrive(&bar->q_conv);
+            }
+            // K runs one tile ahead of V: the logits product of a tile comes first, its V is needed a softmax later
+            for (int e = 0; e < s.cnt && ok; ++e) {
+                ok = convert_k(ring_base + e);
+                if (ok && e > 0) ok = convert_v(ring_base + e - 1);
+            }
+            if (ok) ok = convert_v(ring_base + s.cnt - 1);
+            ring_base += s.cnt;
+            g += s.cnt;
+        }
     }
 
     tc_fence_before();
@@ -720,13 +871,15 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         // barriers of the ring positions it issued last: the copies against them are the only ones that can still be
         // in flight.
         if (warp == 0 && g_begin < g_end) {
-            for (int pos = max(0, k_issued - p.k_stages); pos < k_issued; ++pos)
-                mbar_drain(&bar->k_full[pos % p.k_stages], (pos / p.k_stages) & 1);
+            uint64_t* const k_landed = FP8 ? bar->kq_full : bar->k_full;
+            for (int pos = max(0, k_issued - k_depth); pos < k_issued; ++pos)
+                mbar_drain(&k_landed[pos % k_depth], (pos / k_depth) & 1);
             mbar_drain(&bar->q_full, (q_issued - 1) & 1);
         }
         if (warp == 2 && g_begin < g_end) {
-            for (int pos = max(0, v_issued - p.v_stages); pos < v_issued; ++pos)
-                mbar_drain(&bar->v_full[pos % p.v_stages], (pos / p.v_stages) & 1);
+            uint64_t* const v_landed = FP8 ? bar->vq_full : bar->v_full;
+            for (int pos = max(0, v_issued - v_depth); pos < v_issued; ++pos)
+                mbar_drain(&v_landed[pos % v_depth], (pos / v_depth) & 1);
         }
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
         __syncthreads();
@@ -737,7 +890,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
 }  // namespace
 
 
-int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
+int naive_sm100_tile_tokens(int B, bool fp8) { return (fp8 || B <= 128) ? 64 : 128; }
 
 // Host-side plan (pure function of the sizes): number of tile ranges R and of partial slots.
 //
@@ -748,10 +901,11 @@ int naive_sm100_tile_tokens(int B) { return B <= 128 ? 64 : 128; }
 // pays the fixed cost and a partial slot; with 64-token tiles a further slot per head is also charged
 // the extra read it causes in the combine).  Stream-K is taken when its modelled cost is lower (by at
 // least 5% in the HBM-bound regime of 64-token tiles).
-void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots) {
-    const bool mode_y = B <= 128;
+void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots, bool fp8) {
+    // (8-bit cache: always 64-token tiles, row groups of 64 requests)
+    const bool mode_y = fp8 || B <= 128;
     const int tok = mode_y ? 64 : 128;
-    const int m_groups = mode_y ? 1 : (B + 255) / 256;
+    const int m_groups = fp8 ? (B + 63) / 64 : (mode_y ? 1 : (B + 255) / 256);
     const int n_tiles = (int)((Ls + tok - 1) / tok);
     const long long T = (long long)H * n_tiles;
     if (T <= 0) {
@@ -813,27 +967,28 @@ void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_r
 
 cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     if (a.B <= 0 || a.Ls <= 0 || a.n_ranges <= 0) return cudaSuccess;
+    const bool fp8 = a.fp8_mult != nullptr;
     CUtensorMap tm_qn, tm_qp;
     {
         uint64_t dims[3] = {128, (uint64_t)a.H, (uint64_t)a.B};
         uint64_t str[2] = {128 * 2, (uint64_t)a.H * 128 * 2};
-        uint32_t box[3] = {64, 1, 128};
+        uint32_t box[3] = {64, 1, fp8 ? 64u : 128u};
         cudaError_t e = make_tmap_bf16(&tm_qn, a.q_nope, 3, dims, str, box);
         if (e != cudaSuccess) return e;
     }
     {
         uint64_t dims[3] = {64, (uint64_t)a.H, (uint64_t)a.B};
         uint64_t str[2] = {64 * 2, (uint64_t)a.H * 64 * 2};
-        uint32_t box[3] = {64, 1, 128};
+        uint32_t box[3] = {64, 1, fp8 ? 64u : 128u};
         cudaError_t e = make_tmap_bf16(&tm_qp, a.q_pe, 3, dims, str, box);
         if (e != cudaSuccess) return e;
     }
-    const bool mode_y = a.B <= 128;
+    const bool mode_y = fp8 || a.B <= 128;
     const int tok = mode_y ? 64 : 128;
     NaiveSm100Params p{};
     p.B = a.B; p.H = a.H; p.Ls = a.Ls; p.Ls_pad = (a.Ls + 127) / 128 * 128;
     p.part_rows = a.part_rows > 0 ? a.part_rows : a.B;
-    p.m_groups = mode_y ? 1 : (a.B + 255) / 256;
+    p.m_groups = fp8 ? (a.B + 63) / 64 : (mode_y ? 1 : (a.B + 255) / 256);
     p.n_tiles = (a.Ls + tok - 1) / tok;
     p.n_ranges = a.n_ranges;
     {
@@ -843,26 +998,33 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
         p.rem = (int)(T % a.n_ranges);
     }
     p.n_seg_max = a.n_slots;
-    p.k_stages = mode_y ? 4 : 2;
-    p.v_stages = mode_y ? 4 : 1;
+    p.k_stages = fp8 ? 2 : (mode_y ? 4 : 2);
+    p.v_stages = fp8 ? 2 : (mode_y ? 4 : 1);
+    p.kq_stages = fp8 ? 5 : 0;
+    p.vq_stages = fp8 ? 5 : 0;
+    p.mult = a.fp8_mult;
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = a.status;
-    const int k_tile = tok * 384, v_tile = mode_y ? 16384 : 32768;
-    const int smem = (mode_y ? 1 : 2) * Q_TILE_BYTES + p.k_stages * k_tile + p.v_stages * v_tile + 1024 + (int)sizeof(Barriers) + 64;
+    const int k_tile = fp8 ? 16384 : tok * 384, v_tile = mode_y ? 16384 : 32768;
+    const int smem = (fp8 ? Q_TILE_BYTES / 2 : (mode_y ? 1 : 2) * Q_TILE_BYTES) + p.k_stages * k_tile + p.v_stages * v_tile +
+                     p.kq_stages * 16384 + p.vq_stages * 8192 + 1024 + (int)sizeof(Barriers) + 64;
     dim3 grid(p.n_ranges * p.m_groups, 1, 1);
     if (smem > kNaiveSmemMax) return cudaErrorInvalidValue;
+    if (fp8)
+        return launch_pdl(naive_attn_sm100_kernel<64, true, true>, grid, dim3(512), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     if (mode_y) {
         if (a.B <= 64)   // half-height MMAs: the padding rows 64..127 of the query tile cost tensor-pipe time and power
-            return launch_pdl(naive_attn_sm100_kernel<64, true>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
-        return launch_pdl(naive_attn_sm100_kernel<64, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+            return launch_pdl(naive_attn_sm100_kernel<64, true, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        return launch_pdl(naive_attn_sm100_kernel<64, false, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
     }
-    return launch_pdl(naive_attn_sm100_kernel<128, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+    return launch_pdl(naive_attn_sm100_kernel<128, false, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
 }
 
 cudaError_t set_attrs_naive_sm100() {
-    cudaError_t e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    cudaError_t e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<128, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
     return e;
 }
 
@@ -893,6 +1055,24 @@ cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const vo
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+cudaError_t make_naive_fp8_tmaps(const void* k8, const void* kpe, const void* v8, int H, int64_t Ls_pad,
+                                 CUtensorMap* tm_k8, CUtensorMap* tm_kp, CUtensorMap* tm_v8) {
+    // Both code arrays are [H][Ls_pad rows of 128 bytes]: a 64-token block of K is 64 token rows of 128 dims, a
+    // 64-token block of V^T is 128 dim rows of 64 tokens = 64 rows of 128 bytes.  The copies treat a row as 64
+    // 16-bit elements (the conversion warpgroup undoes the 128-byte swizzle when it reads the block).
+    for (int t = 0; t < 2; ++t) {
+        uint64_t dims[3] = {64, (uint64_t)Ls_pad, (uint64_t)H};
+        uint64_t str[2] = {128, (uint64_t)Ls_pad * 128};
+        uint32_t box[3] = {64, 64, 1};
+        cudaError_t e = make_tmap_bf16(t == 0 ? tm_k8 : tm_v8, t == 0 ? k8 : v8, 3, dims, str, box);
+        if (e != cudaSuccess) return e;
+    }
+    uint64_t dims[2] = {64, (uint64_t)Ls_pad};
+    uint64_t str[1] = {64 * 2};
+    uint32_t box[2] = {64, 64};
+    return make_tmap_bf16(tm_kp, kpe, 2, dims, str, box);
 }
 
 }  // namespace tmla

@@ -87,7 +87,7 @@ extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, 
     const int n_sm = sh->num_sms > 0 ? sh->num_sms : 148;
     int n_ranges = 0, n_slots = 0;
     if (sh->Ls > 0) {
-        naive_sm100_plan(B, H, sh->Ls, n_sm, 0, &n_ranges, &n_slots);
+        naive_sm100_plan(B, H, sh->Ls, n_sm, 0, &n_ranges, &n_slots, sh->fp8 != 0);
         if ((size_t)n_slots * per_split > kScratchBytes) {
             n_ranges = H;
             n_slots = 1;
@@ -104,6 +104,7 @@ extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, 
     if (n_slots > 0) {
         NaiveAttnSm100 na{q_nope, q_pe, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt, B, H, (int)sh->Ls, n_ranges, n_slots,
                           softmax_scale, o_part, lse_part, sh->status, B};
+        if (sh->fp8) na.fp8_mult = sh->fp8_f + 2 * H;
         e = launch_naive_attn_sm100(na, s);
         if (e != cudaSuccess) return api_cuda_fail(e);
         ++launches;

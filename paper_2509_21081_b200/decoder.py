@@ -16,7 +16,7 @@ class TyphoonMLADecoder:
 
     def __init__(self, num_heads: int, ckv_shared: torch.Tensor, kpe_shared: torch.Tensor,
                  w_uk: torch.Tensor, w_uv: torch.Tensor, softmax_scale: float,
-                 max_batch: int, max_pages: int, page_size: int = 64):
+                 max_batch: int, max_pages: int, page_size: int = 64, fp8_shared: bool = False):
         for t in (ckv_shared, kpe_shared, w_uk, w_uv):
             if not t.is_cuda or t.dtype != torch.bfloat16:
                 raise ValueError("all tensors must be bf16 CUDA tensors")
@@ -25,7 +25,8 @@ class TyphoonMLADecoder:
         self.page_size = int(page_size)
         self.max_batch, self.max_pages = int(max_batch), int(max_pages)
         self.w_uk, self.w_uv = w_uk.contiguous(), w_uv.contiguous()
-        self.shared = _b.typhoon_mla_prepare_shared(self.dims, ckv_shared, kpe_shared, self.w_uk, self.w_uv)
+        prepare = _b.typhoon_mla_prepare_shared_fp8 if fp8_shared else _b.typhoon_mla_prepare_shared
+        self.shared = prepare(self.dims, ckv_shared, kpe_shared, self.w_uk, self.w_uv)
         nbytes = _b.typhoon_mla_workspace_bytes(self.shared, self.max_batch, self.max_pages, self.page_size)
         self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
         sbytes = _b.typhoon_mla_host_staging_bytes(self.shared, self.max_batch, self.max_pages)

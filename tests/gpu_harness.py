@@ -13,7 +13,7 @@ LSE_TOL = 2e-2          # natural-log LSE; bf16 inputs, fp32 statistics
 
 
 def run_gpu(inp, mode, page_size=None, pages=None, want_lse=True, poison=True, min_max_pages=0,
-            force_max_pages=None):
+            force_max_pages=None, fp8_shared=False):
     from paper_2509_21081_b200 import binding as b
     from paper_2509_21081_b200.decoder import TyphoonMLADecoder
     cfg = inp.cfg
@@ -22,7 +22,7 @@ def run_gpu(inp, mode, page_size=None, pages=None, want_lse=True, poison=True, m
     dev = "cuda"
     max_pages = pc.block_table.shape[1] if force_max_pages is None else force_max_pages
     dec = TyphoonMLADecoder(cfg.H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), inp.w_uk.to(dev),
-                            inp.w_uv.to(dev), inp.scale, cfg.B, max_pages, ps)
+                            inp.w_uv.to(dev), inp.scale, cfg.B, max_pages, ps, fp8_shared=fp8_shared)
     lse = torch.empty(cfg.B, cfg.H, dtype=torch.float32, device=dev) if want_lse else None
     if force_max_pages == 0:
         out = dec.decode(inp.q_nope.to(dev), inp.q_pe.to(dev), None, None, None, None, mode=mode, lse_out=lse)
@@ -42,6 +42,16 @@ def run_oracle(inp, pairs=None, drop_suffix=False):
     kpe_suf = [f(x[:0] if drop_suffix else x) for x in inp.kpe_suffix]
     return O.mla_decode(f(inp.q_nope), f(inp.q_pe), f(inp.ckv_shared), f(inp.kpe_shared), ckv_suf, kpe_suf,
                         f(inp.w_uk), f(inp.w_uv), inp.scale, pairs=pairs)
+
+
+def run_oracle_fp8(inp, pairs=None, drop_suffix=False):
+    """The checker for a prefix whose expanded K_nope / V are stored as E4M3 codes."""
+    from oracle import fp8_oracle as F
+    f = I.to_f64
+    ckv_suf = [f(x[:0] if drop_suffix else x) for x in inp.ckv_suffix]
+    kpe_suf = [f(x[:0] if drop_suffix else x) for x in inp.kpe_suffix]
+    return F.mla_decode_fp8_shared(f(inp.q_nope), f(inp.q_pe), f(inp.ckv_shared), f(inp.kpe_shared), ckv_suf, kpe_suf,
+                                   f(inp.w_uk), f(inp.w_uv), inp.scale, pairs=pairs)
 
 
 def errors(gpu, ref, mask=None):

@@ -1,0 +1,134 @@
+"""GPU parity of the 8-bit (E4M3) expanded shared-prefix cache: the stored codes against the checker's encoder, and the
+decode step against the checker's operator over the decoded values.  The kernel widens the codes exactly and then
+computes as the 16-bit path does, so the bars are the 16-bit path's (max-abs 2e-2, relative Frobenius 5e-3, LSE 2e-2);
+what the encoding itself costs is measured against the unencoded definition and reported, not asserted tightly."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fp8_oracle as F
+from oracle import mla_oracle as O
+from paper_2509_21081_b200 import inputs as I
+from tests import gpu_harness as G
+
+pytestmark = pytest.mark.gpu
+
+ABSORB, HYBRID, AUTO, NAIVE = 1, 2, 0, 3
+
+
+def _cfg(name, B, H, Ls, lo, hi, seed, page_size=64):
+    return I.MLAConfig(name, B=B, H=H, Ls=Ls, suffix_lo=lo, suffix_hi=hi, seed=seed, page_size=page_size)
+
+
+@pytest.mark.parametrize("H,Ls", [(16, 200), (32, 777)])
+def test_codes_and_scales_match_the_encoder(H, Ls):
+    """Every stored code equals the checker's, except where the 16-bit expansion itself (fp32 accumulation on the GPU,
+    exact in the checker) rounds to a neighbouring bfloat16: there the two codes must be adjacent, and such places must
+    be rare.  Scales are equal exactly; padding tokens hold code 0."""
+    from paper_2509_21081_b200 import binding as b
+    inp = I.make_inputs(_cfg("codes", B=1, H=H, Ls=Ls, lo=0, hi=0, seed=77))
+    dims = b.make_dims(H)
+    w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
+    sh = b.typhoon_mla_prepare_shared_fp8(dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    kc, vc, sc = b.typhoon_mla_shared_export_fp8(sh)
+    assert b.typhoon_mla_check_status(sh) == 0
+    kc, vc, sc = kc.cpu().numpy(), vc.cpu().numpy(), sc.cpu().double().numpy()
+    Lp = kc.shape[1]
+    assert Lp % 128 == 0 and Lp >= Ls
+    f = I.to_f64
+    table = F.e4m3_decode_table()
+    n_diff = 0
+    for h in range(H):
+        K = O.decompress_head(f(inp.ckv_shared), f(inp.w_uk)[h])          # [Ls, 128]
+        V = O.decompress_head(f(inp.ckv_shared), f(inp.w_uv)[h])
+        ck, sk = F.encode_head(K)
+        cv, sv = F.encode_head(V)
+        assert sc[0, h] == sk and sc[1, h] == sv
+        got_k = kc[h, :Ls]                                                  # [Ls, 128]
+        got_v = vc[h].transpose(0, 2, 1).reshape(Lp, 128)[:Ls]              # blocks [128 dims, 64 tok] -> [tok, dim]
+        for got, want in ((got_k, ck), (got_v, cv)):
+            d = got != want
+            n_diff += int(d.sum())
+            if d.any():   # neighbours in value: same sign (or a zero), magnitude codes one apart
+                g, w = got[d].astype(int), want[d].astype(int)
+                assert np.all(np.abs((g & 0x7F) - (w & 0x7F)) <= 1)
+                assert np.all(((g ^ w) & 0x80 == 0) | ((g & 0x7F) + (w & 0x7F) <= 1))
+        assert not kc[h, Ls:].any() and not vc[h].transpose(0, 2, 1).reshape(Lp, 128)[Ls:].any()
+    assert n_diff <= 2e-3 * 2 * H * Ls * 128, n_diff
+    sh.free()
+
+
+@pytest.mark.parametrize("B,H,Ls,hi", [(4, 16, 256, 64), (9, 16, 331, 300), (64, 128, 520, 100), (37, 48, 1000, 70),
+                                       (70, 64, 520, 90), (130, 16, 700, 50), (200, 32, 450, 0)])
+@pytest.mark.parametrize("mode", [HYBRID, NAIVE])
+def test_decode_matches_the_checker_over_decoded_values(B, H, Ls, hi, mode):
+    """One and several 64-request row groups, ragged prefixes, several head counts; HYBRID and (no suffix) NAIVE."""
+    cfg = _cfg("fp8", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=300 + B)
+    inp = I.make_inputs(cfg)
+    drop = mode == NAIVE
+    ref, ref_lse = G.run_oracle_fp8(inp, drop_suffix=drop)
+    out, lse, launches = G.run_gpu(inp, mode, fp8_shared=True, force_max_pages=0 if drop else None)
+    assert launches > 0
+    G.assert_parity(out, ref, lse, ref_lse, what=f"fp8 B={B} H={H} Ls={Ls} mode={mode}")
+    # what the encoding costs against the unencoded definition: well above the kernel's own error, far below 1
+    plain, _ = G.run_oracle(inp, drop_suffix=drop)
+    _, rel = G.errors(ref, plain)
+    assert 1e-3 < rel < 0.1, rel
+
+
+@pytest.mark.parametrize("schedule", [1, 2])
+def test_work_decompositions(schedule):
+    from paper_2509_21081_b200 import binding as b
+    b.typhoon_mla_set_naive_schedule(schedule)
+    try:
+        inp = I.make_inputs(_cfg("fp8s", B=100, H=32, Ls=1500, lo=0, hi=40, seed=311))
+        ref, ref_lse = G.run_oracle_fp8(inp)
+        out, lse, _ = G.run_gpu(inp, HYBRID, fp8_shared=True)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"fp8 schedule {schedule}")
+    finally:
+        b.typhoon_mla_set_naive_schedule(0)
+
+
+def test_absorb_mode_and_empty_prefix_do_not_touch_the_codes():
+    """ABSORB mode attends over the 16-bit latent copy of the prefix: the plain definition is the expected value.
+    An empty prefix has nothing to encode."""
+    inp = I.make_inputs(_cfg("fp8a", B=5, H=32, Ls=400, lo=1, hi=200, seed=312))
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, ABSORB, fp8_shared=True)
+    G.assert_parity(out, ref, lse, ref_lse, what="fp8 handle, ABSORB")
+    inp = I.make_inputs(_cfg("fp8e", B=3, H=16, Ls=0, lo=5, hi=100, seed=313))
+    ref, ref_lse = G.run_oracle(inp)
+    out, lse, _ = G.run_gpu(inp, HYBRID, fp8_shared=True)
+    G.assert_parity(out, ref, lse, ref_lse, what="fp8 handle, no prefix")
+
+
+def test_footprint_is_halved_and_other_paths_refuse():
+    from paper_2509_21081_b200 import binding as b
+    inp = I.make_inputs(_cfg("fp8f", B=2, H=16, Ls=1024, lo=0, hi=10, seed=314))
+    dims = b.make_dims(16)
+    args = (dims, inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), inp.w_uk.cuda(), inp.w_uv.cuda())
+    s16 = b.typhoon_mla_prepare_shared(*args)
+    s8 = b.typhoon_mla_prepare_shared_fp8(*args)
+    _, Lp, own16 = b.typhoon_mla_shared_view(s16)
+    _, _, own8 = b.typhoon_mla_shared_view(s8)
+    expanded16 = 2 * 16 * Lp * 128 * 2
+    assert own16 - own8 == expanded16 // 2 - 16 * 5 * 4      # codes are half the bytes; plus the per-head factors
+    with pytest.raises(b.TyphoonMLAError):
+        b.typhoon_mla_shared_export(s8)
+    with pytest.raises(b.TyphoonMLAError):
+        b.typhoon_mla_shared_export_fp8(s16)
+    # the warp-MMA cross-check kernels have no 8-bit path: refused, nothing launched
+    pc = I.build_pages(inp)
+    ws = torch.empty(b.typhoon_mla_workspace_bytes(s8, 2, pc.block_table.shape[1], 64), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(2, 16, 128, dtype=torch.bfloat16, device="cuda")
+    b.typhoon_mla_set_kernel_path(b.PATH_WARP_MMA)
+    try:
+        with pytest.raises(b.TyphoonMLAError):
+            b.typhoon_mla_decode(s8, inp.q_nope.cuda(), inp.q_pe.cuda(), pc.ckv_pages.cuda(), pc.kpe_pages.cuda(), 64,
+                                 pc.block_table.cuda(), pc.seq_lens.cuda(), inp.scale, out, ws, mode=HYBRID)
+    finally:
+        b.typhoon_mla_set_kernel_path(b.PATH_TCGEN05)
+    torch.cuda.synchronize()
+    assert not out.any()
+    s16.free()
+    s8.free()
