@@ -51,9 +51,9 @@ def _peaks():
 
 
 # ------------------------------------------------------------------ work accounting
-def algorithmic_work(cfg, suffix_lens, mode_name):
+def algorithmic_work(cfg, suffix_lens, mode_name, fp8=False):
     """Algorithmic flops and bytes of one step (Table 1 terms plus the once-only reads of q and the
-    weights and the write of out)."""
+    weights and the write of out); with the 8-bit expanded cache K_nope and V cost one byte per element."""
     H, B, Ls = cfg.H, cfg.B, cfg.Ls
     sum_ln = sum(suffix_lens)
     W = 4 * H * 65536
@@ -62,16 +62,16 @@ def algorithmic_work(cfg, suffix_lens, mode_name):
         bytes_ = 1152 * Ls + W + 1152 * sum_ln + 640 * H * B
     else:
         flops = H * (640 * B * Ls + 2176 * sum_ln + 4 * 65536 * B)
-        bytes_ = (512 * H + 128) * Ls + W + 1152 * sum_ln + 640 * H * B
+        bytes_ = ((256 if fp8 else 512) * H + 128) * Ls + W + 1152 * sum_ln + 640 * H * B
     return flops, bytes_
 
 
-def dominant_kernel(cfg, suffix_lens, mode_name):
+def dominant_kernel(cfg, suffix_lens, mode_name, fp8=False):
     """(kernel id, name, bound, algorithmic bytes per launch, flops per launch) of the kernel that
     carries most of the step's roofline time."""
     H, B, Ls = cfg.H, cfg.B, cfg.Ls
     sum_ln = sum(suffix_lens)
-    naive_bytes = (512 * H + 128) * Ls + 384 * B * H          # expanded K/V + rope keys once, q once
+    naive_bytes = ((256 if fp8 else 512) * H + 128) * Ls + 384 * B * H   # expanded K/V + rope keys once, q once
     naive_flops = 640 * B * H * Ls
     if mode_name == "absorb":
         absorb_bytes = 1152 * (B * Ls + sum_ln) + 1152 * B * H   # latent tokens per request + Q_A|q_pe
@@ -225,7 +225,7 @@ def _workload_name(cfg):
             f"page={cfg.page_size} d=(128,64,128,512) bf16")
 
 
-def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with_e2e=True, max_steps=None):
+def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with_e2e=True, max_steps=None, fp8=False):
     """One configuration: K steps per timed region, the region repeated until MIN_REGION_MS of GPU time
     has been measured (median of the repeats reported; the clock sampler runs over all of them), then
     the dominant kernel's duration inside the step and alone, optionally per-stage times, the end-to-end
@@ -252,7 +252,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         # has paid for context and module loading
         pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         pe0.record()
-        dec = TyphoonMLADecoder(cfg.H, *dev_in, inp.scale, cfg.B, max_pages, pc.page_size)
+        dec = TyphoonMLADecoder(cfg.H, *dev_in, inp.scale, cfg.B, max_pages, pc.page_size, fp8_shared=fp8)
         pe1.record()
         if k == 1:
             torch.cuda.synchronize()
@@ -280,7 +280,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
     torch.cuda.synchronize()
     launches_per_step = b.typhoon_mla_last_launch_count()
     assert b.typhoon_mla_check_status(sets[0]["dec"].shared) == 0 and b.typhoon_mla_check_status(sets[1]["dec"].shared) == 0
-    kid, kname, k_bytes, k_flops = dominant_kernel(cfg, inp.suffix_lens, mode_name)
+    kid, kname, k_bytes, k_flops = dominant_kernel(cfg, inp.suffix_lens, mode_name, fp8)
 
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -341,11 +341,11 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         roof = {"bound": "tensor", "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / pk["bf16_tflops_sustained"], "frac_of_burst_peak": achieved / pk["bf16_tflops"],
                 "burst_peak": pk["bf16_tflops"]}
-    roof.update({"traffic": NCU_TRAFFIC_BYTES.get((cfg.name, kname)), "kernel": kname,
+    roof.update({"traffic": None if fp8 else NCU_TRAFFIC_BYTES.get((cfg.name, kname)), "kernel": kname,
                  "kernel_ms": k_avg_s * 1e3, "launches_timed": k_n,
                  "ms_per_step_with_kernel_events": instrumented_ms_per_step, "peak_source": pk["source"],
                  "algorithmic_bytes": k_bytes, "algorithmic_flops": k_flops})
-    flops, bytes_ = algorithmic_work(cfg, inp.suffix_lens, mode_name)
+    flops, bytes_ = algorithmic_work(cfg, inp.suffix_lens, mode_name, fp8)
     t_lb = max(flops / (pk["bf16_tflops"] * 1e12), bytes_ / (pk["hbm_gbs"] * 1e9))
     roof["step_frac_of_combined_roofline"] = t_lb / (ms_per_step * 1e-3)
     # The same kernel with the side stream switched off (every kernel alone on the GPU), outside the
@@ -406,7 +406,7 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
             s = sets[k % n_sets]
             dec = s["dec"] if k < n_sets else TyphoonMLADecoder(
                 cfg.H, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), s["dec"].w_uk, s["dec"].w_uv, inp.scale,
-                cfg.B, max_pages, pc.page_size)
+                cfg.B, max_pages, pc.page_size, fp8_shared=fp8)
             lanes.append(dict(dec=dec, ckv=s["ckv"], kpe=s["kpe"], stream=torch.cuda.Stream(),
                               h=(inp.q_nope.pin_memory(), inp.q_pe.pin_memory(), pc.block_table.pin_memory(),
                                  pc.seq_lens.pin_memory(),
@@ -483,7 +483,8 @@ def bench_config(cfg, args, mode, rank, world, device_index, with_cpu=True, with
         s["dec"].close()
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
+            "dtype": "bf16" if not fp8 else "bf16 (expanded shared K/V stored as e4m3 codes, widened exactly to f16 operands)",
+            "data": "synthetic",
             # `config` names the workload and how L2 is kept cold; how this arm ran it is in `run`
             "config": {"workload": _workload_name(cfg),
                        "l2": f"{n_sets} full input sets used alternately, each larger than the 126 MB L2"},
@@ -778,6 +779,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
                     help="device time every timed region is repeated up to (0: each region once, e.g. under a profiler)")
+    ap.add_argument("--fp8-shared", action="store_true",
+                    help="extension: expanded shared-prefix K/V stored as E4M3 codes (typhoon_mla_prepare_shared_fp8)")
     ap.add_argument("--no-extra", action="store_true", help="headline configuration only (skip the other configurations' short lines)")
     args = ap.parse_args()
     globals()["MIN_REGION_MS"] = max(args.min_region_ms, 0.0)
@@ -833,9 +836,18 @@ def main():
         if args.batch:
             cfg = cfg.with_batch(args.batch)
         line = bench_config(cfg, args, mode, rank, world, local, with_cpu=not args.no_cpu,
-                            with_e2e=not args.no_e2e)
-        if args.config == "cfg1" and not args.batch and args.mode == "auto" and not args.no_extra:
+                            with_e2e=not args.no_e2e, fp8=args.fp8_shared)
+        if args.config == "cfg1" and not args.batch and args.mode == "auto" and not args.no_extra and not args.fp8_shared:
             line["extra_configs"] = bench_extra_configs(args, rank, world, local)
+            # the headline workload once more with the expanded cache in 8 bits (an extension: not the headline's precision)
+            ln = bench_config(cfg, args, mode, rank, world, local, with_cpu=False, with_e2e=False, max_steps=20, fp8=True)
+            r = ln["roofline"]
+            line["fp8_shared_cache"] = {
+                "workload": ln["config"]["workload"], "storage": ln["dtype"], "mode": ln["run"]["mode"], "value": ln["value"],
+                "ms_per_step": ln["ms_per_step"], "steps": ln["steps"], "timed_regions": ln["timed_regions"],
+                "dominant_kernel": r["kernel"], "bound": r["bound"], "frac": r["frac"], "frac_alone": r["frac_alone"],
+                "kernel_ms": r["kernel_ms"], "kernel_ms_alone": r["kernel_ms_alone"], "algorithmic_bytes": r["algorithmic_bytes"],
+                "step_frac_of_combined_roofline": r["step_frac_of_combined_roofline"]}
         if rank == 0:
             print(json.dumps(line), flush=True)
     if world > 1:

@@ -117,9 +117,11 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims /* host */,
  * fp32 accumulation), so the only error added is that of the encoding.  Queries must be
  * within half precision's range (|q| < 65504).  The handle is used like any other
  * (decode, decode_tree, decode_partial, the no-alloc call; AUTO / ABSORB / HYBRID /
- * NAIVE); the shared-prefix kernel then works on row groups of 64 requests, so for
- * B > 128 it is slower than with the 16-bit cache.  A 16-bit scratch of the size of one
- * expanded tensor is taken from and returned to the stream's memory pool inside the call.
+ * NAIVE).  The option trades speed for memory: widening the codes inside the kernel
+ * costs more than the halved traffic saves, and the shared-prefix kernel then works on
+ * row groups of at most 128 requests (measured on B200: steps 1.3 to 1.7 times as long
+ * as with the 16-bit cache).  A 16-bit scratch of the size of one expanded tensor is taken
+ * from and returned to the stream's memory pool inside the call.
  * Arguments and errors as typhoon_mla_prepare_shared.
  */
 int typhoon_mla_prepare_shared_fp8(const typhoon_mla_dims_t* dims /* host */,

@@ -392,7 +392,7 @@ static int prepare_impl(const typhoon_mla_dims_t* dims, const void* ckv_shared, 
     if (ok_alloc && !sh->fp8) ok_alloc = alloc(&sh->k_nope, b_k) && alloc(&sh->v_t, b_k);
     if (ok_alloc && sh->fp8)
         ok_alloc = alloc(&sh->k8, b_k / 2) && alloc(&sh->v8, b_k / 2) &&
-                   alloc(reinterpret_cast<void**>(&sh->fp8_f), (size_t)H * 5 * sizeof(float));
+                   alloc(reinterpret_cast<void**>(&sh->fp8_f), (size_t)H * 3 * sizeof(float));
     if (!ok_alloc) {
         typhoon_mla_free(sh);
         return TYPHOON_MLA_ERR_ALLOC;
@@ -431,16 +431,16 @@ static int prepare_impl(const typhoon_mla_dims_t* dims, const void* ckv_shared, 
                      (int)Lp, 128, 512, H, false, 0, true};
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
             if (e == cudaSuccess && sh->fp8)
-                e = launch_quantize_e4m3(k_dst, false, H, (int64_t)Lp, sh->k8, reinterpret_cast<uint32_t*>(sh->fp8_f + 4 * H),
-                                         sh->fp8_f, sh->fp8_f + 2 * H, s);
+                e = launch_quantize_e4m3(k_dst, false, H, (int64_t)Lp, sh->k8, reinterpret_cast<uint32_t*>(sh->fp8_f + 2 * H),
+                                         sh->fp8_f, s);
         }
         if (e == cudaSuccess) {  // V^T[h] = W_UV[h] * ckv^T
             GemmTN g{w_uv, 512, 128 * 512, sh->ckv, 512, 0, v_dst, (int64_t)Lp, (int64_t)(128 * Lp),
                      128, (int)Lp, 512, H, false, 64};
             e = tc ? launch_gemm_tn_sm100(g, sh->status, s) : launch_gemm_tn(g, s);
             if (e == cudaSuccess && sh->fp8)
-                e = launch_quantize_e4m3(v_dst, true, H, (int64_t)Lp, sh->v8, reinterpret_cast<uint32_t*>(sh->fp8_f + 4 * H),
-                                         sh->fp8_f + H, sh->fp8_f + 3 * H, s);
+                e = launch_quantize_e4m3(v_dst, true, H, (int64_t)Lp, sh->v8, reinterpret_cast<uint32_t*>(sh->fp8_f + 2 * H),
+                                         sh->fp8_f + H, s);
         }
     }
     if (scratch16) {
@@ -561,8 +561,8 @@ int typhoon_mla_shared_export_fp8(const typhoon_mla_shared_t* sh, void* k_codes_
     const int H = sh->dims.num_heads;
     const size_t n = (size_t)H * (size_t)sh->Ls_pad * 128;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_unpermute_codes(sh->k8, k_codes_dst, n, s);
-    if (e == cudaSuccess) e = launch_unpermute_codes(sh->v8, v_codes_dst, n, s);
+    cudaError_t e = cudaMemcpyAsync(k_codes_dst, sh->k8, n, cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(v_codes_dst, sh->v8, n, cudaMemcpyDeviceToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(scales_dst, sh->fp8_f, (size_t)2 * H * sizeof(float), cudaMemcpyDeviceToDevice, s);
     return e == cudaSuccess ? TYPHOON_MLA_OK : cuda_fail(e);
 }
@@ -659,7 +659,7 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         if (tc) {
             NaiveAttnSm100 na{qn, qp, &jb.sh->tm_kn, &jb.sh->tm_kp, &jb.sh->tm_vt, jb.rows, H, (int)jb.sh->Ls,
                               jb.n_ranges, jb.n_slots_level, softmax_scale, op, lp, sh->status, B};
-            if (jb.sh->fp8) na.fp8_mult = jb.sh->fp8_f + 2 * H;
+            if (jb.sh->fp8) na.fp8_mult = jb.sh->fp8_f;
             e = launch_naive_attn_sm100(na, s);
         } else {
             NaiveAttn na{qn, qp, jb.sh->k_nope, jb.sh->v_t, jb.sh->kpe, B, H, (int)jb.sh->Ls, (int)jb.sh->Ls_pad,

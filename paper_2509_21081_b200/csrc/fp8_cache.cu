@@ -32,8 +32,8 @@ __global__ void amax_kernel(const uint4* __restrict__ src, size_t vec_per_head, 
     if ((threadIdx.x & 31) == 0 && m) atomicMax(&amax_bits[h], m);
 }
 
-// scale[h] = 2^e, mult[h] = 2^(e + 8), e the smallest integer with amax <= 448 * 2^e (e = 0 for an all-zero head)
-__global__ void scale_kernel(const uint32_t* __restrict__ amax_bits, int H, float* __restrict__ scale, float* __restrict__ mult) {
+// scale[h] = 2^e, e the smallest integer with amax <= 448 * 2^e (e = 0 for an all-zero head)
+__global__ void scale_kernel(const uint32_t* __restrict__ amax_bits, int H, float* __restrict__ scale) {
     const int h = blockIdx.x * blockDim.x + threadIdx.x;
     if (h >= H) return;
     const float amax = __uint_as_float(amax_bits[h] << 16);
@@ -44,7 +44,6 @@ __global__ void scale_kernel(const uint32_t* __restrict__ amax_bits, int H, floa
         e = (m <= 1.75f) ? E - 8 : E - 7;                 // 448 = 1.75 * 2^8
     }
     scale[h] = ldexpf(1.f, e);
-    mult[h] = ldexpf(1.f, e + 8);
 }
 
 __device__ __forceinline__ uint32_t encode4(uint2 v, float inv_scale) {
@@ -54,7 +53,7 @@ __device__ __forceinline__ uint32_t encode4(uint2 v, float inv_scale) {
     const uint32_t c1 = __nv_cvt_float_to_fp8(a.y * inv_scale, __NV_SATFINITE, __NV_E4M3);
     const uint32_t c2 = __nv_cvt_float_to_fp8(b.x * inv_scale, __NV_SATFINITE, __NV_E4M3);
     const uint32_t c3 = __nv_cvt_float_to_fp8(b.y * inv_scale, __NV_SATFINITE, __NV_E4M3);
-    return c0 | (c2 << 8) | (c1 << 16) | (c3 << 24);      // stored byte order (0, 2, 1, 3)
+    return c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
 }
 
 // K_nope: bf16 [H, Lp/64, 2 slabs, 64 tokens, 64 dims] -> codes [H, Lp tokens, 128 dims]; one thread per 4 codes
@@ -81,24 +80,17 @@ __global__ void quantize_v_kernel(const uint2* __restrict__ src, const float* __
         dst[(int64_t)h * n + i] = encode4(src[(int64_t)h * n + i], inv);
 }
 
-__global__ void unpermute_kernel(const uint32_t* __restrict__ src, uint32_t* __restrict__ dst, size_t n_words) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += (size_t)gridDim.x * blockDim.x) {
-        const uint32_t w = src[i];
-        dst[i] = (w & 0xff0000ffu) | ((w & 0x0000ff00u) << 8) | ((w & 0x00ff0000u) >> 8);
-    }
-}
-
 }  // namespace
 
 cudaError_t launch_quantize_e4m3(const void* src_bf16, bool is_v, int H, int64_t Ls_pad, void* dst_codes, uint32_t* amax_bits,
-                                 float* scale_out, float* mult_out, cudaStream_t s) {
+                                 float* scale_out, cudaStream_t s) {
     if (H <= 0 || Ls_pad <= 0) return cudaSuccess;
     cudaError_t e = cudaMemsetAsync(amax_bits, 0, (size_t)H * sizeof(uint32_t), s);
     if (e != cudaSuccess) return e;
     const size_t vec_per_head = (size_t)Ls_pad * 128 * 2 / 16;
     const int bx = (int)std::min<size_t>((vec_per_head + 255) / 256, 64);
     amax_kernel<<<dim3(bx, H), 256, 0, s>>>(reinterpret_cast<const uint4*>(src_bf16), vec_per_head, amax_bits);
-    scale_kernel<<<(H + 127) / 128, 128, 0, s>>>(amax_bits, H, scale_out, mult_out);
+    scale_kernel<<<(H + 127) / 128, 128, 0, s>>>(amax_bits, H, scale_out);
     const int qx = (int)std::min<int64_t>((Ls_pad * 32 + 255) / 256, 256);
     if (is_v)
         quantize_v_kernel<<<dim3(qx, H), 256, 0, s>>>(reinterpret_cast<const uint2*>(src_bf16), scale_out, Ls_pad,
@@ -106,14 +98,6 @@ cudaError_t launch_quantize_e4m3(const void* src_bf16, bool is_v, int H, int64_t
     else
         quantize_k_kernel<<<dim3(qx, H), 256, 0, s>>>(reinterpret_cast<const uint2*>(src_bf16), scale_out, Ls_pad,
                                                       reinterpret_cast<uint32_t*>(dst_codes));
-    return cudaGetLastError();
-}
-
-cudaError_t launch_unpermute_codes(const void* src, void* dst, size_t n, cudaStream_t s) {
-    if (n == 0) return cudaSuccess;
-    const size_t words = n / 4;
-    unpermute_kernel<<<(int)std::min<size_t>((words + 255) / 256, 4096), 256, 0, s>>>(reinterpret_cast<const uint32_t*>(src),
-                                                                                       reinterpret_cast<uint32_t*>(dst), words);
     return cudaGetLastError();
 }
 

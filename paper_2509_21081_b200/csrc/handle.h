@@ -30,6 +30,5 @@ struct typhoon_mla_shared {
     int fp8;
     void* k8;       // E4M3 codes [H, Ls_pad, 128]: token rows of 128 dims
     void* v8;       // E4M3 codes [H, Ls_pad/64, 128, 64]: V^T in 64-token blocks
-    float* fp8_f;   // device [4][H] floats: scale of K_nope, scale of V, 2^8 * scale of K_nope, 2^8 * scale of V;
-                    // then [H] words of scratch for the amax reduction
+    float* fp8_f;   // device [2][H] floats: scale of K_nope, scale of V; then [H] words of scratch for the amax reduction
 };

@@ -98,7 +98,7 @@ struct NaiveAttnSm100 {
     float* lse_part; // [slots][part_rows][H]
     int* status;     // device word, set non-zero if a bounded wait expired
     int part_rows = 0;   // rows of the partial arrays; 0 = B (a launch may fill a row range of a larger batch)
-    // 8-bit cache: device [2][H] factors 2^8 * scale of K_nope and V (tm_kn / tm_vt then describe the code arrays,
+    // 8-bit cache: device [2][H] power-of-two scales of K_nope and V (tm_kn / tm_vt then describe the code arrays,
     // see make_naive_fp8_tmaps); null for the 16-bit cache
     const float* fp8_mult = nullptr;
 };
@@ -115,12 +115,10 @@ cudaError_t make_naive_sm100_tmaps(const void* k_nope, const void* kpe, const vo
 cudaError_t make_naive_fp8_tmaps(const void* k8, const void* kpe, const void* v8, int H, int64_t Ls_pad,
                                  CUtensorMap* tm_k8, CUtensorMap* tm_kp, CUtensorMap* tm_v8);
 // Expanded 16-bit cache of one tensor (k_nope or v_t layout) -> per-head power-of-two scale (smallest 2^e with
-// amax / 2^e <= 448) and E4M3 codes (round to nearest even) in the layouts above, the four codes of a group
-// stored in byte order (0, 2, 1, 3).  scale_out[h] = 2^e, mult_out[h] = 2^(e + 8); amax_bits is a scratch of H words.
+// amax / 2^e <= 448) and E4M3 codes (round to nearest even) in the layouts above.  scale_out[h] = 2^e; amax_bits is
+// a scratch of H words.
 cudaError_t launch_quantize_e4m3(const void* src_bf16, bool is_v, int H, int64_t Ls_pad, void* dst_codes, uint32_t* amax_bits,
-                                 float* scale_out, float* mult_out, cudaStream_t s);
-// Codes in the stored byte order -> codes in logical order (tests), n multiple of 4.
-cudaError_t launch_unpermute_codes(const void* src, void* dst, size_t n, cudaStream_t s);
+                                 float* scale_out, cudaStream_t s);
 
 // Absorb attention partials over latent tokens (Algorithm 1 line 6).
 struct AbsorbAttn {

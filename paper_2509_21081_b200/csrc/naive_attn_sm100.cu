@@ -69,7 +69,7 @@ struct NaiveSm100Params {
     int n_seg_max;         // partial slots per head (one per segment of the head)
     int k_stages, v_stages;
     int kq_stages, vq_stages;   // 8-bit cache: depth of the staging rings the copies land in
-    const float* mult;          // 8-bit cache: [2][H] factors 2^8 * scale of K_nope and of V, per head
+    const float* mult;          // 8-bit cache: [2][H] power-of-two scales of K_nope and of V, per head
     float scale_log2;
     float* o_part;     // [n_slots][part_rows][H][128]
     float* lse_part;   // [n_slots][part_rows][H]
@@ -120,9 +120,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
     constexpr int K_SLAB = TOK * 128;                   // bytes of one [TOK][64] K slab
     constexpr int K_TILE_BYTES = (FP8 ? 2 : 3) * K_SLAB;   // (8-bit cache: the rope slab stays in the staging ring)
     constexpr int V_TILE_BYTES = BLK * 16384;           // BLK slabs [128 dims][64 tokens]
-    constexpr int ROWS = FP8 ? 64 : (MODE_Y ? 128 : 256);   // query rows per column
-    static_assert(!FP8 || (M64 && TOK == 64), "the 8-bit cache path is built for 64-row, 64-token tiles");
-    constexpr int Q_SLAB = (FP8 ? 64 : 128) * 128;      // bytes of one [rows][64] slab of the query tile
+    constexpr int ROWS = FP8 ? (M64 ? 64 : 128) : (MODE_Y ? 128 : 256);   // query rows per column
+    static_assert(!FP8 || TOK == 64, "the 8-bit cache path is built for 64-token tiles");
+    constexpr int Q_SLAB = ((FP8 && M64) ? 64 : 128) * 128;   // bytes of one [rows][64] slab of the query tile
     constexpr int Q_BYTES = 3 * Q_SLAB;
     constexpr int KQ_BYTES = 16384, VQ_BYTES = 8192;    // staging slots: K codes 8 KB + rope keys 8 KB; V codes 8 KB
 
@@ -454,7 +454,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const bool warp_has_rows = tile_row0 + (M64 ? (warp & 3) * 16 : lg) < p.B;   // warp-uniform: the warp's first row is a real request
             float m_ref = -INFINITY, m_ref_b = -INFINITY;   // (M = 64: reference exponents of this thread's rows A and B)
             uint64_t l_sum2 = pack_f32x2(0.f, 0.f), l_sum2b = pack_f32x2(0.f, 0.f);   // row sum of the probabilities, as four partial sums
-            // (8-bit cache: the accumulated logits are the true ones divided by 2^8 * scale of this head's K, see below)
+            // (8-bit cache: the accumulated logits are the true ones divided by the scale of this head's K, see below)
             const float scale_l2 = FP8 ? p.scale_log2 * p.mult[s.h] : p.scale_log2;
             const uint64_t scale2 = pack_f32x2(scale_l2, scale_l2);
             for (int j = 0; j < nt && ok; ++j) {
@@ -615,7 +615,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         float x0, x1;
                         unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(src[2 * c]), __uint_as_float(src[2 * c + 1])), scale2, neg_m2), x0, x1);
                         const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                        dst[c] = pack_bf16(p0, p1);
+                        dst[c] = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
                         if (c & 1) l_sum2b = add_f32x2(l_sum2b, pack_f32x2(p0, p1));
                         else l_sum2 = add_f32x2(l_sum2, pack_f32x2(p0, p1));
                     }
@@ -715,7 +715,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     a0 = 1.f / l_sum;
                     lse2 = m_ref + log2f(l_sum);
                 }
-                if (FP8) {   // the accumulators hold P times the V codes' half-precision images: 2^-8 / scale of the true values
+                if (FP8) {   // the accumulators hold P times the V codes' values: the true values divided by the scale
                     const float vm = p.mult[p.H + s.h];
                     a0 *= vm;
                     a1 *= vm;
@@ -762,30 +762,33 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             g += s.cnt;
         }
     } else if (FP8) {
-        // ---------------- conversion warpgroup (warps 12-15; 8-bit cache only).
+        // ---------------- conversion warps (8-bit cache only): warps 12-13 for K and the query tile, warps 14-15 for V.
         // The expanded K_nope and V of the prefix are stored as E4M3 codes with one power-of-two scale per head.
-        // Bulk copies bring 8 KB blocks of codes into staging slots; this warpgroup rewrites each block as the
-        // half-precision operand tile the MMAs read (same 128-byte-swizzled layouts as the 16-bit path).  A code
-        // (s eeee mmm) becomes the half-precision bit pattern s 0eeee mmm0000000: the same number times 2^-8,
-        // subnormal codes included, by two masks, a shift and an OR per pair.  The factors 2^8 * scale go where they
-        // cost nothing.  K: the query's nope part is only converted to half precision (once per segment, here), its
-        // rope part is divided by the factor (a power of two: exact), so the accumulated logits are the true ones
-        // divided by it, and the softmax scale is multiplied by it.  V: into the final normalisation.  The bytes of every 4-code group are stored in the order (0, 2, 1, 3), so
-        // that the pairs (0, 1) and (2, 3) come out of one 32-bit word without a byte shuffle.
-        const int ct = threadIdx.x - 384;
-        auto wg_sync = [] { asm volatile("bar.sync 3, 128;\n" ::: "memory"); };
+        // Bulk copies bring 8 KB blocks of codes into staging slots; these warps rewrite each block as the
+        // half-precision operand tile the MMAs read (same 128-byte-swizzled layouts as the 16-bit path).  Every E4M3
+        // value is a half-precision value, so widening is exact (one conversion instruction per pair of codes).  The
+        // scales go where they cost nothing.  K: the query's nope part is only converted to half precision (once
+        // per segment, here), its rope part is divided by the scale (a power of two: exact), so the accumulated
+        // logits are the true ones divided by it, and the softmax scale is multiplied by it.  V: into the final
+        // normalisation.
+        const bool is_v = warp >= 14;
+        const int ct = threadIdx.x - (is_v ? 448 : 384);          // 0..63 within the pair of warps
+        auto pair_sync = [&] {
+            if (is_v) asm volatile("bar.sync 4, 64;\n" ::: "memory");
+            else asm volatile("bar.sync 3, 64;\n" ::: "memory");
+        };
         auto widen = [](uint32_t w, uint32_t& lo, uint32_t& hi) {
-            const uint32_t v = w << 8;
-            lo = (v & 0x80008000u) | ((v & 0x7f007f00u) >> 1);   // codes 0, 1 of the group
-            hi = (w & 0x80008000u) | ((w & 0x7f007f00u) >> 1);   // codes 2, 3
+            asm("{\n.reg .b16 a, b;\nmov.b32 {a, b}, %2;\ncvt.rn.f16x2.e4m3x2 %0, a;\ncvt.rn.f16x2.e4m3x2 %1, b;\n}\n"
+                : "=r"(lo), "=r"(hi)
+                : "r"(w));
         };
         // one 8 KB staging block (64 rows of 128 bytes, 16-byte chunks swizzled by the row) -> 16 KB operand tile.
         // K: row = token, chunk = 16 dims, tile = two [64 tokens][64 dims] slabs.  V: row = two dims (64 tokens
         // each), chunk = 16 tokens of one dim, tile = [128 dims][64 tokens].
-        auto convert = [&](const uint8_t* src, uint8_t* dst, bool is_v) {
+        auto convert = [&](const uint8_t* src, uint8_t* dst) {
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-                const int u = it * 128 + ct, r = u >> 3, c = u & 7;
+            for (int it = 0; it < 8; ++it) {
+                const int u = it * 64 + ct, r = u >> 3, c = u & 7;
                 const uint4 w = *reinterpret_cast<const uint4*>(src + r * 128 + ((c ^ (r & 7)) << 4));
                 uint4 o0, o1;
                 widen(w.x, o0.x, o0.y);
@@ -800,31 +803,22 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 *reinterpret_cast<uint4*>(d + (((c0 + 1) ^ (row & 7)) << 4)) = o1;
             }
         };
-        auto convert_k = [&](int ring) {
-            const int sq = ring % p.kq_stages, st = ring % p.k_stages;
-            bool ok = __all_sync(0xffffffffu, mbar_wait(&bar->kq_full[sq], (ring / p.kq_stages) & 1, abort_flag));
-            ok = ok && __all_sync(0xffffffffu, mbar_wait(&bar->k_empty[st], ((ring / p.k_stages) & 1) ^ 1, abort_flag));
+        // ring position `ring`: staging slot -> 16-bit slot, then hand both on
+        auto convert_tile = [&](int ring) {
+            const int q_depth = is_v ? p.vq_stages : p.kq_stages, depth = is_v ? p.v_stages : p.k_stages;
+            const int sq = ring % q_depth, st = ring % depth;
+            uint64_t* const staged = is_v ? &bar->vq_full[sq] : &bar->kq_full[sq];
+            uint64_t* const slot_free = is_v ? &bar->v_empty[st] : &bar->k_empty[st];
+            bool ok = __all_sync(0xffffffffu, mbar_wait(staged, (ring / q_depth) & 1, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(slot_free, ((ring / depth) & 1) ^ 1, abort_flag));
             if (!ok) return false;
-            convert(sKq + sq * KQ_BYTES, sK + st * K_TILE_BYTES, false);
+            if (is_v) convert(sVq + sq * VQ_BYTES, sV + st * V_TILE_BYTES);
+            else convert(sKq + sq * KQ_BYTES, sK + st * K_TILE_BYTES);
             fence_proxy_async();   // the MMAs read the tile through the async proxy
-            wg_sync();
+            pair_sync();
             if (ct == 0) {
-                mbar_arrive(&bar->k_full[st]);
-                mbar_arrive(&bar->kq_empty[sq]);
-            }
-            return true;
-        };
-        auto convert_v = [&](int ring) {
-            const int sq = ring % p.vq_stages, st = ring % p.v_stages;
-            bool ok = __all_sync(0xffffffffu, mbar_wait(&bar->vq_full[sq], (ring / p.vq_stages) & 1, abort_flag));
-            ok = ok && __all_sync(0xffffffffu, mbar_wait(&bar->v_empty[st], ((ring / p.v_stages) & 1) ^ 1, abort_flag));
-            if (!ok) return false;
-            convert(sVq + sq * VQ_BYTES, sV + st * V_TILE_BYTES, true);
-            fence_proxy_async();
-            wg_sync();
-            if (ct == 0) {
-                mbar_arrive(&bar->v_full[st]);
-                mbar_arrive(&bar->vq_empty[sq]);
+                mbar_arrive(is_v ? &bar->v_full[st] : &bar->k_full[st]);
+                mbar_arrive(is_v ? &bar->vq_empty[sq] : &bar->kq_empty[sq]);
             }
             return true;
         };
@@ -832,33 +826,30 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         bool ok = true;
         for (int g = g_begin; g < g_end && ok; ++seg) {
             const Segment s = segment_at(g);
-            // query tile (three slabs of 64 rows): nope part to half precision, rope part divided by 2^8 * scale
-            ok = __all_sync(0xffffffffu, mbar_wait(&bar->q_full, seg & 1, abort_flag));
-            if (!ok) break;
-            {
-                const float inv_km = __fdiv_rn(1.f, p.mult[s.h]);   // a power of two: exact
+            if (!is_v) {
+                // query tile (three slabs): nope part to half precision, rope part divided by the K scale
+                ok = __all_sync(0xffffffffu, mbar_wait(&bar->q_full, seg & 1, abort_flag));
+                if (!ok) break;
+                const float inv_ks = __fdiv_rn(1.f, p.mult[s.h]);   // a power of two: exact
 #pragma unroll
-                for (int it = 0; it < 12; ++it) {
-                    uint4* qv = reinterpret_cast<uint4*>(sQ) + it * 128 + ct;
+                constexpr int N_IT = Q_BYTES / 16 / 64;   // 16-byte pieces per thread; the first two thirds are the nope slabs
+#pragma unroll 8
+                for (int it = 0; it < N_IT; ++it) {
+                    uint4* qv = reinterpret_cast<uint4*>(sQ) + it * 64 + ct;
                     uint4 w = *qv;
                     uint32_t* e = reinterpret_cast<uint32_t*>(&w);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&e[k]));
-                        e[k] = it < 8 ? pack_f16(f.x, f.y) : pack_bf16(f.x * inv_km, f.y * inv_km);
+                        e[k] = it < 2 * N_IT / 3 ? pack_f16(f.x, f.y) : pack_bf16(f.x * inv_ks, f.y * inv_ks);
                     }
                     *qv = w;
                 }
                 fence_proxy_async();
-                wg_sync();
+                pair_sync();
                 if (ct == 0) mbar_arrive(&bar->q_conv);
             }
-            // K runs one tile ahead of V: the logits product of a tile comes first, its V is needed a softmax later
-            for (int e = 0; e < s.cnt && ok; ++e) {
-                ok = convert_k(ring_base + e);
-                if (ok && e > 0) ok = convert_v(ring_base + e - 1);
-            }
-            if (ok) ok = convert_v(ring_base + s.cnt - 1);
+            for (int e = 0; e < s.cnt && ok; ++e) ok = convert_tile(ring_base + e);
             ring_base += s.cnt;
             g += s.cnt;
         }
@@ -902,10 +893,10 @@ int naive_sm100_tile_tokens(int B, bool fp8) { return (fp8 || B <= 128) ? 64 : 1
 // the extra read it causes in the combine).  Stream-K is taken when its modelled cost is lower (by at
 // least 5% in the HBM-bound regime of 64-token tiles).
 void naive_sm100_plan(int B, int H, int64_t Ls, int n_sm, int schedule, int* n_ranges, int* n_slots, bool fp8) {
-    // (8-bit cache: always 64-token tiles, row groups of 64 requests)
+    // (8-bit cache: always 64-token tiles, row groups of 128 requests)
     const bool mode_y = fp8 || B <= 128;
     const int tok = mode_y ? 64 : 128;
-    const int m_groups = fp8 ? (B + 63) / 64 : (mode_y ? 1 : (B + 255) / 256);
+    const int m_groups = fp8 ? (B + 127) / 128 : (mode_y ? 1 : (B + 255) / 256);
     const int n_tiles = (int)((Ls + tok - 1) / tok);
     const long long T = (long long)H * n_tiles;
     if (T <= 0) {
@@ -972,14 +963,14 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     {
         uint64_t dims[3] = {128, (uint64_t)a.H, (uint64_t)a.B};
         uint64_t str[2] = {128 * 2, (uint64_t)a.H * 128 * 2};
-        uint32_t box[3] = {64, 1, fp8 ? 64u : 128u};
+        uint32_t box[3] = {64, 1, (fp8 && a.B <= 64) ? 64u : 128u};
         cudaError_t e = make_tmap_bf16(&tm_qn, a.q_nope, 3, dims, str, box);
         if (e != cudaSuccess) return e;
     }
     {
         uint64_t dims[3] = {64, (uint64_t)a.H, (uint64_t)a.B};
         uint64_t str[2] = {64 * 2, (uint64_t)a.H * 64 * 2};
-        uint32_t box[3] = {64, 1, fp8 ? 64u : 128u};
+        uint32_t box[3] = {64, 1, (fp8 && a.B <= 64) ? 64u : 128u};
         cudaError_t e = make_tmap_bf16(&tm_qp, a.q_pe, 3, dims, str, box);
         if (e != cudaSuccess) return e;
     }
@@ -988,7 +979,7 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     NaiveSm100Params p{};
     p.B = a.B; p.H = a.H; p.Ls = a.Ls; p.Ls_pad = (a.Ls + 127) / 128 * 128;
     p.part_rows = a.part_rows > 0 ? a.part_rows : a.B;
-    p.m_groups = fp8 ? (a.B + 63) / 64 : (mode_y ? 1 : (a.B + 255) / 256);
+    p.m_groups = fp8 ? (a.B + 127) / 128 : (mode_y ? 1 : (a.B + 255) / 256);
     p.n_tiles = (a.Ls + tok - 1) / tok;
     p.n_ranges = a.n_ranges;
     {
@@ -1000,18 +991,21 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
     p.n_seg_max = a.n_slots;
     p.k_stages = fp8 ? 2 : (mode_y ? 4 : 2);
     p.v_stages = fp8 ? 2 : (mode_y ? 4 : 1);
-    p.kq_stages = fp8 ? 5 : 0;
-    p.vq_stages = fp8 ? 5 : 0;
+    p.kq_stages = fp8 ? (a.B <= 64 ? 5 : 4) : 0;   // (the 128-row query tile takes 24 KB more)
+    p.vq_stages = fp8 ? (a.B <= 64 ? 5 : 4) : 0;
     p.mult = a.fp8_mult;
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = a.status;
     const int k_tile = fp8 ? 16384 : tok * 384, v_tile = mode_y ? 16384 : 32768;
-    const int smem = (fp8 ? Q_TILE_BYTES / 2 : (mode_y ? 1 : 2) * Q_TILE_BYTES) + p.k_stages * k_tile + p.v_stages * v_tile +
+    const int smem = ((fp8 && a.B <= 64) ? Q_TILE_BYTES / 2 : (mode_y ? 1 : 2) * Q_TILE_BYTES) + p.k_stages * k_tile + p.v_stages * v_tile +
                      p.kq_stages * 16384 + p.vq_stages * 8192 + 1024 + (int)sizeof(Barriers) + 64;
     dim3 grid(p.n_ranges * p.m_groups, 1, 1);
     if (smem > kNaiveSmemMax) return cudaErrorInvalidValue;
-    if (fp8)
-        return launch_pdl(naive_attn_sm100_kernel<64, true, true>, grid, dim3(512), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+    if (fp8) {
+        if (a.B <= 64)
+            return launch_pdl(naive_attn_sm100_kernel<64, true, true>, grid, dim3(512), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+        return launch_pdl(naive_attn_sm100_kernel<64, false, true>, grid, dim3(512), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
+    }
     if (mode_y) {
         if (a.B <= 64)   // half-height MMAs: the padding rows 64..127 of the query tile cost tensor-pipe time and power
             return launch_pdl(naive_attn_sm100_kernel<64, true, false>, grid, dim3(384), smem, s, tm_qn, tm_qp, *a.tm_kn, *a.tm_kp, *a.tm_vt, p);
@@ -1025,6 +1019,7 @@ cudaError_t set_attrs_naive_sm100() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<128, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(naive_attn_sm100_kernel<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kNaiveSmemMax);
     return e;
 }
 

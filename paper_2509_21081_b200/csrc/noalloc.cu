@@ -104,7 +104,7 @@ extern "C" int typhoon_mla_naive_shared_noalloc(const typhoon_mla_shared_t* sh, 
     if (n_slots > 0) {
         NaiveAttnSm100 na{q_nope, q_pe, &sh->tm_kn, &sh->tm_kp, &sh->tm_vt, B, H, (int)sh->Ls, n_ranges, n_slots,
                           softmax_scale, o_part, lse_part, sh->status, B};
-        if (sh->fp8) na.fp8_mult = sh->fp8_f + 2 * H;
+        if (sh->fp8) na.fp8_mult = sh->fp8_f;
         e = launch_naive_attn_sm100(na, s);
         if (e != cudaSuccess) return api_cuda_fail(e);
         ++launches;

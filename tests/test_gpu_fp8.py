@@ -112,7 +112,7 @@ def test_footprint_is_halved_and_other_paths_refuse():
     _, Lp, own16 = b.typhoon_mla_shared_view(s16)
     _, _, own8 = b.typhoon_mla_shared_view(s8)
     expanded16 = 2 * 16 * Lp * 128 * 2
-    assert own16 - own8 == expanded16 // 2 - 16 * 5 * 4      # codes are half the bytes; plus the per-head factors
+    assert own16 - own8 == expanded16 // 2 - 16 * 3 * 4      # codes are half the bytes; plus the per-head scales
     with pytest.raises(b.TyphoonMLAError):
         b.typhoon_mla_shared_export(s8)
     with pytest.raises(b.TyphoonMLAError):
@@ -132,3 +132,38 @@ def test_footprint_is_halved_and_other_paths_refuse():
     assert not out.any()
     s16.free()
     s8.free()
+
+
+def test_tree_with_an_8bit_root_and_16bit_branches():
+    """Several shared prefixes per step, the root stored in 8 bits, the per-group prefixes in 16: the checker encodes
+    the root only (the branches are part of each request's own context there)."""
+    from paper_2509_21081_b200 import binding as b
+    from tests.test_gpu_parity import _tree_problem
+    B, H = 11, 32
+    lens = [0, 3, 64, 65, 130, 7, 200, 1, 90, 64, 30]
+    rows, inp, br = _tree_problem(B, H, 210, [(0, 150), (3, 0), (5, 333), (9, 70)], lens, seed=39)
+    ref, ref_lse = G.run_oracle_fp8(rows)
+    dev = "cuda"
+    w_uk, w_uv = inp.w_uk.to(dev), inp.w_uv.to(dev)
+    dims = b.make_dims(H)
+    root = b.typhoon_mla_prepare_shared_fp8(dims, inp.ckv_shared.to(dev), inp.kpe_shared.to(dev), w_uk, w_uv)
+    handles = [root]
+    prefixes = []
+    for _, _, c, r in br:
+        if c.shape[0] > 0:
+            handles.append(b.typhoon_mla_prepare_shared(dims, c.to(dev), r.to(dev), w_uk, w_uv))
+            prefixes.append(handles[-1])
+        else:
+            prefixes.append(None)
+    levels = [([root], [0, B]), (prefixes, [b0 for b0, _, _, _ in br] + [B])]
+    pc = I.build_pages(inp)
+    ws = torch.empty(b.typhoon_mla_tree_workspace_bytes(levels, B, pc.block_table.shape[1], 64), dtype=torch.uint8, device=dev)
+    out = torch.empty(B, H, 128, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(B, H, dtype=torch.float32, device=dev)
+    b.typhoon_mla_decode_tree(levels, inp.q_nope.to(dev), inp.q_pe.to(dev), pc.ckv_pages.to(dev), pc.kpe_pages.to(dev), 64,
+                              pc.block_table.to(dev), pc.seq_lens.to(dev), inp.scale, out, ws, lse_out=lse)
+    for h in handles:
+        assert b.typhoon_mla_check_status(h) == 0
+    G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse, what="tree, 8-bit root")
+    for h in handles:
+        h.free()

@@ -94,3 +94,21 @@ def test_noalloc_rejects_oversized_problem():
     assert bool((out == 7.0).all()) and bool((lse == 7.0).all()), "a refused call wrote to its outputs"
     assert b.typhoon_mla_last_launch_count() == 0
     sh.free()
+
+
+def test_noalloc_with_an_8bit_expanded_cache():
+    """The same entry point on a handle whose expanded cache is stored as E4M3 codes: against the checker's operator
+    over the decoded values, prefix alone."""
+    from paper_2509_21081_b200 import binding as b
+    cfg = I.MLAConfig("noalloc8", B=70, H=16, Ls=900, suffix_lo=0, suffix_hi=0, seed=78)
+    inp = I.make_inputs(cfg)
+    w_uk, w_uv = inp.w_uk.cuda(), inp.w_uv.cuda()
+    sh = b.typhoon_mla_prepare_shared_fp8(b.make_dims(cfg.H), inp.ckv_shared.cuda(), inp.kpe_shared.cuda(), w_uk, w_uv)
+    ora, ora_lse = G.run_oracle_fp8(inp, drop_suffix=True)
+    out = torch.full((cfg.B, cfg.H, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((cfg.B, cfg.H), float("nan"), dtype=torch.float32, device="cuda")
+    b.typhoon_mla_naive_shared_noalloc(sh, inp.q_nope.cuda(), inp.q_pe.cuda(), inp.scale, out, lse)
+    assert b.typhoon_mla_check_status(sh) == 0
+    G.assert_parity(out.float().cpu().double().numpy(), ora, lse.cpu().double().numpy(), ora_lse,
+                    what="allocation-free entry point, 8-bit cache")
+    sh.free()
