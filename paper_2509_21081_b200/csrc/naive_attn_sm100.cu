@@ -788,7 +788,11 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
         auto convert = [&](const uint8_t* src, uint8_t* dst) {
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
-                const int u = it * 64 + ct, r = u >> 3, c = u & 7;
+                // Eight consecutive lanes take chunks 0-3 of one row and chunks 4-7 of the next (or the other way round):
+                // their eight 16-byte reads fall on eight different bank groups, and so do their writes (the two
+                // rows' swizzles differ in the lowest bit, the two halves of a K row go to different slabs).
+                const int u = it * 64 + ct, j = u & 7, grp = u >> 3;
+                const int r = 2 * (grp >> 1) + (j >> 2), c = (j & 3) + 4 * ((j >> 2) ^ (grp & 1));
                 const uint4 w = *reinterpret_cast<const uint4*>(src + r * 128 + ((c ^ (r & 7)) << 4));
                 uint4 o0, o1;
                 widen(w.x, o0.x, o0.y);
@@ -989,10 +993,10 @@ cudaError_t launch_naive_attn_sm100(const NaiveAttnSm100& a, cudaStream_t s) {
         p.rem = (int)(T % a.n_ranges);
     }
     p.n_seg_max = a.n_slots;
-    p.k_stages = fp8 ? 2 : (mode_y ? 4 : 2);
-    p.v_stages = fp8 ? 2 : (mode_y ? 4 : 1);
-    p.kq_stages = fp8 ? (a.B <= 64 ? 5 : 4) : 0;   // (the 128-row query tile takes 24 KB more)
-    p.vq_stages = fp8 ? (a.B <= 64 ? 5 : 4) : 0;
+    p.k_stages = fp8 ? (a.B <= 64 ? 3 : 2) : (mode_y ? 4 : 2);   // (8-bit cache: the 128-row query tile takes 24 KB more)
+    p.v_stages = fp8 ? (a.B <= 64 ? 3 : 2) : (mode_y ? 4 : 1);
+    p.kq_stages = fp8 ? 4 : 0;
+    p.vq_stages = fp8 ? 4 : 0;
     p.mult = a.fp8_mult;
     p.scale_log2 = a.scale * kLog2e;
     p.o_part = a.o_part; p.lse_part = a.lse_part; p.status = a.status;
