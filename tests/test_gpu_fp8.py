@@ -167,3 +167,22 @@ def test_tree_with_an_8bit_root_and_16bit_branches():
     G.assert_parity(out.float().cpu().double().numpy(), ref, lse.cpu().double().numpy(), ref_lse, what="tree, 8-bit root")
     for h in handles:
         h.free()
+
+
+@pytest.mark.parametrize("name,batch", [("cfg1", 0), ("cfg4", 512)])
+def test_full_size_configurations(name, batch):
+    """The benchmark's headline configuration (64-row instance, one tile range per head) and the fan-out sweep at
+    B = 512 (128-row instance, four row groups, equal tile ranges over all SMs) on an 8-bit handle, in the launch
+    configuration the benchmark times: all heads of at least 16 requests against the checker's operator."""
+    from tests.test_gpu_parity import _checked_requests
+    cfg = I.CONFIGS[name].with_batch(batch) if batch else I.CONFIGS[name]
+    inp = I.make_inputs(cfg)
+    reqs = _checked_requests(cfg, inp)
+    reqs = sorted(set(reqs) | {r for g0 in range(0, cfg.B, 128) for r in (g0, min(g0 + 127, cfg.B - 1))})   # every 128-row group
+    pairs = [(r, h) for r in reqs for h in range(cfg.H)]
+    ref, ref_lse = G.run_oracle_fp8(inp, pairs=pairs)
+    mask = ~np.isnan(ref_lse)
+    assert mask.sum() == len(reqs) * cfg.H
+    out, lse, _ = G.run_gpu(inp, HYBRID, fp8_shared=True)
+    assert np.isfinite(out).all()
+    G.assert_parity(out, ref, lse, ref_lse, mask=mask, what=f"fp8 {cfg.name} full size")
