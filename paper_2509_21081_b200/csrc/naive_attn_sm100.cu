@@ -115,6 +115,11 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         const __grid_constant__ CUtensorMap tm_kn, const __grid_constant__ CUtensorMap tm_kp,
                         const __grid_constant__ CUtensorMap tm_vt, NaiveSm100Params p) {
     constexpr bool MODE_Y = TOK == 64;
+    // 128-token tiles (compute-bound regime): pairs of exponentials computed on the FMA pipe instead of the
+    // special-function unit, by position of the pair within a group of eight (bit set = polynomial).  Measured at
+    // B = 512: one pair in four is the best mix (-4 % kernel time); one in eight and three in eight gain 1-2 %, every
+    // second pair changes the compiler's register allocation for the worse (+5 %).
+    constexpr unsigned kPolyExpMask = TOK == 128 ? 0x88u : 0u;
     constexpr int NB = MODE_Y ? 2 : 1;                  // S buffers per stream
     constexpr int BLK = TOK / 64;                       // 64-token blocks per tile
     constexpr int K_SLAB = TOK * 128;                   // bytes of one [TOK][64] K slab
@@ -614,7 +619,13 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                         // two logits per instruction: distance to the reference exponent, probabilities, running sums
                         float x0, x1;
                         unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(src[2 * c]), __uint_as_float(src[2 * c + 1])), scale2, neg_m2), x0, x1);
-                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        float p0, p1;
+                        if ((kPolyExpMask >> (c & 7)) & 1) {
+                            exp2_poly_x2(x0, x1, p0, p1);
+                        } else {
+                            p0 = fast_exp2(x0);
+                            p1 = fast_exp2(x1);
+                        }
                         dst[c] = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
                         if (c & 1) l_sum2b = add_f32x2(l_sum2b, pack_f32x2(p0, p1));
                         else l_sum2 = add_f32x2(l_sum2, pack_f32x2(p0, p1));

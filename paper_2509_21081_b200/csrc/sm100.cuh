@@ -297,6 +297,25 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
     asm("mul.rn.f32x2 %0, %1, %2;\n" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// 2^x for a pair of values on the FMA and ALU pipes instead of the special-function unit (16 results per clock and
+// SM): x (clamped to >= -126, so that the result stays a normal number; -inf gives 2^-126) is split into its nearest
+// integer j (adding and subtracting 1.5 * 2^23 rounds to nearest) and a fraction f in [-0.5, 0.5]; 2^f comes from a
+// degree-3 polynomial (largest relative error 7.5e-5, far below the 2^-9 of the 16-bit probabilities it feeds), and j
+// is added to the exponent field as an integer.  Twelve instructions per pair.
+__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& p0, float& p1) {
+    const uint64_t x = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const uint64_t t = add_f32x2(x, pack_f32x2(12582912.f, 12582912.f));     // integer part in the low mantissa bits
+    const uint64_t r = add_f32x2(t, pack_f32x2(-12582912.f, -12582912.f));   // ... as a float
+    const uint64_t f = fma_f32x2(r, pack_f32x2(-1.f, -1.f), x);
+    uint64_t q = fma_f32x2(pack_f32x2(0.05517164617776871f, 0.05517164617776871f), f, pack_f32x2(0.2426111251115799f, 0.2426111251115799f));
+    q = fma_f32x2(q, f, pack_f32x2(0.6932609677314758f, 0.6932609677314758f));
+    q = fma_f32x2(q, f, pack_f32x2(0.9999280571937561f, 0.9999280571937561f));
+    float t0, t1, q0, q1;
+    unpack_f32x2(t, t0, t1);
+    unpack_f32x2(q, q0, q1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
