@@ -284,7 +284,10 @@ int typhoon_mla_set_absorb_efficiency(double fraction) {
     return TYPHOON_MLA_OK;
 }
 
-int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int32_t B, int64_t total_suffix_tokens) {
+// `naive_time_factor`: how much longer the shared-prefix kernel takes than the model says (1 for the 16-bit cache; the
+// 8-bit cache's kernel is bound by its widening step: measured 1.4-1.7 times the 16-bit kernel's time)
+static int choose_mode_impl(const typhoon_mla_dims_t* dims, int64_t Ls, int32_t B, int64_t total_suffix_tokens,
+                            double naive_time_factor) {
     if (!dims || B < 1 || Ls <= 0) return TYPHOON_MLA_MODE_ABSORB;
     if (total_suffix_tokens == 0) return TYPHOON_MLA_MODE_NAIVE;
     // Shared-prefix part only: the suffix part is identical in both modes.
@@ -302,14 +305,18 @@ int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int3
     // The absorb kernel re-reads the prefix per request and runs M = 64 tiles: measured on B200 it
     // reaches about half of the tensor throughput the naive kernel does, hence the factor.
     const double T = g_tensor_flops.load(), M = g_hbm_bytes.load();
-    const double t_hybrid = std::max(f_naive / T, by_naive / M) + g_hybrid_fixed_s.load();
+    const double t_hybrid = naive_time_factor * std::max(f_naive / T, by_naive / M) + g_hybrid_fixed_s.load();
     const double t_absorb = std::max(f_absorb / (g_absorb_efficiency.load() * T), by_absorb / M);
     return t_hybrid < t_absorb ? TYPHOON_MLA_MODE_HYBRID : TYPHOON_MLA_MODE_ABSORB;
 }
 
+int typhoon_mla_choose_mode_for(const typhoon_mla_dims_t* dims, int64_t Ls, int32_t B, int64_t total_suffix_tokens) {
+    return choose_mode_impl(dims, Ls, B, total_suffix_tokens, 1.0);
+}
+
 int typhoon_mla_choose_mode(const typhoon_mla_shared_t* sh, int32_t B, int64_t total_suffix_tokens) {
     if (!sh) return TYPHOON_MLA_MODE_ABSORB;
-    return typhoon_mla_choose_mode_for(&sh->dims, sh->Ls, B, total_suffix_tokens);
+    return choose_mode_impl(&sh->dims, sh->Ls, B, total_suffix_tokens, sh->fp8 ? 1.5 : 1.0);
 }
 
 int typhoon_mla_free(typhoon_mla_shared_t* sh) {
