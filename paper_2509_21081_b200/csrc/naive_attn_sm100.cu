@@ -39,6 +39,10 @@
 // The expanded cache is stored in 64-token blocks: K_nope [H, L/64, 2 slabs, 64, 64],
 // V^T [H, L/64, 128, 64], rope keys [L, 64]; every TMA box is a contiguous 8 or 16 KB.
 //
+// With the expanded cache stored as E4M3 codes (template flag FP8; 64-token tiles, row groups of at most 128
+// requests) four more warps (12-15, 512 threads) widen the copied code blocks into half-precision operand
+// tiles; see the conversion warps below.
+//
 // Every mbarrier wait has a deadline; on expiry all roles fall through to the common teardown
 // and the status word is set.
 #include <cstddef>
