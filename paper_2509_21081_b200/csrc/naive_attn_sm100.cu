@@ -265,9 +265,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             for (int i = lane; i < n_bars; i += 32) {
                 uint64_t* m = all + i;
                 const bool wg = (m >= &bar->p_ready[0][0] && m < &bar->sbuf_free[0][0]) || (m >= &bar->o_free[0] && m < &bar->o_done[0][0]);   // o_free, merge_ready
-                // (a K staging slot is released by two parties: the conversion warpgroup and the S products that read its rope keys)
-                const bool two = FP8 && m >= &bar->kq_empty[0] && m < &bar->vq_full[0];
-                mbar_init(m, wg ? 128 : (two ? 2 : 1));
+                mbar_init(m, wg ? 128 : 1);
             }
             if (lane == 0) bar->abort_flag = 0;
             fence_mbar_init();
@@ -351,19 +349,25 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     if (j >= (i == 0 ? s.n_str0 : s.n_str1)) continue;
                     const int ring = ring_base + entry_of(j, i);
                     const int st = ring % p.k_stages;
-                    if (MODE_Y || i == 0) {                       // mode X: stream 1 reuses stream 0's tile
-                        ok = mbar_wait_warp(&bar->k_full[st], (ring / p.k_stages) & 1, abort_flag);
-                        if (!ok) break;
-                        if (FP8) {   // the rope keys of the tile are read from the staging slot itself
-                            ok = mbar_wait_warp(&bar->kq_full[ring % p.kq_stages], (ring / p.kq_stages) & 1, abort_flag);
-                            if (!ok) break;
-                        }
-                    }
+                    // Awaited: the K tile (mode X: stream 1 reuses stream 0's), with the 8-bit cache also the staging slot
+                    // whose rope keys the product reads, and, from the NB-th use on, the PV product that read P from this
+                    // S buffer NB uses ago.  The barriers are tested together: each test of a barrier costs about 200
+                    // clocks even when its phase is complete, and this warp's loop is the pace of the 64-token kernels.
                     const int u = (i == 0 ? used0 : used1) + j;
-                    if (u >= NB) {   // the PV product that read P from this S buffer NB uses ago must be done
-                        ok = mbar_wait_warp(&bar->sbuf_free[i][u % NB], ((u / NB) - 1) & 1, abort_flag);
-                        if (!ok) break;
-                    }
+                    const bool need_k = MODE_Y || i == 0, need_s = u >= NB;
+                    uint64_t* const kf = &bar->k_full[st];
+                    uint64_t* const kq = &bar->kq_full[FP8 ? ring % p.kq_stages : 0];
+                    uint64_t* const sf = &bar->sbuf_free[i][u % NB];
+                    const uint32_t kf_par = (ring / p.k_stages) & 1, kq_par = FP8 ? (ring / p.kq_stages) & 1 : 0;
+                    const uint32_t sf_par = ((u / NB) - 1) & 1;
+                    if (need_k && need_s)
+                        ok = FP8 ? mbar_wait3_warp(kf, kf_par, kq, kq_par, sf, sf_par, abort_flag)
+                                 : mbar_wait2_warp(kf, kf_par, sf, sf_par, abort_flag);
+                    else if (need_k)
+                        ok = FP8 ? mbar_wait2_warp(kf, kf_par, kq, kq_par, abort_flag) : mbar_wait_warp(kf, kf_par, abort_flag);
+                    else if (need_s)
+                        ok = mbar_wait_warp(sf, sf_par, abort_flag);
+                    if (!ok) break;
                     tc_fence_after();
                     const uint32_t qa = smem_u32(sQ + (MODE_Y ? 0 : i) * Q_BYTES);
                     const uint32_t ka = smem_u32(sK + st * K_TILE_BYTES);
@@ -380,7 +384,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     }
                     umma_commit_if(ld, &bar->s_ready[i][u % NB]);
                     if (last_user) umma_commit_if(ld, &bar->k_empty[st]);   // last user releases the ring slot
-                    if (FP8) umma_commit_if(ld, &bar->kq_empty[ring % p.kq_stages]);   // ... and its share of the staging slot
+                    if (FP8) umma_commit_if(ld, &bar->kq_empty[ring % p.kq_stages]);   // ... and the staging slot (rope keys read, codes widened before)
                 }
             }
             umma_commit_if(ld, &bar->q_free);                     // the Q tile may be replaced
@@ -403,13 +407,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                     if (j >= (i == 0 ? s.n_str0 : s.n_str1)) continue;
                     const int ring = ring_base + entry_of(j, i);
                     const int st = ring % p.v_stages;
-                    if (MODE_Y || i == 0) {
-                        ok = mbar_wait_warp(&bar->v_full[st], (ring / p.v_stages) & 1, abort_flag);
-                        if (!ok) break;
-                    }
+                    // the V tile and the probabilities, tested together (see the S issuer)
                     const int u = (i == 0 ? used0 : used1) + j;
-                    ok = MODE_Y ? mbar_wait_warp(&bar->p_ready[i][u % NB], (u / NB) & 1, abort_flag)
-                                : mbar_wait_warp(&bar->p_half[i], u & 1, abort_flag);
+                    uint64_t* const pf = MODE_Y ? &bar->p_ready[i][u % NB] : &bar->p_half[i];
+                    const uint32_t pf_par = MODE_Y ? (u / NB) & 1 : u & 1;
+                    if (MODE_Y || i == 0) ok = mbar_wait2_warp(&bar->v_full[st], (ring / p.v_stages) & 1, pf, pf_par, abort_flag);
+                    else ok = mbar_wait_warp(pf, pf_par, abort_flag);
                     if (!ok) break;
                     if (j == 0 && seg > 0) {   // the previous segment's epilogue has read this accumulator
                         ok = mbar_wait_warp(&bar->o_free[i], (seg - 1) & 1, abort_flag);
@@ -828,8 +831,12 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const int sq = ring % q_depth, st = ring % depth;
             uint64_t* const staged = is_v ? &bar->vq_full[sq] : &bar->kq_full[sq];
             uint64_t* const slot_free = is_v ? &bar->v_empty[st] : &bar->k_empty[st];
-            bool ok = __all_sync(0xffffffffu, mbar_wait(staged, (ring / q_depth) & 1, abort_flag));
-            ok = ok && __all_sync(0xffffffffu, mbar_wait(slot_free, ((ring / depth) & 1) ^ 1, abort_flag));
+            // (both barriers tested together first: in the steady state both phases are complete)
+            bool ok = __all_sync(0xffffffffu, mbar_try_wait2(staged, (ring / q_depth) & 1, slot_free, ((ring / depth) & 1) ^ 1));
+            if (!ok) {
+                ok = __all_sync(0xffffffffu, mbar_wait(staged, (ring / q_depth) & 1, abort_flag));
+                ok = ok && __all_sync(0xffffffffu, mbar_wait(slot_free, ((ring / depth) & 1) ^ 1, abort_flag));
+            }
             if (!ok) return false;
             if (is_v) convert(sVq + sq * VQ_BYTES, sV + st * V_TILE_BYTES);
             else convert(sKq + sq * KQ_BYTES, sK + st * K_TILE_BYTES);
@@ -837,7 +844,9 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             pair_sync();
             if (ct == 0) {
                 mbar_arrive(is_v ? &bar->v_full[st] : &bar->k_full[st]);
-                mbar_arrive(is_v ? &bar->vq_empty[sq] : &bar->kq_empty[sq]);
+                // A K staging slot is released by the logits product that reads its rope keys: that product waits for
+                // this tile's k_full, so it cannot complete before the codes have been read.
+                if (is_v) mbar_arrive(&bar->vq_empty[sq]);
             }
             return true;
         };

@@ -34,6 +34,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// Two barriers tested together (a test of a completed phase still takes about 200 clocks; the two tests overlap):
+// true if both phases are complete.
+__device__ __forceinline__ bool mbar_try_wait2(uint64_t* bar_a, uint32_t parity_a, uint64_t* bar_b, uint32_t parity_b) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p, q;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 q, [%3], %4;\n"
+        "and.pred p, p, q;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(smem_u32(bar_a)), "r"(parity_a), "r"(smem_u32(bar_b)), "r"(parity_b) : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ bool mbar_try_wait3(uint64_t* bar_a, uint32_t parity_a, uint64_t* bar_b, uint32_t parity_b,
+                                               uint64_t* bar_c, uint32_t parity_c) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p, q, r;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 q, [%3], %4;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 r, [%5], %6;\n"
+        "and.pred p, p, q;\n"
+        "and.pred p, p, r;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar_a)), "r"(parity_a), "r"(smem_u32(bar_b)), "r"(parity_b), "r"(smem_u32(bar_c)), "r"(parity_c)
+        : "memory");
+    return ok != 0;
+}
+
 // Wait with a deadline (about one second of SM clocks).  On expiry, or when
 // another thread of the CTA has already given up, returns false; the caller
 // then skips its remaining work and falls through to the common teardown.
@@ -71,6 +102,19 @@ __device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t parity) {
 // and coordinates in uniform registers) and elect one lane only for the issuing instruction.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
+// Two (three) barriers awaited by a role warp.  In the steady state of a pipeline the awaited phases are usually
+// complete already; testing them together costs one test latency (about 200 clocks) instead of one per barrier.
+__device__ __forceinline__ bool mbar_wait2_warp(uint64_t* bar_a, uint32_t parity_a, uint64_t* bar_b, uint32_t parity_b,
+                                                volatile int* abort_flag) {
+    if (__all_sync(0xffffffffu, mbar_try_wait2(bar_a, parity_a, bar_b, parity_b))) return true;
+    return mbar_wait_warp(bar_a, parity_a, abort_flag) && mbar_wait_warp(bar_b, parity_b, abort_flag);
+}
+__device__ __forceinline__ bool mbar_wait3_warp(uint64_t* bar_a, uint32_t parity_a, uint64_t* bar_b, uint32_t parity_b,
+                                                uint64_t* bar_c, uint32_t parity_c, volatile int* abort_flag) {
+    if (__all_sync(0xffffffffu, mbar_try_wait3(bar_a, parity_a, bar_b, parity_b, bar_c, parity_c))) return true;
+    return mbar_wait_warp(bar_a, parity_a, abort_flag) && mbar_wait_warp(bar_b, parity_b, abort_flag) &&
+           mbar_wait_warp(bar_c, parity_c, abort_flag);
 }
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
