@@ -119,7 +119,7 @@ int typhoon_mla_prepare_shared(const typhoon_mla_dims_t* dims /* host */,
  * (decode, decode_tree, decode_partial, the no-alloc call; AUTO / ABSORB / HYBRID /
  * NAIVE).  The option trades speed for memory: widening the codes inside the kernel
  * costs more than the halved traffic saves, and the shared-prefix kernel then works on
- * row groups of at most 128 requests (measured on B200: steps 1.3 to 1.7 times as long
+ * row groups of at most 128 requests (measured on B200: steps 1.15 to 1.6 times as long
  * as with the 16-bit cache).  A 16-bit scratch of the size of one expanded tensor is taken
  * from and returned to the stream's memory pool inside the call.
  * Arguments and errors as typhoon_mla_prepare_shared.
