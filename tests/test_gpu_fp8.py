@@ -186,3 +186,25 @@ def test_full_size_configurations(name, batch):
     out, lse, _ = G.run_gpu(inp, HYBRID, fp8_shared=True)
     assert np.isfinite(out).all()
     G.assert_parity(out, ref, lse, ref_lse, mask=mask, what=f"fp8 {cfg.name} full size")
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes(seed):
+    """Seeded random sizes, head counts, page sizes and work decompositions on an 8-bit handle (ring wrap-around with the
+    staging and operand rings, several segments per CTA, odd tile counts, partial row groups)."""
+    import random
+    from paper_2509_21081_b200 import binding as b
+    rnd = random.Random(7000 + seed)
+    H = rnd.choice([16, 32, 48, 64, 128])
+    B = rnd.choice([rnd.randint(1, 8), rnd.randint(9, 64), rnd.randint(65, 128), rnd.randint(129, 300)])
+    Ls = rnd.choice([rnd.randint(1, 200), rnd.randint(200, 1500), rnd.randint(1500, 2600) if H <= 32 else rnd.randint(64, 900)])
+    hi = rnd.choice([0, 5, 70, 200])
+    page_size = rnd.choice([64, 128])
+    b.typhoon_mla_set_naive_schedule(rnd.choice([0, 1, 2]))
+    try:
+        inp = I.make_inputs(_cfg("fp8rand", B=B, H=H, Ls=Ls, lo=0, hi=hi, seed=900 + seed, page_size=page_size))
+        ref, ref_lse = G.run_oracle_fp8(inp)
+        out, lse, _ = G.run_gpu(inp, HYBRID, page_size=page_size, fp8_shared=True)
+        G.assert_parity(out, ref, lse, ref_lse, what=f"fp8 random {seed}: B={B} H={H} Ls={Ls} hi={hi} ps={page_size}")
+    finally:
+        b.typhoon_mla_set_naive_schedule(0)
