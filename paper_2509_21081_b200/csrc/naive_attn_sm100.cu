@@ -795,6 +795,18 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             if (is_v) asm volatile("bar.sync 4, 64;\n" ::: "memory");
             else asm volatile("bar.sync 3, 64;\n" ::: "memory");
         };
+        // The two warps of a pair must take the same decision before either of them goes to the pair's barrier: one
+        // may have seen the abort flag in a wait that the other left through its fast path.
+        auto pair_vote_or = [&](bool pred) {
+            uint32_t r;
+            if (is_v)
+                asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 q, %1, 0;\nbar.red.or.pred p, 4, 64, q;\nselp.u32 %0, 1, 0, p;\n}\n"
+                             : "=r"(r) : "r"(pred ? 1u : 0u) : "memory");
+            else
+                asm volatile("{\n.reg .pred p, q;\nsetp.ne.b32 q, %1, 0;\nbar.red.or.pred p, 3, 64, q;\nselp.u32 %0, 1, 0, p;\n}\n"
+                             : "=r"(r) : "r"(pred ? 1u : 0u) : "memory");
+            return r != 0;
+        };
         auto widen = [](uint32_t w, uint32_t& lo, uint32_t& hi) {
             asm("{\n.reg .b16 a, b;\nmov.b32 {a, b}, %2;\ncvt.rn.f16x2.e4m3x2 %0, a;\ncvt.rn.f16x2.e4m3x2 %1, b;\n}\n"
                 : "=r"(lo), "=r"(hi)
@@ -837,7 +849,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
                 ok = __all_sync(0xffffffffu, mbar_wait(staged, (ring / q_depth) & 1, abort_flag));
                 ok = ok && __all_sync(0xffffffffu, mbar_wait(slot_free, ((ring / depth) & 1) ^ 1, abort_flag));
             }
-            if (!ok) return false;
+            if (pair_vote_or(!ok)) return false;
             if (is_v) convert(sVq + sq * VQ_BYTES, sV + st * V_TILE_BYTES);
             else convert(sKq + sq * KQ_BYTES, sK + st * K_TILE_BYTES);
             fence_proxy_async();   // the MMAs read the tile through the async proxy
@@ -856,7 +868,7 @@ naive_attn_sm100_kernel(const __grid_constant__ CUtensorMap tm_qn, const __grid_
             const Segment s = segment_at(g);
             if (!is_v) {
                 // query tile (three slabs): nope part to half precision, rope part divided by the K scale
-                ok = __all_sync(0xffffffffu, mbar_wait(&bar->q_full, seg & 1, abort_flag));
+                ok = !pair_vote_or(!__all_sync(0xffffffffu, mbar_wait(&bar->q_full, seg & 1, abort_flag)));
                 if (!ok) break;
                 const float inv_ks = __fdiv_rn(1.f, p.mult[s.h]);   // a power of two: exact
 #pragma unroll
