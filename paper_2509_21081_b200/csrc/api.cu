@@ -697,7 +697,21 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
         prof_before(TYPHOON_MLA_KERNEL_Q_ABSORB, s);
         if (tc) {
             if (order) desc = reinterpret_cast<int32_t*>(ws + pl.off_desc);
-            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->num_sms, sh->status, order ? seq_lens : nullptr, order,
+            // Beside the shared-prefix kernel the absorb branch has the SMs that kernel's CTAs leave free: if those are few,
+            // that many CTAs walk through the heads (each resident for the whole launch) instead of one CTA per head
+            // queueing for them.
+            int walk_ctas = 0;
+            if (forked) {
+                int naive_ctas = 0;
+                for (int j = 0; j < n_jobs; ++j) {
+                    const int rows = jobs[j].rows;
+                    const int groups = jobs[j].sh->fp8 ? (rows + 127) / 128 : (rows <= 128 ? 1 : (rows + 255) / 256);
+                    naive_ctas = std::max(naive_ctas, jobs[j].n_ranges * groups);
+                }
+                const int free_sms = sh->num_sms - naive_ctas;
+                if (n_jobs == 1 && free_sms >= 8 && free_sms < H) walk_ctas = free_sms;
+            }
+            e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->num_sms, walk_ctas, sh->status, order ? seq_lens : nullptr, order,
                                       block_table, max_pages, page_size, desc, s);
         } else {
             GemmTN g1{q_nope, (int64_t)H * 128, 128, sh->w_uk_t, 128, 512 * 128, q_abs, (int64_t)H * 512, 512,

@@ -72,7 +72,9 @@ cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w);
 // With seq_lens and order given (B <= 4096) one extra block also writes the longest-first request order and,
 // with desc given, one int4 per launch position {request, clamped suffix length, first page, second page}
 // (-1 where the block table has no such column) that saves the absorb kernel three dependent loads.
-cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int n_sm, int* status,
+// walk_ctas > 0 (and B <= 128): that many CTAs walk through the heads instead of one CTA per head (for launches that share the
+// GPU with a kernel that leaves only a few SMs free).
+cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int n_sm, int walk_ctas, int* status,
                                   const int32_t* seq_lens, int32_t* order, const int32_t* block_table, int max_pages,
                                   int page_size, int32_t* desc, cudaStream_t s);
 

@@ -4,7 +4,10 @@
 // S-th tile of 128 requests (S CTAs per head when there are more SMs than heads).  The head's transposed weight
 // (128 KB) is loaded once and stays in shared memory; the query tiles (32 KB) stream through one buffer that is
 // refilled as soon as the products that read it have completed, i.e. while the previous tile's result is still
-// being written.  The 512-wide result of a tile is accumulated in all 512 tensor-memory columns (four N = 128
+// being written.  With at most 128 requests (one tile per head) the grid may instead be a few CTAs that each walk
+// through every G-th head ("walk" mode): in a hybrid step the kernel runs on the few SMs the shared-prefix kernel
+// leaves free, and a CTA that stays resident loads the next head's weights while the previous head's result is
+// being written, instead of paying launch, barrier set-up and tensor-memory allocation once per head.  The 512-wide result of a tile is accumulated in all 512 tensor-memory columns (four N = 128
 // blocks).  The epilogue packs each block to bf16 into a 128-byte-swizzled staging buffer (two of them, used
 // alternately) and writes it with tiled bulk stores, so that global memory sees whole 128-byte lines instead
 // of one 16-byte piece per thread.  The step is bound by reading the weights once (16.8 MB at 128 heads) and
@@ -31,6 +34,7 @@ struct QAbsorbParams {
     void* q_abs;   // bf16 [B, H, 512]
     int B, H;
     int n_tiles, splits;   // tiles of 128 requests; CTAs per head (CTA s takes tiles s, s + splits, ...)
+    int walk_ctas;         // > 0: walk mode with this many working CTAs (1-D grid, block walk_ctas is the ordering block)
     int* status;
     // optional: one extra block (blockIdx.y == H) computes the longest-first request order that the
     // absorb attention kernel launched next uses, saving a launch on the absorb branch
@@ -49,8 +53,9 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     pdl_trigger();
     pdl_wait();
-    if ((int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
-        if (blockIdx.x == 0) {
+    const bool walk = p.walk_ctas > 0;
+    if (walk ? (int)blockIdx.x == p.walk_ctas : (int)blockIdx.y == p.H) {   // the ordering block (whole block takes this branch)
+        if (walk || blockIdx.x == 0) {
             block_order_by_length(p.seq_lens, p.B, p.order, reinterpret_cast<unsigned long long*>(smem));
             if (p.desc != nullptr) {
                 __syncthreads();   // perm[] written by this block is read back below
@@ -75,9 +80,19 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
     const int warp = warp_index_uniform(), lane = threadIdx.x & 31;
-    const int h = blockIdx.y;
-    const int n_my = ((int)blockIdx.x < p.n_tiles) ? (p.n_tiles - 1 - (int)blockIdx.x) / p.splits + 1 : 0;   // tiles of this CTA
-    auto tile_of = [&](int k) { return (int)blockIdx.x + k * p.splits; };
+    // work items of this CTA: (head, request tile).  Walk mode: heads blockIdx.x, + walk_ctas, ..., tile 0 each.
+    const int n_my = walk ? (((int)blockIdx.x < p.H) ? (p.H - 1 - (int)blockIdx.x) / p.walk_ctas + 1 : 0)
+                          : (((int)blockIdx.x < p.n_tiles) ? (p.n_tiles - 1 - (int)blockIdx.x) / p.splits + 1 : 0);
+    auto tile_of = [&](int k) { return walk ? 0 : (int)blockIdx.x + k * p.splits; };
+    auto head_of = [&](int k) { return walk ? (int)blockIdx.x + k * p.walk_ctas : (int)blockIdx.y; };
+    auto issue_weights = [&](uint32_t ld, int h) {   // barrier n completes when weight block n has landed
+#pragma unroll 1
+        for (int n = 0; n < 4; ++n) {
+            mbar_arrive_expect_tx_if(ld, &w_full[n], W_BYTES / 4);
+            tma_load_3d_if(ld, sW + n * 32768, &tm_w, &w_full[n], 0, n * 128, h);
+            tma_load_3d_if(ld, sW + n * 32768 + 16384, &tm_w, &w_full[n], 64, n * 128, h);
+        }
+    };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -89,16 +104,11 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         __syncwarp();
         if (n_my > 0) {
             const uint32_t ld = elect_one() ? 1u : 0u;
-            // the first query tile and the weights, all at once; barrier n completes when weight block n has landed
+            // the first query tile and the weights, all at once
             mbar_arrive_expect_tx_if(ld, q_full, A_BYTES);
-            tma_load_3d_if(ld, sA, &tm_q, q_full, 0, h, tile_of(0) * 128);
-            tma_load_3d_if(ld, sA + 16384, &tm_q, q_full, 64, h, tile_of(0) * 128);
-#pragma unroll 1
-            for (int n = 0; n < 4; ++n) {
-                mbar_arrive_expect_tx_if(ld, &w_full[n], W_BYTES / 4);
-                tma_load_3d_if(ld, sW + n * 32768, &tm_w, &w_full[n], 0, n * 128, h);
-                tma_load_3d_if(ld, sW + n * 32768 + 16384, &tm_w, &w_full[n], 64, n * 128, h);
-            }
+            tma_load_3d_if(ld, sA, &tm_q, q_full, 0, head_of(0), tile_of(0) * 128);
+            tma_load_3d_if(ld, sA + 16384, &tm_q, q_full, 64, head_of(0), tile_of(0) * 128);
+            issue_weights(ld, head_of(0));
         }
     }
     if (warp == 1) tmem_alloc(tmem_holder, 512);
@@ -109,13 +119,15 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
     int q_issued = n_my > 0 ? 1 : 0;   // producer warp: query tiles issued, for the abort path
     if (warp == 0) {
-        // the remaining query tiles: tile k goes into the buffer once the products of tile k - 1 have read it
+        // the remaining items: item k goes into the buffers once the products of item k - 1 have read them (walk mode:
+        // the next head's weights as well)
         const uint32_t ld = elect_one() ? 1u : 0u;
         for (int k = 1; k < n_my; ++k) {
             if (!mbar_wait_warp(acc_full, (k - 1) & 1, abort_flag)) break;
             mbar_arrive_expect_tx_if(ld, q_full, A_BYTES);
-            tma_load_3d_if(ld, sA, &tm_q, q_full, 0, h, tile_of(k) * 128);
-            tma_load_3d_if(ld, sA + 16384, &tm_q, q_full, 64, h, tile_of(k) * 128);
+            tma_load_3d_if(ld, sA, &tm_q, q_full, 0, head_of(k), tile_of(k) * 128);
+            tma_load_3d_if(ld, sA + 16384, &tm_q, q_full, 64, head_of(k), tile_of(k) * 128);
+            if (walk) issue_weights(ld, head_of(k));
             q_issued = k + 1;
         }
     } else if (warp == 1) {
@@ -128,8 +140,8 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             if (!ok) break;
             tc_fence_after();
             for (int n = 0; n < 4 && ok; ++n) {
-                if (k == 0) {
-                    ok = mbar_wait_warp(&w_full[n], 0, abort_flag);
+                if (k == 0 || walk) {
+                    ok = mbar_wait_warp(&w_full[n], walk ? (k & 1) : 0, abort_flag);
                     if (!ok) break;
                 }
 #pragma unroll
@@ -154,6 +166,7 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             if (!ok) break;
             tc_fence_after();
             const int b0 = tile_of(k) * 128;
+            const int h = head_of(k);
             if (p.B <= 32) {
                 // A handful of requests (one warp's rows at most): the staged store's two block-wide barriers per
                 // result block cost more than they save; every thread writes its own row.
@@ -224,7 +237,7 @@ q_absorb_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         // A wait gave up: the copies that can still be in flight are the weight blocks and the query tile issued last;
         // wait for them (with a limit) before the shared memory is released, then report.
         if (warp == 0 && n_my > 0) {
-            for (int n = 0; n < 4; ++n) mbar_drain(&w_full[n], 0);
+            for (int n = 0; n < 4; ++n) mbar_drain(&w_full[n], walk ? (q_issued - 1) & 1 : 0);
             mbar_drain(q_full, (q_issued - 1) & 1);
         }
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, 4);
@@ -246,7 +259,7 @@ cudaError_t make_q_absorb_tmap(const void* w_uk_t, int H, CUtensorMap* tm_w) {
     return make_tmap_bf16(tm_w, w_uk_t, 3, dims, str, box);
 }
 
-cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int n_sm, int* status,
+cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, void* q_abs, int B, int H, int n_sm, int walk_ctas, int* status,
                                   const int32_t* seq_lens, int32_t* order, const int32_t* block_table, int max_pages,
                                   int page_size, int32_t* desc, cudaStream_t s) {
     if (B <= 0) return cudaSuccess;
@@ -270,9 +283,11 @@ cudaError_t launch_q_absorb_sm100(const void* q_nope, const CUtensorMap* tm_w, v
     // one CTA per head keeps the head's weights resident over all of its request tiles; with more SMs than heads
     // the tiles of a head are dealt to several CTAs
     const int splits = std::max(1, std::min(n_tiles, std::max(n_sm, 1) / H));
-    QAbsorbParams p{q_abs, B, H, n_tiles, splits, status, seq_lens, order, block_table, max_pages, page_size,
+    // walk mode only with one request tile per head and fewer working CTAs than heads
+    const int walk = (n_tiles == 1 && walk_ctas > 0 && walk_ctas < H) ? walk_ctas : 0;
+    QAbsorbParams p{q_abs, B, H, n_tiles, splits, walk, status, seq_lens, order, block_table, max_pages, page_size,
                     (with_order && block_table != nullptr) ? reinterpret_cast<int4*>(desc) : nullptr};
-    dim3 grid(splits, H + (with_order ? 1 : 0), 1);
+    const dim3 grid = walk ? dim3(walk + (with_order ? 1 : 0), 1, 1) : dim3(splits, H + (with_order ? 1 : 0), 1);
     return launch_pdl(q_absorb_sm100_kernel, grid, dim3(192), SMEM_BYTES, s, tm_q, *tm_w, tm_out, p);
 }
 
