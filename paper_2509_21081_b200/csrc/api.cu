@@ -709,7 +709,16 @@ static int decode_core(const Settings& cfg, const typhoon_mla_shared* sh, const 
                     naive_ctas = std::max(naive_ctas, jobs[j].n_ranges * groups);
                 }
                 const int free_sms = sh->num_sms - naive_ctas;
-                if (n_jobs == 1 && free_sms >= 8 && free_sms < H) walk_ctas = free_sms;
+                if (n_jobs == 1 && free_sms >= 8 && free_sms < H) {
+                    // ... but only if the shared-prefix kernel lasts about as long as the walk (measured: about 5 us per head
+                    // for a walking CTA, 0.7 us per 64-token tile for a shared-prefix CTA; B = 64, H = 128: the walk wins
+                    // from 3072 prefix tokens on and loses at 2048); under a short shared-prefix kernel one CTA per head,
+                    // which spreads over the whole GPU as soon as that kernel ends, is faster.
+                    const int64_t tok = jobs[0].rows <= 128 || jobs[0].sh->fp8 ? 64 : 128;
+                    const int64_t tiles_per_cta = ((jobs[0].sh->Ls + tok - 1) / tok * H + jobs[0].n_ranges - 1) / jobs[0].n_ranges;
+                    const int heads_per_cta = (H + free_sms - 1) / free_sms;
+                    if ((double)tiles_per_cta * (tok == 64 ? 0.7 : 3.0) >= 4.0 * heads_per_cta) walk_ctas = free_sms;
+                }
             }
             e = launch_q_absorb_sm100(q_nope, &sh->tm_wuk_t, q_abs, B, H, sh->num_sms, walk_ctas, sh->status, order ? seq_lens : nullptr, order,
                                       block_table, max_pages, page_size, desc, s);
